@@ -1,0 +1,189 @@
+/*
+ * libtbn -- inference forward of Tiled Bit Network layers on NVIDIA B200 (sm_100a).
+ *
+ * A tiled layer (Tiled Bit Networks, Sec. 3) stores ONE binary tile t of q = N/k
+ * bits plus one scaling factor alpha per layer (Eq. 6) or per tile (Eq. 7-8).  The
+ * layer's N-element weight tensor is the tile repeated k times, reshaped in
+ * row-major order (Eq. 4-5), each repetition scaled by its alpha:
+ *
+ *     B_hat[f] = alpha[f / q] * (bit(t, f % q) ? +1 : -1),   f = row-major flat index
+ *
+ * (k here is the paper's compression factor p.)  The library never materialises
+ * B_hat in device memory except in tbn_expand_tile, which exists for testing.
+ *
+ * General conventions
+ *   - Every pointer is a DEVICE pointer unless its name ends in _host or the
+ *     comment says "host".  The caller owns every buffer; the library allocates
+ *     no device memory, keeps no reference after the call returns and frees nothing.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     All work is enqueued on it and the call returns without synchronising,
+ *     except the *_host entry points, which synchronise the stream before returning.
+ *   - Base pointers must be 16-byte aligned.  Matrices are dense row-major with no
+ *     row padding.
+ *   - Return value: a tbn_status.  Argument errors are detected on the host before
+ *     anything is launched.  No entry point throws, aborts or exits.
+ *   - Same inputs give the same bits out on every call (no order-dependent atomics).
+ *   - Packed tile format: bit i of the tile is bit (i % 32) of 32-bit word (i / 32),
+ *     least-significant bit first; 1 encodes +1, 0 encodes -1.  A packed tile
+ *     occupies tbn_tile_words(q) words (a multiple of 4, i.e. of 128 bits); the
+ *     padding bits are zero.
+ */
+#ifndef TBN_H_
+#define TBN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    TBN_OK = 0,
+    TBN_ERR_INVALID_ARG = -1, /* null pointer, negative size, unknown enum value, misaligned pointer */
+    TBN_ERR_SHAPE = -2,       /* k does not divide N (Sec. 3 requires k*q = N), or sizes inconsistent */
+    TBN_ERR_UNSUPPORTED = -3, /* a combination the library does not implement */
+    TBN_ERR_WORKSPACE = -4,   /* workspace missing or smaller than the matching *_workspace_bytes() */
+    TBN_ERR_CUDA = -5,        /* a CUDA runtime / driver call failed */
+    TBN_ERR_TIMEOUT = -6      /* a device-side bounded wait gave up (see tbn_last_device_status) */
+} tbn_status;
+
+typedef enum { TBN_F32 = 0, TBN_BF16 = 1 } tbn_dtype;
+typedef enum { TBN_ALPHA_PER_LAYER = 0, TBN_ALPHA_PER_TILE = 1 } tbn_alpha_mode; /* 1 or k floats */
+typedef enum { TBN_ACT_NONE = 0, TBN_ACT_RELU = 1, TBN_ACT_GELU = 2 } tbn_act;   /* GELU: exact erf form */
+
+/* Which kernel family executes a forward call.  AUTO picks by shape. */
+typedef enum {
+    TBN_PATH_AUTO = 0,
+    TBN_PATH_GENERIC = 1, /* CUDA-core kernel; any shape and any alignment of q against the row length */
+    TBN_PATH_SMALL = 2,   /* small-batch kernel; needs q % in_features == 0 */
+    TBN_PATH_TENSOR = 3   /* tcgen05 / TMEM kernel; needs q % in_features == 0 and in_features % 8 == 0 */
+} tbn_path;
+
+/* ceil(q/32) rounded up to a multiple of 4: the number of uint32 words of a packed tile. */
+int64_t tbn_tile_words(int64_t q);
+
+const char *tbn_status_string(int status);
+
+/* ------------------------------------------------------------------------------------------------
+ * Tile construction (Sec. 3, Eq. 1-3 and Eq. 6-8).
+ *
+ *   s_i     = sum_{j<k} W[j*q + i]      fp32, added sequentially in increasing j     (Eq. 1-2)
+ *   bit_i   = (s_i > 0)                 zero, negative zero and NaN give 0 (= -1)    (Eq. 3)
+ *   alpha   = ||S||_1 / N               per layer                                    (Eq. 6)
+ *   alpha_j = ||S[j*q, (j+1)*q)||_1 / q per tile, j < k                              (Eq. 7-8)
+ * where S = A when A is not NULL (the paper's separate tensor for alpha), else W.
+ *
+ * W, A      : N fp32 values, the layer's weight tensor in row-major order.
+ * tile_bits : out, tbn_tile_words(N/k) words.
+ * alpha     : out, 1 float (per layer) or k floats (per tile).
+ * workspace : scratch of at least tbn_aggregate_workspace_bytes(N, k) bytes; contents undefined after.
+ * Errors    : N % k != 0 -> TBN_ERR_SHAPE; N == 0 is TBN_ERR_INVALID_ARG.
+ * The bits equal the CPU definition exactly; alpha is accumulated in fp64 in a fixed order.
+ */
+size_t tbn_aggregate_workspace_bytes(int64_t N, int32_t k);
+int tbn_aggregate_tile(const float *W, const float *A, int64_t N, int32_t k, int alpha_mode,
+                       uint32_t *tile_bits, float *alpha, void *workspace, size_t workspace_bytes,
+                       void *stream);
+
+/* Pack an existing real-valued tile (Sec. 5.1: tiles are stored one bit per element):
+ * src[i] > 0 -> bit 1, else 0.  src: q fp32 values.  tile_bits: tbn_tile_words(q) words. */
+int tbn_pack_tile(const float *src, int64_t q, uint32_t *tile_bits, void *stream);
+
+/* Testing aid, not on the hot path: write B_hat (Eq. 4-5 plus the alpha scaling) as N fp32 values. */
+int tbn_expand_tile(const uint32_t *tile_bits, int64_t N, int32_t k, const float *alpha, int alpha_mode,
+                    float *B_hat, void *stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Fully-connected forward (Sec. 3 "B_hat is used for the operation on the inputs"; Algorithm 1):
+ *
+ *     y[t][o] = act( sum_j B_hat[o][j] * x[t][j] + bias[o] ),   B_hat is out_f x in_f (row-major)
+ *
+ * x    : T x in_f, fp32 or bf16 (x_dtype).      y : T x out_f, fp32 or bf16 (y_dtype).
+ * tile_bits, k, alpha, alpha_mode: as produced by tbn_aggregate_tile with N = out_f*in_f.
+ * bias : out_f fp32 values or NULL (the paper uses none).
+ * Products are accumulated in fp32.  On the TENSOR path fp32 activations are rounded to bf16 first
+ * (into the workspace); the other paths use them as given.
+ * Where the tile spans whole rows (q % in_f == 0) only the q/in_f distinct rows are contracted and the
+ * result is written k times, each copy scaled by its alpha (Sec. 4.1, replicated channels).
+ * workspace: at least tbn_linear_workspace_bytes(...) bytes (may be NULL when that is 0).
+ * T == 0 is a successful no-op.
+ */
+size_t tbn_linear_workspace_bytes(int64_t T, int32_t in_f, int32_t out_f, int32_t k, int x_dtype);
+int tbn_linear_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, int32_t out_f,
+                   const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                   const float *bias, int act, void *y, int y_dtype,
+                   void *workspace, size_t workspace_bytes, void *stream);
+/* Same, with the kernel family forced (TBN_ERR_UNSUPPORTED if the shape does not qualify). */
+int tbn_linear_fwd_path(const void *x, int x_dtype, int64_t T, int32_t in_f, int32_t out_f,
+                        const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                        const float *bias, int act, void *y, int y_dtype,
+                        void *workspace, size_t workspace_bytes, void *stream, int path);
+/* The family TBN_PATH_AUTO resolves to for this shape (a tbn_path), or a negative tbn_status. */
+int tbn_linear_select_path(int64_t T, int32_t in_f, int32_t out_f, int32_t k, int x_dtype);
+
+/* Same layer with HOST activations: x_host and y_host are host buffers (pinned memory recommended).
+ * The call copies x to the device, runs tbn_linear_fwd, copies y back and synchronises `stream`.
+ * workspace (device) must hold tbn_linear_host_workspace_bytes(...) bytes: staging for x and y plus
+ * the forward's own scratch.  tile_bits, alpha and bias stay device pointers (model state). */
+size_t tbn_linear_host_workspace_bytes(int64_t T, int32_t in_f, int32_t out_f, int32_t k,
+                                       int x_dtype, int y_dtype);
+int tbn_linear_fwd_host(const void *x_host, int x_dtype, int64_t T, int32_t in_f, int32_t out_f,
+                        const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                        const float *bias, int act, void *y_host, int y_dtype,
+                        void *workspace, size_t workspace_bytes, void *stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * 2-D convolution forward.  The paper defines tiling for convolutional layers (Sec. 3: the tile
+ * fills the whole weight tensor) but ships no convolution kernel (Sec. 6 lists it as future work).
+ * The weight tensor is (Cout, Cin, kh, kw) in row-major order, N = Cout*Cin*kh*kw:
+ *
+ *   y[b][co][oh][ow] = act( sum_{ci,u,v} B_hat[co][ci][u][v] * x[b][ci][oh*stride+u-pad][ow*stride+v-pad]
+ *                           + bias[co] )
+ *
+ * Cross-correlation (no kernel flip), zero padding, same stride and padding in both directions,
+ * dilation 1, one group.  x: NCHW (Nb, Cin, H, Wd).  y: NCHW (Nb, Cout, Ho, Wo) with
+ * Ho = (H + 2*pad - kh)/stride + 1, Wo likewise.  Where the tile spans whole filters
+ * (q % (Cin*kh*kw) == 0) each distinct filter is applied once and its output channel is written k
+ * times with the k alphas (Sec. 4.1).
+ */
+size_t tbn_conv2d_workspace_bytes(int32_t Nb, int32_t Cin, int32_t H, int32_t Wd, int32_t Cout,
+                                  int32_t kh, int32_t kw, int32_t stride, int32_t pad, int32_t k,
+                                  int x_dtype);
+int tbn_conv2d_fwd(const void *x, int x_dtype, int32_t Nb, int32_t Cin, int32_t H, int32_t Wd,
+                   int32_t Cout, int32_t kh, int32_t kw, int32_t stride, int32_t pad,
+                   const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                   const float *bias, int act, void *y, int y_dtype,
+                   void *workspace, size_t workspace_bytes, void *stream);
+int tbn_conv2d_fwd_path(const void *x, int x_dtype, int32_t Nb, int32_t Cin, int32_t H, int32_t Wd,
+                        int32_t Cout, int32_t kh, int32_t kw, int32_t stride, int32_t pad,
+                        const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                        const float *bias, int act, void *y, int y_dtype,
+                        void *workspace, size_t workspace_bytes, void *stream, int path);
+
+/* ------------------------------------------------------------------------------------------------
+ * Chain of L fully-connected tiled layers (Sec. 5.1: an MLP with a fused ReLU):
+ *     h_0 = x;  h_{l+1} = hidden_act(layer_l(h_l)) for l < L-1;  y = layer_{L-1}(h_{L-1}).
+ * dims (host, L+1 ints): dims[l] -> dims[l+1] is layer l.  ks, alpha_modes: host arrays of L values.
+ * tiles, alphas: HOST arrays of L DEVICE pointers.  No biases.  Hidden tensors are kept in bf16 in
+ * the workspace.  x: T x dims[0];  y: T x dims[L].
+ */
+size_t tbn_mlp_workspace_bytes(int64_t T, int32_t L, const int32_t *dims, const int32_t *ks, int x_dtype);
+int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t *dims,
+                const uint32_t *const *tiles, const int32_t *ks, const float *const *alphas,
+                const int *alpha_modes, int hidden_act, void *y, int y_dtype,
+                void *workspace, size_t workspace_bytes, void *stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Device-side status.  Kernels that wait on hardware barriers bound every wait; when a wait gives
+ * up the kernel records TBN_ERR_TIMEOUT and a detail word (which barrier, which block), abandons
+ * its remaining work and returns normally.  This call synchronises `stream`, reads the record of
+ * the current device into *code / *detail (TBN_OK when nothing was recorded) and clears it.
+ * Returns TBN_OK, or TBN_ERR_CUDA if the synchronisation or the copy failed.
+ */
+int tbn_last_device_status(void *stream, int *code, int *detail);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TBN_H_ */

@@ -1,0 +1,377 @@
+// C entry points of libtbn: argument validation, path selection, workspace carving.
+// Every step of the computation runs in the kernels of the other translation units; nothing here
+// touches the data on the host, and there is no CPU fallback.
+#include <cstring>
+
+#include "common.cuh"
+
+namespace tbn {
+
+// Device-side status record: {code, detail, reserved, reserved}.  Kernels receive its address.
+__device__ int g_device_status[4];
+
+namespace {
+
+int *device_status_ptr()
+{
+    // one address per device, looked up lazily (the symbol has a distinct instance on each device)
+    static int *cache[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!cache[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) return nullptr;
+        cache[dev] = static_cast<int *>(p);
+    }
+    return cache[dev];
+}
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool valid_dtype(int d) { return d == TBN_F32 || d == TBN_BF16; }
+inline bool valid_alpha_mode(int a) { return a == TBN_ALPHA_PER_LAYER || a == TBN_ALPHA_PER_TILE; }
+inline bool valid_act(int a) { return a == TBN_ACT_NONE || a == TBN_ACT_RELU || a == TBN_ACT_GELU; }
+inline size_t dtype_bytes(int d) { return d == TBN_BF16 ? 2 : 4; }
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Validation shared by the fully-connected and convolution entry points.
+int check_layer_common(const void *x, int x_dtype, const uint32_t *tile, int32_t k, const float *alpha,
+                       int alpha_mode, const float *bias, int act, const void *y, int y_dtype, int path)
+{
+    if (!x || !tile || !alpha || !y) return TBN_ERR_INVALID_ARG;
+    if (!valid_dtype(x_dtype) || !valid_dtype(y_dtype) || !valid_alpha_mode(alpha_mode) || !valid_act(act))
+        return TBN_ERR_INVALID_ARG;
+    if (path < TBN_PATH_AUTO || path > TBN_PATH_TENSOR) return TBN_ERR_INVALID_ARG;
+    if (k <= 0) return TBN_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(y) || !aligned16(tile)) return TBN_ERR_INVALID_ARG;
+    if (bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) return TBN_ERR_INVALID_ARG;
+    return TBN_OK;
+}
+
+int select_linear_path(const LayerArgs &a)
+{
+    if (tensor_path_supported(a) && a.T >= 32) return TBN_PATH_TENSOR;
+    if (small_batch_supported(a)) return TBN_PATH_SMALL;
+    if (tensor_path_supported(a)) return TBN_PATH_TENSOR;
+    return TBN_PATH_GENERIC;
+}
+
+size_t tensor_scratch_bytes(int64_t T, int32_t in_f, int x_dtype)
+{
+    // fp32 activations are rounded to bf16 before the tensor-core kernel stages them with TMA
+    return x_dtype == TBN_F32 ? round_up((size_t)T * (size_t)in_f * 2, 256) : 0;
+}
+
+// Runs one layer on the chosen path.  `a` is fully validated.
+int run_layer(LayerArgs a, int path, void *workspace, size_t workspace_bytes, cudaStream_t s)
+{
+    if (a.T == 0) return TBN_OK;
+    if (path == TBN_PATH_AUTO) path = a.is_conv ? TBN_PATH_GENERIC : select_linear_path(a);
+    cudaError_t e = cudaSuccess;
+    switch (path) {
+    case TBN_PATH_GENERIC:
+        e = launch_generic(a, s);
+        break;
+    case TBN_PATH_SMALL:
+        if (a.is_conv || !small_batch_supported(a)) return TBN_ERR_UNSUPPORTED;
+        e = launch_small_batch(a, s);
+        break;
+    case TBN_PATH_TENSOR: {
+        if (a.is_conv || !tensor_path_supported(a)) return TBN_ERR_UNSUPPORTED;
+        if (a.x_dtype == TBN_F32) {
+            const size_t need = tensor_scratch_bytes(a.T, a.n, a.x_dtype);
+            if (!workspace || workspace_bytes < need || !aligned16(workspace)) return TBN_ERR_WORKSPACE;
+            e = launch_f32_to_bf16(static_cast<const float *>(a.x), static_cast<__nv_bfloat16 *>(workspace),
+                                   a.T * (int64_t)a.n, s);
+            if (e != cudaSuccess) return TBN_ERR_CUDA;
+            a.x = workspace;
+            a.x_dtype = TBN_BF16;
+        }
+        int *st = device_status_ptr();
+        if (!st) return TBN_ERR_CUDA;
+        return launch_tensor_linear(a, st, s);
+    }
+    default:
+        return TBN_ERR_INVALID_ARG;
+    }
+    return e == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+}
+
+int fill_linear(LayerArgs &a, const void *x, int x_dtype, int64_t T, int32_t in_f, int32_t out_f,
+                const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                const float *bias, int act, void *y, int y_dtype, int path)
+{
+    if (T < 0 || in_f <= 0 || out_f <= 0) return TBN_ERR_INVALID_ARG;
+    int rc = check_layer_common(x, x_dtype, tile_bits, k, alpha, alpha_mode, bias, act, y, y_dtype, path);
+    if (rc != TBN_OK) return rc;
+    const int64_t N = (int64_t)in_f * out_f;
+    if (N % k != 0) return TBN_ERR_SHAPE;
+    std::memset(&a, 0, sizeof(a));
+    a.x = x; a.y = y; a.tile = tile_bits; a.alpha = alpha; a.bias = bias;
+    a.T = T; a.n = in_f; a.m = out_f; a.k = k; a.q = N / k;
+    a.x_dtype = x_dtype; a.y_dtype = y_dtype; a.alpha_mode = alpha_mode; a.act = act;
+    a.is_conv = 0;
+    return TBN_OK;
+}
+
+int check_mlp(int64_t T, int32_t L, const int32_t *dims, const int32_t *ks)
+{
+    if (T < 0 || L <= 0 || !dims || !ks) return TBN_ERR_INVALID_ARG;
+    for (int32_t l = 0; l <= L; ++l)
+        if (dims[l] <= 0) return TBN_ERR_INVALID_ARG;
+    for (int32_t l = 0; l < L; ++l) {
+        if (ks[l] <= 0) return TBN_ERR_INVALID_ARG;
+        if (((int64_t)dims[l] * dims[l + 1]) % ks[l] != 0) return TBN_ERR_SHAPE;
+    }
+    return TBN_OK;
+}
+
+}  // namespace
+}  // namespace tbn
+
+using namespace tbn;
+
+extern "C" {
+
+int64_t tbn_tile_words(int64_t q)
+{
+    if (q <= 0) return 0;
+    return ((q + 31) / 32 + 3) / 4 * 4;
+}
+
+const char *tbn_status_string(int status)
+{
+    switch (status) {
+    case TBN_OK: return "ok";
+    case TBN_ERR_INVALID_ARG: return "invalid argument";
+    case TBN_ERR_SHAPE: return "shape error: k must divide the number of weights";
+    case TBN_ERR_UNSUPPORTED: return "unsupported combination";
+    case TBN_ERR_WORKSPACE: return "workspace missing or too small";
+    case TBN_ERR_CUDA: return "CUDA call failed";
+    case TBN_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+    }
+}
+
+size_t tbn_aggregate_workspace_bytes(int64_t N, int32_t k)
+{
+    if (N <= 0 || k <= 0 || N % k != 0) return 0;
+    return round_up(aggregate_workspace_bytes(N, k), 256);
+}
+
+int tbn_aggregate_tile(const float *W, const float *A, int64_t N, int32_t k, int alpha_mode,
+                       uint32_t *tile_bits, float *alpha, void *workspace, size_t workspace_bytes,
+                       void *stream)
+{
+    if (!W || !tile_bits || !alpha || N <= 0 || k <= 0 || !valid_alpha_mode(alpha_mode))
+        return TBN_ERR_INVALID_ARG;
+    if (N % k != 0) return TBN_ERR_SHAPE;
+    if (!aligned16(W) || (A && !aligned16(A)) || !aligned16(tile_bits)) return TBN_ERR_INVALID_ARG;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < aggregate_workspace_bytes(N, k))
+        return TBN_ERR_WORKSPACE;
+    cudaError_t e = launch_aggregate(W, A, N, k, alpha_mode == TBN_ALPHA_PER_TILE, tile_bits, alpha,
+                                     workspace, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+}
+
+int tbn_pack_tile(const float *src, int64_t q, uint32_t *tile_bits, void *stream)
+{
+    if (!src || !tile_bits || q <= 0) return TBN_ERR_INVALID_ARG;
+    if (!aligned16(tile_bits)) return TBN_ERR_INVALID_ARG;
+    cudaError_t e = launch_pack(src, q, tile_bits, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+}
+
+int tbn_expand_tile(const uint32_t *tile_bits, int64_t N, int32_t k, const float *alpha, int alpha_mode,
+                    float *B_hat, void *stream)
+{
+    if (!tile_bits || !alpha || !B_hat || N <= 0 || k <= 0 || !valid_alpha_mode(alpha_mode))
+        return TBN_ERR_INVALID_ARG;
+    if (N % k != 0) return TBN_ERR_SHAPE;
+    cudaError_t e = launch_expand(tile_bits, N, k, alpha, alpha_mode == TBN_ALPHA_PER_TILE, B_hat,
+                                  static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+}
+
+size_t tbn_linear_workspace_bytes(int64_t T, int32_t in_f, int32_t out_f, int32_t k, int x_dtype)
+{
+    (void)out_f; (void)k;
+    if (T <= 0 || in_f <= 0) return 0;
+    return tensor_scratch_bytes(T, in_f, x_dtype);
+}
+
+int tbn_linear_select_path(int64_t T, int32_t in_f, int32_t out_f, int32_t k, int x_dtype)
+{
+    if (T < 0 || in_f <= 0 || out_f <= 0 || k <= 0 || !valid_dtype(x_dtype)) return TBN_ERR_INVALID_ARG;
+    if (((int64_t)in_f * out_f) % k != 0) return TBN_ERR_SHAPE;
+    LayerArgs a;
+    std::memset(&a, 0, sizeof(a));
+    a.T = T; a.n = in_f; a.m = out_f; a.k = k; a.q = (int64_t)in_f * out_f / k;
+    a.x_dtype = x_dtype; a.y_dtype = TBN_BF16;
+    return select_linear_path(a);
+}
+
+int tbn_linear_fwd_path(const void *x, int x_dtype, int64_t T, int32_t in_f, int32_t out_f,
+                        const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                        const float *bias, int act, void *y, int y_dtype,
+                        void *workspace, size_t workspace_bytes, void *stream, int path)
+{
+    LayerArgs a;
+    int rc = fill_linear(a, x, x_dtype, T, in_f, out_f, tile_bits, k, alpha, alpha_mode, bias, act, y,
+                         y_dtype, path);
+    if (rc != TBN_OK) return rc;
+    return run_layer(a, path, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+int tbn_linear_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, int32_t out_f,
+                   const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                   const float *bias, int act, void *y, int y_dtype,
+                   void *workspace, size_t workspace_bytes, void *stream)
+{
+    return tbn_linear_fwd_path(x, x_dtype, T, in_f, out_f, tile_bits, k, alpha, alpha_mode, bias, act, y,
+                               y_dtype, workspace, workspace_bytes, stream, TBN_PATH_AUTO);
+}
+
+size_t tbn_linear_host_workspace_bytes(int64_t T, int32_t in_f, int32_t out_f, int32_t k,
+                                       int x_dtype, int y_dtype)
+{
+    if (T <= 0 || in_f <= 0 || out_f <= 0 || !valid_dtype(x_dtype) || !valid_dtype(y_dtype)) return 0;
+    return round_up((size_t)T * in_f * dtype_bytes(x_dtype), 256) +
+           round_up((size_t)T * out_f * dtype_bytes(y_dtype), 256) +
+           tbn_linear_workspace_bytes(T, in_f, out_f, k, x_dtype);
+}
+
+int tbn_linear_fwd_host(const void *x_host, int x_dtype, int64_t T, int32_t in_f, int32_t out_f,
+                        const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                        const float *bias, int act, void *y_host, int y_dtype,
+                        void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!x_host || !y_host || !valid_dtype(x_dtype) || !valid_dtype(y_dtype) || T < 0 || in_f <= 0 ||
+        out_f <= 0)
+        return TBN_ERR_INVALID_ARG;
+    if (T == 0) return TBN_OK;
+    const size_t xb = round_up((size_t)T * in_f * dtype_bytes(x_dtype), 256);
+    const size_t yb = round_up((size_t)T * out_f * dtype_bytes(y_dtype), 256);
+    const size_t inner = tbn_linear_workspace_bytes(T, in_f, out_f, k, x_dtype);
+    if (!workspace || !aligned16(workspace) || workspace_bytes < xb + yb + inner) return TBN_ERR_WORKSPACE;
+    char *ws = static_cast<char *>(workspace);
+    void *x_dev = ws, *y_dev = ws + xb, *inner_ws = ws + xb + yb;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(x_dev, x_host, (size_t)T * in_f * dtype_bytes(x_dtype), cudaMemcpyHostToDevice, s) !=
+        cudaSuccess)
+        return TBN_ERR_CUDA;
+    int rc = tbn_linear_fwd(x_dev, x_dtype, T, in_f, out_f, tile_bits, k, alpha, alpha_mode, bias, act, y_dev,
+                            y_dtype, inner_ws, inner, stream);
+    if (rc != TBN_OK) return rc;
+    if (cudaMemcpyAsync(y_host, y_dev, (size_t)T * out_f * dtype_bytes(y_dtype), cudaMemcpyDeviceToHost, s) !=
+        cudaSuccess)
+        return TBN_ERR_CUDA;
+    return cudaStreamSynchronize(s) == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+}
+
+size_t tbn_conv2d_workspace_bytes(int32_t, int32_t, int32_t, int32_t, int32_t, int32_t, int32_t, int32_t,
+                                  int32_t, int32_t, int)
+{
+    return 0;
+}
+
+int tbn_conv2d_fwd_path(const void *x, int x_dtype, int32_t Nb, int32_t Cin, int32_t H, int32_t Wd,
+                        int32_t Cout, int32_t kh, int32_t kw, int32_t stride, int32_t pad,
+                        const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                        const float *bias, int act, void *y, int y_dtype,
+                        void *workspace, size_t workspace_bytes, void *stream, int path)
+{
+    if (Nb < 0 || Cin <= 0 || H <= 0 || Wd <= 0 || Cout <= 0 || kh <= 0 || kw <= 0 || stride <= 0 || pad < 0)
+        return TBN_ERR_INVALID_ARG;
+    int rc = check_layer_common(x, x_dtype, tile_bits, k, alpha, alpha_mode, bias, act, y, y_dtype, path);
+    if (rc != TBN_OK) return rc;
+    if (H + 2 * pad < kh || Wd + 2 * pad < kw) return TBN_ERR_SHAPE;
+    const int64_t n = (int64_t)Cin * kh * kw;
+    if (n > 0x7fffffffLL) return TBN_ERR_UNSUPPORTED;
+    const int64_t N = n * Cout;
+    if (N % k != 0) return TBN_ERR_SHAPE;
+    LayerArgs a;
+    std::memset(&a, 0, sizeof(a));
+    a.x = x; a.y = y; a.tile = tile_bits; a.alpha = alpha; a.bias = bias;
+    a.n = (int32_t)n; a.m = Cout; a.k = k; a.q = N / k;
+    a.x_dtype = x_dtype; a.y_dtype = y_dtype; a.alpha_mode = alpha_mode; a.act = act;
+    a.is_conv = 1;
+    a.Nb = Nb; a.Cin = Cin; a.H = H; a.Wd = Wd; a.kh = kh; a.kw = kw; a.stride = stride; a.pad = pad;
+    a.Ho = (H + 2 * pad - kh) / stride + 1;
+    a.Wo = (Wd + 2 * pad - kw) / stride + 1;
+    a.T = (int64_t)Nb * a.Ho * a.Wo;
+    return run_layer(a, path, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+int tbn_conv2d_fwd(const void *x, int x_dtype, int32_t Nb, int32_t Cin, int32_t H, int32_t Wd,
+                   int32_t Cout, int32_t kh, int32_t kw, int32_t stride, int32_t pad,
+                   const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                   const float *bias, int act, void *y, int y_dtype,
+                   void *workspace, size_t workspace_bytes, void *stream)
+{
+    return tbn_conv2d_fwd_path(x, x_dtype, Nb, Cin, H, Wd, Cout, kh, kw, stride, pad, tile_bits, k, alpha,
+                               alpha_mode, bias, act, y, y_dtype, workspace, workspace_bytes, stream,
+                               TBN_PATH_AUTO);
+}
+
+size_t tbn_mlp_workspace_bytes(int64_t T, int32_t L, const int32_t *dims, const int32_t *ks, int x_dtype)
+{
+    if (check_mlp(T, L, dims, ks) != TBN_OK || T == 0) return 0;
+    // two ping-pong bf16 hidden buffers sized for the widest hidden layer + the first layer's scratch
+    int32_t widest = 0;
+    for (int32_t l = 1; l < L; ++l) widest = dims[l] > widest ? dims[l] : widest;
+    const size_t hidden = round_up((size_t)T * widest * 2, 256);
+    return 2 * hidden + tbn_linear_workspace_bytes(T, dims[0], dims[1], ks[0], x_dtype);
+}
+
+int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t *dims,
+                const uint32_t *const *tiles, const int32_t *ks, const float *const *alphas,
+                const int *alpha_modes, int hidden_act, void *y, int y_dtype,
+                void *workspace, size_t workspace_bytes, void *stream)
+{
+    int rc = check_mlp(T, L, dims, ks);
+    if (rc != TBN_OK) return rc;
+    if (!x || !y || !tiles || !alphas || !alpha_modes || !valid_act(hidden_act)) return TBN_ERR_INVALID_ARG;
+    for (int32_t l = 0; l < L; ++l)
+        if (!tiles[l] || !alphas[l] || !valid_alpha_mode(alpha_modes[l])) return TBN_ERR_INVALID_ARG;
+    if (T == 0) return TBN_OK;
+    const size_t need = tbn_mlp_workspace_bytes(T, L, dims, ks, x_dtype);
+    if (need > 0 && (!workspace || !aligned16(workspace) || workspace_bytes < need)) return TBN_ERR_WORKSPACE;
+    int32_t widest = 0;
+    for (int32_t l = 1; l < L; ++l) widest = dims[l] > widest ? dims[l] : widest;
+    const size_t hidden = round_up((size_t)T * widest * 2, 256);
+    char *ws = static_cast<char *>(workspace);
+    void *buf[2] = {ws, ws + hidden};
+    void *scratch = ws + 2 * hidden;
+    const size_t scratch_bytes = need - 2 * hidden;
+
+    const void *cur = x;
+    int cur_dtype = x_dtype;
+    for (int32_t l = 0; l < L; ++l) {
+        const bool last = l == L - 1;
+        void *out = last ? y : buf[l & 1];
+        rc = tbn_linear_fwd(cur, cur_dtype, T, dims[l], dims[l + 1], tiles[l], ks[l], alphas[l],
+                            alpha_modes[l], nullptr, last ? TBN_ACT_NONE : hidden_act, out,
+                            last ? y_dtype : TBN_BF16, scratch, l == 0 ? scratch_bytes : 0, stream);
+        if (rc != TBN_OK) return rc;
+        cur = out;
+        cur_dtype = TBN_BF16;
+    }
+    return TBN_OK;
+}
+
+int tbn_last_device_status(void *stream, int *code, int *detail)
+{
+    if (!code || !detail) return TBN_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int *st = device_status_ptr();
+    if (!st) return TBN_ERR_CUDA;
+    int host[4] = {0, 0, 0, 0};
+    if (cudaStreamSynchronize(s) != cudaSuccess) return TBN_ERR_CUDA;
+    if (cudaMemcpy(host, st, sizeof(host), cudaMemcpyDeviceToHost) != cudaSuccess) return TBN_ERR_CUDA;
+    *code = host[0];
+    *detail = host[1];
+    if (host[0] != 0 && cudaMemset(st, 0, sizeof(host)) != cudaSuccess) return TBN_ERR_CUDA;
+    return TBN_OK;
+}
+
+}  // extern "C"

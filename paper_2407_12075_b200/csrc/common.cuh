@@ -1,0 +1,69 @@
+// Shared declarations of the libtbn translation units (internal; the public surface is include/tbn.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "tbn.h"
+
+namespace tbn {
+
+// ---- scalar helpers ---------------------------------------------------------------------------
+__device__ __forceinline__ float load_as_float(const float *p, int64_t i) { return p[i]; }
+__device__ __forceinline__ float load_as_float(const __nv_bfloat16 *p, int64_t i) {
+    return __bfloat162float(p[i]);
+}
+__device__ __forceinline__ void store_from_float(float *p, int64_t i, float v) { p[i] = v; }
+__device__ __forceinline__ void store_from_float(__nv_bfloat16 *p, int64_t i, float v) {
+    p[i] = __float2bfloat16_rn(v);
+}
+
+__device__ __forceinline__ float apply_act(float v, int act) {
+    if (act == TBN_ACT_RELU) return fmaxf(v, 0.0f);
+    if (act == TBN_ACT_GELU) return 0.5f * v * (1.0f + erff(v * 0.70710678118654752440f));
+    return v;
+}
+
+// One bit of a packed tile (LSB-first 32-bit words).
+__device__ __forceinline__ uint32_t tile_bit(const uint32_t *__restrict__ words, int64_t i) {
+    return (__ldg(words + (i >> 5)) >> (uint32_t)(i & 31)) & 1u;
+}
+
+// ---- description of one layer call, filled by the C entry points --------------------------------
+struct LayerArgs {
+    const void *x;
+    void *y;
+    const uint32_t *tile;
+    const float *alpha;
+    const float *bias;
+    int64_t T;       // rows of the contraction: tokens, or Nb*Ho*Wo output pixels
+    int32_t n;       // contraction length: in_features or Cin*kh*kw
+    int32_t m;       // output features / channels
+    int32_t k;       // number of tile repetitions
+    int64_t q;       // tile length in bits
+    int x_dtype, y_dtype, alpha_mode, act;
+    // convolution geometry (is_conv == 0 for fully-connected)
+    int is_conv;
+    int32_t Nb, Cin, H, Wd, kh, kw, stride, pad, Ho, Wo;
+};
+
+// ---- launchers implemented in the other translation units ---------------------------------------
+cudaError_t launch_aggregate(const float *W, const float *A, int64_t N, int32_t k, int per_tile,
+                             uint32_t *tile_bits, float *alpha, void *workspace, cudaStream_t s);
+size_t aggregate_workspace_bytes(int64_t N, int32_t k);
+cudaError_t launch_pack(const float *src, int64_t q, uint32_t *tile_bits, cudaStream_t s);
+cudaError_t launch_expand(const uint32_t *tile_bits, int64_t N, int32_t k, const float *alpha,
+                          int per_tile, float *B_hat, cudaStream_t s);
+cudaError_t launch_f32_to_bf16(const float *src, __nv_bfloat16 *dst, int64_t count, cudaStream_t s);
+
+cudaError_t launch_generic(const LayerArgs &a, cudaStream_t s);
+
+bool small_batch_supported(const LayerArgs &a);
+cudaError_t launch_small_batch(const LayerArgs &a, cudaStream_t s);
+
+// The tensor-core path reports through a tbn_status because it also uses the driver API.
+bool tensor_path_supported(const LayerArgs &a);
+int launch_tensor_linear(const LayerArgs &a, int *device_status, cudaStream_t s);
+
+}  // namespace tbn

@@ -1,0 +1,204 @@
+// Tile construction kernels: chunk-sum + threshold + bit packing (Eq. 1-3), scaling factors
+// (Eq. 6-8), packing of an existing tile, and the test-only expansion (Eq. 4-5).
+//
+// All of them are streaming, HBM-bound kernels: W (and A) are read exactly once with coalesced
+// 128-byte warp accesses, the packed tile is written once.
+#include "common.cuh"
+
+namespace tbn {
+
+namespace {
+
+constexpr int kAggThreads = 256;
+constexpr int kAggIter = 4;                               // columns per thread
+constexpr int kAggCols = kAggThreads * kAggIter;          // columns per block (multiple of 32)
+
+struct AggScratch {          // layout of the caller's workspace
+    unsigned int ticket;     // blocks that have published their partial sums
+    unsigned int pad[3];
+    // followed by k * gridDim.x doubles: partial[j * blocks + b]
+};
+
+// Block b owns columns [b*kAggCols, (b+1)*kAggCols) of the k x q view of W.  For every column it
+// forms s = ((0 + W[0][c]) + W[1][c]) + ... in fp32, one rounding per add, exactly the sequential
+// sum the CPU definition uses, so the sign -- and therefore the bit -- is identical.  Alongside, the
+// block accumulates |S| per tile in fp64 and publishes it; the last block to finish adds the
+// partials of all blocks in a fixed order, which makes alpha reproducible from run to run.
+__global__ void __launch_bounds__(kAggThreads)
+aggregate_kernel(const float *__restrict__ W, const float *__restrict__ A, int64_t q, int32_t k,
+                 int per_tile, uint32_t *__restrict__ tile_bits, int64_t n_words,
+                 float *__restrict__ alpha, AggScratch *scratch)
+{
+    __shared__ double warp_part[2][kAggThreads / 32];
+    __shared__ double red[kAggThreads];
+    __shared__ unsigned int s_ticket;
+
+    const int tid = threadIdx.x;
+    const int lane = tid & 31, warp = tid >> 5;
+    const int64_t base = (int64_t)blockIdx.x * kAggCols;
+    double *partial = reinterpret_cast<double *>(scratch + 1);
+    const unsigned int blocks = gridDim.x;
+
+    float s[kAggIter];
+#pragma unroll
+    for (int it = 0; it < kAggIter; ++it) s[it] = 0.0f;
+
+    for (int32_t j = 0; j < k; ++j) {
+        const int64_t row = (int64_t)j * q;
+        float a_abs = 0.0f;
+#pragma unroll
+        for (int it = 0; it < kAggIter; ++it) {
+            const int64_t c = base + it * kAggThreads + tid;
+            if (c < q) {
+                const float w = __ldg(W + row + c);
+                s[it] = __fadd_rn(s[it], w);             // never fused, never reassociated
+                a_abs += fabsf(A ? __ldg(A + row + c) : w);
+            }
+        }
+        double d = (double)a_abs;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
+        if (lane == 0) warp_part[j & 1][warp] = d;
+        __syncthreads();
+        if (tid == 0) {
+            double t = 0.0;
+#pragma unroll
+            for (int w = 0; w < kAggThreads / 32; ++w) t += warp_part[j & 1][w];
+            partial[(int64_t)j * blocks + blockIdx.x] = t;
+        }
+    }
+
+    // Eq. 3 + packing: lane l of a warp holds column (32*g + l); the ballot is the packed word.
+#pragma unroll
+    for (int it = 0; it < kAggIter; ++it) {
+        const int64_t c0 = base + it * kAggThreads + warp * 32;
+        const uint32_t word = __ballot_sync(0xffffffffu, s[it] > 0.0f);   // NaN and +-0 give 0
+        const int64_t widx = c0 >> 5;
+        if (lane == 0 && widx < n_words) tile_bits[widx] = word;
+    }
+
+    // Publish, then let the last block reduce.
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_ticket = atomicAdd(&scratch->ticket, 1u);
+    __syncthreads();
+    if (s_ticket != blocks - 1) return;
+    __threadfence();
+
+    const volatile double *vp = partial;
+    if (per_tile) {
+        for (int32_t j = 0; j < k; ++j) {
+            double t = 0.0;
+            for (unsigned int b = tid; b < blocks; b += kAggThreads) t += vp[(int64_t)j * blocks + b];
+            red[tid] = t;
+            __syncthreads();
+            for (int off = kAggThreads / 2; off > 0; off >>= 1) {
+                if (tid < off) red[tid] += red[tid + off];
+                __syncthreads();
+            }
+            if (tid == 0) alpha[j] = (float)(red[0] / (double)q);
+            __syncthreads();
+        }
+    } else {
+        double t = 0.0;
+        const int64_t total = (int64_t)k * blocks;
+        for (int64_t b = tid; b < total; b += kAggThreads) t += vp[b];
+        red[tid] = t;
+        __syncthreads();
+        for (int off = kAggThreads / 2; off > 0; off >>= 1) {
+            if (tid < off) red[tid] += red[tid + off];
+            __syncthreads();
+        }
+        if (tid == 0) alpha[0] = (float)(red[0] / ((double)q * (double)k));
+    }
+}
+
+__global__ void __launch_bounds__(256)
+pack_kernel(const float *__restrict__ src, int64_t q, uint32_t *__restrict__ tile_bits, int64_t n_words)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warp_global = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t warps_total = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t w = warp_global; w < n_words; w += warps_total) {
+        const int64_t i = w * 32 + lane;
+        const bool pos = (i < q) && (__ldg(src + i) > 0.0f);
+        const uint32_t word = __ballot_sync(0xffffffffu, pos);
+        if (lane == 0) tile_bits[w] = word;
+    }
+}
+
+__global__ void __launch_bounds__(256)
+expand_kernel(const uint32_t *__restrict__ tile_bits, int64_t N, int64_t q, const float *__restrict__ alpha,
+              int per_tile, float *__restrict__ B_hat)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t f = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; f < N; f += stride) {
+        const int64_t i = f % q;
+        const float a = per_tile ? __ldg(alpha + f / q) : __ldg(alpha);
+        B_hat[f] = tile_bit(tile_bits, i) ? a : -a;
+    }
+}
+
+__global__ void __launch_bounds__(256)
+f32_to_bf16_kernel(const float *__restrict__ src, __nv_bfloat16 *__restrict__ dst, int64_t count)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t pairs = count >> 1;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < pairs; i += stride) {
+        const float2 v = __ldg(reinterpret_cast<const float2 *>(src) + i);
+        reinterpret_cast<__nv_bfloat162 *>(dst)[i] = __floats2bfloat162_rn(v.x, v.y);
+    }
+    if ((count & 1) && blockIdx.x == 0 && threadIdx.x == 0)
+        dst[count - 1] = __float2bfloat16_rn(src[count - 1]);
+}
+
+int grid_for(int64_t work_items, int threads, int cap_blocks)
+{
+    int64_t b = (work_items + threads - 1) / threads;
+    if (b < 1) b = 1;
+    if (b > cap_blocks) b = cap_blocks;
+    return (int)b;
+}
+
+}  // namespace
+
+size_t aggregate_workspace_bytes(int64_t N, int32_t k)
+{
+    const int64_t q = N / k;
+    const int64_t blocks = (q + kAggCols - 1) / kAggCols;
+    return sizeof(AggScratch) + (size_t)k * (size_t)blocks * sizeof(double);
+}
+
+cudaError_t launch_aggregate(const float *W, const float *A, int64_t N, int32_t k, int per_tile,
+                             uint32_t *tile_bits, float *alpha, void *workspace, cudaStream_t s)
+{
+    const int64_t q = N / k;
+    const int64_t blocks = (q + kAggCols - 1) / kAggCols;
+    cudaError_t e = cudaMemsetAsync(workspace, 0, sizeof(AggScratch), s);
+    if (e != cudaSuccess) return e;
+    aggregate_kernel<<<(unsigned)blocks, kAggThreads, 0, s>>>(
+        W, A, q, k, per_tile, tile_bits, tbn_tile_words(q), alpha, static_cast<AggScratch *>(workspace));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pack(const float *src, int64_t q, uint32_t *tile_bits, cudaStream_t s)
+{
+    const int64_t n_words = tbn_tile_words(q);
+    pack_kernel<<<grid_for(n_words * 32, 256, 148 * 8), 256, 0, s>>>(src, q, tile_bits, n_words);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_expand(const uint32_t *tile_bits, int64_t N, int32_t k, const float *alpha,
+                          int per_tile, float *B_hat, cudaStream_t s)
+{
+    expand_kernel<<<grid_for(N, 256, 148 * 8), 256, 0, s>>>(tile_bits, N, N / k, alpha, per_tile, B_hat);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_f32_to_bf16(const float *src, __nv_bfloat16 *dst, int64_t count, cudaStream_t s)
+{
+    f32_to_bf16_kernel<<<grid_for(count / 2 + 1, 256, 148 * 8), 256, 0, s>>>(src, dst, count);
+    return cudaGetLastError();
+}
+
+}  // namespace tbn

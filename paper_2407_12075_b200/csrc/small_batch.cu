@@ -1,0 +1,160 @@
+// Small-batch forward (a handful of tokens): the matrix-vector regime of Algorithm 1.
+//
+// Needs the tile to span whole rows (q % n == 0), so only r = q/n distinct rows exist; each is
+// contracted once and written k times with the k alphas (Sec. 4.1, replicated channels).
+//
+// One warp owns RW distinct rows.  Lane l walks the row in groups of 256 weights and takes the 8
+// weights [256*i + 8*l, +8): one 16-byte (bf16) or two 16-byte (fp32) coalesced activation loads per
+// token, shared by the warp's RW rows, and one byte of tile bits per row (32 consecutive bytes per
+// warp).  A weight bit becomes the float +-1 by OR-ing its inverted value into the sign position of
+// 1.0f, so the inner operation is a single FMA per token.  Lanes are combined with warp shuffles.
+#include "common.cuh"
+
+namespace tbn {
+
+namespace {
+
+constexpr int kWarps = 4;
+
+template <typename XT> struct XVec;
+template <> struct XVec<__nv_bfloat16> {
+    static __device__ __forceinline__ void load8(const __nv_bfloat16 *p, float (&v)[8]) {
+        const uint4 u = __ldg(reinterpret_cast<const uint4 *>(p));
+        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            v[2 * i] = __uint_as_float(w[i] << 16);
+            v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
+    }
+};
+template <> struct XVec<float> {
+    static __device__ __forceinline__ void load8(const float *p, float (&v)[8]) {
+        const float4 a = __ldg(reinterpret_cast<const float4 *>(p));
+        const float4 b = __ldg(reinterpret_cast<const float4 *>(p) + 1);
+        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+        v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    }
+};
+
+template <typename XT, int RW, int TT>
+__global__ void __launch_bounds__(kWarps * 32)
+small_batch_kernel(const LayerArgs a, int32_t r)
+{
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int32_t row0 = (blockIdx.x * kWarps + warp) * RW;      // first distinct row of this warp
+    const int64_t t0 = (int64_t)blockIdx.y * TT;
+    if (row0 >= r) return;
+
+    const XT *x = static_cast<const XT *>(a.x);
+    const uint8_t *bits = reinterpret_cast<const uint8_t *>(a.tile);
+    const int32_t n = a.n;
+    const int32_t row_bytes = n >> 3;
+
+    float acc[RW][TT];
+#pragma unroll
+    for (int rr = 0; rr < RW; ++rr)
+#pragma unroll
+        for (int t = 0; t < TT; ++t) acc[rr][t] = 0.0f;
+
+    for (int32_t e0 = lane * 8; e0 < n; e0 += 256) {
+        float xv[TT][8];
+#pragma unroll
+        for (int t = 0; t < TT; ++t) {
+            if (t0 + t < a.T) {
+                XVec<XT>::load8(x + (t0 + t) * n + e0, xv[t]);
+            } else {
+#pragma unroll
+                for (int b = 0; b < 8; ++b) xv[t][b] = 0.0f;
+            }
+        }
+#pragma unroll
+        for (int rr = 0; rr < RW; ++rr) {
+            const int32_t row = min(row0 + rr, r - 1);            // clamp: extra rows are not stored
+            const uint32_t nb = ~(uint32_t)__ldg(bits + (int64_t)row * row_bytes + (e0 >> 3));
+#pragma unroll
+            for (int b = 0; b < 8; ++b) {
+                const float sgn = __uint_as_float(0x3f800000u | ((nb << (31 - b)) & 0x80000000u));
+#pragma unroll
+                for (int t = 0; t < TT; ++t) acc[rr][t] = fmaf(sgn, xv[t][b], acc[rr][t]);
+            }
+        }
+    }
+
+#pragma unroll
+    for (int rr = 0; rr < RW; ++rr)
+#pragma unroll
+        for (int t = 0; t < TT; ++t) {
+            float v = acc[rr][t];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+            acc[rr][t] = v;
+        }
+
+    // every lane now holds all sums; spread the k x RW x TT stores over the lanes
+    const bool per_tile = a.alpha_mode == TBN_ALPHA_PER_TILE;
+    const int total = a.k * RW * TT;
+    for (int e = lane; e < total; e += 32) {
+        const int t = e % TT;
+        const int rr = (e / TT) % RW;
+        const int j = e / (TT * RW);
+        const int32_t row = row0 + rr;
+        if (row >= r || t0 + t >= a.T) continue;
+        float z = 0.0f;
+#pragma unroll
+        for (int r2 = 0; r2 < RW; ++r2)
+#pragma unroll
+            for (int t2 = 0; t2 < TT; ++t2)
+                if (r2 == rr && t2 == t) z = acc[r2][t2];
+        const int32_t o = j * r + row;
+        const float al = per_tile ? __ldg(a.alpha + j) : __ldg(a.alpha);
+        const float v = apply_act(fmaf(al, z, a.bias ? __ldg(a.bias + o) : 0.0f), a.act);
+        const int64_t yi = (t0 + t) * a.m + o;
+        if (a.y_dtype == TBN_BF16) store_from_float(static_cast<__nv_bfloat16 *>(a.y), yi, v);
+        else store_from_float(static_cast<float *>(a.y), yi, v);
+    }
+}
+
+template <typename XT, int RW>
+cudaError_t launch_tt(const LayerArgs &a, int32_t r, cudaStream_t s)
+{
+    const int rows_per_block = kWarps * RW;
+    const unsigned gx = (unsigned)((r + rows_per_block - 1) / rows_per_block);
+    if (a.T <= 1) {
+        small_batch_kernel<XT, RW, 1><<<dim3(gx, 1), kWarps * 32, 0, s>>>(a, r);
+    } else if (a.T <= 2) {
+        small_batch_kernel<XT, RW, 2><<<dim3(gx, 1), kWarps * 32, 0, s>>>(a, r);
+    } else {
+        small_batch_kernel<XT, RW, 4><<<dim3(gx, (unsigned)((a.T + 3) / 4)), kWarps * 32, 0, s>>>(a, r);
+    }
+    return cudaGetLastError();
+}
+
+template <typename XT>
+cudaError_t launch_rw(const LayerArgs &a, int32_t r, cudaStream_t s)
+{
+    // more rows per warp reuse each activation load more often, but small layers need the blocks
+    if (r >= 148 * 4 * kWarps * 4) return launch_tt<XT, 4>(a, r, s);
+    if (r >= 148 * 2 * kWarps * 2) return launch_tt<XT, 2>(a, r, s);
+    return launch_tt<XT, 1>(a, r, s);
+}
+
+}  // namespace
+
+bool small_batch_supported(const LayerArgs &a)
+{
+    if (a.is_conv) return false;
+    if (a.q % a.n != 0) return false;          // tile must span whole rows
+    if (a.n % 8 != 0) return false;            // 16-byte activation vectors, byte-aligned bit rows
+    if (a.T > 65535 * 4) return false;
+    return true;
+}
+
+cudaError_t launch_small_batch(const LayerArgs &a, cudaStream_t s)
+{
+    const int32_t r = (int32_t)(a.q / a.n);
+    return a.x_dtype == TBN_BF16 ? launch_rw<__nv_bfloat16>(a, r, s) : launch_rw<float>(a, r, s);
+}
+
+}  // namespace tbn
