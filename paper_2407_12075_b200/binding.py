@@ -1,0 +1,234 @@
+"""ctypes binding of libtbn.so: the same entry points as include/tbn.h, argument marshalling only.
+
+Tensors are torch tensors (device memory and streams come from torch; every step of the
+computation runs inside the library's kernels).  There is no fallback: if the shared library is
+missing or a call returns a non-zero status, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtbn.so")
+
+OK = 0
+F32, BF16 = 0, 1
+ALPHA_PER_LAYER, ALPHA_PER_TILE = 0, 1
+ACT_NONE, ACT_RELU, ACT_GELU = 0, 1, 2
+PATH_AUTO, PATH_GENERIC, PATH_SMALL, PATH_TENSOR = 0, 1, 2, 3
+
+c_i32, c_i64, c_int, c_vp, c_sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t
+
+_LINEAR_ARGS = [c_vp, c_int, c_i64, c_i32, c_i32, c_vp, c_i32, c_vp, c_int, c_vp, c_int, c_vp, c_int,
+                c_vp, c_sz, c_vp]
+_CONV_ARGS = [c_vp, c_int] + [c_i32] * 9 + [c_vp, c_i32, c_vp, c_int, c_vp, c_int, c_vp, c_int, c_vp, c_sz, c_vp]
+
+SIGNATURES = {
+    "tbn_tile_words": (c_i64, [c_i64]),
+    "tbn_status_string": (ctypes.c_char_p, [c_int]),
+    "tbn_aggregate_workspace_bytes": (c_sz, [c_i64, c_i32]),
+    "tbn_aggregate_tile": (c_int, [c_vp, c_vp, c_i64, c_i32, c_int, c_vp, c_vp, c_vp, c_sz, c_vp]),
+    "tbn_pack_tile": (c_int, [c_vp, c_i64, c_vp, c_vp]),
+    "tbn_expand_tile": (c_int, [c_vp, c_i64, c_i32, c_vp, c_int, c_vp, c_vp]),
+    "tbn_linear_workspace_bytes": (c_sz, [c_i64, c_i32, c_i32, c_i32, c_int]),
+    "tbn_linear_fwd": (c_int, _LINEAR_ARGS),
+    "tbn_linear_fwd_path": (c_int, _LINEAR_ARGS + [c_int]),
+    "tbn_linear_select_path": (c_int, [c_i64, c_i32, c_i32, c_i32, c_int]),
+    "tbn_linear_host_workspace_bytes": (c_sz, [c_i64, c_i32, c_i32, c_i32, c_int, c_int]),
+    "tbn_linear_fwd_host": (c_int, _LINEAR_ARGS),
+    "tbn_conv2d_workspace_bytes": (c_sz, [c_i32] * 10 + [c_int]),
+    "tbn_conv2d_fwd": (c_int, _CONV_ARGS),
+    "tbn_conv2d_fwd_path": (c_int, _CONV_ARGS + [c_int]),
+    "tbn_mlp_workspace_bytes": (c_sz, [c_i64, c_i32, c_vp, c_vp, c_int]),
+    "tbn_mlp_fwd": (c_int, [c_vp, c_int, c_i64, c_i32, c_vp, c_vp, c_vp, c_vp, c_vp, c_int, c_vp, c_int,
+                            c_vp, c_sz, c_vp]),
+    "tbn_last_device_status": (c_int, [c_vp, c_vp, c_vp]),
+}
+
+_lib = None
+
+
+class TbnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().tbn_status_string(status).decode() if _lib is not None else "?"
+        super().__init__(f"{where}: status {status} ({msg})")
+
+
+def lib() -> ctypes.CDLL:
+    """Load libtbn.so (built in-tree by paper_2407_12075_b200.build); raise if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} not found: build it with `python -m paper_2407_12075_b200.build`; "
+                               "there is no fallback path")
+        L = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise TbnError(status, where)
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    assert t.is_contiguous(), "tensors must be contiguous"
+    return t.data_ptr()
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _torch_dtype(code: int):
+    return torch.bfloat16 if code == BF16 else torch.float32
+
+
+def _ws(nbytes: int, device):
+    return torch.empty(max(int(nbytes), 16), dtype=torch.uint8, device=device)
+
+
+# ------------------------------------------------------------------------------------------------
+def tbn_tile_words(q: int) -> int:
+    return int(lib().tbn_tile_words(q))
+
+
+def tbn_aggregate_tile(W: torch.Tensor, k: int, alpha_mode: int = ALPHA_PER_TILE, A: torch.Tensor | None = None,
+                       workspace: torch.Tensor | None = None):
+    """Eq. 1-3 and Eq. 6-8 on the device.  Returns (tile_bits int32[words], alpha float32[1 or k])."""
+    N = W.numel()
+    if k <= 0 or N % k:
+        raise TbnError(-2, "tbn_aggregate_tile")
+    tile = torch.empty(tbn_tile_words(N // k), dtype=torch.int32, device=W.device)
+    alpha = torch.empty(k if alpha_mode == ALPHA_PER_TILE else 1, dtype=torch.float32, device=W.device)
+    need = lib().tbn_aggregate_workspace_bytes(N, k)
+    ws = workspace if workspace is not None else _ws(need, W.device)
+    _check(lib().tbn_aggregate_tile(_ptr(W), _ptr(A), N, k, alpha_mode, _ptr(tile), _ptr(alpha), _ptr(ws),
+                                    ws.numel(), _stream()), "tbn_aggregate_tile")
+    return tile, alpha
+
+
+def tbn_pack_tile(src: torch.Tensor) -> torch.Tensor:
+    q = src.numel()
+    tile = torch.empty(tbn_tile_words(q), dtype=torch.int32, device=src.device)
+    _check(lib().tbn_pack_tile(_ptr(src), q, _ptr(tile), _stream()), "tbn_pack_tile")
+    return tile
+
+
+def tbn_expand_tile(tile: torch.Tensor, N: int, k: int, alpha: torch.Tensor, alpha_mode: int) -> torch.Tensor:
+    out = torch.empty(N, dtype=torch.float32, device=tile.device)
+    _check(lib().tbn_expand_tile(_ptr(tile), N, k, _ptr(alpha), alpha_mode, _ptr(out), _stream()),
+           "tbn_expand_tile")
+    return out
+
+
+def tbn_linear_workspace_bytes(T, in_f, out_f, k, x_dtype) -> int:
+    return int(lib().tbn_linear_workspace_bytes(T, in_f, out_f, k, x_dtype))
+
+
+def tbn_linear_select_path(T, in_f, out_f, k, x_dtype) -> int:
+    return int(lib().tbn_linear_select_path(T, in_f, out_f, k, x_dtype))
+
+
+def tbn_linear_fwd(x: torch.Tensor, out_f: int, tile: torch.Tensor, k: int, alpha: torch.Tensor,
+                   alpha_mode: int, bias: torch.Tensor | None = None, act: int = ACT_NONE,
+                   y_dtype: int | None = None, path: int = PATH_AUTO, y: torch.Tensor | None = None,
+                   workspace: torch.Tensor | None = None) -> torch.Tensor:
+    T, in_f = x.shape
+    xd = _dtype_code(x)
+    yd = xd if y_dtype is None else y_dtype
+    if y is None:
+        y = torch.empty((T, out_f), dtype=_torch_dtype(yd), device=x.device)
+    ws = workspace if workspace is not None else _ws(tbn_linear_workspace_bytes(T, in_f, out_f, k, xd), x.device)
+    _check(lib().tbn_linear_fwd_path(_ptr(x), xd, T, in_f, out_f, _ptr(tile), k, _ptr(alpha), alpha_mode,
+                                     _ptr(bias), act, _ptr(y), yd, _ptr(ws), ws.numel(), _stream(), path),
+           "tbn_linear_fwd")
+    return y
+
+
+def tbn_linear_host_workspace_bytes(T, in_f, out_f, k, x_dtype, y_dtype) -> int:
+    return int(lib().tbn_linear_host_workspace_bytes(T, in_f, out_f, k, x_dtype, y_dtype))
+
+
+def tbn_linear_fwd_host(x_host: torch.Tensor, y_host: torch.Tensor, tile, k, alpha, alpha_mode,
+                        workspace: torch.Tensor, bias=None, act=ACT_NONE):
+    """x_host / y_host are HOST tensors (pinned); workspace, tile, alpha live on the device."""
+    T, in_f = x_host.shape
+    out_f = y_host.shape[1]
+    _check(lib().tbn_linear_fwd_host(_ptr(x_host), _dtype_code(x_host), T, in_f, out_f, _ptr(tile), k,
+                                     _ptr(alpha), alpha_mode, _ptr(bias), act, _ptr(y_host),
+                                     _dtype_code(y_host), _ptr(workspace), workspace.numel(), _stream()),
+           "tbn_linear_fwd_host")
+    return y_host
+
+
+def tbn_conv2d_fwd(x: torch.Tensor, Cout: int, kh: int, kw: int, stride: int, pad: int, tile, k, alpha,
+                   alpha_mode, bias=None, act=ACT_NONE, y_dtype=None, path=PATH_AUTO) -> torch.Tensor:
+    Nb, Cin, H, Wd = x.shape
+    xd = _dtype_code(x)
+    yd = xd if y_dtype is None else y_dtype
+    Ho = (H + 2 * pad - kh) // stride + 1
+    Wo = (Wd + 2 * pad - kw) // stride + 1
+    y = torch.empty((Nb, Cout, max(Ho, 0), max(Wo, 0)), dtype=_torch_dtype(yd), device=x.device)
+    need = lib().tbn_conv2d_workspace_bytes(Nb, Cin, H, Wd, Cout, kh, kw, stride, pad, k, xd)
+    ws = _ws(need, x.device)
+    _check(lib().tbn_conv2d_fwd_path(_ptr(x), xd, Nb, Cin, H, Wd, Cout, kh, kw, stride, pad, _ptr(tile), k,
+                                     _ptr(alpha), alpha_mode, _ptr(bias), act, _ptr(y), yd, _ptr(ws),
+                                     ws.numel(), _stream(), path), "tbn_conv2d_fwd")
+    return y
+
+
+def _i32_array(vals):
+    return (c_i32 * len(vals))(*[int(v) for v in vals])
+
+
+def tbn_mlp_workspace_bytes(T, dims, ks, x_dtype) -> int:
+    L = len(ks)
+    return int(lib().tbn_mlp_workspace_bytes(T, L, ctypes.cast(_i32_array(dims), c_vp),
+                                             ctypes.cast(_i32_array(ks), c_vp), x_dtype))
+
+
+def tbn_mlp_fwd(x: torch.Tensor, dims, tiles, ks, alphas, alpha_modes, hidden_act=ACT_RELU, y_dtype=None,
+                workspace: torch.Tensor | None = None, y: torch.Tensor | None = None) -> torch.Tensor:
+    T = x.shape[0]
+    L = len(ks)
+    xd = _dtype_code(x)
+    yd = xd if y_dtype is None else y_dtype
+    if y is None:
+        y = torch.empty((T, dims[-1]), dtype=_torch_dtype(yd), device=x.device)
+    ws = workspace if workspace is not None else _ws(tbn_mlp_workspace_bytes(T, dims, ks, xd), x.device)
+    d_arr, k_arr = _i32_array(dims), _i32_array(ks)
+    m_arr = (c_int * L)(*[int(v) for v in alpha_modes])
+    t_arr = (c_vp * L)(*[_ptr(t) for t in tiles])
+    a_arr = (c_vp * L)(*[_ptr(a) for a in alphas])
+    _check(lib().tbn_mlp_fwd(_ptr(x), xd, T, L, ctypes.cast(d_arr, c_vp), ctypes.cast(t_arr, c_vp),
+                             ctypes.cast(k_arr, c_vp), ctypes.cast(a_arr, c_vp), ctypes.cast(m_arr, c_vp),
+                             hidden_act, _ptr(y), yd, _ptr(ws), ws.numel(), _stream()), "tbn_mlp_fwd")
+    return y
+
+
+def tbn_last_device_status():
+    code, detail = c_int(0), c_int(0)
+    _check(lib().tbn_last_device_status(_stream(), ctypes.byref(code), ctypes.byref(detail)),
+           "tbn_last_device_status")
+    return int(code.value), int(detail.value)
