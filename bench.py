@@ -1,0 +1,317 @@
+#!/usr/bin/env python
+"""Benchmark of the tiled-layer forward on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--tokens T]
+
+Workload (default): the large fully-connected sweep at its largest batch -- in = out = 8192,
+T = 16384 bf16 tokens ~N(0,1), W ~N(0, 0.02^2) aggregated to a tile, per-tile alpha, seed 4.
+One step = one forward for each k in {2, 4, 8, 16} on the same activations (4 kernel launches).
+The activation and output tensors (268 MB each) are larger than L2, so nothing is cache-resident
+from one launch to the next.  Metric: algorithmic TFLOP/s = sum_k 2*T*(8192/k)*8192 / time, i.e. the
+flops of the distinct rows only (the k-fold replication is a store, not a contraction).
+
+With --gpus N > 1 (under torchrun) every rank runs the same workload on its own GPU: the path has
+no exchange step, so ranks are independent replicas and the value is the sum over ranks.
+
+--impl reference times the CPU oracle (plain C, fp64, never tuned) on a bounded sample of the same
+workload, on the host cores of the machine.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+N_FEAT = 8192
+KS = (2, 4, 8, 16)
+SEED = 4
+METRIC = "tbn_layer_fwd_algorithmic_tflops"
+UNIT = "TFLOP/s"
+
+
+def algorithmic_flops(T: int, k: int) -> float:
+    """2*T*r*n with r = out/k distinct rows (tile spans whole rows for every k here)."""
+    return 2.0 * T * (N_FEAT // k) * N_FEAT
+
+
+def algorithmic_bytes(T: int, k: int) -> float:
+    """activations in + outputs out (bf16) + packed tile + alphas."""
+    return 2.0 * T * N_FEAT * 2 + (N_FEAT * N_FEAT // k) / 8 + 4 * k
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def oracle_sample(x_bits: np.ndarray, W: np.ndarray, k: int, rows: int, seed: int = 0):
+    """Time the CPU oracle (expand the tile, naive fp64 product) on `rows` seeded token rows."""
+    from oracle import tbn_oracle as O
+    T = x_bits.shape[0]
+    pick = np.sort(np.random.default_rng(seed).choice(T, size=min(rows, T), replace=False))
+    words, al = O.prepare(W, k, True)
+    xs = np.ascontiguousarray(x_bits[pick])
+    t0 = time.perf_counter()
+    O.linear(xs, words, k, al, True, N_FEAT, N_FEAT)
+    dt = time.perf_counter() - t0
+    return dt, len(pick), O.num_threads()
+
+
+def run_reference(args, T: int):
+    """--impl reference: the oracle as it stands, on the host cores, on a bounded sample per step."""
+    from paper_2407_12075_b200 import synth
+    rows = 64
+    x = synth.to_bf16_bits(synth.normal(SEED, 0, rows * N_FEAT).reshape(rows, N_FEAT))
+    W = synth.normal(SEED, 1, N_FEAT * N_FEAT, 0.02).reshape(N_FEAT, N_FEAT)
+    times, cores = [], 1
+    for step in range(args.warmup + args.steps):
+        t = 0.0
+        for k in KS:
+            dt, n, cores = oracle_sample(x, W, k, rows)
+            t += dt
+        if step >= args.warmup:
+            times.append(t)
+    ms = 1e3 * float(np.mean(times))
+    flops = sum(algorithmic_flops(rows, k) for k in KS)
+    value = flops / (ms * 1e-3) / 1e12
+    sample = (f"{rows} of {T} token rows x all 8192 outputs, each k in {list(KS)}; dense fp64 product "
+              f"(the oracle never uses the replicated-row shortcut); value counts algorithmic flops")
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
+                ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64",
+                data="synthetic", impl="reference",
+                config=dict(workload=f"large linear sweep 8192x8192, T={T}, k in {list(KS)}, per-tile alpha, seed {SEED}",
+                            l2="n/a (CPU)"),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                gpu_launches=0)
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--tokens", type=int, default=16384, help="development override of the batch size")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args, args.tokens)
+        return
+
+    run_ours(args, rank, world, local_rank)
+
+
+
+def run_ours(args, rank: int, world: int, local_rank: int):
+    import torch
+    from paper_2407_12075_b200 import binding as B
+    from paper_2407_12075_b200 import build as tbn_build
+    from paper_2407_12075_b200 import synth
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        tbn_build.build()
+    if world > 1:
+        dist.barrier()
+    B.lib()
+
+    T = args.tokens
+    peaks = read_peaks()
+    # ---- seeded synthetic inputs, resident in HBM before the timed region -----------------------
+    x_np = synth.to_bf16_bits(synth.normal(SEED, 0, T * N_FEAT).reshape(T, N_FEAT))
+    W_np = synth.normal(SEED, 1, N_FEAT * N_FEAT, 0.02).reshape(N_FEAT, N_FEAT)
+    x = torch.from_numpy(x_np.view(np.int16)).view(torch.bfloat16).to(dev)
+    Wd = torch.from_numpy(W_np).to(dev)
+    layers = {}
+    for k in KS:
+        layers[k] = B.tbn_aggregate_tile(Wd, k, B.ALPHA_PER_TILE)
+    del Wd
+    y = torch.empty((T, N_FEAT), dtype=torch.bfloat16, device=dev)
+    ws = torch.empty(max(B.tbn_linear_workspace_bytes(T, N_FEAT, N_FEAT, 2, B.BF16), 16), dtype=torch.uint8, device=dev)
+    path_names = {1: "generic", 2: "small-batch", 3: "tensor (tcgen05)"}
+    path = path_names.get(B.tbn_linear_select_path(T, N_FEAT, N_FEAT, 2, B.BF16), "?")
+
+    def step(events=None):
+        for i, k in enumerate(KS):
+            tile, alpha = layers[k]
+            if events is not None:
+                events[i][0].record()
+            B.tbn_linear_fwd(x, N_FEAT, tile, k, alpha, B.ALPHA_PER_TILE, y=y, workspace=ws)
+            if events is not None:
+                events[i][1].record()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    code, detail = B.tbn_last_device_status()
+    if code != 0:
+        raise SystemExit(f"device-side status {code} (detail {detail}) after warm-up")
+
+    # ---- timed region: K steps, CUDA events on the launching stream, clocks sampled meanwhile ----
+    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in KS]
+          for _ in range(args.steps)]
+    t_beg, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    t_beg.record()
+    for s in range(args.steps):
+        step(ev[s])
+    t_end.record()
+    barrier()
+    clocks = sampler.stop()
+    total_ms = t_beg.elapsed_time(t_end)
+    if world > 1:
+        tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / args.steps
+    per_k_ms = {k: float(np.mean([ev[s][i][0].elapsed_time(ev[s][i][1]) for s in range(args.steps)]))
+                for i, k in enumerate(KS)}
+    flops_step = sum(algorithmic_flops(T, k) for k in KS)
+    value = world * flops_step / (ms_per_step * 1e-3) / 1e12
+
+    # ---- roofline of the dominant kernel (the forward kernel, averaged over the four k) --------
+    kern_ms = float(np.mean(list(per_k_ms.values())))
+    achieved = flops_step / len(KS) / (kern_ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops_sustained"]
+    per_k = {}
+    for k in KS:
+        tf = algorithmic_flops(T, k) / (per_k_ms[k] * 1e-3) / 1e12
+        gbs = algorithmic_bytes(T, k) / (per_k_ms[k] * 1e-3) / 1e9
+        t_bound = max(algorithmic_flops(T, k) / (peak * 1e12), algorithmic_bytes(T, k) / (peaks["hbm_gbs"] * 1e9))
+        per_k[str(k)] = dict(ms=per_k_ms[k], alg_tflops=tf, dense_equiv_tflops=tf * k, alg_gbs=gbs,
+                             frac_of_binding_roofline=t_bound / (per_k_ms[k] * 1e-3))
+    roofline = dict(bound="tensor", achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak,
+                    traffic=None, peak_source=f"{peaks['source']} (sustained bf16 GEMM)", kernel_path=path)
+
+    # ---- end to end: host buffers through the C-ABI, copies inside the timed region -------------
+    e2e = None
+    if rank == 0 or world > 1:
+        xh = torch.from_numpy(x_np.view(np.int16)).view(torch.bfloat16).pin_memory()
+        yh = torch.empty((T, N_FEAT), dtype=torch.bfloat16).pin_memory()
+        hws = torch.empty(B.tbn_linear_host_workspace_bytes(T, N_FEAT, N_FEAT, 2, B.BF16, B.BF16),
+                          dtype=torch.uint8, device=dev)
+        def host_step():
+            for k in KS:
+                tile, alpha = layers[k]
+                B.tbn_linear_fwd_host(xh, yh, tile, k, alpha, B.ALPHA_PER_TILE, hws)
+        host_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            host_step()
+        torch.cuda.synchronize()
+        dt = (time.perf_counter() - t0) / args.e2e_steps
+        if world > 1:
+            tt = torch.tensor([dt], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            dt = float(tt.item())
+        nbytes = T * N_FEAT * 2 * len(KS)
+        e2e = dict(value=world * flops_step / dt / 1e12, unit=UNIT, h2d_bytes_per_step=nbytes,
+                   d2h_bytes_per_step=nbytes, ms_per_step=dt * 1e3, steps=args.e2e_steps)
+
+    # ---- the oracle on the host cores, rank 0 at N = 1 only ---------------------------------------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        rows = 96
+        dt, n, cores = oracle_sample(x_np, W_np, 4, rows)
+        cpu = dict(value=algorithmic_flops(n, 4) / dt / 1e12, unit=UNIT, cores=cores, kind="oracle",
+                   sample=f"{n} seeded token rows of {T} x all 8192 outputs at k=4, {dt:.1f} s; the oracle does the "
+                          f"dense fp64 product ({2.0 * n * N_FEAT * N_FEAT / dt / 1e9:.2f} dense GFLOP/s), value "
+                          f"counts algorithmic flops")
+
+    if rank == 0:
+        line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                    ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
+                    dtype="bf16", data="synthetic",
+                    config=dict(workload=f"large linear sweep 8192x8192, T={T}, k in {list(KS)}, per-tile alpha, seed {SEED}",
+                                step="one forward per k (4 launches)", l2="inputs larger than L2 (x and y 268 MB each)",
+                                multi_gpu="replicas only (no exchange step in the path)"),
+                    clocks=clocks, e2e=e2e, gpu_launches=args.steps * len(KS), roofline=roofline,
+                    cpu_baseline=cpu, per_k=per_k)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,93 @@
+"""GPU parity: tiled convolution and the MLP chain against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import tbn_oracle as O
+from paper_2407_12075_b200 import binding as B
+from paper_2407_12075_b200 import synth
+from tests.util import DEV, assert_close, to_dev, to_np64
+
+pytestmark = pytest.mark.gpu
+
+# (Nb, Cout, Cin, kh, kw, k, stride, pad, H)
+CONVS = [
+    (3, 2, 1, 3, 3, 2, 1, 1, 5),        # the paper's replicated-channel example
+    (2, 128, 64, 3, 3, 4, 1, 1, 32),
+    (2, 128, 64, 3, 3, 4, 2, 1, 32),
+    (2, 256, 128, 3, 3, 4, 2, 1, 16),
+    (3, 16, 8, 1, 1, 4, 1, 0, 7),
+    (2, 8, 3, 3, 3, 2, 2, 1, 9),        # q = 108: four filters of 27
+    (2, 4, 3, 3, 3, 3, 2, 1, 9),        # q = 36: a tile ends inside a filter
+]
+
+
+@pytest.mark.parametrize("Nb,Cout,Cin,kh,kw,k,stride,pad,H", CONVS)
+@pytest.mark.parametrize("per_tile", [False, True])
+def test_conv_matches_oracle(Nb, Cout, Cin, kh, kw, k, stride, pad, H, per_tile):
+    x, W = synth.conv_layer(2, Nb, Cin, H, H, Cout, kh, kw)
+    words, al = O.prepare(W, k, per_tile)
+    ref = O.conv2d(x, words, k, al, per_tile, Cout, Cin, kh, kw, stride, pad, act=O.ACT_RELU)
+    for path in (B.PATH_GENERIC, B.PATH_AUTO):
+        y = B.tbn_conv2d_fwd(to_dev(x), Cout, kh, kw, stride, pad, to_dev(words), k, to_dev(al), int(per_tile),
+                             act=B.ACT_RELU, path=path)
+        torch.cuda.synchronize()
+        assert_close(to_np64(y), ref, f"conv path {path}")
+
+
+def test_conv_replicated_channels_are_bit_identical():
+    # Sec. 4.1: single alpha, no bias -> the k copies of a filter give identical channels
+    x, W = synth.conv_layer(5, 4, 8, 12, 12, 32, 3, 3)
+    words, al = O.prepare(W, 4, False)
+    y = B.tbn_conv2d_fwd(to_dev(x), 32, 3, 3, 1, 1, to_dev(words), 4, to_dev(al), 0)
+    for j in range(1, 4):
+        assert torch.equal(y[:, :8], y[:, 8 * j:8 * (j + 1)])
+
+
+def test_conv_fp32_in_out_and_bias():
+    x, W = synth.conv_layer(6, 2, 4, 9, 9, 8, 3, 3, x_bf16=False)
+    bias = synth.normal(6, 200, 8)
+    words, al = O.prepare(W, 2, True)
+    ref = O.conv2d(x, words, 2, al, True, 8, 4, 3, 3, 2, 1, bias=bias.astype(np.float64))
+    y = B.tbn_conv2d_fwd(to_dev(x), 8, 3, 3, 2, 1, to_dev(words), 2, to_dev(al), 1, bias=to_dev(bias))
+    assert y.dtype == torch.float32
+    assert_close(to_np64(y), ref, "conv fp32")
+
+
+def _mlp_layers(Ws, ks):
+    layers, tiles, alphas = [], [], []
+    for W, k in zip(Ws, ks):
+        m, n = W.shape
+        words, al = O.prepare(W, k, True)
+        layers.append(dict(words=words, p=k, alphas=al, per_tile=True, m=m, n=n))
+        tiles.append(to_dev(words))
+        alphas.append(to_dev(al))
+    return layers, tiles, alphas
+
+
+@pytest.mark.parametrize("T", [1, 7, 200])
+def test_mlp_small_matches_oracle(T):
+    dims, ks = [64, 128, 96, 10], [4, 8, 1]
+    x = synth.to_bf16_bits(synth.normal(1, 0, T * dims[0]).reshape(T, dims[0]))
+    Ws = [synth.normal(1, 1 + l, dims[l + 1] * dims[l], 0.1).reshape(dims[l + 1], dims[l]) for l in range(3)]
+    layers, tiles, alphas = _mlp_layers(Ws, ks)
+    ref = O.mlp(x, layers)
+    y = B.tbn_mlp_fwd(to_dev(x), dims, tiles, ks, alphas, [1, 1, 1])
+    torch.cuda.synchronize()
+    assert_close(to_np64(y), ref, f"mlp T={T}")
+
+
+def test_mlp_benchmark_config_sampled_rows():
+    # 1024 -> 2048 -> 2048 -> 10, k = 8 on the hidden layers, batch 4096: all rows on the GPU,
+    # a seeded sample of rows through the oracle
+    c = synth.config_mlp(T=4096)
+    layers, tiles, alphas = _mlp_layers(c["Ws"], c["ks"])
+    y = B.tbn_mlp_fwd(to_dev(c["x"]), c["dims"], tiles, c["ks"], alphas, [1, 1, 1])
+    torch.cuda.synchronize()
+    rows = np.sort(np.random.default_rng(0).choice(4096, 48, replace=False))
+    ref = O.mlp(c["x"][rows], layers)
+    assert_close(to_np64(y)[rows], ref, "mlp config")
+    # tiles built on the GPU equal the oracle's
+    for W, k, t in zip(c["Ws"], c["ks"], tiles):
+        t2, _ = B.tbn_aggregate_tile(to_dev(W), k, B.ALPHA_PER_TILE)
+        assert torch.equal(t2, t)

@@ -1,0 +1,108 @@
+"""GPU parity, fully-connected forward: every kernel family against the CPU oracle on the same
+seeded inputs, element by element, within max|err| <= 1e-2 * (1 + |ref|)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import tbn_oracle as O
+from paper_2407_12075_b200 import binding as B
+from paper_2407_12075_b200 import synth
+from tests.util import DEV, assert_close, make_linear_case, to_dev, to_np64
+
+pytestmark = pytest.mark.gpu
+
+# (m, n, k): the survey's shape zoo -- aligned, misaligned, several tiles per row, nothing divides
+ZOO = [(8, 8, 1), (8, 8, 2), (8, 8, 8), (128, 784, 4), (10, 128, 1), (512, 512, 4), (2304, 768, 8),
+       (96, 40, 6), (6, 64, 4), (4, 64, 8), (7, 33, 3)]
+TOKENS = [1, 2, 3, 17, 64, 129]
+
+
+def run(path, x, words, al, per_tile, m, k, act=B.ACT_NONE, bias=None, y_dtype=None):
+    y = B.tbn_linear_fwd(to_dev(x), m, to_dev(words), k, to_dev(al), int(per_tile),
+                         bias=None if bias is None else to_dev(bias), act=act, y_dtype=y_dtype, path=path)
+    torch.cuda.synchronize()
+    return to_np64(y)
+
+
+@pytest.mark.parametrize("m,n,k", ZOO)
+@pytest.mark.parametrize("T", TOKENS)
+def test_generic_path_matches_oracle(m, n, k, T):
+    for per_tile in (False, True):
+        for x_bf16 in (False, True):
+            x, W, words, al = make_linear_case(100 + T, T, m, n, k, per_tile, x_bf16, w_sigma=1.0)
+            ref = O.linear(x, words, k, al, per_tile, m, n)
+            got = run(B.PATH_GENERIC, x, words, al, per_tile, m, k, y_dtype=B.F32)
+            assert_close(got, ref, f"generic {m}x{n} k={k} T={T}")
+
+
+ALIGNED = [(m, n, k) for (m, n, k) in ZOO if (m * n // k) % n == 0 and n % 8 == 0]
+
+
+@pytest.mark.parametrize("m,n,k", ALIGNED + [(2048, 1024, 8), (64, 8200, 2)])
+@pytest.mark.parametrize("T", [1, 2, 3, 5, 17])
+def test_small_batch_path_matches_oracle(m, n, k, T):
+    for per_tile in (False, True):
+        for x_bf16 in (False, True):
+            x, W, words, al = make_linear_case(200 + T, T, m, n, k, per_tile, x_bf16)
+            ref = O.linear(x, words, k, al, per_tile, m, n, act=O.ACT_RELU)
+            got = run(B.PATH_SMALL, x, words, al, per_tile, m, k, act=B.ACT_RELU)
+            assert_close(got, ref, f"small {m}x{n} k={k} T={T}")
+
+
+def test_small_batch_rejects_misaligned_tiles():
+    x, W, words, al = make_linear_case(1, 2, 6, 64, 4)
+    with pytest.raises(B.TbnError) as e:
+        run(B.PATH_SMALL, x, words, al, True, 6, 4)
+    assert e.value.status == -3
+
+
+@pytest.mark.parametrize("act", [B.ACT_NONE, B.ACT_RELU, B.ACT_GELU])
+@pytest.mark.parametrize("path", [B.PATH_GENERIC, B.PATH_SMALL, B.PATH_AUTO])
+def test_bias_activation_and_output_dtypes(act, path):
+    m, n, k, T = 64, 128, 4, 5
+    x, W, words, al = make_linear_case(7, T, m, n, k, True, True, w_sigma=1.0)
+    bias = synth.normal(7, 200, m)
+    ref = O.linear(x, words, k, al, True, m, n, bias=bias.astype(np.float64), act=act)
+    for yd in (B.F32, B.BF16):
+        got = run(path, x, words, al, True, m, k, act=act, bias=bias, y_dtype=yd)
+        assert_close(got, ref, f"act={act} path={path} yd={yd}")
+
+
+def test_single_fc_config_all_paths_agree():
+    # single layer 512 -> 512, k = 4, batch 64, fp32 activations, W ~ N(0, 0.02), seed 0
+    c = synth.config_single_fc()
+    words, al = O.prepare(c["W"], c["k"], True)
+    tile, alpha = B.tbn_aggregate_tile(to_dev(c["W"]), c["k"], B.ALPHA_PER_TILE)
+    assert np.array_equal(tile.cpu().numpy().view(np.uint32), words)
+    ref = O.linear(c["x"], words, c["k"], al, True, c["m"], c["n"])
+    xd = to_dev(c["x"])
+    outs = {}
+    for path in (B.PATH_GENERIC, B.PATH_SMALL, B.PATH_AUTO):
+        y = B.tbn_linear_fwd(xd, c["m"], tile, c["k"], alpha, B.ALPHA_PER_TILE, path=path)
+        outs[path] = to_np64(y)
+        assert_close(outs[path], ref, f"config 1 path {path}")
+    # shortcut kernels vs the generic kernel (which never uses the shortcut): fp32 reassociation only
+    assert np.allclose(outs[B.PATH_SMALL], outs[B.PATH_GENERIC], rtol=1e-4, atol=1e-5)
+
+
+def test_zero_tokens_is_a_noop_and_zero_alpha_gives_zeros():
+    m, n, k = 16, 32, 2
+    x, W, words, al = make_linear_case(3, 4, m, n, k)
+    y = B.tbn_linear_fwd(torch.empty((0, n), dtype=torch.bfloat16, device=DEV), m, to_dev(words), k,
+                         to_dev(al), B.ALPHA_PER_TILE)
+    assert y.shape == (0, m)
+    got = run(B.PATH_AUTO, x, words, np.zeros(k, np.float32), True, m, k)
+    assert np.all(got == 0)
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    m, n, k, T = 256, 512, 4, 33
+    x, W, words, al = make_linear_case(9, T, m, n, k)
+    xh = torch.from_numpy(x.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+    yh = torch.empty((T, m), dtype=torch.bfloat16).pin_memory()
+    ws = torch.empty(B.tbn_linear_host_workspace_bytes(T, n, m, k, B.BF16, B.BF16), dtype=torch.uint8, device=DEV)
+    tile, alpha = to_dev(words), to_dev(al)
+    B.tbn_linear_fwd_host(xh, yh, tile, k, alpha, B.ALPHA_PER_TILE, ws)
+    yd = B.tbn_linear_fwd(xh.to(DEV), m, tile, k, alpha, B.ALPHA_PER_TILE)
+    assert torch.equal(yh, yd.cpu())
+    assert_close(to_np64(yh), O.linear(x, words, k, al, True, m, n), "host entry point")

@@ -1,0 +1,79 @@
+"""GPU parity, tile construction: aggregate / pack / expand must equal the oracle bit for bit;
+alpha within 1e-6 relative (its reduction order is free)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import tbn_oracle as O
+from paper_2407_12075_b200 import binding as B
+from paper_2407_12075_b200 import synth
+from tests.util import DEV, to_dev, words_np
+
+pytestmark = pytest.mark.gpu
+
+CASES = [  # (N, k)
+    (64, 1), (64, 2), (64, 8), (100352, 4), (1280, 1), (262144, 4), (2304 * 768, 8),
+    (96 * 40, 6), (7 * 33, 3), (1024 * 4, 4), (1025 * 3, 3), (4097 * 2, 2), (73728, 4), (1 << 22, 16),
+]
+
+
+@pytest.mark.parametrize("N,k", CASES)
+@pytest.mark.parametrize("per_tile", [False, True])
+def test_aggregate_bits_exact_alpha_close(N, k, per_tile):
+    W = synth.normal(10 + k, 1, N, 0.02)
+    W[::97] = 0.0
+    tile, alpha = B.tbn_aggregate_tile(to_dev(W), k, B.ALPHA_PER_TILE if per_tile else B.ALPHA_PER_LAYER)
+    torch.cuda.synchronize()
+    words_ref, al_ref = O.prepare(W, k, per_tile)
+    assert np.array_equal(words_np(tile), words_ref)
+    assert np.allclose(alpha.cpu().numpy(), al_ref, rtol=1e-6, atol=0)
+
+
+def test_aggregate_separate_alpha_tensor_and_determinism():
+    N, k = 512 * 512, 4
+    W = synth.normal(0, 1, N, 0.02)
+    A = synth.normal(0, 101, N, 0.05)
+    Wd, Ad = to_dev(W), to_dev(A)
+    tile, alpha = B.tbn_aggregate_tile(Wd, k, B.ALPHA_PER_TILE, A=Ad)
+    words_ref, al_ref = O.prepare(W, k, True, A=A)
+    assert np.array_equal(words_np(tile), words_ref)
+    assert np.allclose(alpha.cpu().numpy(), al_ref, rtol=1e-6)
+    for _ in range(3):
+        t2, a2 = B.tbn_aggregate_tile(Wd, k, B.ALPHA_PER_TILE, A=Ad)
+        assert torch.equal(t2, tile) and torch.equal(a2, alpha)      # bit-identical from run to run
+
+
+def test_aggregate_near_cancelling_sums_follow_fp32_order():
+    # columns whose fp32 sequential sum and fp64 sum disagree in sign, plus ties and NaN
+    q = 4096
+    W = np.zeros((3, q), dtype=np.float32)
+    W[0], W[1], W[2] = 1e8, 1.0, -1e8                # fp32: 0 -> bit 0 ; fp64: 1
+    W[:, 1::4] = np.array([[1e8], [-1e8], [1.0]], dtype=np.float32)   # (1e8-1e8)+1 = 1 -> bit 1
+    W[:, 2::4] = 0.0
+    W[0, 3::4] = np.nan
+    tile, _ = B.tbn_aggregate_tile(to_dev(W.reshape(-1)), 3, B.ALPHA_PER_LAYER)
+    bits_ref, mism = O.aggregate(W.reshape(-1), 3)
+    assert mism == q // 4
+    assert np.array_equal(words_np(tile), O.pack_bits(bits_ref))
+
+
+@pytest.mark.parametrize("q", [1, 31, 32, 33, 127, 129, 1000, 65536, 100003])
+def test_pack_exact(q):
+    src = synth.normal(q, 1, q)
+    src[::5] = 0.0
+    tile = B.tbn_pack_tile(to_dev(src))
+    assert np.array_equal(words_np(tile), O.pack(src))
+
+
+@pytest.mark.parametrize("N,k,per_tile", [(64, 2, True), (262144, 4, True), (7 * 33, 3, False), (96 * 40, 6, True)])
+def test_expand_exact(N, k, per_tile):
+    W = synth.normal(3, 1, N, 0.02)
+    words, al = O.prepare(W, k, per_tile)
+    out = B.tbn_expand_tile(to_dev(words), N, k, to_dev(al), int(per_tile))
+    assert np.array_equal(out.cpu().numpy(), O.expand(words, N, k, al, per_tile))
+
+
+def test_shape_errors_surface_as_exceptions():
+    W = torch.zeros(10, device=DEV)
+    with pytest.raises(B.TbnError):
+        B.tbn_aggregate_tile(W, 3)
