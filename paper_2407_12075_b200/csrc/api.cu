@@ -35,9 +35,11 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Validation shared by the fully-connected and convolution entry points.
 int check_layer_common(const void *x, int x_dtype, const uint32_t *tile, int32_t k, const float *alpha,
-                       int alpha_mode, const float *bias, int act, const void *y, int y_dtype, int path)
+                       int alpha_mode, const float *bias, int act, const void *y, int y_dtype, int path,
+                       bool empty)
 {
-    if (!x || !tile || !alpha || !y) return TBN_ERR_INVALID_ARG;
+    if (!tile || !alpha) return TBN_ERR_INVALID_ARG;
+    if (!empty && (!x || !y)) return TBN_ERR_INVALID_ARG;   // an empty batch may come with null data pointers
     if (!valid_dtype(x_dtype) || !valid_dtype(y_dtype) || !valid_alpha_mode(alpha_mode) || !valid_act(act))
         return TBN_ERR_INVALID_ARG;
     if (path < TBN_PATH_AUTO || path > TBN_PATH_TENSOR) return TBN_ERR_INVALID_ARG;
@@ -101,7 +103,7 @@ int fill_linear(LayerArgs &a, const void *x, int x_dtype, int64_t T, int32_t in_
                 const float *bias, int act, void *y, int y_dtype, int path)
 {
     if (T < 0 || in_f <= 0 || out_f <= 0) return TBN_ERR_INVALID_ARG;
-    int rc = check_layer_common(x, x_dtype, tile_bits, k, alpha, alpha_mode, bias, act, y, y_dtype, path);
+    int rc = check_layer_common(x, x_dtype, tile_bits, k, alpha, alpha_mode, bias, act, y, y_dtype, path, T == 0);
     if (rc != TBN_OK) return rc;
     const int64_t N = (int64_t)in_f * out_f;
     if (N % k != 0) return TBN_ERR_SHAPE;
@@ -282,7 +284,7 @@ int tbn_conv2d_fwd_path(const void *x, int x_dtype, int32_t Nb, int32_t Cin, int
 {
     if (Nb < 0 || Cin <= 0 || H <= 0 || Wd <= 0 || Cout <= 0 || kh <= 0 || kw <= 0 || stride <= 0 || pad < 0)
         return TBN_ERR_INVALID_ARG;
-    int rc = check_layer_common(x, x_dtype, tile_bits, k, alpha, alpha_mode, bias, act, y, y_dtype, path);
+    int rc = check_layer_common(x, x_dtype, tile_bits, k, alpha, alpha_mode, bias, act, y, y_dtype, path, Nb == 0);
     if (rc != TBN_OK) return rc;
     if (H + 2 * pad < kh || Wd + 2 * pad < kw) return TBN_ERR_SHAPE;
     const int64_t n = (int64_t)Cin * kh * kw;

@@ -1,6 +1,551 @@
-// placeholder until the tcgen05 kernel lands
+// Tensor-core forward of a tiled fully-connected layer on sm_100a: tcgen05.mma with the decoded
+// weights as the A operand in tensor memory and the activations as the B operand in shared memory.
+//
+// Problem.  The tile spans r = q/n whole rows, so only Z[T, r] = X[T, n] * Wd[r, n]^T has to be
+// contracted (Wd = the r distinct +-1 rows, Sec. 4.1); the output is Y[:, j*r + c] = act(alpha_j *
+// Z[:, c] + bias) for the k repetitions j.  The kernel computes Z^T tiles: the UMMA M dimension (the
+// 128 TMEM lanes) runs over weight rows, the N dimension over tokens.
+//
+// Why the weights go to tensor memory.  The packed tile is 1/16 of the bf16 weight bytes and is
+// expanded in registers; writing the expansion with tcgen05.st into TMEM costs no shared-memory
+// bandwidth, and tcgen05.mma then reads A from TMEM and only the activation operand from shared
+// memory.  Each decoded 128 x 64 block is reused for all NTOK tokens of the CTA tile, and each
+// activation stage is reused by NA blocks of 128 weight rows.
+//
+// Warp roles (10 warps): 0 = TMA producer (activation stages, 128-byte swizzle), 1 = MMA issuer and
+// TMEM owner, 2-5 = tile decode (bits -> +-1 bf16 pairs -> tcgen05.st), 6-9 = epilogue (tcgen05.ld ->
+// alpha/bias/activation -> k-fold replicated stores).  All hand-offs are mbarriers; every wait is
+// bounded by a wall-clock limit, after which the CTA records TBN_ERR_TIMEOUT, drains and returns.
+#include <cuda.h>
+
 #include "common.cuh"
+
 namespace tbn {
-bool tensor_path_supported(const LayerArgs &) { return false; }
-int launch_tensor_linear(const LayerArgs &, int *, cudaStream_t) { return TBN_ERR_UNSUPPORTED; }
+
+namespace {
+
+constexpr int kThreads = 320;
+constexpr int kStageK = 64;            // contraction elements per pipeline stage (= one 128-byte swizzle row)
+constexpr int kAStages = 2;            // decoded-weight stages in tensor memory
+constexpr int kMaxAlpha = 64;          // alphas cached in shared memory
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: orders of magnitude above any legitimate wait
+
+// ---- PTX wrappers -----------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
 }
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+__device__ __forceinline__ void fence_barrier_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int32_t c0, int32_t c1,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]^T, bf16 x bf16 -> fp32, M = 128
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// 32 lanes x 32 consecutive 32-bit columns: thread l of the warp owns TMEM lane (quadrant base + l)
+__device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr),
+          "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+// 16 tile bits (low half of h, upper half zero) -> 8 registers of two bf16 each: bit 2j in the low half,
+// bit 2j+1 in the high half; bit 1 -> +1.0 (0x3F80), bit 0 -> -1.0 (0xBF80).  v keeps the even bits at
+// positions 2j and moves the odd bits to 2j+16, so one shift lines both up with the two sign positions.
+__device__ __forceinline__ void decode16(uint32_t h, uint32_t *out) {
+    const uint32_t v = (h | (h << 15)) & 0x55555555u;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) out[j] = ((v << (15 - 2 * j)) & 0x80008000u) ^ 0xBF80BF80u;
+}
+// 64 consecutive tile bits (b0 = first 32) -> one 128-lane x 32-column row of the A operand
+__device__ __forceinline__ void decode64(uint32_t b0, uint32_t b1, uint32_t (&v)[32]) {
+    decode16(b0 & 0xffffu, v);
+    decode16(b0 >> 16, v + 8);
+    decode16(b1 & 0xffffu, v + 16);
+    decode16(b1 >> 16, v + 24);
+}
+
+// ---- shared-memory control block -----------------------------------------------------------------
+template <int SX>
+struct Control {
+    uint64_t x_full[SX], x_empty[SX];
+    uint64_t a_full[kAStages], a_empty[kAStages];
+    uint64_t d_full, d_empty;
+    uint32_t tmem_base;
+    int abort_flag;
+    float alpha[kMaxAlpha];
+};
+
+struct Pipe {
+    uint32_t stage = 0, phase = 0;
+    __device__ __forceinline__ void advance(uint32_t n) { if (++stage == n) { stage = 0; phase ^= 1u; } }
+};
+
+// Bounded wait on an mbarrier phase.  Returns false when the CTA is aborting (this or another thread
+// ran out of time); the first thread to time out records the status for the host.
+__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
+                                       int detail) {
+    const uint64_t t0 = global_timer_ns();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 63u) == 0) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                if (atomicCAS(status, 0, (int)TBN_ERR_TIMEOUT) == 0) status[1] = detail;
+                __threadfence();
+                return false;
+            }
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
+                                         int detail) {
+    // every lane of the calling warp waits; the verdict is made warp-uniform so that the warp stays
+    // converged for the .sync.aligned tcgen05 instructions that follow
+    bool r = mbar_try_wait(bar, parity) != 0;
+    if (!r) r = wait_slow(bar, parity, abort_flag, status, detail);
+    return __all_sync(0xffffffffu, r) != 0;
+}
+
+struct TcParams {
+    const uint32_t *tile;
+    const float *alpha;
+    const float *bias;
+    void *y;
+    int *status;
+    int64_t T;
+    int64_t n_words;     // words of the packed tile
+    int32_t n, m, r, k;
+    int32_t k_stages;    // ceil(n / 64)
+    int32_t w_tiles, t_tiles;
+    int per_tile, act, y_bf16;
+};
+
+__host__ __device__ constexpr uint32_t next_pow2_cols(uint32_t c) {
+    uint32_t p = 32;
+    while (p < c) p <<= 1;
+    return p;
+}
+
+// Shared-memory matrix descriptor of one activation stage: K-major, 128-byte swizzle, rows of 128 bytes,
+// 8-row groups 1024 bytes apart.  `addr` may point 32*kk bytes into the first row to select a K slice.
+__device__ __forceinline__ uint64_t make_b_desc(uint32_t addr) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// Quiet bounded wait used only while draining after an abort.
+__device__ __forceinline__ void drain_wait(uint32_t bar, uint32_t parity) {
+    const uint64_t t0 = global_timer_ns();
+    while (!mbar_try_wait(bar, parity)) {
+        if (global_timer_ns() - t0 > 20000000ull) break;   // 20 ms
+    }
+}
+
+template <int NTOK, int NA, int SX>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
+{
+    static_assert(NTOK % 32 == 0 && NTOK >= 32 && NTOK <= 256, "token tile");
+    constexpr uint32_t kStageBytes = NTOK * 128;
+    constexpr uint32_t kDCols = NA * NTOK;
+    constexpr uint32_t kACols = NA * 32;
+    constexpr uint32_t kTmemCols = next_pow2_cols(kDCols + kAStages * kACols);
+    static_assert(kTmemCols <= 512, "tensor memory budget");
+    // instruction descriptor: D fp32, A and B bf16, both K-major, N = NTOK, M = 128
+    constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NTOK >> 3) << 17) | (8u << 24);
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    uint8_t *smem = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
+    Control<SX> *ctl = reinterpret_cast<Control<SX> *>(smem + SX * kStageBytes);
+    const uint32_t stage0 = smem_u32(smem);
+    volatile int *abort_flag = &ctl->abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int bid = blockIdx.x;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < SX; ++s) { mbar_init(smem_u32(&ctl->x_full[s]), 1); mbar_init(smem_u32(&ctl->x_empty[s]), 1); }
+        for (int s = 0; s < kAStages; ++s) { mbar_init(smem_u32(&ctl->a_full[s]), 128); mbar_init(smem_u32(&ctl->a_empty[s]), 1); }
+        mbar_init(smem_u32(&ctl->d_full), 1);
+        mbar_init(smem_u32(&ctl->d_empty), 128);
+        ctl->abort_flag = 0;
+        fence_barrier_init();
+        fence_proxy_async();
+    }
+    if (threadIdx.x < kMaxAlpha && (int)threadIdx.x < p.k)
+        ctl->alpha[threadIdx.x] = p.per_tile ? __ldg(p.alpha + threadIdx.x) : __ldg(p.alpha);
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    const int32_t n_tiles = p.w_tiles * p.t_tiles;
+    bool ok = true;
+
+    if (warp == 0) {
+        // ---------------- TMA producer: activation stages ----------------
+        Pipe px;
+        uint32_t issued_mask = 0, issued_phase = 0;
+        for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
+            const int32_t tok0 = (tile / p.w_tiles) * NTOK;
+            for (int32_t ks = 0; ks < p.k_stages && ok; ++ks) {
+                ok = wait_bar(smem_u32(&ctl->x_empty[px.stage]), px.phase ^ 1u, abort_flag, p.status,
+                              (1 << 24) | (px.stage << 16) | (bid & 0xffff));
+                if (!ok) break;
+                if (lane == 0) {
+                    const uint32_t bar = smem_u32(&ctl->x_full[px.stage]);
+                    mbar_arrive_expect_tx(bar, kStageBytes);
+                    tma_load_2d(stage0 + px.stage * kStageBytes, &x_map, ks * kStageK, tok0, bar);
+                }
+                issued_mask |= 1u << px.stage;
+                issued_phase = (issued_phase & ~(1u << px.stage)) | (px.phase << px.stage);
+                __syncwarp();
+                px.advance(SX);
+            }
+        }
+        if (!ok) {   // let copies in flight land before the CTA's shared memory goes away
+            for (int s = 0; s < SX; ++s)
+                if (issued_mask & (1u << s)) drain_wait(smem_u32(&ctl->x_full[s]), (issued_phase >> s) & 1u);
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        Pipe px, pa;
+        uint32_t dphase = 0;
+        for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
+            ok = wait_bar(smem_u32(&ctl->d_empty), dphase ^ 1u, abort_flag, p.status, (2 << 24) | (bid & 0xffff));
+            if (!ok) break;
+            tc_fence_after();
+            for (int32_t ks = 0; ks < p.k_stages && ok; ++ks) {
+                ok = wait_bar(smem_u32(&ctl->x_full[px.stage]), px.phase, abort_flag, p.status,
+                              (3 << 24) | (px.stage << 16) | (bid & 0xffff));
+                ok = ok && wait_bar(smem_u32(&ctl->a_full[pa.stage]), pa.phase, abort_flag, p.status,
+                                    (4 << 24) | (pa.stage << 16) | (bid & 0xffff));
+                if (!ok) break;
+                tc_fence_after();
+                if (lane == 0) {
+                    const int32_t rem = p.n - ks * kStageK;
+                    const int kk_end = rem >= kStageK ? 4 : (rem + 15) >> 4;
+                    const uint32_t b_addr = stage0 + px.stage * kStageBytes;
+                    const uint32_t a_addr = tmem_base + kDCols + pa.stage * kACols;
+#pragma unroll
+                    for (int a = 0; a < NA; ++a)
+                        for (int kk = 0; kk < kk_end; ++kk)
+                            tc_mma_ts(tmem_base + a * NTOK, a_addr + a * 32 + kk * 8, make_b_desc(b_addr + kk * 32),
+                                      kIdesc, (ks > 0 || kk > 0) ? 1u : 0u);
+                    tc_commit(smem_u32(&ctl->x_empty[px.stage]));
+                    tc_commit(smem_u32(&ctl->a_empty[pa.stage]));
+                }
+                __syncwarp();
+                px.advance(SX);
+                pa.advance(kAStages);
+            }
+            if (ok && lane == 0) tc_commit(smem_u32(&ctl->d_full));
+            __syncwarp();
+            dphase ^= 1u;
+        }
+    } else if (warp < 6) {
+        // ---------------- tile decode: bits -> +-1 bf16 pairs -> tensor memory ----------------
+        const int qd = warp & 3;
+        const int L = qd * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
+        const int64_t last_word = p.n_words - 1;
+        Pipe pa;
+        for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
+            const int32_t row_base = (tile % p.w_tiles) * (NA * 128) + L;
+            int64_t bitoff[NA];
+            uint32_t w0[NA], w1[NA], w2[NA];
+#pragma unroll
+            for (int a = 0; a < NA; ++a) {
+                const int32_t row = min(row_base + a * 128, p.r - 1);
+                bitoff[a] = (int64_t)row * p.n;
+                const int64_t wi = bitoff[a] >> 5;
+                w0[a] = __ldg(p.tile + min(wi, last_word));
+                w1[a] = __ldg(p.tile + min(wi + 1, last_word));
+                w2[a] = __ldg(p.tile + min(wi + 2, last_word));
+            }
+            for (int32_t ks = 0; ks < p.k_stages && ok; ++ks) {
+                uint32_t b0[NA], b1[NA];
+#pragma unroll
+                for (int a = 0; a < NA; ++a) {
+                    const uint32_t sh = (uint32_t)(bitoff[a] + (int64_t)ks * kStageK) & 31u;
+                    b0[a] = __funnelshift_r(w0[a], w1[a], sh);
+                    b1[a] = __funnelshift_r(w1[a], w2[a], sh);
+                    // fetch the next stage's words while this one is decoded
+                    const int64_t wi = (bitoff[a] + (int64_t)(ks + 1) * kStageK) >> 5;
+                    w0[a] = w2[a];
+                    if (ks + 1 < p.k_stages) {
+                        w1[a] = __ldg(p.tile + min(wi + 1, last_word));
+                        w2[a] = __ldg(p.tile + min(wi + 2, last_word));
+                    }
+                }
+                ok = wait_bar(smem_u32(&ctl->a_empty[pa.stage]), pa.phase ^ 1u, abort_flag, p.status,
+                              (5 << 24) | (pa.stage << 16) | (bid & 0xffff));
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int a = 0; a < NA; ++a) {
+                    uint32_t v[32];
+                    decode64(b0[a], b1[a], v);
+                    tmem_st_32x32(tmem_base + lane_base + kDCols + pa.stage * kACols + a * 32, v);
+                }
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(smem_u32(&ctl->a_full[pa.stage]));
+                pa.advance(kAStages);
+            }
+        }
+    } else {
+        // ---------------- epilogue: TMEM -> alpha / bias / activation -> k replicated stores ----------------
+        const int qd = warp & 3;
+        const int L = qd * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
+        uint32_t dphase = 0;
+        for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
+            const int64_t tok0 = (int64_t)(tile / p.w_tiles) * NTOK;
+            const int32_t row_base = (tile % p.w_tiles) * (NA * 128) + L;
+            ok = wait_bar(smem_u32(&ctl->d_full), dphase, abort_flag, p.status, (6 << 24) | (bid & 0xffff));
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int a = 0; a < NA; ++a) {
+                const int32_t row = row_base + a * 128;
+                const bool valid = row < p.r;
+                for (int c0 = 0; c0 < NTOK; c0 += 32) {
+                    if (tok0 + c0 >= p.T) break;                      // uniform: rest of the tile is padding
+                    uint32_t v[32];
+                    tmem_ld_32x32(tmem_base + lane_base + a * NTOK + c0, v);
+                    tc_wait_ld();
+                    if (!valid) continue;
+                    const int nt = (int)min((int64_t)32, p.T - tok0 - c0);
+                    for (int32_t j = 0; j < p.k; ++j) {
+                        const int32_t o = j * p.r + row;
+                        const float al = j < kMaxAlpha ? ctl->alpha[j]
+                                                       : (p.per_tile ? __ldg(p.alpha + j) : __ldg(p.alpha));
+                        const float b = p.bias ? __ldg(p.bias + o) : 0.0f;
+                        if (p.y_bf16) {
+                            __nv_bfloat16 *yp = static_cast<__nv_bfloat16 *>(p.y) + (tok0 + c0) * p.m + o;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                if (i < nt)
+                                    yp[(int64_t)i * p.m] =
+                                        __float2bfloat16_rn(apply_act(fmaf(al, __uint_as_float(v[i]), b), p.act));
+                        } else {
+                            float *yp = static_cast<float *>(p.y) + (tok0 + c0) * p.m + o;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                if (i < nt) yp[(int64_t)i * p.m] = apply_act(fmaf(al, __uint_as_float(v[i]), b), p.act);
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(smem_u32(&ctl->d_empty));
+            dphase ^= 1u;
+        }
+    }
+
+    // ---------------- teardown ----------------
+    if (warp == 1 && *abort_flag) {
+        // make sure no MMA is still reading shared or tensor memory before they are released
+        if (lane == 0) tc_commit(smem_u32(&ctl->x_empty[0]));
+        __syncwarp();
+        drain_wait(smem_u32(&ctl->x_empty[0]), 0);
+        drain_wait(smem_u32(&ctl->x_empty[0]), 1);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ---- host side -----------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+int sm_count()
+{
+    static int cache[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (!cache[dev]) cudaDeviceGetAttribute(&cache[dev], cudaDevAttrMultiProcessorCount, dev);
+    return cache[dev];
+}
+
+template <int NTOK, int NA, int SX>
+int launch_config(const LayerArgs &a, TcParams p, int *device_status, cudaStream_t s)
+{
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return TBN_ERR_CUDA;
+    CUtensorMap map;
+    const cuuint64_t dims[2] = {(cuuint64_t)a.n, (cuuint64_t)a.T};
+    const cuuint64_t strides[1] = {(cuuint64_t)a.n * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kStageK, (cuuint32_t)NTOK};
+    const cuuint32_t estr[2] = {1, 1};
+    if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(a.x), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return TBN_ERR_CUDA;
+
+    p.w_tiles = (p.r + NA * 128 - 1) / (NA * 128);
+    p.t_tiles = (int32_t)((a.T + NTOK - 1) / NTOK);
+    p.status = device_status;
+    const size_t smem = (size_t)SX * NTOK * 128 + sizeof(Control<SX>) + 1024;
+    auto kern = tc_linear_kernel<NTOK, NA, SX>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return TBN_ERR_CUDA;
+    const int sms = sm_count();
+    if (sms <= 0) return TBN_ERR_CUDA;
+    const int64_t tiles = (int64_t)p.w_tiles * p.t_tiles;
+    const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
+    kern<<<grid, kThreads, smem, s>>>(map, p);
+    return cudaGetLastError() == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+}
+
+}  // namespace
+
+bool tensor_path_supported(const LayerArgs &a)
+{
+    if (a.is_conv) return false;
+    if (a.q % a.n != 0) return false;            // the tile must span whole rows
+    if (a.n % 8 != 0) return false;              // TMA: row pitch a multiple of 16 bytes
+    if (a.T >= (int64_t)1 << 31) return false;   // TMA coordinates are 32-bit
+    return true;
+}
+
+int launch_tensor_linear(const LayerArgs &a, int *device_status, cudaStream_t s)
+{
+    if (a.x_dtype != TBN_BF16) return TBN_ERR_UNSUPPORTED;
+    TcParams p;
+    p.tile = a.tile; p.alpha = a.alpha; p.bias = a.bias; p.y = a.y; p.status = device_status;
+    p.T = a.T; p.n_words = tbn_tile_words(a.q);
+    p.n = a.n; p.m = a.m; p.r = (int32_t)(a.q / a.n); p.k = a.k;
+    p.k_stages = (a.n + kStageK - 1) / kStageK;
+    p.w_tiles = 0; p.t_tiles = 0;
+    p.per_tile = a.alpha_mode == TBN_ALPHA_PER_TILE; p.act = a.act; p.y_bf16 = a.y_dtype == TBN_BF16;
+
+    // Tile shape: estimated cycles = waves * NA * max(2*NTOK, decode floor) per stage; pick the cheapest.
+    const int sms = sm_count() > 0 ? sm_count() : 148;
+    struct Cand { int ntok, na; };
+    const Cand cands[] = {{192, 2}, {128, 2}, {256, 1}, {128, 1}, {64, 1}, {32, 1}};
+    int best = 0;
+    double best_cost = 1e300;
+    for (int i = 0; i < 6; ++i) {
+        const int64_t wt = (p.r + cands[i].na * 128 - 1) / (cands[i].na * 128);
+        const int64_t tt = (a.T + cands[i].ntok - 1) / cands[i].ntok;
+        const int64_t waves = (wt * tt + sms - 1) / sms;
+        const double stage = cands[i].na * (double)(2 * cands[i].ntok > 160 ? 2 * cands[i].ntok : 160);
+        const double epi = (double)cands[i].na * cands[i].ntok * a.k * 1.5;
+        const double cost = (double)waves * (stage * p.k_stages + epi);
+        if (cost < best_cost) { best_cost = cost; best = i; }
+    }
+    switch (best) {
+    case 0: return launch_config<192, 2, 6>(a, p, device_status, s);
+    case 1: return launch_config<128, 2, 8>(a, p, device_status, s);
+    case 2: return launch_config<256, 1, 5>(a, p, device_status, s);
+    case 3: return launch_config<128, 1, 8>(a, p, device_status, s);
+    case 4: return launch_config<64, 1, 8>(a, p, device_status, s);
+    default: return launch_config<32, 1, 8>(a, p, device_status, s);
+    }
+}
+
+}  // namespace tbn

@@ -106,3 +106,44 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     yd = B.tbn_linear_fwd(xh.to(DEV), m, tile, k, alpha, B.ALPHA_PER_TILE)
     assert torch.equal(yh, yd.cpu())
     assert_close(to_np64(yh), O.linear(x, words, k, al, True, m, n), "host entry point")
+
+
+# ------------------------------------------------------------------------------------------------
+# tensor-core (tcgen05) path
+TENSOR_SHAPES = ALIGNED + [(2048, 1024, 8), (64, 8200, 2), (256, 72, 1), (1024, 4096, 2)]
+
+
+@pytest.mark.parametrize("m,n,k", TENSOR_SHAPES)
+@pytest.mark.parametrize("T", [1, 3, 17, 64, 129, 200, 500])
+def test_tensor_path_matches_oracle(m, n, k, T):
+    for per_tile in (False, True):
+        x, W, words, al = make_linear_case(300 + T, T, m, n, k, per_tile, True)
+        ref = O.linear(x, words, k, al, per_tile, m, n, act=O.ACT_RELU)
+        got = run(B.PATH_TENSOR, x, words, al, per_tile, m, k, act=B.ACT_RELU)
+        assert_close(got, ref, f"tensor {m}x{n} k={k} T={T}")
+    assert B.tbn_last_device_status() == (0, 0)
+
+
+def test_tensor_path_fp32_activations_bias_fp32_out():
+    m, n, k, T = 512, 512, 4, 64
+    x, W, words, al = make_linear_case(0, T, m, n, k, True, False)
+    bias = synth.normal(0, 200, m, 0.1)
+    ref = O.linear(x, words, k, al, True, m, n, bias=bias.astype(np.float64), act=O.ACT_GELU)
+    got = run(B.PATH_TENSOR, x, words, al, True, m, k, act=B.ACT_GELU, bias=bias, y_dtype=B.F32)
+    assert_close(got, ref, "tensor fp32 in/out")
+
+
+@pytest.mark.parametrize("k", [2, 16])
+def test_tensor_path_many_tiles_sampled_rows(k):
+    # several waves of CTA tiles, ragged token tail; a seeded sample of rows through the oracle
+    m, n, T = 4096, 2048, 3000
+    x, W, words, al = make_linear_case(11, T, m, n, k, True, True)
+    got = run(B.PATH_TENSOR, x, words, al, True, m, k)
+    rows = np.sort(np.random.default_rng(1).choice(T, 40, replace=False))
+    rows[-1] = T - 1
+    ref = O.linear(x[rows], words, k, al, True, m, n)
+    assert_close(got[rows], ref, f"tensor many tiles k={k}")
+    # and the whole output against the generic kernel (no shortcut, CUDA cores)
+    gen = run(B.PATH_GENERIC, x, words, al, True, m, k)
+    assert_close(got, gen, "tensor vs generic")
+    assert B.tbn_last_device_status() == (0, 0)
