@@ -154,8 +154,12 @@ def main():
     ap.add_argument("--tokens", type=int, default=16384, help="development override of the batch size")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ks", default="", help="development override: comma-separated subset of k values")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.ks:
+        global KS
+        KS = tuple(int(v) for v in args.ks.split(","))
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -265,7 +269,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
 
     # ---- end to end: host buffers through the C-ABI, copies inside the timed region -------------
     e2e = None
-    if rank == 0 or world > 1:
+    if args.e2e_steps > 0:
         xh = torch.from_numpy(x_np.view(np.int16)).view(torch.bfloat16).pin_memory()
         yh = torch.empty((T, N_FEAT), dtype=torch.bfloat16).pin_memory()
         hws = torch.empty(B.tbn_linear_host_workspace_bytes(T, N_FEAT, N_FEAT, 2, B.BF16, B.BF16),
