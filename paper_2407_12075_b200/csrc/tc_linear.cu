@@ -18,6 +18,8 @@
 // bounded by a wall-clock limit, after which the CTA records TBN_ERR_TIMEOUT, drains and returns.
 #include <cuda.h>
 
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace tbn {
@@ -25,7 +27,7 @@ namespace tbn {
 namespace {
 
 constexpr int kThreads = 320;
-constexpr int kStageK = 64;            // contraction elements per pipeline stage (= one 128-byte swizzle row)
+constexpr int kAtomK = 64;             // contraction elements per 128-byte swizzle row (one TMA box, 4 MMA K steps)
 constexpr int kAStages = 2;            // decoded-weight stages in tensor memory
 constexpr int kMaxAlpha = 64;          // alphas cached in shared memory
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: orders of magnitude above any legitimate wait
@@ -89,14 +91,16 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                  : "memory");
 }
-// D[tmem] (+)= A[tmem] * B[smem]^T, bf16 x bf16 -> fp32, M = 128
-__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate) {
+// D[tmem] (+)= A[tmem] * B[smem]^T, bf16 x bf16 -> fp32, M = 128.  The shared-memory descriptor is passed
+// as its two 32-bit halves so that stepping along K is a single 32-bit add on the low word.
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_desc_lo, uint32_t b_desc_hi,
+                                          uint32_t idesc, uint32_t accumulate) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+        "{\n\t.reg .pred p;\n\t.reg .b64 bd;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 bd, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], bd, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_desc_lo), "r"(b_desc_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -205,11 +209,11 @@ __host__ __device__ constexpr uint32_t next_pow2_cols(uint32_t c) {
     return p;
 }
 
-// Shared-memory matrix descriptor of one activation stage: K-major, 128-byte swizzle, rows of 128 bytes,
-// 8-row groups 1024 bytes apart.  `addr` may point 32*kk bytes into the first row to select a K slice.
-__device__ __forceinline__ uint64_t make_b_desc(uint32_t addr) {
-    return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
-}
+// Shared-memory matrix descriptor of the activation operand: K-major, 128-byte swizzle, rows of 128 bytes,
+// 8-row groups 1024 bytes apart (stride offset 64 x 16 bytes), descriptor version 1, leading offset 1.
+// The low word carries the start address in 16-byte units; advancing it by 2 selects the next 16-element
+// K slice inside the swizzled row.
+constexpr uint64_t kBDescHi = (64ull << 32) | (1ull << 46) | (2ull << 61);
 
 // Quiet bounded wait used only while draining after an abort.
 __device__ __forceinline__ void drain_wait(uint32_t bar, uint32_t parity) {
@@ -219,14 +223,26 @@ __device__ __forceinline__ void drain_wait(uint32_t bar, uint32_t parity) {
     }
 }
 
-template <int NTOK, int NA, int SX>
+// Single-thread bounded wait (the MMA issuer runs on one lane).
+__device__ __forceinline__ bool wait_one(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
+                                         int detail) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return wait_slow(bar, parity, abort_flag, status, detail);
+}
+
+// NTOK tokens x (NA x 128) weight rows per CTA tile; KA 64-element K atoms per pipeline stage; SX activation
+// stages in shared memory.  Tensor memory: NA accumulators of NTOK columns, then kAStages decoded-weight
+// stages of NA x KA x 32 columns.
+template <int NTOK, int NA, int KA, int SX>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
 {
     static_assert(NTOK % 32 == 0 && NTOK >= 32 && NTOK <= 256, "token tile");
-    constexpr uint32_t kStageBytes = NTOK * 128;
+    constexpr uint32_t kAtomBytes = NTOK * 128;
+    constexpr uint32_t kStageBytes = KA * kAtomBytes;
+    constexpr int kStageK = KA * kAtomK;
     constexpr uint32_t kDCols = NA * NTOK;
-    constexpr uint32_t kACols = NA * 32;
+    constexpr uint32_t kACols = NA * KA * 32;
     constexpr uint32_t kTmemCols = next_pow2_cols(kDCols + kAStages * kACols);
     static_assert(kTmemCols <= 512, "tensor memory budget");
     // instruction descriptor: D fp32, A and B bf16, both K-major, N = NTOK, M = 128
@@ -278,7 +294,10 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                 if (lane == 0) {
                     const uint32_t bar = smem_u32(&ctl->x_full[px.stage]);
                     mbar_arrive_expect_tx(bar, kStageBytes);
-                    tma_load_2d(stage0 + px.stage * kStageBytes, &x_map, ks * kStageK, tok0, bar);
+#pragma unroll
+                    for (int at = 0; at < KA; ++at)   // a box that lies past the last column is zero-filled
+                        tma_load_2d(stage0 + px.stage * kStageBytes + at * kAtomBytes, &x_map,
+                                    ks * kStageK + at * kAtomK, tok0, bar);
                 }
                 issued_mask |= 1u << px.stage;
                 issued_phase = (issued_phase & ~(1u << px.stage)) | (px.phase << px.stage);
@@ -291,43 +310,80 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                 if (issued_mask & (1u << s)) drain_wait(smem_u32(&ctl->x_full[s]), (issued_phase >> s) & 1u);
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        Pipe px, pa;
-        uint32_t dphase = 0;
-        for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
-            ok = wait_bar(smem_u32(&ctl->d_empty), dphase ^ 1u, abort_flag, p.status, (2 << 24) | (bid & 0xffff));
-            if (!ok) break;
-            tc_fence_after();
-            for (int32_t ks = 0; ks < p.k_stages && ok; ++ks) {
-                ok = wait_bar(smem_u32(&ctl->x_full[px.stage]), px.phase, abort_flag, p.status,
-                              (3 << 24) | (px.stage << 16) | (bid & 0xffff));
-                ok = ok && wait_bar(smem_u32(&ctl->a_full[pa.stage]), pa.phase, abort_flag, p.status,
-                                    (4 << 24) | (pa.stage << 16) | (bid & 0xffff));
+        // ---------------- MMA issuer (lane 0) ----------------
+        // tcgen05.mma is issued by one thread, and that thread's instructions execute back to back with no
+        // other warp to hide their latency: every instruction between two MMAs is dead time for the tensor
+        // cores once their small queue has drained.  So the K steps of a full stage are unrolled with all
+        // offsets immediate (two adds per MMA), the NEXT stage's barriers are polled in the middle of the
+        // current stage (if they are already complete, the common case, the next stage starts at once),
+        // and the other 31 lanes stay out of the loop.
+        if (lane == 0) {
+            Pipe px, pa;
+            uint32_t dphase = 0;
+            bool ready = false;
+            constexpr uint32_t kDescHi = (uint32_t)(kBDescHi >> 32);
+            constexpr int kSteps = KA * 4;             // 16-element K steps per full stage
+            for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
+                ok = wait_one(smem_u32(&ctl->d_empty), dphase ^ 1u, abort_flag, p.status, (2 << 24) | (bid & 0xffff));
                 if (!ok) break;
                 tc_fence_after();
-                if (lane == 0) {
-                    const int32_t rem = p.n - ks * kStageK;
-                    const int kk_end = rem >= kStageK ? 4 : (rem + 15) >> 4;
-                    const uint32_t b_addr = stage0 + px.stage * kStageBytes;
+                for (int32_t ks = 0; ks < p.k_stages; ++ks) {
+                    if (!ready) {
+                        ok = wait_one(smem_u32(&ctl->x_full[px.stage]), px.phase, abort_flag, p.status,
+                                      (3 << 24) | (px.stage << 16) | (bid & 0xffff)) &&
+                             wait_one(smem_u32(&ctl->a_full[pa.stage]), pa.phase, abort_flag, p.status,
+                                      (4 << 24) | (pa.stage << 16) | (bid & 0xffff));
+                        if (!ok) break;
+                    }
+                    tc_fence_after();
+                    // descriptor low word: start address in 16-byte units | leading offset 1 << 16
+                    const uint32_t b_lo = (((stage0 + px.stage * kStageBytes) & 0x3FFFFu) >> 4) | (1u << 16);
                     const uint32_t a_addr = tmem_base + kDCols + pa.stage * kACols;
+                    Pipe nx = px, na = pa;
+                    nx.advance(SX);
+                    na.advance(kAStages);
+                    const int32_t rem = p.n - ks * kStageK;
+                    if (rem >= kStageK) {
 #pragma unroll
-                    for (int a = 0; a < NA; ++a)
-                        for (int kk = 0; kk < kk_end; ++kk)
-                            tc_mma_ts(tmem_base + a * NTOK, a_addr + a * 32 + kk * 8, make_b_desc(b_addr + kk * 32),
-                                      kIdesc, (ks > 0 || kk > 0) ? 1u : 0u);
+                        for (int st = 0; st < kSteps; ++st) {
+                            const int at = st >> 2, kk = st & 3;
+#pragma unroll
+                            for (int a = 0; a < NA; ++a)
+                                tc_mma_ts(tmem_base + a * NTOK, a_addr + (a * KA + at) * 32 + kk * 8,
+                                          b_lo + at * (kAtomBytes >> 4) + kk * 2, kDescHi, kIdesc,
+                                          st > 0 ? 1u : (uint32_t)(ks > 0));
+                            if (st == kSteps / 2 - 1)
+                                ready = mbar_try_wait(smem_u32(&ctl->x_full[nx.stage]), nx.phase) &&
+                                        mbar_try_wait(smem_u32(&ctl->a_full[na.stage]), na.phase);
+                        }
+                    } else {                              // ragged last stage: only the K steps that hold data
+                        const int steps = (rem + 15) >> 4;
+                        for (int st = 0; st < steps; ++st) {
+                            const int at = st >> 2, kk = st & 3;
+#pragma unroll
+                            for (int a = 0; a < NA; ++a)
+                                tc_mma_ts(tmem_base + a * NTOK, a_addr + (a * KA + at) * 32 + kk * 8,
+                                          b_lo + at * (kAtomBytes >> 4) + kk * 2, kDescHi, kIdesc,
+                                          (ks > 0 || st > 0) ? 1u : 0u);
+                        }
+                        ready = false;
+                    }
                     tc_commit(smem_u32(&ctl->x_empty[px.stage]));
                     tc_commit(smem_u32(&ctl->a_empty[pa.stage]));
+                    if (ks == p.k_stages - 1) tc_commit(smem_u32(&ctl->d_full));
+                    px = nx;
+                    pa = na;
                 }
-                __syncwarp();
-                px.advance(SX);
-                pa.advance(kAStages);
+                dphase ^= 1u;
             }
-            if (ok && lane == 0) tc_commit(smem_u32(&ctl->d_full));
-            __syncwarp();
-            dphase ^= 1u;
         }
+        __syncwarp();
     } else if (warp < 6) {
         // ---------------- tile decode: bits -> +-1 bf16 pairs -> tensor memory ----------------
+        // Thread (quadrant qd, lane) owns TMEM lane L = 32*qd + lane, i.e. weight row L of each of the NA
+        // blocks.  Per stage it needs 64*KA consecutive bits of each row; the words for the next stage are
+        // requested before this stage is decoded, so their latency overlaps the ALU work.
+        constexpr int kW = 2 * KA;                 // 32-bit words of tile bits per row and stage
         const int qd = warp & 3;
         const int L = qd * 32 + lane;
         const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
@@ -336,29 +392,27 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
         for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
             const int32_t row_base = (tile % p.w_tiles) * (NA * 128) + L;
             int64_t bitoff[NA];
-            uint32_t w0[NA], w1[NA], w2[NA];
+            uint32_t w[NA][kW + 1];
 #pragma unroll
             for (int a = 0; a < NA; ++a) {
-                const int32_t row = min(row_base + a * 128, p.r - 1);
+                const int32_t row = min(row_base + a * 128, p.r - 1);   // rows past the end are never stored
                 bitoff[a] = (int64_t)row * p.n;
                 const int64_t wi = bitoff[a] >> 5;
-                w0[a] = __ldg(p.tile + min(wi, last_word));
-                w1[a] = __ldg(p.tile + min(wi + 1, last_word));
-                w2[a] = __ldg(p.tile + min(wi + 2, last_word));
+#pragma unroll
+                for (int i = 0; i <= kW; ++i) w[a][i] = __ldg(p.tile + min(wi + i, last_word));
             }
             for (int32_t ks = 0; ks < p.k_stages && ok; ++ks) {
-                uint32_t b0[NA], b1[NA];
+                uint32_t b[NA][kW];
 #pragma unroll
                 for (int a = 0; a < NA; ++a) {
-                    const uint32_t sh = (uint32_t)(bitoff[a] + (int64_t)ks * kStageK) & 31u;
-                    b0[a] = __funnelshift_r(w0[a], w1[a], sh);
-                    b1[a] = __funnelshift_r(w1[a], w2[a], sh);
-                    // fetch the next stage's words while this one is decoded
-                    const int64_t wi = (bitoff[a] + (int64_t)(ks + 1) * kStageK) >> 5;
-                    w0[a] = w2[a];
+                    const uint32_t sh = (uint32_t)bitoff[a] & 31u;      // constant along the row: stages are 64*KA bits
+#pragma unroll
+                    for (int i = 0; i < kW; ++i) b[a][i] = __funnelshift_r(w[a][i], w[a][i + 1], sh);
+                    w[a][0] = w[a][kW];
                     if (ks + 1 < p.k_stages) {
-                        w1[a] = __ldg(p.tile + min(wi + 1, last_word));
-                        w2[a] = __ldg(p.tile + min(wi + 2, last_word));
+                        const int64_t wi = (bitoff[a] + (int64_t)(ks + 1) * kStageK) >> 5;
+#pragma unroll
+                        for (int i = 1; i <= kW; ++i) w[a][i] = __ldg(p.tile + min(wi + i, last_word));
                     }
                 }
                 ok = wait_bar(smem_u32(&ctl->a_empty[pa.stage]), pa.phase ^ 1u, abort_flag, p.status,
@@ -367,9 +421,12 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                 tc_fence_after();
 #pragma unroll
                 for (int a = 0; a < NA; ++a) {
-                    uint32_t v[32];
-                    decode64(b0[a], b1[a], v);
-                    tmem_st_32x32(tmem_base + lane_base + kDCols + pa.stage * kACols + a * 32, v);
+#pragma unroll
+                    for (int at = 0; at < KA; ++at) {
+                        uint32_t v[32];
+                        decode64(b[a][2 * at], b[a][2 * at + 1], v);
+                        tmem_st_32x32(tmem_base + lane_base + kDCols + pa.stage * kACols + (a * KA + at) * 32, v);
+                    }
                 }
                 tc_wait_st();
                 tc_fence_before();
@@ -471,7 +528,7 @@ int sm_count()
     return cache[dev];
 }
 
-template <int NTOK, int NA, int SX>
+template <int NTOK, int NA, int KA, int SX>
 int launch_config(const LayerArgs &a, TcParams p, int *device_status, cudaStream_t s)
 {
     EncodeTiledFn encode = encode_tiled_fn();
@@ -479,7 +536,7 @@ int launch_config(const LayerArgs &a, TcParams p, int *device_status, cudaStream
     CUtensorMap map;
     const cuuint64_t dims[2] = {(cuuint64_t)a.n, (cuuint64_t)a.T};
     const cuuint64_t strides[1] = {(cuuint64_t)a.n * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kStageK, (cuuint32_t)NTOK};
+    const cuuint32_t box[2] = {(cuuint32_t)kAtomK, (cuuint32_t)NTOK};
     const cuuint32_t estr[2] = {1, 1};
     if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(a.x), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -488,9 +545,10 @@ int launch_config(const LayerArgs &a, TcParams p, int *device_status, cudaStream
 
     p.w_tiles = (p.r + NA * 128 - 1) / (NA * 128);
     p.t_tiles = (int32_t)((a.T + NTOK - 1) / NTOK);
+    p.k_stages = (a.n + KA * kAtomK - 1) / (KA * kAtomK);
     p.status = device_status;
-    const size_t smem = (size_t)SX * NTOK * 128 + sizeof(Control<SX>) + 1024;
-    auto kern = tc_linear_kernel<NTOK, NA, SX>;
+    const size_t smem = (size_t)SX * KA * NTOK * 128 + sizeof(Control<SX>) + 1024;
+    auto kern = tc_linear_kernel<NTOK, NA, KA, SX>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return TBN_ERR_CUDA;
     const int sms = sm_count();
@@ -519,32 +577,38 @@ int launch_tensor_linear(const LayerArgs &a, int *device_status, cudaStream_t s)
     p.tile = a.tile; p.alpha = a.alpha; p.bias = a.bias; p.y = a.y; p.status = device_status;
     p.T = a.T; p.n_words = tbn_tile_words(a.q);
     p.n = a.n; p.m = a.m; p.r = (int32_t)(a.q / a.n); p.k = a.k;
-    p.k_stages = (a.n + kStageK - 1) / kStageK;
+    p.k_stages = 0;
     p.w_tiles = 0; p.t_tiles = 0;
     p.per_tile = a.alpha_mode == TBN_ALPHA_PER_TILE; p.act = a.act; p.y_bf16 = a.y_dtype == TBN_BF16;
 
-    // Tile shape: estimated cycles = waves * NA * max(2*NTOK, decode floor) per stage; pick the cheapest.
+    // Tile shape.  Cost model in tensor-pipe cycles per CTA: every 64-element K atom costs 4 MMAs of
+    // NTOK/2 cycles per block of 128 rows, but never less than the decode of that atom (~170 cycles per
+    // block); the epilogue adds about 1.5 cycles per stored element per warp quadrant.  The cheapest
+    // candidate over whole waves of CTAs wins.
     const int sms = sm_count() > 0 ? sm_count() : 148;
     struct Cand { int ntok, na; };
-    const Cand cands[] = {{192, 2}, {128, 2}, {256, 1}, {128, 1}, {64, 1}, {32, 1}};
+    const Cand cands[] = {{128, 2}, {192, 2}, {256, 1}, {128, 1}, {64, 1}, {32, 1}};
+    const int n_cands = 6;
     int best = 0;
     double best_cost = 1e300;
-    for (int i = 0; i < 6; ++i) {
+    const char *force = getenv("TBN_TC_CONFIG");     // tuning aid: force a candidate by index
+    for (int i = 0; i < n_cands; ++i) {
         const int64_t wt = (p.r + cands[i].na * 128 - 1) / (cands[i].na * 128);
         const int64_t tt = (a.T + cands[i].ntok - 1) / cands[i].ntok;
         const int64_t waves = (wt * tt + sms - 1) / sms;
-        const double stage = cands[i].na * (double)(2 * cands[i].ntok > 160 ? 2 * cands[i].ntok : 160);
+        const double atom = cands[i].na * (double)(2 * cands[i].ntok > 170 ? 2 * cands[i].ntok : 170);
         const double epi = (double)cands[i].na * cands[i].ntok * a.k * 1.5;
-        const double cost = (double)waves * (stage * p.k_stages + epi);
+        const double cost = (double)waves * (atom * ((a.n + kAtomK - 1) / kAtomK) + epi);
         if (cost < best_cost) { best_cost = cost; best = i; }
     }
+    if (force && force[0] >= '0' && force[0] < '0' + n_cands && force[1] == 0) best = force[0] - '0';
     switch (best) {
-    case 0: return launch_config<192, 2, 6>(a, p, device_status, s);
-    case 1: return launch_config<128, 2, 8>(a, p, device_status, s);
-    case 2: return launch_config<256, 1, 5>(a, p, device_status, s);
-    case 3: return launch_config<128, 1, 8>(a, p, device_status, s);
-    case 4: return launch_config<64, 1, 8>(a, p, device_status, s);
-    default: return launch_config<32, 1, 8>(a, p, device_status, s);
+    case 0: return launch_config<128, 2, 2, 5>(a, p, device_status, s);
+    case 1: return launch_config<192, 2, 1, 6>(a, p, device_status, s);
+    case 2: return launch_config<256, 1, 2, 3>(a, p, device_status, s);
+    case 3: return launch_config<128, 1, 2, 6>(a, p, device_status, s);
+    case 4: return launch_config<64, 1, 2, 8>(a, p, device_status, s);
+    default: return launch_config<32, 1, 2, 8>(a, p, device_status, s);
     }
 }
 
