@@ -150,10 +150,11 @@ template <int SX>
 struct Control {
     uint64_t x_full[SX], x_empty[SX];
     uint64_t a_full[kAStages], a_empty[kAStages];
-    uint64_t d_full, d_empty;
+    uint64_t d_full[2], d_empty[2];
     uint32_t tmem_base;
     int abort_flag;
     float alpha[kMaxAlpha];
+    uint32_t transpose[4][32 * 33];      // one padded 32 x 32 block per epilogue warp
 };
 
 struct Pipe {
@@ -231,9 +232,10 @@ __device__ __forceinline__ bool wait_one(uint32_t bar, uint32_t parity, volatile
 }
 
 // NTOK tokens x (NA x 128) weight rows per CTA tile; KA 64-element K atoms per pipeline stage; SX activation
-// stages in shared memory.  Tensor memory: NA accumulators of NTOK columns, then kAStages decoded-weight
-// stages of NA x KA x 32 columns.
-template <int NTOK, int NA, int KA, int SX>
+// stages in shared memory; DB accumulator buffers (2 = the epilogue of one tile overlaps the main loop of the
+// next).  Tensor memory: DB x NA accumulators of NTOK columns, then kAStages decoded-weight stages of
+// NA x KA x 32 columns.
+template <int NTOK, int NA, int KA, int SX, int DB>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
 {
@@ -243,7 +245,8 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
     constexpr int kStageK = KA * kAtomK;
     constexpr uint32_t kDCols = NA * NTOK;
     constexpr uint32_t kACols = NA * KA * 32;
-    constexpr uint32_t kTmemCols = next_pow2_cols(kDCols + kAStages * kACols);
+    constexpr uint32_t kABase = DB * kDCols;             // first column of the decoded-weight stages
+    constexpr uint32_t kTmemCols = next_pow2_cols(kABase + kAStages * kACols);
     static_assert(kTmemCols <= 512, "tensor memory budget");
     // instruction descriptor: D fp32, A and B bf16, both K-major, N = NTOK, M = 128
     constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NTOK >> 3) << 17) | (8u << 24);
@@ -261,8 +264,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
     if (threadIdx.x == 0) {
         for (int s = 0; s < SX; ++s) { mbar_init(smem_u32(&ctl->x_full[s]), 1); mbar_init(smem_u32(&ctl->x_empty[s]), 1); }
         for (int s = 0; s < kAStages; ++s) { mbar_init(smem_u32(&ctl->a_full[s]), 128); mbar_init(smem_u32(&ctl->a_empty[s]), 1); }
-        mbar_init(smem_u32(&ctl->d_full), 1);
-        mbar_init(smem_u32(&ctl->d_empty), 128);
+        for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&ctl->d_full[s]), 1); mbar_init(smem_u32(&ctl->d_empty[s]), 128); }
         ctl->abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async();
@@ -318,15 +320,16 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
         // current stage (if they are already complete, the common case, the next stage starts at once),
         // and the other 31 lanes stay out of the loop.
         if (lane == 0) {
-            Pipe px, pa;
-            uint32_t dphase = 0;
+            Pipe px, pa, pd;
             bool ready = false;
             constexpr uint32_t kDescHi = (uint32_t)(kBDescHi >> 32);
             constexpr int kSteps = KA * 4;             // 16-element K steps per full stage
             for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
-                ok = wait_one(smem_u32(&ctl->d_empty), dphase ^ 1u, abort_flag, p.status, (2 << 24) | (bid & 0xffff));
+                ok = wait_one(smem_u32(&ctl->d_empty[pd.stage]), pd.phase ^ 1u, abort_flag, p.status,
+                              (2 << 24) | (bid & 0xffff));
                 if (!ok) break;
                 tc_fence_after();
+                const uint32_t d_addr = tmem_base + pd.stage * kDCols;
                 for (int32_t ks = 0; ks < p.k_stages; ++ks) {
                     if (!ready) {
                         ok = wait_one(smem_u32(&ctl->x_full[px.stage]), px.phase, abort_flag, p.status,
@@ -338,7 +341,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                     tc_fence_after();
                     // descriptor low word: start address in 16-byte units | leading offset 1 << 16
                     const uint32_t b_lo = (((stage0 + px.stage * kStageBytes) & 0x3FFFFu) >> 4) | (1u << 16);
-                    const uint32_t a_addr = tmem_base + kDCols + pa.stage * kACols;
+                    const uint32_t a_addr = tmem_base + kABase + pa.stage * kACols;
                     Pipe nx = px, na = pa;
                     nx.advance(SX);
                     na.advance(kAStages);
@@ -349,7 +352,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                             const int at = st >> 2, kk = st & 3;
 #pragma unroll
                             for (int a = 0; a < NA; ++a)
-                                tc_mma_ts(tmem_base + a * NTOK, a_addr + (a * KA + at) * 32 + kk * 8,
+                                tc_mma_ts(d_addr + a * NTOK, a_addr + (a * KA + at) * 32 + kk * 8,
                                           b_lo + at * (kAtomBytes >> 4) + kk * 2, kDescHi, kIdesc,
                                           st > 0 ? 1u : (uint32_t)(ks > 0));
                             if (st == kSteps / 2 - 1)
@@ -362,7 +365,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                             const int at = st >> 2, kk = st & 3;
 #pragma unroll
                             for (int a = 0; a < NA; ++a)
-                                tc_mma_ts(tmem_base + a * NTOK, a_addr + (a * KA + at) * 32 + kk * 8,
+                                tc_mma_ts(d_addr + a * NTOK, a_addr + (a * KA + at) * 32 + kk * 8,
                                           b_lo + at * (kAtomBytes >> 4) + kk * 2, kDescHi, kIdesc,
                                           (ks > 0 || st > 0) ? 1u : 0u);
                         }
@@ -370,11 +373,11 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                     }
                     tc_commit(smem_u32(&ctl->x_empty[px.stage]));
                     tc_commit(smem_u32(&ctl->a_empty[pa.stage]));
-                    if (ks == p.k_stages - 1) tc_commit(smem_u32(&ctl->d_full));
+                    if (ks == p.k_stages - 1) tc_commit(smem_u32(&ctl->d_full[pd.stage]));
                     px = nx;
                     pa = na;
                 }
-                dphase ^= 1u;
+                pd.advance(DB);
             }
         }
         __syncwarp();
@@ -425,7 +428,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                     for (int at = 0; at < KA; ++at) {
                         uint32_t v[32];
                         decode64(b[a][2 * at], b[a][2 * at + 1], v);
-                        tmem_st_32x32(tmem_base + lane_base + kDCols + pa.stage * kACols + (a * KA + at) * 32, v);
+                        tmem_st_32x32(tmem_base + lane_base + kABase + pa.stage * kACols + (a * KA + at) * 32, v);
                     }
                 }
                 tc_wait_st();
@@ -435,52 +438,83 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
             }
         }
     } else {
-        // ---------------- epilogue: TMEM -> alpha / bias / activation -> k replicated stores ----------------
+        // ---------------- epilogue: TMEM -> transpose -> alpha / bias / activation -> k replicated stores ------
+        // tcgen05.ld hands thread (quadrant qd, lane) one weight row and 32 consecutive tokens.  The output is
+        // row-major [token][feature], so each 32 x 32 block goes through a private padded shared-memory buffer
+        // and comes back with thread = token holding 32 consecutive output features: every repetition j is then
+        // one multiply per element (fp32), a pack to bf16 and four 16-byte stores per thread.
         const int qd = warp & 3;
-        const int L = qd * 32 + lane;
         const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
-        uint32_t dphase = 0;
+        uint32_t *tbuf = ctl->transpose[warp - 6];
+        Pipe pd;                                          // accumulator buffer (stage) and its phase
+        const bool vec_ok = (p.m % 8 == 0) && (p.r % 8 == 0);
         for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
             const int64_t tok0 = (int64_t)(tile / p.w_tiles) * NTOK;
-            const int32_t row_base = (tile % p.w_tiles) * (NA * 128) + L;
-            ok = wait_bar(smem_u32(&ctl->d_full), dphase, abort_flag, p.status, (6 << 24) | (bid & 0xffff));
+            ok = wait_bar(smem_u32(&ctl->d_full[pd.stage]), pd.phase, abort_flag, p.status, (6 << 24) | (bid & 0xffff));
             if (!ok) break;
             tc_fence_after();
-#pragma unroll
+            const int n_chunks = (int)min((int64_t)(NTOK / 32), (p.T - tok0 + 31) / 32);
+#pragma unroll 1
             for (int a = 0; a < NA; ++a) {
-                const int32_t row = row_base + a * 128;
-                const bool valid = row < p.r;
-                for (int c0 = 0; c0 < NTOK; c0 += 32) {
-                    if (tok0 + c0 >= p.T) break;                      // uniform: rest of the tile is padding
+                const int32_t row0 = (tile % p.w_tiles) * (NA * 128) + a * 128 + qd * 32;
+                const int rows_valid = max(0, min(32, p.r - row0));
+#pragma unroll 1
+                for (int ch = 0; ch < n_chunks; ++ch) {
+                    __syncwarp();                                 // reconverge before the warp-wide TMEM load
                     uint32_t v[32];
-                    tmem_ld_32x32(tmem_base + lane_base + a * NTOK + c0, v);
+                    tmem_ld_32x32(tmem_base + lane_base + pd.stage * kDCols + a * NTOK + ch * 32, v);
                     tc_wait_ld();
-                    if (!valid) continue;
-                    const int nt = (int)min((int64_t)32, p.T - tok0 - c0);
+                    if (a == NA - 1 && ch == n_chunks - 1) {      // accumulator fully read: hand it back early
+                        tc_fence_before();
+                        mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));
+                    }
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) tbuf[i * 33 + lane] = v[i];
+                    __syncwarp();
+                    float z[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) z[i] = __uint_as_float(tbuf[lane * 33 + i]);
+                    __syncwarp();
+                    const int64_t tok = tok0 + ch * 32 + lane;
+                    if (tok >= p.T || rows_valid == 0) continue;
+                    if (p.act == TBN_ACT_RELU && p.bias == nullptr) {
+                        // alpha >= 0, so relu(alpha * z) = alpha * relu(z): clamp once, outside the k loop
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) z[i] = fmaxf(z[i], 0.0f);
+                    }
+                    const bool plain = p.bias == nullptr && (p.act == TBN_ACT_NONE || p.act == TBN_ACT_RELU);
                     for (int32_t j = 0; j < p.k; ++j) {
-                        const int32_t o = j * p.r + row;
                         const float al = j < kMaxAlpha ? ctl->alpha[j]
                                                        : (p.per_tile ? __ldg(p.alpha + j) : __ldg(p.alpha));
-                        const float b = p.bias ? __ldg(p.bias + o) : 0.0f;
-                        if (p.y_bf16) {
-                            __nv_bfloat16 *yp = static_cast<__nv_bfloat16 *>(p.y) + (tok0 + c0) * p.m + o;
+                        const int64_t o0 = (int64_t)j * p.r + row0;
+                        const int64_t yi = tok * p.m + o0;
+                        if (rows_valid == 32 && vec_ok && plain && p.y_bf16) {
+                            uint4 *dst = reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(p.y) + yi);
 #pragma unroll
-                            for (int i = 0; i < 32; ++i)
-                                if (i < nt)
-                                    yp[(int64_t)i * p.m] =
-                                        __float2bfloat16_rn(apply_act(fmaf(al, __uint_as_float(v[i]), b), p.act));
+                            for (int g = 0; g < 4; ++g) {
+                                uint32_t pk[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const __nv_bfloat162 h =
+                                        __floats2bfloat162_rn(al * z[g * 8 + 2 * e], al * z[g * 8 + 2 * e + 1]);
+                                    pk[e] = *reinterpret_cast<const uint32_t *>(&h);
+                                }
+                                dst[g] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                            }
                         } else {
-                            float *yp = static_cast<float *>(p.y) + (tok0 + c0) * p.m + o;
-#pragma unroll
-                            for (int i = 0; i < 32; ++i)
-                                if (i < nt) yp[(int64_t)i * p.m] = apply_act(fmaf(al, __uint_as_float(v[i]), b), p.act);
+                            for (int i = 0; i < rows_valid; ++i) {
+                                // general path: own column of the transpose buffer (unclamped accumulator)
+                                const float zz = __uint_as_float(tbuf[lane * 33 + i]);
+                                const float b = p.bias ? __ldg(p.bias + o0 + i) : 0.0f;
+                                const float val = apply_act(fmaf(al, zz, b), p.act);
+                                if (p.y_bf16) static_cast<__nv_bfloat16 *>(p.y)[yi + i] = __float2bfloat16_rn(val);
+                                else static_cast<float *>(p.y)[yi + i] = val;
+                            }
                         }
                     }
                 }
             }
-            tc_fence_before();
-            mbar_arrive(smem_u32(&ctl->d_empty));
-            dphase ^= 1u;
+            pd.advance(DB);
         }
     }
 
@@ -528,7 +562,7 @@ int sm_count()
     return cache[dev];
 }
 
-template <int NTOK, int NA, int KA, int SX>
+template <int NTOK, int NA, int KA, int SX, int DB>
 int launch_config(const LayerArgs &a, TcParams p, int *device_status, cudaStream_t s)
 {
     EncodeTiledFn encode = encode_tiled_fn();
@@ -548,7 +582,7 @@ int launch_config(const LayerArgs &a, TcParams p, int *device_status, cudaStream
     p.k_stages = (a.n + KA * kAtomK - 1) / (KA * kAtomK);
     p.status = device_status;
     const size_t smem = (size_t)SX * KA * NTOK * 128 + sizeof(Control<SX>) + 1024;
-    auto kern = tc_linear_kernel<NTOK, NA, KA, SX>;
+    auto kern = tc_linear_kernel<NTOK, NA, KA, SX, DB>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return TBN_ERR_CUDA;
     const int sms = sm_count();
@@ -581,34 +615,37 @@ int launch_tensor_linear(const LayerArgs &a, int *device_status, cudaStream_t s)
     p.w_tiles = 0; p.t_tiles = 0;
     p.per_tile = a.alpha_mode == TBN_ALPHA_PER_TILE; p.act = a.act; p.y_bf16 = a.y_dtype == TBN_BF16;
 
-    // Tile shape.  Cost model in tensor-pipe cycles per CTA: every 64-element K atom costs 4 MMAs of
-    // NTOK/2 cycles per block of 128 rows, but never less than the decode of that atom (~170 cycles per
-    // block); the epilogue adds about 1.5 cycles per stored element per warp quadrant.  The cheapest
-    // candidate over whole waves of CTAs wins.
+    // Tile shape.  Cost model in nanoseconds per CTA, fitted to measurements on B200 at T = 16384, n = 8192:
+    // one MMA of N tokens takes about 0.45*N + 14 ns, a pipeline stage adds about 150 ns of hand-offs, the
+    // epilogue costs about 2 ns per instruction of one warp (100 per 32 x 32 block + 52 per repetition).
+    // With two accumulator buffers the epilogue hides behind the next tile's main loop except once.
     const int sms = sm_count() > 0 ? sm_count() : 148;
-    struct Cand { int ntok, na; };
-    const Cand cands[] = {{128, 2}, {192, 2}, {256, 1}, {128, 1}, {64, 1}, {32, 1}};
+    struct Cand { int ntok, na, ka, db; };
+    const Cand cands[] = {{256, 1, 2, 1}, {192, 1, 2, 2}, {128, 2, 2, 1}, {128, 1, 2, 2}, {64, 1, 2, 2}, {32, 1, 2, 2}};
     const int n_cands = 6;
     int best = 0;
     double best_cost = 1e300;
     const char *force = getenv("TBN_TC_CONFIG");     // tuning aid: force a candidate by index
+    const double atoms = (double)((a.n + kAtomK - 1) / kAtomK);
     for (int i = 0; i < n_cands; ++i) {
-        const int64_t wt = (p.r + cands[i].na * 128 - 1) / (cands[i].na * 128);
-        const int64_t tt = (a.T + cands[i].ntok - 1) / cands[i].ntok;
+        const Cand &c = cands[i];
+        const int64_t wt = (p.r + c.na * 128 - 1) / (c.na * 128);
+        const int64_t tt = (a.T + c.ntok - 1) / c.ntok;
         const int64_t waves = (wt * tt + sms - 1) / sms;
-        const double atom = cands[i].na * (double)(2 * cands[i].ntok > 170 ? 2 * cands[i].ntok : 170);
-        const double epi = (double)cands[i].na * cands[i].ntok * a.k * 1.5;
-        const double cost = (double)waves * (atom * ((a.n + kAtomK - 1) / kAtomK) + epi);
+        const double stage = c.na * c.ka * 4 * (0.45 * c.ntok + 14.0) + 150.0;
+        const double mainloop = atoms / c.ka * stage;
+        const double epi = c.na * (c.ntok / 32.0) * (100.0 + 52.0 * a.k) * 2.0;
+        const double cost = c.db == 2 ? waves * (mainloop > epi ? mainloop : epi) + epi : waves * (mainloop + epi);
         if (cost < best_cost) { best_cost = cost; best = i; }
     }
     if (force && force[0] >= '0' && force[0] < '0' + n_cands && force[1] == 0) best = force[0] - '0';
     switch (best) {
-    case 0: return launch_config<128, 2, 2, 5>(a, p, device_status, s);
-    case 1: return launch_config<192, 2, 1, 6>(a, p, device_status, s);
-    case 2: return launch_config<256, 1, 2, 3>(a, p, device_status, s);
-    case 3: return launch_config<128, 1, 2, 6>(a, p, device_status, s);
-    case 4: return launch_config<64, 1, 2, 8>(a, p, device_status, s);
-    default: return launch_config<32, 1, 2, 8>(a, p, device_status, s);
+    case 0: return launch_config<256, 1, 2, 3, 1>(a, p, device_status, s);
+    case 1: return launch_config<192, 1, 2, 4, 2>(a, p, device_status, s);
+    case 2: return launch_config<128, 2, 2, 5, 1>(a, p, device_status, s);
+    case 3: return launch_config<128, 1, 2, 6, 2>(a, p, device_status, s);
+    case 4: return launch_config<64, 1, 2, 8, 2>(a, p, device_status, s);
+    default: return launch_config<32, 1, 2, 8, 2>(a, p, device_status, s);
     }
 }
 
