@@ -86,6 +86,25 @@ int tbn_aggregate_tile(const float *W, const float *A, int64_t N, int32_t k, int
                        uint32_t *tile_bits, float *alpha, void *workspace, size_t workspace_bytes,
                        void *stream);
 
+/* Variant of tbn_aggregate_tile for callers that cannot provide scratch memory.  (The paper has no
+ * counterpart: this is a convenience of this library.)  Some callers run where device allocation is not
+ * an option -- inside a latency-critical serving loop that must never hit the allocator, in a plug-in that
+ * is handed its input and output buffers and nothing else, or under a memory manager that forbids
+ * cudaMalloc after start-up.  For them the scratch lives in an array built into the library: 1 MiB per GPU
+ * that loads the library, held until the process exits.  The call allocates nothing and calls no
+ * allocating routine.
+ *   Limit : tbn_aggregate_workspace_bytes(N, k) must not exceed 1 MiB (N up to about 134 million weights);
+ *           larger layers are refused with TBN_ERR_WORKSPACE before anything is launched.
+ *   Set-up: the first call on a device looks up the array's device address.  Make that first call with
+ *           the device current and before any stream capture begins.
+ *   Sharing: every call on a device uses the same array.  The call clears the part that must start at
+ *           zero, so calls that follow one another on a stream are fine; calls that may overlap on the GPU
+ *           (different streams, no ordering between them) race on the array and must be serialised by the
+ *           caller.
+ * Arguments, results and the remaining errors are those of tbn_aggregate_tile without the workspace pair. */
+int tbn_aggregate_tile_static(const float *W, const float *A, int64_t N, int32_t k, int alpha_mode,
+                              uint32_t *tile_bits, float *alpha, void *stream);
+
 /* Pack an existing real-valued tile (Sec. 5.1: tiles are stored one bit per element):
  * src[i] > 0 -> bit 1, else 0.  src: q fp32 values.  tile_bits: tbn_tile_words(q) words. */
 int tbn_pack_tile(const float *src, int64_t q, uint32_t *tile_bits, void *stream);

@@ -31,6 +31,7 @@ SIGNATURES = {
     "tbn_status_string": (ctypes.c_char_p, [c_int]),
     "tbn_aggregate_workspace_bytes": (c_sz, [c_i64, c_i32]),
     "tbn_aggregate_tile": (c_int, [c_vp, c_vp, c_i64, c_i32, c_int, c_vp, c_vp, c_vp, c_sz, c_vp]),
+    "tbn_aggregate_tile_static": (c_int, [c_vp, c_vp, c_i64, c_i32, c_int, c_vp, c_vp, c_vp]),
     "tbn_pack_tile": (c_int, [c_vp, c_i64, c_vp, c_vp]),
     "tbn_expand_tile": (c_int, [c_vp, c_i64, c_i32, c_vp, c_int, c_vp, c_vp]),
     "tbn_linear_workspace_bytes": (c_sz, [c_i64, c_i32, c_i32, c_i32, c_int]),
@@ -125,6 +126,18 @@ def tbn_aggregate_tile(W: torch.Tensor, k: int, alpha_mode: int = ALPHA_PER_TILE
     ws = workspace if workspace is not None else _ws(need, W.device)
     _check(lib().tbn_aggregate_tile(_ptr(W), _ptr(A), N, k, alpha_mode, _ptr(tile), _ptr(alpha), _ptr(ws),
                                     ws.numel(), _stream()), "tbn_aggregate_tile")
+    return tile, alpha
+
+
+def tbn_aggregate_tile_static(W: torch.Tensor, k: int, tile: torch.Tensor, alpha: torch.Tensor,
+                              alpha_mode: int = ALPHA_PER_TILE, A: torch.Tensor | None = None):
+    """Same result as tbn_aggregate_tile, for callers that cannot allocate: the scratch is an array built
+    into the library (1 MiB per GPU), so this wrapper allocates nothing either -- the caller passes the
+    output tensors.  Layers whose scratch need exceeds 1 MiB raise TbnError(-4).  Calls that could overlap
+    on the GPU share the array and must be ordered by the caller; make the first call on a device before
+    any stream capture."""
+    _check(lib().tbn_aggregate_tile_static(_ptr(W), _ptr(A), W.numel(), k, alpha_mode, _ptr(tile), _ptr(alpha),
+                                           _stream()), "tbn_aggregate_tile_static")
     return tile, alpha
 
 

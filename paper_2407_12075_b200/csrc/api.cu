@@ -175,6 +175,20 @@ int tbn_aggregate_tile(const float *W, const float *A, int64_t N, int32_t k, int
     return e == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
 }
 
+int tbn_aggregate_tile_static(const float *W, const float *A, int64_t N, int32_t k, int alpha_mode,
+                              uint32_t *tile_bits, float *alpha, void *stream)
+{
+    if (!W || !tile_bits || !alpha || N <= 0 || k <= 0 || !valid_alpha_mode(alpha_mode))
+        return TBN_ERR_INVALID_ARG;
+    if (N % k != 0) return TBN_ERR_SHAPE;
+    if (!aligned16(W) || (A && !aligned16(A)) || !aligned16(tile_bits)) return TBN_ERR_INVALID_ARG;
+    if (aggregate_workspace_bytes(N, k) > aggregate_static_scratch_capacity())
+        return TBN_ERR_WORKSPACE;           // the layer needs more scratch than the built-in array holds
+    cudaError_t e = launch_aggregate_static(W, A, N, k, alpha_mode == TBN_ALPHA_PER_TILE, tile_bits, alpha,
+                                            static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+}
+
 int tbn_pack_tile(const float *src, int64_t q, uint32_t *tile_bits, void *stream)
 {
     if (!src || !tile_bits || q <= 0) return TBN_ERR_INVALID_ARG;

@@ -52,6 +52,9 @@ struct LayerArgs {
 cudaError_t launch_aggregate(const float *W, const float *A, int64_t N, int32_t k, int per_tile,
                              uint32_t *tile_bits, float *alpha, void *workspace, cudaStream_t s);
 size_t aggregate_workspace_bytes(int64_t N, int32_t k);
+size_t aggregate_static_scratch_capacity();
+cudaError_t launch_aggregate_static(const float *W, const float *A, int64_t N, int32_t k, int per_tile,
+                                    uint32_t *tile_bits, float *alpha, cudaStream_t s);
 cudaError_t launch_pack(const float *src, int64_t q, uint32_t *tile_bits, cudaStream_t s);
 cudaError_t launch_expand(const uint32_t *tile_bits, int64_t N, int32_t k, const float *alpha,
                           int per_tile, float *B_hat, cudaStream_t s);

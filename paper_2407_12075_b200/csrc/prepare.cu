@@ -181,6 +181,34 @@ cudaError_t launch_aggregate(const float *W, const float *A, int64_t N, int32_t 
     return cudaGetLastError();
 }
 
+// ---- built-in scratch for callers that cannot allocate ---------------------------------------------
+// One array per device that loads the library, held until the process exits.  Host code must not hand
+// the symbol itself to a kernel (on the host it is only a stand-in); the device address is looked up
+// once per device with cudaGetSymbolAddress and cached.
+constexpr size_t kStaticScratchBytes = 1u << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+size_t aggregate_static_scratch_capacity() { return kStaticScratchBytes; }
+
+cudaError_t launch_aggregate_static(const float *W, const float *A, int64_t N, int32_t k, int per_tile,
+                                    uint32_t *tile_bits, float *alpha, cudaStream_t s)
+{
+    static void *cache[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!cache[dev]) {                       // set-up: first call on this device, with the device current
+        void *ptr = nullptr;
+        e = cudaGetSymbolAddress((void **)&ptr, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        cache[dev] = ptr;
+    }
+    // launch_aggregate clears the ticket word that must start at zero; the partial sums are written
+    // before they are read, so the previous call's contents do not matter.
+    return launch_aggregate(W, A, N, k, per_tile, tile_bits, alpha, cache[dev], s);
+}
+
 cudaError_t launch_pack(const float *src, int64_t q, uint32_t *tile_bits, cudaStream_t s)
 {
     const int64_t n_words = tbn_tile_words(q);
