@@ -102,6 +102,12 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], bd, %4, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "r"(b_desc_lo), "r"(b_desc_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
+// 256-bit global store: one full 32-byte sector per thread and instruction
+__device__ __forceinline__ void st_global_v8(void *ptr, const uint32_t *v) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(ptr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
+}
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
@@ -447,7 +453,8 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
         const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
         uint32_t *tbuf = ctl->transpose[warp - 6];
         Pipe pd;                                          // accumulator buffer (stage) and its phase
-        const bool vec_ok = (p.m % 8 == 0) && (p.r % 8 == 0);
+        const bool vec_ok = (p.m % 8 == 0) && (p.r % 8 == 0);       // 16-byte aligned rows of 32 features
+        const bool wide_ok = (p.m % 16 == 0) && (p.r % 16 == 0);    // 32-byte aligned: 256-bit stores
         for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
             const int64_t tok0 = (int64_t)(tile / p.w_tiles) * NTOK;
             ok = wait_bar(smem_u32(&ctl->d_full[pd.stage]), pd.phase, abort_flag, p.status, (6 << 24) | (bid & 0xffff));
@@ -489,17 +496,21 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                         const int64_t o0 = (int64_t)j * p.r + row0;
                         const int64_t yi = tok * p.m + o0;
                         if (rows_valid == 32 && vec_ok && plain && p.y_bf16) {
-                            uint4 *dst = reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(p.y) + yi);
+                            uint32_t pk[16];
 #pragma unroll
-                            for (int g = 0; g < 4; ++g) {
-                                uint32_t pk[4];
+                            for (int e = 0; e < 16; ++e) {
+                                const __nv_bfloat162 h = __floats2bfloat162_rn(al * z[2 * e], al * z[2 * e + 1]);
+                                pk[e] = *reinterpret_cast<const uint32_t *>(&h);
+                            }
+                            __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.y) + yi;
+                            if (wide_ok) {          // two full 32-byte sectors per thread
+                                st_global_v8(dst, pk);
+                                st_global_v8(dst + 16, pk + 8);
+                            } else {
 #pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const __nv_bfloat162 h =
-                                        __floats2bfloat162_rn(al * z[g * 8 + 2 * e], al * z[g * 8 + 2 * e + 1]);
-                                    pk[e] = *reinterpret_cast<const uint32_t *>(&h);
-                                }
-                                dst[g] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                                for (int g = 0; g < 4; ++g)
+                                    reinterpret_cast<uint4 *>(dst)[g] =
+                                        make_uint4(pk[4 * g], pk[4 * g + 1], pk[4 * g + 2], pk[4 * g + 3]);
                             }
                         } else {
                             for (int i = 0; i < rows_valid; ++i) {
