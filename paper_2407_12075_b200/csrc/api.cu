@@ -67,7 +67,8 @@ size_t tensor_scratch_bytes(int64_t T, int32_t in_f, int x_dtype)
 int run_layer(LayerArgs a, int path, void *workspace, size_t workspace_bytes, cudaStream_t s)
 {
     if (a.T == 0) return TBN_OK;
-    if (path == TBN_PATH_AUTO) path = a.is_conv ? TBN_PATH_GENERIC : select_linear_path(a);
+    if (path == TBN_PATH_AUTO)
+        path = a.is_conv ? (tensor_conv_supported(a) ? TBN_PATH_TENSOR : TBN_PATH_GENERIC) : select_linear_path(a);
     cudaError_t e = cudaSuccess;
     switch (path) {
     case TBN_PATH_GENERIC:
@@ -78,19 +79,20 @@ int run_layer(LayerArgs a, int path, void *workspace, size_t workspace_bytes, cu
         e = launch_small_batch(a, s);
         break;
     case TBN_PATH_TENSOR: {
-        if (a.is_conv || !tensor_path_supported(a)) return TBN_ERR_UNSUPPORTED;
+        if (a.is_conv ? !tensor_conv_supported(a) : !tensor_path_supported(a)) return TBN_ERR_UNSUPPORTED;
+        const int64_t x_count = a.is_conv ? (int64_t)a.Nb * a.Cin * a.H * a.Wd : a.T * (int64_t)a.n;
         if (a.x_dtype == TBN_F32) {
-            const size_t need = tensor_scratch_bytes(a.T, a.n, a.x_dtype);
+            const size_t need = round_up((size_t)x_count * 2, 256);
             if (!workspace || workspace_bytes < need || !aligned16(workspace)) return TBN_ERR_WORKSPACE;
             e = launch_f32_to_bf16(static_cast<const float *>(a.x), static_cast<__nv_bfloat16 *>(workspace),
-                                   a.T * (int64_t)a.n, s);
+                                   x_count, s);
             if (e != cudaSuccess) return TBN_ERR_CUDA;
             a.x = workspace;
             a.x_dtype = TBN_BF16;
         }
         int *st = device_status_ptr();
         if (!st) return TBN_ERR_CUDA;
-        return launch_tensor_linear(a, st, s);
+        return a.is_conv ? launch_tensor_conv(a, st, s) : launch_tensor_linear(a, st, s);
     }
     default:
         return TBN_ERR_INVALID_ARG;
@@ -284,10 +286,12 @@ int tbn_linear_fwd_host(const void *x_host, int x_dtype, int64_t T, int32_t in_f
     return cudaStreamSynchronize(s) == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
 }
 
-size_t tbn_conv2d_workspace_bytes(int32_t, int32_t, int32_t, int32_t, int32_t, int32_t, int32_t, int32_t,
-                                  int32_t, int32_t, int)
+size_t tbn_conv2d_workspace_bytes(int32_t Nb, int32_t Cin, int32_t H, int32_t Wd, int32_t, int32_t, int32_t,
+                                  int32_t, int32_t, int32_t, int x_dtype)
 {
-    return 0;
+    // the tensor-core path rounds fp32 activations to bf16 first
+    if (x_dtype != TBN_F32 || Nb <= 0 || Cin <= 0 || H <= 0 || Wd <= 0) return 0;
+    return round_up((size_t)Nb * Cin * H * Wd * 2, 256);
 }
 
 int tbn_conv2d_fwd_path(const void *x, int x_dtype, int32_t Nb, int32_t Cin, int32_t H, int32_t Wd,

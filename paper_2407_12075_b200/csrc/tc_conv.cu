@@ -1,0 +1,423 @@
+// Tensor-core forward of a tiled 3x3 convolution on sm_100a (implicit GEMM without im2col duplication).
+//
+// GEMM view: D[channel][position] = sum over (ci, u, v) of W[channel][(ci,u,v)] * X[ci][position shifted by (u,v)].
+// As in the fully-connected kernel the decoded +-1 weights are the tcgen05.mma A operand in tensor memory
+// (UMMA M = 128 output channels) and the activations are the B operand in shared memory (UMMA N = output
+// positions).  What is new is how the B operand is staged.
+//
+// Shifted windows instead of im2col.  For each 16-channel K step the producers copy the input patch of the
+// CTA tile ONCE into shared memory as [8-channel chunk][patch position][8 channels] (16 bytes per position;
+// the un-swizzled K-major UMMA layout with consecutive positions 16 bytes apart).  Because positions are
+// linear with the patch row pitch PW, the operand of filter tap (u,v) is the same buffer read from a start
+// address advanced by (du*PW + dv) positions: nine MMAs per K step read nine shifted views of one staged
+// patch, so shared memory holds each input element once and HBM/L2 traffic is not multiplied by 9.  The MMA
+// N index runs over patch positions, halo columns included; outputs at halo positions are discarded by
+// the epilogue.  For stride 2 the patch is split into its 4 parity planes (row parity, column parity): all
+// inputs of one tap lie in one plane with unit pitch.
+//
+// The weight bits of 16 consecutive input channels and all 9 taps are 144 consecutive tile bits (row-major
+// (Cout, Cin, kh, kw)); the decode warps gather bit ci*9 + tap for each tap into that tap's A block.  The
+// K order inside the kernel is therefore (channel group, tap, channel), which the MMA does not care about.
+//
+// Lanes are output channels (not distinct filters): channel o uses tile row o mod r and alpha[o div r], so
+// the k-fold replication of Sec. 4.1 costs no epilogue work here.  (With r < 128, as in the benchmark's
+// conv layers, the tensor core would idle on the missing lanes anyway.)
+//
+// Warp roles (13 warps): 0-3 patch producers, 4 MMA issuer / TMEM owner, 5-8 tile decode, 9-12 epilogue.
+// Two accumulator buffers: the epilogue of one tile overlaps the main loop of the next.  Every wait is
+// bounded (see tc_common.cuh).
+#include "tc_common.cuh"
+
+namespace tbn {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kConvThreads = 13 * 32;
+constexpr int kTaps = 9;               // 3 x 3
+constexpr int kChanPerStage = 16;      // one UMMA K step per tap and stage
+constexpr int kNMax = 176;             // max positions per tile: 2 x 176 accumulator columns + 2 x 72 weight columns <= 512
+constexpr int kSX = 4;                 // patch stages in shared memory
+constexpr int kACols = kTaps * 8;      // 72 columns per decoded-weight stage
+constexpr int kABase = 2 * kNMax;      // first weight column
+constexpr uint32_t kConvTmemCols = 512;
+
+struct ConvParams {
+    const __nv_bfloat16 *x;
+    void *y;
+    const uint32_t *tile;
+    const float *alpha;
+    const float *bias;
+    int *status;
+    int64_t n_words;
+    int32_t Nb, Cin, H, W, Ho, Wo, m, r, k, n;   // n = Cin * 9
+    int32_t stride, pad;
+    int32_t planes;            // stride * stride
+    int32_t du_min, dv_min;    // smallest plane-row / plane-column offset over the taps
+    int32_t PW;                // patch pitch (positions per patch row) = Wo + column offset range
+    int32_t PHt;               // patch rows per image slot = R + row offset range
+    int32_t R;                 // output rows per image slot
+    int32_t G;                 // image slots per tile (G > 1 only when R == Ho)
+    int32_t bands;             // row bands per image = ceil(Ho / R)
+    int32_t n_pos;             // UMMA N: positions per tile, a multiple of 16, <= kNMax
+    int32_t slot_pos;          // PHt * PW
+    int32_t buf_pos;           // positions held per (plane, chunk) buffer >= n_pos + largest tap offset
+    int32_t tap_plane[kTaps];  // parity plane read by tap t
+    int32_t tap_off[kTaps];    // start offset (positions) of tap t inside its plane
+    int32_t m_blocks, s_tiles; // 128-channel blocks, spatial tiles
+    int32_t k_stages;          // Cin / 16
+    int per_tile, act, y_bf16;
+};
+
+struct ConvControl {
+    uint64_t x_full[kSX], x_empty[kSX];
+    uint64_t a_full[2], a_empty[2];
+    uint64_t d_full[2], d_empty[2];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+__global__ void __launch_bounds__(kConvThreads, 1)
+tc_conv3x3_kernel(const ConvParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    uint8_t *smem = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
+    const uint32_t stage_bytes = (uint32_t)p.planes * 2u * (uint32_t)p.buf_pos * 16u;
+    ConvControl *ctl = reinterpret_cast<ConvControl *>(smem + kSX * stage_bytes);
+    const uint32_t stage0 = smem_u32(smem);
+    volatile int *abort_flag = &ctl->abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int bid = blockIdx.x;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kSX; ++s) { mbar_init(smem_u32(&ctl->x_full[s]), 128); mbar_init(smem_u32(&ctl->x_empty[s]), 1); }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(smem_u32(&ctl->a_full[s]), 128); mbar_init(smem_u32(&ctl->a_empty[s]), 1);
+            mbar_init(smem_u32(&ctl->d_full[s]), 1);   mbar_init(smem_u32(&ctl->d_empty[s]), 128);
+        }
+        ctl->abort_flag = 0;
+        fence_barrier_init();
+        fence_proxy_async();
+    }
+    if (warp == 4) {
+        tmem_alloc(smem_u32(&ctl->tmem_base), kConvTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    const int32_t n_tiles = p.m_blocks * p.s_tiles;
+    bool ok = true;
+
+    if (warp < 4) {
+        // ---------------- patch producers: NCHW global -> [plane][chunk][position][8 channels] ----------------
+        const int tid = threadIdx.x;                       // 0..127
+        const int32_t fill_pos = p.G * p.slot_pos;
+        const int32_t items = p.planes * 2 * fill_pos;
+        const int64_t plane_elems = (int64_t)p.H * p.W;
+        const unsigned short *xs = reinterpret_cast<const unsigned short *>(p.x);
+        Pipe px;
+        for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
+            const int32_t st = tile / p.m_blocks;
+            const int32_t img0 = p.G > 1 ? st * p.G : st / p.bands;
+            const int32_t oh0 = p.G > 1 ? 0 : (st % p.bands) * p.R;
+            for (int32_t ks = 0; ks < p.k_stages && ok; ++ks) {
+                ok = wait_bar(smem_u32(&ctl->x_empty[px.stage]), px.phase ^ 1u, abort_flag, p.status,
+                              (1 << 24) | (px.stage << 16) | (bid & 0xffff));
+                if (!ok) break;
+                uint8_t *stage = smem + px.stage * stage_bytes;
+                for (int32_t id = tid; id < items; id += 128) {
+                    const int32_t pos = id % fill_pos;
+                    const int32_t pc = id / fill_pos;
+                    const int32_t chunk = pc & 1, plane = pc >> 1;
+                    const int32_t g = pos / p.slot_pos;
+                    const int32_t rem = pos - g * p.slot_pos;
+                    const int32_t a_l = rem / p.PW, b_l = rem - a_l * p.PW;
+                    const int32_t py = plane / p.stride, pxx = plane - py * p.stride;
+                    const int32_t ih = p.stride * (oh0 + a_l + p.du_min) + py;
+                    const int32_t iw = p.stride * (b_l + p.dv_min) + pxx;
+                    const int32_t img = img0 + g;
+                    uint32_t v[4] = {0u, 0u, 0u, 0u};
+                    if (img < p.Nb && ih >= 0 && ih < p.H && iw >= 0 && iw < p.W) {
+                        const unsigned short *src =
+                            xs + ((int64_t)img * p.Cin + ks * kChanPerStage + chunk * 8) * plane_elems + (int64_t)ih * p.W + iw;
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const uint32_t lo = __ldg(src + (2 * c) * plane_elems);
+                            const uint32_t hi = __ldg(src + (2 * c + 1) * plane_elems);
+                            v[c] = lo | (hi << 16);
+                        }
+                    }
+                    *reinterpret_cast<uint4 *>(stage + ((size_t)(plane * 2 + chunk) * p.buf_pos + pos) * 16) =
+                        make_uint4(v[0], v[1], v[2], v[3]);
+                }
+                fence_proxy_async();                       // generic-proxy stores -> visible to the tensor core
+                mbar_arrive(smem_u32(&ctl->x_full[px.stage]));
+                px.advance(kSX);
+            }
+        }
+    } else if (warp == 4) {
+        // ---------------- MMA issuer (lane 0): 9 shifted-window MMAs per 16-channel stage ----------------
+        if (lane == 0) {
+            Pipe px, pa, pd;
+            bool ready = false;
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_pos >> 3) << 17) | (8u << 24);
+            // un-swizzled K-major descriptor: stride offset 128 bytes (next 8 positions), leading offset =
+            // distance between the two 8-channel chunks, version 1
+            const uint32_t desc_hi = 8u | (1u << 14);
+            const uint32_t lbo = (uint32_t)p.buf_pos << 16;
+            for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
+                ok = wait_one(smem_u32(&ctl->d_empty[pd.stage]), pd.phase ^ 1u, abort_flag, p.status,
+                              (2 << 24) | (bid & 0xffff));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_addr = tmem_base + pd.stage * kNMax;
+                for (int32_t ks = 0; ks < p.k_stages; ++ks) {
+                    if (!ready) {
+                        ok = wait_one(smem_u32(&ctl->x_full[px.stage]), px.phase, abort_flag, p.status,
+                                      (3 << 24) | (px.stage << 16) | (bid & 0xffff)) &&
+                             wait_one(smem_u32(&ctl->a_full[pa.stage]), pa.phase, abort_flag, p.status,
+                                      (4 << 24) | (pa.stage << 16) | (bid & 0xffff));
+                        if (!ok) break;
+                    }
+                    tc_fence_after();
+                    const uint32_t b_base = ((stage0 + px.stage * stage_bytes) & 0x3FFFFu) >> 4;   // 16-byte units
+                    const uint32_t a_addr = tmem_base + kABase + pa.stage * kACols;
+                    Pipe nx = px, na = pa;
+                    nx.advance(kSX);
+                    na.advance(2);
+#pragma unroll
+                    for (int t = 0; t < kTaps; ++t) {
+                        const uint32_t b_lo = (b_base + (uint32_t)(p.tap_plane[t] * 2 * p.buf_pos + p.tap_off[t])) | lbo;
+                        tc_mma_ts(d_addr, a_addr + t * 8, b_lo, desc_hi, idesc, t > 0 ? 1u : (uint32_t)(ks > 0));
+                        if (t == 4)
+                            ready = mbar_try_wait(smem_u32(&ctl->x_full[nx.stage]), nx.phase) &&
+                                    mbar_try_wait(smem_u32(&ctl->a_full[na.stage]), na.phase);
+                    }
+                    tc_commit(smem_u32(&ctl->x_empty[px.stage]));
+                    tc_commit(smem_u32(&ctl->a_empty[pa.stage]));
+                    if (ks == p.k_stages - 1) tc_commit(smem_u32(&ctl->d_full[pd.stage]));
+                    px = nx;
+                    pa = na;
+                }
+                pd.advance(2);
+            }
+        }
+        __syncwarp();
+    } else if (warp < 9) {
+        // ---------------- tile decode: 144 bits (16 channels x 9 taps) -> nine 128 x 16 A blocks ----------------
+        const int qd = warp & 3;
+        const int L = qd * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
+        const int64_t last_word = p.n_words - 1;
+        Pipe pa;
+        for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
+            const int32_t o = min((tile % p.m_blocks) * 128 + L, p.m - 1);   // channels past the end are never stored
+            const int64_t row_bit = (int64_t)(o % p.r) * p.n;                  // tile row of this channel
+            uint32_t w[6];
+            {
+                const int64_t wi = row_bit >> 5;
+#pragma unroll
+                for (int i = 0; i < 6; ++i) w[i] = __ldg(p.tile + min(wi + i, last_word));
+            }
+            for (int32_t ks = 0; ks < p.k_stages && ok; ++ks) {
+                const int64_t off = row_bit + (int64_t)ks * (kChanPerStage * kTaps);
+                const uint32_t sh = (uint32_t)off & 31u;
+                uint32_t b[5];
+#pragma unroll
+                for (int i = 0; i < 5; ++i) b[i] = __funnelshift_r(w[i], w[i + 1], sh);
+                if (ks + 1 < p.k_stages) {                       // next stage's words, in flight during the decode
+                    const int64_t wi = (off + kChanPerStage * kTaps) >> 5;
+#pragma unroll
+                    for (int i = 0; i < 6; ++i) w[i] = __ldg(p.tile + min(wi + i, last_word));
+                }
+                ok = wait_bar(smem_u32(&ctl->a_empty[pa.stage]), pa.phase ^ 1u, abort_flag, p.status,
+                              (5 << 24) | (pa.stage << 16) | (bid & 0xffff));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_addr = tmem_base + lane_base + kABase + pa.stage * kACols;
+#pragma unroll
+                for (int t = 0; t < kTaps; ++t) {
+                    uint32_t v[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        // channels 2i and 2i+1 of the stage at tap t: bits (2i)*9 + t and (2i+1)*9 + t
+                        const int pe = (2 * i) * kTaps + t, po = pe + kTaps;
+                        const uint32_t be = (b[pe >> 5] >> (pe & 31)) & 1u;
+                        const uint32_t bo = (b[po >> 5] >> (po & 31)) & 1u;
+                        v[i] = ((be << 15) | (bo << 31)) ^ 0xBF80BF80u;       // bit 1 -> +1.0, bit 0 -> -1.0
+                    }
+                    tmem_st_32x8(a_addr + t * 8, v);
+                }
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(smem_u32(&ctl->a_full[pa.stage]));
+                pa.advance(2);
+            }
+        }
+    } else {
+        // ---------------- epilogue: thread = output channel, 32 patch positions per TMEM load ----------------
+        const int qd = warp & 3;
+        const int L = qd * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
+        Pipe pd;
+        const int n_chunks = (p.n_pos + 31) / 32;
+        const int64_t out_plane = (int64_t)p.Ho * p.Wo;
+        for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
+            const int32_t st = tile / p.m_blocks;
+            const int32_t img0 = p.G > 1 ? st * p.G : st / p.bands;
+            const int32_t oh0 = p.G > 1 ? 0 : (st % p.bands) * p.R;
+            const int32_t o = (tile % p.m_blocks) * 128 + L;
+            const bool ch_valid = o < p.m;
+            const float al = ch_valid ? (p.per_tile ? __ldg(p.alpha + o / p.r) : __ldg(p.alpha)) : 0.0f;
+            const float bs = (ch_valid && p.bias) ? __ldg(p.bias + o) : 0.0f;
+            ok = wait_bar(smem_u32(&ctl->d_full[pd.stage]), pd.phase, abort_flag, p.status, (6 << 24) | (bid & 0xffff));
+            if (!ok) break;
+            tc_fence_after();
+            int32_t g = 0, oh = 0, ow = 0;                     // patch coordinates of the next position
+#pragma unroll 1
+            for (int ch = 0; ch < n_chunks; ++ch) {
+                __syncwarp();
+                uint32_t v[32];
+                tmem_ld_32x32(tmem_base + lane_base + pd.stage * kNMax + ch * 32, v);
+                tc_wait_ld();
+                if (ch == n_chunks - 1) {                        // accumulator fully read: hand it back early
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));
+                }
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int32_t img = img0 + g, row = oh0 + oh;
+                    if (ch_valid && g < p.G && img < p.Nb && oh < p.R && row < p.Ho && ow < p.Wo) {
+                        const float val = apply_act(fmaf(al, __uint_as_float(v[i]), bs), p.act);
+                        const int64_t yi = ((int64_t)img * p.m + o) * out_plane + (int64_t)row * p.Wo + ow;
+                        if (p.y_bf16) static_cast<__nv_bfloat16 *>(p.y)[yi] = __float2bfloat16_rn(val);
+                        else static_cast<float *>(p.y)[yi] = val;
+                    }
+                    if (++ow == p.PW) { ow = 0; if (++oh == p.PHt) { oh = 0; ++g; } }
+                }
+            }
+            pd.advance(2);
+        }
+    }
+
+    // ---------------- teardown ----------------
+    if (warp == 4 && *abort_flag) {
+        if (lane == 0) tc_commit(smem_u32(&ctl->x_empty[0]));
+        __syncwarp();
+        drain_wait(smem_u32(&ctl->x_empty[0]), 0);
+        drain_wait(smem_u32(&ctl->x_empty[0]), 1);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kConvTmemCols);
+    }
+}
+
+inline int floor_div(int a, int b) { return (a >= 0) ? a / b : -((-a + b - 1) / b); }
+
+int conv_sm_count()
+{
+    static int cache[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (!cache[dev]) cudaDeviceGetAttribute(&cache[dev], cudaDevAttrMultiProcessorCount, dev);
+    return cache[dev];
+}
+
+// Geometry of the shifted-window staging for one call; false when the shape does not fit this kernel.
+bool plan_conv(const LayerArgs &a, ConvParams &p)
+{
+    if (!a.is_conv || a.kh != 3 || a.kw != 3) return false;
+    if (a.stride != 1 && a.stride != 2) return false;
+    if (a.pad < 0 || a.pad > 2) return false;
+    if (a.q % a.n != 0) return false;                 // the tile must span whole filters
+    if (a.Cin % kChanPerStage != 0) return false;
+    if (a.Nb <= 0 || a.Ho <= 0 || a.Wo <= 0) return false;
+    const int s = a.stride;
+    int du[3], py[3];
+    int dmin = 1 << 30, dmax = -(1 << 30);
+    for (int u = 0; u < 3; ++u) {
+        du[u] = floor_div(u - a.pad, s);
+        py[u] = (u - a.pad) - s * du[u];
+        dmin = du[u] < dmin ? du[u] : dmin;
+        dmax = du[u] > dmax ? du[u] : dmax;
+    }
+    const int range = dmax - dmin;                    // same for rows and columns (square filter, same padding)
+    p.stride = s; p.pad = a.pad; p.planes = s * s;
+    p.du_min = dmin; p.dv_min = dmin;
+    p.PW = a.Wo + range;
+    if (p.PW > kNMax) return false;
+    const int slot_full = (a.Ho + range) * p.PW;
+    if ((a.Ho * p.PW) <= kNMax) {                     // whole images: possibly several per tile
+        p.R = a.Ho;
+        p.PHt = a.Ho + range;
+        p.G = (kNMax - p.R * p.PW) / slot_full + 1;
+        if (p.G > a.Nb) p.G = a.Nb;
+        p.bands = 1;
+    } else {                                          // row bands of one image
+        p.G = 1;
+        int R = kNMax / p.PW;
+        p.bands = (a.Ho + R - 1) / R;
+        p.R = (a.Ho + p.bands - 1) / p.bands;
+        p.PHt = p.R + range;
+    }
+    p.slot_pos = p.PHt * p.PW;
+    const int used = (p.G - 1) * p.slot_pos + p.R * p.PW;
+    p.n_pos = (used + 15) / 16 * 16;
+    if (p.n_pos > kNMax || p.n_pos < 16) return false;
+    const int max_off = range * p.PW + range;
+    int need = p.n_pos + max_off;
+    if (need < p.G * p.slot_pos) need = p.G * p.slot_pos;
+    p.buf_pos = (need + 7) / 8 * 8;
+    for (int u = 0; u < 3; ++u)
+        for (int v = 0; v < 3; ++v) {
+            p.tap_plane[u * 3 + v] = py[u] * s + py[v];
+            p.tap_off[u * 3 + v] = (du[u] - dmin) * p.PW + (du[v] - dmin);
+        }
+    p.s_tiles = p.G > 1 ? (a.Nb + p.G - 1) / p.G : a.Nb * p.bands;
+    p.m_blocks = (a.m + 127) / 128;
+    p.k_stages = a.Cin / kChanPerStage;
+    const size_t smem = (size_t)kSX * p.planes * 2 * p.buf_pos * 16 + sizeof(ConvControl) + 1024;
+    if (smem > 227 * 1024) return false;
+    return true;
+}
+
+}  // namespace
+
+bool tensor_conv_supported(const LayerArgs &a)
+{
+    ConvParams p;
+    return plan_conv(a, p);
+}
+
+int launch_tensor_conv(const LayerArgs &a, int *device_status, cudaStream_t s)
+{
+    if (a.x_dtype != TBN_BF16) return TBN_ERR_UNSUPPORTED;
+    ConvParams p;
+    if (!plan_conv(a, p)) return TBN_ERR_UNSUPPORTED;
+    p.x = static_cast<const __nv_bfloat16 *>(a.x); p.y = a.y; p.tile = a.tile; p.alpha = a.alpha; p.bias = a.bias;
+    p.status = device_status;
+    p.n_words = tbn_tile_words(a.q);
+    p.Nb = a.Nb; p.Cin = a.Cin; p.H = a.H; p.W = a.Wd; p.Ho = a.Ho; p.Wo = a.Wo;
+    p.m = a.m; p.r = (int32_t)(a.q / a.n); p.k = a.k; p.n = a.n;
+    p.per_tile = a.alpha_mode == TBN_ALPHA_PER_TILE; p.act = a.act; p.y_bf16 = a.y_dtype == TBN_BF16;
+    const size_t smem = (size_t)kSX * p.planes * 2 * p.buf_pos * 16 + sizeof(ConvControl) + 1024;
+    if (cudaFuncSetAttribute(tc_conv3x3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return TBN_ERR_CUDA;
+    const int sms = conv_sm_count();
+    if (sms <= 0) return TBN_ERR_CUDA;
+    const int64_t tiles = (int64_t)p.m_blocks * p.s_tiles;
+    const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
+    tc_conv3x3_kernel<<<grid, kConvThreads, smem, s>>>(p);
+    return cudaGetLastError() == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+}
+
+}  // namespace tbn

@@ -91,3 +91,51 @@ def test_mlp_benchmark_config_sampled_rows():
     for W, k, t in zip(c["Ws"], c["ks"], tiles):
         t2, _ = B.tbn_aggregate_tile(to_dev(W), k, B.ALPHA_PER_TILE)
         assert torch.equal(t2, t)
+
+
+# (Nb, Cout, Cin, k, stride, pad, H, W): shapes the tensor-core 3x3 kernel takes
+TENSOR_CONVS = [
+    (2, 128, 64, 4, 1, 1, 32, 32),     # row bands of one image
+    (3, 128, 64, 4, 2, 1, 32, 32),
+    (7, 256, 128, 4, 2, 1, 16, 16),    # two images per tile, odd batch (ragged last group)
+    (5, 32, 16, 2, 1, 1, 4, 4),        # five whole images per tile
+    (2, 200, 32, 4, 1, 1, 12, 20),     # ragged channel block, non-square image
+    (3, 32, 16, 2, 1, 0, 10, 10),      # no padding
+    (3, 32, 16, 2, 2, 0, 11, 13),      # stride 2 without padding
+    (2, 64, 48, 1, 2, 2, 9, 9),        # padding 2, k = 1
+    (1, 16, 16, 16, 1, 1, 40, 170),    # widest row that still fits, one distinct filter
+]
+
+
+@pytest.mark.parametrize("Nb,Cout,Cin,k,stride,pad,H,W", TENSOR_CONVS)
+def test_tensor_conv_matches_oracle(Nb, Cout, Cin, k, stride, pad, H, W):
+    x, Wt = synth.conv_layer(3, Nb, Cin, H, W, Cout, 3, 3)
+    for per_tile in (False, True):
+        words, al = O.prepare(Wt, k, per_tile)
+        ref = O.conv2d(x, words, k, al, per_tile, Cout, Cin, 3, 3, stride, pad, act=O.ACT_RELU)
+        y = B.tbn_conv2d_fwd(to_dev(x), Cout, 3, 3, stride, pad, to_dev(words), k, to_dev(al), int(per_tile),
+                             act=B.ACT_RELU, path=B.PATH_TENSOR)
+        torch.cuda.synchronize()
+        assert_close(to_np64(y), ref, f"tensor conv {Cout}x{Cin} s{stride} p{pad} {H}x{W}")
+    assert B.tbn_last_device_status() == (0, 0)
+
+
+def test_tensor_conv_fp32_bias_and_agrees_with_generic():
+    x, Wt = synth.conv_layer(8, 3, 32, 14, 14, 64, 3, 3, x_bf16=False)
+    bias = synth.normal(8, 200, 64)
+    words, al = O.prepare(Wt, 4, True)
+    ref = O.conv2d(x, words, 4, al, True, 64, 32, 3, 3, 1, 1, bias=bias.astype(np.float64), act=O.ACT_GELU)
+    args = (to_dev(x), 64, 3, 3, 1, 1, to_dev(words), 4, to_dev(al), 1)
+    yt = B.tbn_conv2d_fwd(*args, bias=to_dev(bias), act=B.ACT_GELU, path=B.PATH_TENSOR)
+    yg = B.tbn_conv2d_fwd(*args, bias=to_dev(bias), act=B.ACT_GELU, path=B.PATH_GENERIC)
+    assert yt.dtype == torch.float32
+    assert_close(to_np64(yt), ref, "tensor conv fp32")
+    assert_close(to_np64(yt), to_np64(yg), "tensor conv vs generic")
+
+
+def test_tensor_conv_rejects_what_it_cannot_take():
+    x, Wt = synth.conv_layer(2, 1, 8, 6, 6, 8, 3, 3)          # 8 input channels: not a multiple of 16
+    words, al = O.prepare(Wt, 2, True)
+    with pytest.raises(B.TbnError) as e:
+        B.tbn_conv2d_fwd(to_dev(x), 8, 3, 3, 1, 1, to_dev(words), 2, to_dev(al), 1, path=B.PATH_TENSOR)
+    assert e.value.status == -3
