@@ -93,7 +93,7 @@ int tbn_aggregate_tile(const float *W, const float *A, int64_t N, int32_t k, int
  * cudaMalloc after start-up.  For them the scratch lives in an array built into the library: 1 MiB per GPU
  * that loads the library, held until the process exits.  The call allocates nothing and calls no
  * allocating routine.
- *   Limit : tbn_aggregate_workspace_bytes(N, k) must not exceed 1 MiB (N up to about 134 million weights);
+ *   Limit : tbn_aggregate_workspace_bytes(N, k) must not exceed 1 MiB (N up to about 500 million weights);
  *           larger layers are refused with TBN_ERR_WORKSPACE before anything is launched.
  *   Set-up: the first call on a device looks up the array's device address.  Make that first call with
  *           the device current and before any stream capture begins.

@@ -10,8 +10,10 @@ namespace tbn {
 namespace {
 
 constexpr int kAggThreads = 256;
-constexpr int kAggIter = 4;                               // columns per thread
-constexpr int kAggCols = kAggThreads * kAggIter;          // columns per block (multiple of 32)
+constexpr int kAggVec = 4;                                // columns per 16-byte load
+constexpr int kAggIter = 4;                               // 16-byte loads per thread and tile repetition
+constexpr int kAggCols = kAggThreads * kAggVec * kAggIter;   // columns per block (4096)
+constexpr int kAggJB = 8;                                 // repetitions whose |.| sums are reduced together
 
 struct AggScratch {          // layout of the caller's workspace
     unsigned int ticket;     // blocks that have published their partial sums
@@ -19,17 +21,20 @@ struct AggScratch {          // layout of the caller's workspace
     // followed by k * gridDim.x doubles: partial[j * blocks + b]
 };
 
-// Block b owns columns [b*kAggCols, (b+1)*kAggCols) of the k x q view of W.  For every column it
-// forms s = ((0 + W[0][c]) + W[1][c]) + ... in fp32, one rounding per add, exactly the sequential
-// sum the CPU definition uses, so the sign -- and therefore the bit -- is identical.  Alongside, the
-// block accumulates |S| per tile in fp64 and publishes it; the last block to finish adds the
-// partials of all blocks in a fixed order, which makes alpha reproducible from run to run.
+// Block b owns columns [b*kAggCols, (b+1)*kAggCols) of the k x q view of W; a thread owns kAggIter groups
+// of 4 consecutive columns.  For every column it forms s = ((0 + W[0][c]) + W[1][c]) + ... in fp32, one
+// rounding per add, exactly the sequential sum the CPU definition uses, so the sign -- and therefore the
+// bit -- is identical.  Alongside, the block accumulates |S| per tile in fp64 and publishes it (one
+// block-level reduction per kAggJB repetitions, so up to 32 independent 16-byte loads per thread are in
+// flight between synchronisations); the last block to finish adds the partials of all blocks in a fixed
+// order, which makes alpha reproducible from run to run.  VEC selects 16-byte loads (q % 4 == 0).
+template <bool VEC>
 __global__ void __launch_bounds__(kAggThreads)
 aggregate_kernel(const float *__restrict__ W, const float *__restrict__ A, int64_t q, int32_t k,
                  int per_tile, uint32_t *__restrict__ tile_bits, int64_t n_words,
                  float *__restrict__ alpha, AggScratch *scratch)
 {
-    __shared__ double warp_part[2][kAggThreads / 32];
+    __shared__ double warp_part[kAggJB][kAggThreads / 32];
     __shared__ double red[kAggThreads];
     __shared__ unsigned int s_ticket;
 
@@ -39,42 +44,82 @@ aggregate_kernel(const float *__restrict__ W, const float *__restrict__ A, int64
     double *partial = reinterpret_cast<double *>(scratch + 1);
     const unsigned int blocks = gridDim.x;
 
-    float s[kAggIter];
+    float s[kAggIter][kAggVec];
 #pragma unroll
-    for (int it = 0; it < kAggIter; ++it) s[it] = 0.0f;
+    for (int it = 0; it < kAggIter; ++it)
+#pragma unroll
+        for (int e = 0; e < kAggVec; ++e) s[it][e] = 0.0f;
 
-    for (int32_t j = 0; j < k; ++j) {
-        const int64_t row = (int64_t)j * q;
-        float a_abs = 0.0f;
+    for (int32_t j0 = 0; j0 < k; j0 += kAggJB) {
+        float a_abs[kAggJB];
 #pragma unroll
-        for (int it = 0; it < kAggIter; ++it) {
-            const int64_t c = base + it * kAggThreads + tid;
-            if (c < q) {
-                const float w = __ldg(W + row + c);
-                s[it] = __fadd_rn(s[it], w);             // never fused, never reassociated
-                a_abs += fabsf(A ? __ldg(A + row + c) : w);
+        for (int jj = 0; jj < kAggJB; ++jj) {
+            a_abs[jj] = 0.0f;
+            const int32_t j = j0 + jj;
+            if (j >= k) continue;
+            const int64_t row = (int64_t)j * q;
+#pragma unroll
+            for (int it = 0; it < kAggIter; ++it) {
+                const int64_t c = base + ((int64_t)it * kAggThreads + tid) * kAggVec;
+                float w[kAggVec], av[kAggVec];
+                if (VEC) {
+                    if (c < q) {                       // q % 4 == 0: the whole group is in range
+                        const float4 t = __ldg(reinterpret_cast<const float4 *>(W + row + c));
+                        w[0] = t.x; w[1] = t.y; w[2] = t.z; w[3] = t.w;
+                        if (A) {
+                            const float4 u = __ldg(reinterpret_cast<const float4 *>(A + row + c));
+                            av[0] = u.x; av[1] = u.y; av[2] = u.z; av[3] = u.w;
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < kAggVec; ++e) { w[e] = 0.0f; av[e] = 0.0f; }
+                    }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < kAggVec; ++e) {
+                        const bool in = c + e < q;
+                        w[e] = in ? __ldg(W + row + c + e) : 0.0f;
+                        av[e] = (in && A) ? __ldg(A + row + c + e) : 0.0f;
+                    }
+                }
+#pragma unroll
+                for (int e = 0; e < kAggVec; ++e) {
+                    s[it][e] = __fadd_rn(s[it][e], w[e]);          // never fused, never reassociated
+                    a_abs[jj] += fabsf(A ? av[e] : w[e]);
+                }
             }
         }
-        double d = (double)a_abs;
+        // block-level reduction of the group's |.| sums
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
-        if (lane == 0) warp_part[j & 1][warp] = d;
+        for (int jj = 0; jj < kAggJB; ++jj) {
+            double d = (double)a_abs[jj];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
+            if (lane == 0) warp_part[jj][warp] = d;
+        }
         __syncthreads();
-        if (tid == 0) {
+        if (tid < kAggJB && j0 + tid < k) {
             double t = 0.0;
 #pragma unroll
-            for (int w = 0; w < kAggThreads / 32; ++w) t += warp_part[j & 1][w];
-            partial[(int64_t)j * blocks + blockIdx.x] = t;
+            for (int w = 0; w < kAggThreads / 32; ++w) t += warp_part[tid][w];
+            partial[(int64_t)(j0 + tid) * blocks + blockIdx.x] = t;
         }
+        __syncthreads();
     }
 
-    // Eq. 3 + packing: lane l of a warp holds column (32*g + l); the ballot is the packed word.
+    // Eq. 3 + packing: a thread holds 4 consecutive columns (a nibble), 8 lanes make one 32-bit word.
 #pragma unroll
     for (int it = 0; it < kAggIter; ++it) {
-        const int64_t c0 = base + it * kAggThreads + warp * 32;
-        const uint32_t word = __ballot_sync(0xffffffffu, s[it] > 0.0f);   // NaN and +-0 give 0
+        uint32_t nib = 0;
+#pragma unroll
+        for (int e = 0; e < kAggVec; ++e) nib |= (s[it][e] > 0.0f ? 1u : 0u) << e;   // NaN and +-0 give 0
+        uint32_t word = nib << (4 * (lane & 7));
+        word |= __shfl_xor_sync(0xffffffffu, word, 1);
+        word |= __shfl_xor_sync(0xffffffffu, word, 2);
+        word |= __shfl_xor_sync(0xffffffffu, word, 4);
+        const int64_t c0 = base + ((int64_t)it * kAggThreads + (tid & ~7)) * kAggVec;   // first column of the word
         const int64_t widx = c0 >> 5;
-        if (lane == 0 && widx < n_words) tile_bits[widx] = word;
+        if ((lane & 7) == 0 && widx < n_words) tile_bits[widx] = word;
     }
 
     // Publish, then let the last block reduce.
@@ -176,8 +221,12 @@ cudaError_t launch_aggregate(const float *W, const float *A, int64_t N, int32_t 
     const int64_t blocks = (q + kAggCols - 1) / kAggCols;
     cudaError_t e = cudaMemsetAsync(workspace, 0, sizeof(AggScratch), s);
     if (e != cudaSuccess) return e;
-    aggregate_kernel<<<(unsigned)blocks, kAggThreads, 0, s>>>(
-        W, A, q, k, per_tile, tile_bits, tbn_tile_words(q), alpha, static_cast<AggScratch *>(workspace));
+    if (q % kAggVec == 0)      // every repetition then starts on a 16-byte boundary (W and A are 16-byte aligned)
+        aggregate_kernel<true><<<(unsigned)blocks, kAggThreads, 0, s>>>(
+            W, A, q, k, per_tile, tile_bits, tbn_tile_words(q), alpha, static_cast<AggScratch *>(workspace));
+    else
+        aggregate_kernel<false><<<(unsigned)blocks, kAggThreads, 0, s>>>(
+            W, A, q, k, per_tile, tile_bits, tbn_tile_words(q), alpha, static_cast<AggScratch *>(workspace));
     return cudaGetLastError();
 }
 

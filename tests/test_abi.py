@@ -61,8 +61,8 @@ def test_argument_errors_are_found_on_the_host(lib):
     assert lib.tbn_aggregate_tile(dummy, None, 10, 3, 0, dummy, dummy, dummy, 1 << 20, None) == -2
     assert lib.tbn_aggregate_tile(dummy, None, 12, 3, 0, dummy, dummy, None, 0, None) == -4
     assert lib.tbn_pack_tile(None, 8, dummy, None) == -1
-    # the scratch-free variant refuses layers beyond its built-in 1 MiB array (needs ~N/128 bytes)
-    assert lib.tbn_aggregate_tile_static(dummy, None, 1 << 28, 2, 0, dummy, dummy, None) == -4
+    # the scratch-free variant refuses layers beyond its built-in 1 MiB array (it needs about N/512 bytes)
+    assert lib.tbn_aggregate_tile_static(dummy, None, 1 << 31, 2, 0, dummy, dummy, None) == -4
     assert lib.tbn_aggregate_tile_static(dummy, None, 10, 3, 0, dummy, dummy, None) == -2
     assert lib.tbn_linear_select_path(4, 64, 64, 3, B.BF16) == -2
     conv = [dummy, B.BF16, 1, 3, 8, 8, 4, 3, 3, 1, 1, dummy, 5, dummy, 0, None, 0, dummy, B.BF16, None, 0, None]
