@@ -42,6 +42,8 @@ constexpr int kSX = 4;                 // patch stages in shared memory
 constexpr int kACols = kTaps * 8;      // 72 columns per decoded-weight stage
 constexpr int kABase = 2 * kNMax;      // first weight column
 constexpr uint32_t kConvTmemCols = 512;
+constexpr int kStagePitchWords = 97;   // epilogue staging: 194 bf16 per lane (6 chunks of 32 + 2), odd word pitch
+constexpr int kStageOutBytes = 4 * 32 * kStagePitchWords * 4;   // four epilogue warps
 
 struct ConvParams {
     const __nv_bfloat16 *x;
@@ -77,6 +79,7 @@ struct ConvControl {
     uint32_t tmem_base;
     int abort_flag;
 };
+constexpr int kCtlBytes = (sizeof(ConvControl) + 15) / 16 * 16;
 
 __global__ void __launch_bounds__(kConvThreads, 1)
 tc_conv3x3_kernel(const ConvParams p)
@@ -268,6 +271,11 @@ tc_conv3x3_kernel(const ConvParams p)
         Pipe pd;
         const int n_chunks = (p.n_pos + 31) / 32;
         const int64_t out_plane = (int64_t)p.Ho * p.Wo;
+        // bf16 outputs whose rows are whole 16-byte pieces go through a per-warp staging buffer, so that the
+        // global stores are 16 / 32-byte pieces of a channel's contiguous rows instead of 2-byte scatters
+        const bool staged = p.y_bf16 && (p.Wo % 8 == 0);
+        uint32_t *stg = reinterpret_cast<uint32_t *>(reinterpret_cast<uint8_t *>(ctl) + kCtlBytes) +
+                        (warp - 9) * 32 * kStagePitchWords;
         for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
             const int32_t st = tile / p.m_blocks;
             const int32_t img0 = p.G > 1 ? st * p.G : st / p.bands;
@@ -279,6 +287,61 @@ tc_conv3x3_kernel(const ConvParams p)
             ok = wait_bar(smem_u32(&ctl->d_full[pd.stage]), pd.phase, abort_flag, p.status, (6 << 24) | (bid & 0xffff));
             if (!ok) break;
             tc_fence_after();
+            if (staged) {
+                // (a) accumulator -> alpha / bias / activation -> bf16 -> this lane's row of the staging buffer
+                uint32_t *my = stg + lane * kStagePitchWords;
+#pragma unroll 1
+                for (int ch = 0; ch < n_chunks; ++ch) {
+                    __syncwarp();
+                    uint32_t v[32];
+                    tmem_ld_32x32(tmem_base + lane_base + pd.stage * kNMax + ch * 32, v);
+                    tc_wait_ld();
+                    if (ch == n_chunks - 1) {                    // accumulator fully read: hand it back early
+                        tc_fence_before();
+                        mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));
+                    }
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float v0 = apply_act(fmaf(al, __uint_as_float(v[2 * i]), bs), p.act);
+                        const float v1 = apply_act(fmaf(al, __uint_as_float(v[2 * i + 1]), bs), p.act);
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+                        my[ch * 16 + i] = *reinterpret_cast<const uint32_t *>(&h);
+                    }
+                }
+                // (b) the output rows of a channel are contiguous in y: copy them out in 16 / 32-byte pieces
+                //     (each lane reads back only what it wrote itself, so no synchronisation is needed)
+                if (ch_valid) {
+                    const unsigned short *my16 = reinterpret_cast<const unsigned short *>(my);
+                    const int32_t rows_here = min(p.R, p.Ho - oh0);
+                    const int32_t gran_per_row = p.Wo >> 3;
+                    const int32_t n_gran = rows_here * gran_per_row;
+                    for (int32_t g = 0; g < p.G; ++g) {
+                        const int32_t img = img0 + g;
+                        if (img >= p.Nb) break;
+                        __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.y) +
+                                             ((int64_t)img * p.m + o) * out_plane + (int64_t)oh0 * p.Wo;
+                        const int32_t slot0 = g * p.slot_pos;
+                        int32_t oh = 0, gx = 0;
+                        for (int32_t gi = 0; gi < n_gran;) {
+                            uint32_t pk[8];
+                            const bool two = (gi + 1 < n_gran) && ((((uintptr_t)(dst + gi * 8)) & 31u) == 0);
+                            const int pieces = two ? 2 : 1;
+                            for (int h = 0; h < pieces; ++h) {
+                                const unsigned short *src = my16 + slot0 + oh * p.PW + gx * 8;
+#pragma unroll
+                                for (int e = 0; e < 4; ++e)
+                                    pk[h * 4 + e] = (uint32_t)src[2 * e] | ((uint32_t)src[2 * e + 1] << 16);
+                                if (++gx == gran_per_row) { gx = 0; ++oh; }
+                            }
+                            if (two) st_global_v8(dst + gi * 8, pk);
+                            else *reinterpret_cast<uint4 *>(dst + gi * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                            gi += pieces;
+                        }
+                    }
+                }
+                pd.advance(2);
+                continue;
+            }
             int32_t g = 0, oh = 0, ow = 0;                     // patch coordinates of the next position
 #pragma unroll 1
             for (int ch = 0; ch < n_chunks; ++ch) {
@@ -385,7 +448,7 @@ bool plan_conv(const LayerArgs &a, ConvParams &p)
     p.s_tiles = p.G > 1 ? (a.Nb + p.G - 1) / p.G : a.Nb * p.bands;
     p.m_blocks = (a.m + 127) / 128;
     p.k_stages = a.Cin / kChanPerStage;
-    const size_t smem = (size_t)kSX * p.planes * 2 * p.buf_pos * 16 + sizeof(ConvControl) + 1024;
+    const size_t smem = (size_t)kSX * p.planes * 2 * p.buf_pos * 16 + kCtlBytes + kStageOutBytes + 1024;
     if (smem > 227 * 1024) return false;
     return true;
 }
@@ -409,7 +472,7 @@ int launch_tensor_conv(const LayerArgs &a, int *device_status, cudaStream_t s)
     p.Nb = a.Nb; p.Cin = a.Cin; p.H = a.H; p.W = a.Wd; p.Ho = a.Ho; p.Wo = a.Wo;
     p.m = a.m; p.r = (int32_t)(a.q / a.n); p.k = a.k; p.n = a.n;
     p.per_tile = a.alpha_mode == TBN_ALPHA_PER_TILE; p.act = a.act; p.y_bf16 = a.y_dtype == TBN_BF16;
-    const size_t smem = (size_t)kSX * p.planes * 2 * p.buf_pos * 16 + sizeof(ConvControl) + 1024;
+    const size_t smem = (size_t)kSX * p.planes * 2 * p.buf_pos * 16 + kCtlBytes + kStageOutBytes + 1024;
     if (cudaFuncSetAttribute(tc_conv3x3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return TBN_ERR_CUDA;
     const int sms = conv_sm_count();
