@@ -23,9 +23,12 @@
 // the k-fold replication of Sec. 4.1 costs no epilogue work here.  (With r < 128, as in the benchmark's
 // conv layers, the tensor core would idle on the missing lanes anyway.)
 //
-// Warp roles (13 warps): 0-3 patch producers, 4 MMA issuer / TMEM owner, 5-8 tile decode, 9-12 epilogue.
+// Warp roles (14 warps): 0-3 patch producers, 4 MMA issuer / TMEM owner, 5-8 tile decode, 9-12 epilogue,
+// 13 TMA loader of raw patches.
 // Two accumulator buffers: the epilogue of one tile overlaps the main loop of the next.  Every wait is
 // bounded (see tc_common.cuh).
+#include <cstring>
+
 #include "tc_common.cuh"
 
 namespace tbn {
@@ -34,11 +37,12 @@ namespace {
 
 using namespace tc;
 
-constexpr int kConvThreads = 13 * 32;
+constexpr int kConvThreads = 14 * 32;
 constexpr int kTaps = 9;               // 3 x 3
 constexpr int kChanPerStage = 16;      // one UMMA K step per tap and stage
 constexpr int kNMax = 176;             // max positions per tile: 2 x 176 accumulator columns + 2 x 72 weight columns <= 512
 constexpr int kSX = 4;                 // patch stages in shared memory
+constexpr int kRS = 3;                 // raw (untransposed) patch stages in shared memory
 constexpr int kACols = kTaps * 8;      // 72 columns per decoded-weight stage
 constexpr int kABase = 2 * kNMax;      // first weight column
 constexpr uint32_t kConvTmemCols = 512;
@@ -65,6 +69,9 @@ struct ConvParams {
     int32_t n_pos;             // UMMA N: positions per tile, a multiple of 16, <= kNMax
     int32_t slot_pos;          // PHt * PW
     int32_t buf_pos;           // positions held per (plane, chunk) buffer >= n_pos + largest tap offset
+    int32_t wide;              // 1: W % 8 == 0, raw patches arrive by TMA
+    int32_t raw_rows;          // input rows per image slot and stage = stride * PHt
+    uint32_t raw_slot_bytes, raw_stage_bytes;   // 16 channels x raw_rows x W bf16 (per slot / per stage)
     int32_t tap_plane[kTaps];  // parity plane read by tap t
     int32_t tap_off[kTaps];    // start offset (positions) of tap t inside its plane
     int32_t m_blocks, s_tiles; // 128-channel blocks, spatial tiles
@@ -76,13 +83,14 @@ struct ConvControl {
     uint64_t x_full[kSX], x_empty[kSX];
     uint64_t a_full[2], a_empty[2];
     uint64_t d_full[2], d_empty[2];
+    uint64_t raw_full[kRS], raw_empty[kRS];
     uint32_t tmem_base;
     int abort_flag;
 };
 constexpr int kCtlBytes = (sizeof(ConvControl) + 15) / 16 * 16;
 
 __global__ void __launch_bounds__(kConvThreads, 1)
-tc_conv3x3_kernel(const ConvParams p)
+tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -90,6 +98,7 @@ tc_conv3x3_kernel(const ConvParams p)
     const uint32_t stage_bytes = (uint32_t)p.planes * 2u * (uint32_t)p.buf_pos * 16u;
     ConvControl *ctl = reinterpret_cast<ConvControl *>(smem + kSX * stage_bytes);
     const uint32_t stage0 = smem_u32(smem);
+    const uint32_t raw_off = (kSX * stage_bytes + kCtlBytes + kStageOutBytes + 127u) & ~127u;   // raw ring, 128-byte aligned
     volatile int *abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -101,6 +110,7 @@ tc_conv3x3_kernel(const ConvParams p)
             mbar_init(smem_u32(&ctl->a_full[s]), 128); mbar_init(smem_u32(&ctl->a_empty[s]), 1);
             mbar_init(smem_u32(&ctl->d_full[s]), 1);   mbar_init(smem_u32(&ctl->d_empty[s]), 128);
         }
+        for (int s = 0; s < kRS; ++s) { mbar_init(smem_u32(&ctl->raw_full[s]), 1); mbar_init(smem_u32(&ctl->raw_empty[s]), 128); }
         ctl->abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async();
@@ -118,13 +128,23 @@ tc_conv3x3_kernel(const ConvParams p)
     bool ok = true;
 
     if (warp < 4) {
-        // ---------------- patch producers: NCHW global -> [plane][chunk][position][8 channels] ----------------
+        // ---------------- patch producers: -> [plane][chunk][position][8 channels] ----------------
+        // Wide rows (W % 8 == 0): a TMA warp brings the raw NCHW patch of the stage ([16 channels][rows][W],
+        // rows outside the image and images outside the batch zero-filled) into a shared-memory ring, so HBM
+        // latency is hidden by the ring depth.  These four warps transpose shared memory -> shared memory: a
+        // unit is 8 consecutive pixels of one raw row for 8 channels -- eight 16-byte loads, an 8 x 8
+        // transpose of 16-bit values in registers (byte permutes), eight 16-byte stores.  Patch positions that
+        // no pixel maps to (the zero padding left and right) are zeroed once, before the first stage.
+        // Other widths: gather straight from global memory with 2-byte loads.
         const int tid = threadIdx.x;                       // 0..127
         const int32_t fill_pos = p.G * p.slot_pos;
         const int32_t items = p.planes * 2 * fill_pos;
         const int64_t plane_elems = (int64_t)p.H * p.W;
         const unsigned short *xs = reinterpret_cast<const unsigned short *>(p.x);
-        Pipe px;
+        if (p.wide) {
+            for (uint32_t off = tid * 16u; off < kSX * stage_bytes; off += 128u * 16u) sts_v4(stage0 + off, 0u, 0u, 0u, 0u);
+        }
+        Pipe px, pr;
         for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
             const int32_t st = tile / p.m_blocks;
             const int32_t img0 = p.G > 1 ? st * p.G : st / p.bands;
@@ -134,30 +154,73 @@ tc_conv3x3_kernel(const ConvParams p)
                               (1 << 24) | (px.stage << 16) | (bid & 0xffff));
                 if (!ok) break;
                 uint8_t *stage = smem + px.stage * stage_bytes;
-                for (int32_t id = tid; id < items; id += 128) {
-                    const int32_t pos = id % fill_pos;
-                    const int32_t pc = id / fill_pos;
-                    const int32_t chunk = pc & 1, plane = pc >> 1;
-                    const int32_t g = pos / p.slot_pos;
-                    const int32_t rem = pos - g * p.slot_pos;
-                    const int32_t a_l = rem / p.PW, b_l = rem - a_l * p.PW;
-                    const int32_t py = plane / p.stride, pxx = plane - py * p.stride;
-                    const int32_t ih = p.stride * (oh0 + a_l + p.du_min) + py;
-                    const int32_t iw = p.stride * (b_l + p.dv_min) + pxx;
-                    const int32_t img = img0 + g;
-                    uint32_t v[4] = {0u, 0u, 0u, 0u};
-                    if (img < p.Nb && ih >= 0 && ih < p.H && iw >= 0 && iw < p.W) {
-                        const unsigned short *src =
-                            xs + ((int64_t)img * p.Cin + ks * kChanPerStage + chunk * 8) * plane_elems + (int64_t)ih * p.W + iw;
+                if (p.wide) {
+                    ok = wait_bar(smem_u32(&ctl->raw_full[pr.stage]), pr.phase, abort_flag, p.status,
+                                  (7 << 24) | (pr.stage << 16) | (bid & 0xffff));
+                    if (!ok) break;
+                    const uint32_t raw_addr = stage0 + raw_off + pr.stage * p.raw_stage_bytes;   // shared addresses
+                    const uint32_t stage_addr = stage0 + px.stage * stage_bytes;
+                    const uint32_t ch_bytes = (uint32_t)(p.raw_rows * p.W) * 2u;                 // between channels
+                    const uint32_t chunk_bytes = (uint32_t)p.buf_pos * 16u;                      // between (plane, chunk) buffers
+                    const int32_t gw = p.W >> 3;
+                    const int32_t units = 2 * p.G * gw * p.raw_rows;
+                    for (int32_t u = tid; u < units; u += 128) {
+                        // unit -> (chunk, image slot, pixel group, raw row); the row varies fastest across lanes
+                        const int32_t rr = u % p.raw_rows;
+                        int32_t t = u / p.raw_rows;
+                        const int32_t gx = t % gw;
+                        t /= gw;
+                        const int32_t g = t % p.G, chunk = t / p.G;
+                        const uint32_t src = raw_addr + (uint32_t)(((g * 16 + chunk * 8) * p.raw_rows + rr) * p.W + gx * 8) * 2u;
+                        uint32_t rg[8][4];
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            const uint32_t lo = __ldg(src + (2 * c) * plane_elems);
-                            const uint32_t hi = __ldg(src + (2 * c + 1) * plane_elems);
-                            v[c] = lo | (hi << 16);
+                        for (int c = 0; c < 8; ++c) {
+                            const uint4 q4 = lds_v4(src + c * ch_bytes);
+                            rg[c][0] = q4.x; rg[c][1] = q4.y; rg[c][2] = q4.z; rg[c][3] = q4.w;
+                        }
+                        const int32_t py = rr % p.stride, a_l = rr / p.stride;
+                        const uint32_t row_dst = stage_addr + (uint32_t)chunk * chunk_bytes +
+                                                 (uint32_t)(g * p.slot_pos + a_l * p.PW) * 16u;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            const int32_t iw = gx * 8 + e;
+                            const int32_t pxx = iw % p.stride;
+                            const int32_t b_l = (iw - pxx) / p.stride - p.dv_min;
+                            if (b_l < 0 || b_l >= p.PW) continue;
+                            const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;      // high or low halves of the pixel pair
+                            sts_v4(row_dst + (uint32_t)((py * p.stride + pxx) * 2) * chunk_bytes + (uint32_t)b_l * 16u,
+                                   __byte_perm(rg[0][e >> 1], rg[1][e >> 1], sel), __byte_perm(rg[2][e >> 1], rg[3][e >> 1], sel),
+                                   __byte_perm(rg[4][e >> 1], rg[5][e >> 1], sel), __byte_perm(rg[6][e >> 1], rg[7][e >> 1], sel));
                         }
                     }
-                    *reinterpret_cast<uint4 *>(stage + ((size_t)(plane * 2 + chunk) * p.buf_pos + pos) * 16) =
-                        make_uint4(v[0], v[1], v[2], v[3]);
+                    mbar_arrive(smem_u32(&ctl->raw_empty[pr.stage]));   // raw stage consumed by this thread
+                    pr.advance(kRS);
+                } else {
+                    for (int32_t id = tid; id < items; id += 128) {
+                        const int32_t pos = id % fill_pos;
+                        const int32_t pc = id / fill_pos;
+                        const int32_t chunk = pc & 1, plane = pc >> 1;
+                        const int32_t g = pos / p.slot_pos;
+                        const int32_t rem = pos - g * p.slot_pos;
+                        const int32_t a_l = rem / p.PW, b_l = rem - a_l * p.PW;
+                        const int32_t py = plane / p.stride, pxx = plane - py * p.stride;
+                        const int32_t ih = p.stride * (oh0 + a_l + p.du_min) + py;
+                        const int32_t iw = p.stride * (b_l + p.dv_min) + pxx;
+                        const int32_t img = img0 + g;
+                        uint32_t v[4] = {0u, 0u, 0u, 0u};
+                        if (img < p.Nb && ih >= 0 && ih < p.H && iw >= 0 && iw < p.W) {
+                            const unsigned short *src =
+                                xs + ((int64_t)img * p.Cin + ks * kChanPerStage + chunk * 8) * plane_elems + (int64_t)ih * p.W + iw;
+    #pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                const uint32_t lo = __ldg(src + (2 * c) * plane_elems);
+                                const uint32_t hi = __ldg(src + (2 * c + 1) * plane_elems);
+                                v[c] = lo | (hi << 16);
+                            }
+                        }
+                        *reinterpret_cast<uint4 *>(stage + ((size_t)(plane * 2 + chunk) * p.buf_pos + pos) * 16) =
+                            make_uint4(v[0], v[1], v[2], v[3]);
+                    }
                 }
                 fence_proxy_async();                       // generic-proxy stores -> visible to the tensor core
                 mbar_arrive(smem_u32(&ctl->x_full[px.stage]));
@@ -263,7 +326,7 @@ tc_conv3x3_kernel(const ConvParams p)
                 pa.advance(2);
             }
         }
-    } else {
+    } else if (warp < 13) {
         // ---------------- epilogue: thread = output channel, 32 patch positions per TMEM load ----------------
         const int qd = warp & 3;
         const int L = qd * 32 + lane;
@@ -367,6 +430,38 @@ tc_conv3x3_kernel(const ConvParams p)
             }
             pd.advance(2);
         }
+    } else {
+        // ---------------- TMA loader (warp 13): raw input patches into the shared-memory ring ----------------
+        if (p.wide) {
+            Pipe pr;
+            uint32_t issued_mask = 0, issued_phase = 0;
+            for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
+                const int32_t st = tile / p.m_blocks;
+                const int32_t img0 = p.G > 1 ? st * p.G : st / p.bands;
+                const int32_t oh0 = p.G > 1 ? 0 : (st % p.bands) * p.R;
+                const int32_t ih_lo = p.stride * (oh0 + p.du_min);     // may be negative: those rows are zero-filled
+                for (int32_t ks = 0; ks < p.k_stages && ok; ++ks) {
+                    ok = wait_bar(smem_u32(&ctl->raw_empty[pr.stage]), pr.phase ^ 1u, abort_flag, p.status,
+                                  (8 << 24) | (pr.stage << 16) | (bid & 0xffff));
+                    if (!ok) break;
+                    if (lane == 0) {
+                        const uint32_t bar = smem_u32(&ctl->raw_full[pr.stage]);
+                        mbar_arrive_expect_tx(bar, p.raw_stage_bytes);
+                        for (int32_t g = 0; g < p.G; ++g)                // images past the batch are zero-filled
+                            tma_load_4d(stage0 + raw_off + pr.stage * p.raw_stage_bytes + g * p.raw_slot_bytes, &x_map, 0,
+                                        ih_lo, ks * kChanPerStage, img0 + g, bar);
+                    }
+                    issued_mask |= 1u << pr.stage;
+                    issued_phase = (issued_phase & ~(1u << pr.stage)) | (pr.phase << pr.stage);
+                    __syncwarp();
+                    pr.advance(kRS);
+                }
+            }
+            if (!ok) {   // let copies in flight land before the CTA's shared memory goes away
+                for (int s = 0; s < kRS; ++s)
+                    if (issued_mask & (1u << s)) drain_wait(smem_u32(&ctl->raw_full[s]), (issued_phase >> s) & 1u);
+            }
+        }
     }
 
     // ---------------- teardown ----------------
@@ -382,6 +477,13 @@ tc_conv3x3_kernel(const ConvParams p)
         tc_fence_after();
         tmem_dealloc(tmem_base, kConvTmemCols);
     }
+}
+
+size_t conv_smem_bytes(const ConvParams &p)
+{
+    size_t b = (size_t)kSX * p.planes * 2 * p.buf_pos * 16 + kCtlBytes + kStageOutBytes + 128;
+    if (p.wide) b += (size_t)kRS * p.raw_stage_bytes;
+    return b + 1024;
 }
 
 inline int floor_div(int a, int b) { return (a >= 0) ? a / b : -((-a + b - 1) / b); }
@@ -448,8 +550,12 @@ bool plan_conv(const LayerArgs &a, ConvParams &p)
     p.s_tiles = p.G > 1 ? (a.Nb + p.G - 1) / p.G : a.Nb * p.bands;
     p.m_blocks = (a.m + 127) / 128;
     p.k_stages = a.Cin / kChanPerStage;
-    const size_t smem = (size_t)kSX * p.planes * 2 * p.buf_pos * 16 + kCtlBytes + kStageOutBytes + 1024;
-    if (smem > 227 * 1024) return false;
+    p.raw_rows = s * p.PHt;
+    p.raw_slot_bytes = (uint32_t)(kChanPerStage * p.raw_rows * a.Wd * 2);
+    p.raw_stage_bytes = p.raw_slot_bytes * (uint32_t)p.G;           // a multiple of 256 when W % 8 == 0
+    p.wide = (a.Wd % 8 == 0 && a.Wd <= 256 && p.raw_rows <= 256) ? 1 : 0;
+    if (p.wide && conv_smem_bytes(p) > 227 * 1024) p.wide = 0;      // no room for the raw ring: gather from global
+    if (conv_smem_bytes(p) > 227 * 1024) return false;
     return true;
 }
 
@@ -472,14 +578,30 @@ int launch_tensor_conv(const LayerArgs &a, int *device_status, cudaStream_t s)
     p.Nb = a.Nb; p.Cin = a.Cin; p.H = a.H; p.W = a.Wd; p.Ho = a.Ho; p.Wo = a.Wo;
     p.m = a.m; p.r = (int32_t)(a.q / a.n); p.k = a.k; p.n = a.n;
     p.per_tile = a.alpha_mode == TBN_ALPHA_PER_TILE; p.act = a.act; p.y_bf16 = a.y_dtype == TBN_BF16;
-    const size_t smem = (size_t)kSX * p.planes * 2 * p.buf_pos * 16 + kCtlBytes + kStageOutBytes + 1024;
+    const size_t smem = conv_smem_bytes(p);
     if (cudaFuncSetAttribute(tc_conv3x3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return TBN_ERR_CUDA;
+    // tensor map of x as (W, H, Cin, Nb); one box = all columns x raw_rows rows x 16 channels of one image
+    CUtensorMap map;
+    std::memset(&map, 0, sizeof(map));
+    if (p.wide) {
+        EncodeTiledFn encode = encode_tiled_fn();
+        if (!encode) return TBN_ERR_CUDA;
+        const cuuint64_t dims[4] = {(cuuint64_t)a.Wd, (cuuint64_t)a.H, (cuuint64_t)a.Cin, (cuuint64_t)a.Nb};
+        const cuuint64_t strides[3] = {(cuuint64_t)a.Wd * 2, (cuuint64_t)a.H * a.Wd * 2,
+                                       (cuuint64_t)a.Cin * a.H * a.Wd * 2};
+        const cuuint32_t box[4] = {(cuuint32_t)a.Wd, (cuuint32_t)p.raw_rows, (cuuint32_t)kChanPerStage, 1};
+        const cuuint32_t estr[4] = {1, 1, 1, 1};
+        if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(a.x), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return TBN_ERR_CUDA;
+    }
     const int sms = conv_sm_count();
     if (sms <= 0) return TBN_ERR_CUDA;
     const int64_t tiles = (int64_t)p.m_blocks * p.s_tiles;
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
-    tc_conv3x3_kernel<<<grid, kConvThreads, smem, s>>>(p);
+    tc_conv3x3_kernel<<<grid, kConvThreads, smem, s>>>(map, p);
     return cudaGetLastError() == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
 }
 
