@@ -72,6 +72,7 @@ struct ConvParams {
     int32_t wide;              // 1: W % 8 == 0, raw patches arrive by TMA
     int32_t raw_rows;          // input rows per image slot and stage = stride * PHt
     uint32_t raw_slot_bytes, raw_stage_bytes;   // 16 channels x raw_rows x W bf16 (per slot / per stage)
+    uint32_t magic_rows, magic_gw;   // floor(2^32 / d) + 1 for d = raw_rows, W / 8: x / d == umulhi(x, magic) for small x
     int32_t tap_plane[kTaps];  // parity plane read by tap t
     int32_t tap_off[kTaps];    // start offset (positions) of tap t inside its plane
     int32_t m_blocks, s_tiles; // 128-channel blocks, spatial tiles
@@ -164,13 +165,15 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                     const uint32_t chunk_bytes = (uint32_t)p.buf_pos * 16u;                      // between (plane, chunk) buffers
                     const int32_t gw = p.W >> 3;
                     const int32_t units = 2 * p.G * gw * p.raw_rows;
+                    const int32_t ssh = p.stride - 1;          // stride is 1 or 2: x / stride == x >> ssh, x % stride == x & ssh
                     for (int32_t u = tid; u < units; u += 128) {
                         // unit -> (chunk, image slot, pixel group, raw row); the row varies fastest across lanes
-                        const int32_t rr = u % p.raw_rows;
-                        int32_t t = u / p.raw_rows;
-                        const int32_t gx = t % gw;
-                        t /= gw;
-                        const int32_t g = t % p.G, chunk = t / p.G;
+                        int32_t t = (int32_t)__umulhi((uint32_t)u, p.magic_rows);
+                        const int32_t rr = u - t * p.raw_rows;
+                        const int32_t t2 = gw == 1 ? t : (int32_t)__umulhi((uint32_t)t, p.magic_gw);
+                        const int32_t gx = t - t2 * gw;
+                        const int32_t chunk = t2 >= p.G ? 1 : 0;
+                        const int32_t g = t2 - chunk * p.G;
                         const uint32_t src = raw_addr + (uint32_t)(((g * 16 + chunk * 8) * p.raw_rows + rr) * p.W + gx * 8) * 2u;
                         uint32_t rg[8][4];
 #pragma unroll
@@ -178,17 +181,19 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                             const uint4 q4 = lds_v4(src + c * ch_bytes);
                             rg[c][0] = q4.x; rg[c][1] = q4.y; rg[c][2] = q4.z; rg[c][3] = q4.w;
                         }
-                        const int32_t py = rr % p.stride, a_l = rr / p.stride;
+                        const int32_t py = rr & ssh, a_l = rr >> ssh;
+                        // destination of pixel e: plane (py, iw & ssh), column ((iw >> ssh) - dv_min)
                         const uint32_t row_dst = stage_addr + (uint32_t)chunk * chunk_bytes +
-                                                 (uint32_t)(g * p.slot_pos + a_l * p.PW) * 16u;
+                                                 (uint32_t)(g * p.slot_pos + a_l * p.PW) * 16u +
+                                                 (uint32_t)(py * p.stride * 2) * chunk_bytes;
+                        const int32_t b0 = ((gx * 8) >> ssh) - p.dv_min;     // column of pixel 0 (gx*8 is even)
 #pragma unroll
                         for (int e = 0; e < 8; ++e) {
-                            const int32_t iw = gx * 8 + e;
-                            const int32_t pxx = iw % p.stride;
-                            const int32_t b_l = (iw - pxx) / p.stride - p.dv_min;
+                            const int32_t pxx = e & ssh;
+                            const int32_t b_l = b0 + (e >> ssh);
                             if (b_l < 0 || b_l >= p.PW) continue;
                             const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;      // high or low halves of the pixel pair
-                            sts_v4(row_dst + (uint32_t)((py * p.stride + pxx) * 2) * chunk_bytes + (uint32_t)b_l * 16u,
+                            sts_v4(row_dst + (uint32_t)(pxx * 2) * chunk_bytes + (uint32_t)b_l * 16u,
                                    __byte_perm(rg[0][e >> 1], rg[1][e >> 1], sel), __byte_perm(rg[2][e >> 1], rg[3][e >> 1], sel),
                                    __byte_perm(rg[4][e >> 1], rg[5][e >> 1], sel), __byte_perm(rg[6][e >> 1], rg[7][e >> 1], sel));
                         }
@@ -352,7 +357,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
             tc_fence_after();
             if (staged) {
                 // (a) accumulator -> alpha / bias / activation -> bf16 -> this lane's row of the staging buffer
-                uint32_t *my = stg + lane * kStagePitchWords;
+                const uint32_t my_addr = smem_u32(stg + lane * kStagePitchWords);
 #pragma unroll 1
                 for (int ch = 0; ch < n_chunks; ++ch) {
                     __syncwarp();
@@ -363,18 +368,33 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                         tc_fence_before();
                         mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));
                     }
+                    if (p.act == TBN_ACT_RELU && p.bias == nullptr) {          // the common case: 2 ops per value
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const float v0 = apply_act(fmaf(al, __uint_as_float(v[2 * i]), bs), p.act);
-                        const float v1 = apply_act(fmaf(al, __uint_as_float(v[2 * i + 1]), bs), p.act);
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
-                        my[ch * 16 + i] = *reinterpret_cast<const uint32_t *>(&h);
+                        for (int i = 0; i < 16; ++i) {
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(fmaxf(al * __uint_as_float(v[2 * i]), 0.0f),
+                                                                           fmaxf(al * __uint_as_float(v[2 * i + 1]), 0.0f));
+                            sts_b32(my_addr + (ch * 16 + i) * 4, *reinterpret_cast<const uint32_t *>(&h));
+                        }
+                    } else if (p.act == TBN_ACT_NONE) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(fmaf(al, __uint_as_float(v[2 * i]), bs),
+                                                                           fmaf(al, __uint_as_float(v[2 * i + 1]), bs));
+                            sts_b32(my_addr + (ch * 16 + i) * 4, *reinterpret_cast<const uint32_t *>(&h));
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const float v0 = apply_act(fmaf(al, __uint_as_float(v[2 * i]), bs), p.act);
+                            const float v1 = apply_act(fmaf(al, __uint_as_float(v[2 * i + 1]), bs), p.act);
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+                            sts_b32(my_addr + (ch * 16 + i) * 4, *reinterpret_cast<const uint32_t *>(&h));
+                        }
                     }
                 }
                 // (b) the output rows of a channel are contiguous in y: copy them out in 16 / 32-byte pieces
                 //     (each lane reads back only what it wrote itself, so no synchronisation is needed)
                 if (ch_valid) {
-                    const unsigned short *my16 = reinterpret_cast<const unsigned short *>(my);
                     const int32_t rows_here = min(p.R, p.Ho - oh0);
                     const int32_t gran_per_row = p.Wo >> 3;
                     const int32_t n_gran = rows_here * gran_per_row;
@@ -390,10 +410,10 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                             const bool two = (gi + 1 < n_gran) && ((((uintptr_t)(dst + gi * 8)) & 31u) == 0);
                             const int pieces = two ? 2 : 1;
                             for (int h = 0; h < pieces; ++h) {
-                                const unsigned short *src = my16 + slot0 + oh * p.PW + gx * 8;
+                                const uint32_t src = my_addr + (uint32_t)(slot0 + oh * p.PW + gx * 8) * 2u;
 #pragma unroll
                                 for (int e = 0; e < 4; ++e)
-                                    pk[h * 4 + e] = (uint32_t)src[2 * e] | ((uint32_t)src[2 * e + 1] << 16);
+                                    pk[h * 4 + e] = lds_u16(src + 4 * e) | (lds_u16(src + 4 * e + 2) << 16);
                                 if (++gx == gran_per_row) { gx = 0; ++oh; }
                             }
                             if (two) st_global_v8(dst + gi * 8, pk);
@@ -554,6 +574,8 @@ bool plan_conv(const LayerArgs &a, ConvParams &p)
     p.raw_slot_bytes = (uint32_t)(kChanPerStage * p.raw_rows * a.Wd * 2);
     p.raw_stage_bytes = p.raw_slot_bytes * (uint32_t)p.G;           // a multiple of 256 when W % 8 == 0
     p.wide = (a.Wd % 8 == 0 && a.Wd <= 256 && p.raw_rows <= 256) ? 1 : 0;
+    p.magic_rows = (uint32_t)(0x100000000ull / (uint32_t)p.raw_rows) + 1u;
+    p.magic_gw = (a.Wd >= 16) ? (uint32_t)(0x100000000ull / (uint32_t)(a.Wd / 8)) + 1u : 0u;   // W / 8 == 1 needs no division
     if (p.wide && conv_smem_bytes(p) > 227 * 1024) p.wide = 0;      // no room for the raw ring: gather from global
     if (conv_smem_bytes(p) > 227 * 1024) return false;
     return true;
