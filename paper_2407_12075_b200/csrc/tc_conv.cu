@@ -46,8 +46,7 @@ constexpr int kRS = 3;                 // raw (untransposed) patch stages in sha
 constexpr int kACols = kTaps * 8;      // 72 columns per decoded-weight stage
 constexpr int kABase = 2 * kNMax;      // first weight column
 constexpr uint32_t kConvTmemCols = 512;
-constexpr int kStagePitchWords = 97;   // epilogue staging: 194 bf16 per lane (6 chunks of 32 + 2), odd word pitch
-constexpr int kStageOutBytes = 4 * 32 * kStagePitchWords * 4;   // four epilogue warps
+constexpr int kStageOutBytes = 0;       // (no epilogue staging in shared memory)
 
 struct ConvParams {
     const __nv_bfloat16 *x;
@@ -339,11 +338,8 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
         Pipe pd;
         const int n_chunks = (p.n_pos + 31) / 32;
         const int64_t out_plane = (int64_t)p.Ho * p.Wo;
-        // bf16 outputs whose rows are whole 16-byte pieces go through a per-warp staging buffer, so that the
-        // global stores are 16 / 32-byte pieces of a channel's contiguous rows instead of 2-byte scatters
-        const bool staged = p.y_bf16 && (p.Wo % 8 == 0);
-        uint32_t *stg = reinterpret_cast<uint32_t *>(reinterpret_cast<uint8_t *>(ctl) + kCtlBytes) +
-                        (warp - 9) * 32 * kStagePitchWords;
+        // bf16 outputs whose rows are whole 16-byte pieces are stored straight from the accumulator rows
+        const bool rows_direct = p.y_bf16 && (p.Wo % 8 == 0);
         for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
             const int32_t st = tile / p.m_blocks;
             const int32_t img0 = p.G > 1 ? st * p.G : st / p.bands;
@@ -355,73 +351,54 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
             ok = wait_bar(smem_u32(&ctl->d_full[pd.stage]), pd.phase, abort_flag, p.status, (6 << 24) | (bid & 0xffff));
             if (!ok) break;
             tc_fence_after();
-            if (staged) {
-                // (a) accumulator -> alpha / bias / activation -> bf16 -> this lane's row of the staging buffer
-                const uint32_t my_addr = smem_u32(stg + lane * kStagePitchWords);
-#pragma unroll 1
-                for (int ch = 0; ch < n_chunks; ++ch) {
-                    __syncwarp();
-                    uint32_t v[32];
-                    tmem_ld_32x32(tmem_base + lane_base + pd.stage * kNMax + ch * 32, v);
-                    tc_wait_ld();
-                    if (ch == n_chunks - 1) {                    // accumulator fully read: hand it back early
-                        tc_fence_before();
-                        mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));
-                    }
-                    if (p.act == TBN_ACT_RELU && p.bias == nullptr) {          // the common case: 2 ops per value
+            if (rows_direct) {
+                // One TMEM load per output row piece: 8 consecutive accumulator columns starting at the row's first
+                // position are 8 consecutive output pixels of this thread's channel -> one 16-byte store (two
+                // pieces that share a 32-byte sector go out as one 32-byte store).  All loops are warp-uniform.
+                const int32_t rows_here = min(p.R, p.Ho - oh0);
+                const int32_t pieces = p.Wo >> 3;
+                for (int32_t g = 0; g < p.G && img0 + g < p.Nb; ++g) {
+                    __nv_bfloat16 *img_dst = static_cast<__nv_bfloat16 *>(p.y) +
+                                             ((int64_t)(img0 + g) * p.m + (ch_valid ? o : 0)) * out_plane + (int64_t)oh0 * p.Wo;
+                    for (int32_t oh = 0; oh < rows_here; ++oh) {
+                        const uint32_t col0 = tmem_base + lane_base + pd.stage * kNMax + g * p.slot_pos + oh * p.PW;
+                        __nv_bfloat16 *row_dst = img_dst + oh * p.Wo;
+                        for (int32_t pc = 0; pc < pieces; pc += 2) {
+                            uint32_t v[16];
+                            const bool two = pc + 1 < pieces;
+                            __syncwarp();
+                            if (two) {
+                                tmem_ld_32x16(col0 + pc * 8, v);
+                            } else {
+                                uint32_t v8[8];
+                                tmem_ld_32x8(col0 + pc * 8, v8);
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const __nv_bfloat162 h = __floats2bfloat162_rn(fmaxf(al * __uint_as_float(v[2 * i]), 0.0f),
-                                                                           fmaxf(al * __uint_as_float(v[2 * i + 1]), 0.0f));
-                            sts_b32(my_addr + (ch * 16 + i) * 4, *reinterpret_cast<const uint32_t *>(&h));
-                        }
-                    } else if (p.act == TBN_ACT_NONE) {
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const __nv_bfloat162 h = __floats2bfloat162_rn(fmaf(al, __uint_as_float(v[2 * i]), bs),
-                                                                           fmaf(al, __uint_as_float(v[2 * i + 1]), bs));
-                            sts_b32(my_addr + (ch * 16 + i) * 4, *reinterpret_cast<const uint32_t *>(&h));
-                        }
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const float v0 = apply_act(fmaf(al, __uint_as_float(v[2 * i]), bs), p.act);
-                            const float v1 = apply_act(fmaf(al, __uint_as_float(v[2 * i + 1]), bs), p.act);
-                            const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
-                            sts_b32(my_addr + (ch * 16 + i) * 4, *reinterpret_cast<const uint32_t *>(&h));
-                        }
-                    }
-                }
-                // (b) the output rows of a channel are contiguous in y: copy them out in 16 / 32-byte pieces
-                //     (each lane reads back only what it wrote itself, so no synchronisation is needed)
-                if (ch_valid) {
-                    const int32_t rows_here = min(p.R, p.Ho - oh0);
-                    const int32_t gran_per_row = p.Wo >> 3;
-                    const int32_t n_gran = rows_here * gran_per_row;
-                    for (int32_t g = 0; g < p.G; ++g) {
-                        const int32_t img = img0 + g;
-                        if (img >= p.Nb) break;
-                        __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.y) +
-                                             ((int64_t)img * p.m + o) * out_plane + (int64_t)oh0 * p.Wo;
-                        const int32_t slot0 = g * p.slot_pos;
-                        int32_t oh = 0, gx = 0;
-                        for (int32_t gi = 0; gi < n_gran;) {
-                            uint32_t pk[8];
-                            const bool two = (gi + 1 < n_gran) && ((((uintptr_t)(dst + gi * 8)) & 31u) == 0);
-                            const int pieces = two ? 2 : 1;
-                            for (int h = 0; h < pieces; ++h) {
-                                const uint32_t src = my_addr + (uint32_t)(slot0 + oh * p.PW + gx * 8) * 2u;
-#pragma unroll
-                                for (int e = 0; e < 4; ++e)
-                                    pk[h * 4 + e] = lds_u16(src + 4 * e) | (lds_u16(src + 4 * e + 2) << 16);
-                                if (++gx == gran_per_row) { gx = 0; ++oh; }
+                                for (int i = 0; i < 8; ++i) { v[i] = v8[i]; v[i + 8] = 0u; }
                             }
-                            if (two) st_global_v8(dst + gi * 8, pk);
-                            else *reinterpret_cast<uint4 *>(dst + gi * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                            gi += pieces;
+                            tc_wait_ld();
+                            uint32_t pk[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                float v0 = fmaf(al, __uint_as_float(v[2 * i]), bs), v1 = fmaf(al, __uint_as_float(v[2 * i + 1]), bs);
+                                if (p.act == TBN_ACT_RELU) { v0 = fmaxf(v0, 0.0f); v1 = fmaxf(v1, 0.0f); }
+                                else if (p.act == TBN_ACT_GELU) { v0 = apply_act(v0, TBN_ACT_GELU); v1 = apply_act(v1, TBN_ACT_GELU); }
+                                const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+                                pk[i] = *reinterpret_cast<const uint32_t *>(&h);
+                            }
+                            if (ch_valid) {
+                                __nv_bfloat16 *dst = row_dst + pc * 8;
+                                if (two && (((uintptr_t)dst) & 31u) == 0) {
+                                    st_global_v8(dst, pk);
+                                } else {
+                                    *reinterpret_cast<uint4 *>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                                    if (two) *reinterpret_cast<uint4 *>(dst + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                                }
+                            }
                         }
                     }
                 }
+                tc_fence_before();
+                mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));      // accumulator fully read
                 pd.advance(2);
                 continue;
             }
