@@ -23,8 +23,8 @@
 // the k-fold replication of Sec. 4.1 costs no epilogue work here.  (With r < 128, as in the benchmark's
 // conv layers, the tensor core would idle on the missing lanes anyway.)
 //
-// Warp roles (14 warps): 0-3 patch producers, 4 MMA issuer / TMEM owner, 5-8 tile decode, 9-12 epilogue,
-// 13 TMA loader of raw patches.
+// Warp roles (16 warps): 0-5 patch producers, 6 MMA issuer / TMEM owner, 7-10 tile decode, 11-14 epilogue,
+// 15 TMA loader of raw patches.
 // Two accumulator buffers: the epilogue of one tile overlaps the main loop of the next.  Every wait is
 // bounded (see tc_common.cuh).
 #include <cstring>
@@ -37,7 +37,10 @@ namespace {
 
 using namespace tc;
 
-constexpr int kConvThreads = 14 * 32;
+constexpr int kProdWarps = 6;           // patch producers
+constexpr int kProdThreads = kProdWarps * 32;
+constexpr int kMmaWarp = kProdWarps;    // then 4 decode warps, 4 epilogue warps, 1 TMA warp
+constexpr int kConvThreads = (kProdWarps + 10) * 32;
 constexpr int kTaps = 9;               // 3 x 3
 constexpr int kChanPerStage = 16;      // one UMMA K step per tap and stage
 constexpr int kNMax = 176;             // max positions per tile: 2 x 176 accumulator columns + 2 x 72 weight columns <= 512
@@ -105,17 +108,17 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
     const int bid = blockIdx.x;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kSX; ++s) { mbar_init(smem_u32(&ctl->x_full[s]), 128); mbar_init(smem_u32(&ctl->x_empty[s]), 1); }
+        for (int s = 0; s < kSX; ++s) { mbar_init(smem_u32(&ctl->x_full[s]), kProdThreads); mbar_init(smem_u32(&ctl->x_empty[s]), 1); }
         for (int s = 0; s < 2; ++s) {
             mbar_init(smem_u32(&ctl->a_full[s]), 128); mbar_init(smem_u32(&ctl->a_empty[s]), 1);
             mbar_init(smem_u32(&ctl->d_full[s]), 1);   mbar_init(smem_u32(&ctl->d_empty[s]), 128);
         }
-        for (int s = 0; s < kRS; ++s) { mbar_init(smem_u32(&ctl->raw_full[s]), 1); mbar_init(smem_u32(&ctl->raw_empty[s]), 128); }
+        for (int s = 0; s < kRS; ++s) { mbar_init(smem_u32(&ctl->raw_full[s]), 1); mbar_init(smem_u32(&ctl->raw_empty[s]), kProdThreads); }
         ctl->abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async();
     }
-    if (warp == 4) {
+    if (warp == kMmaWarp) {
         tmem_alloc(smem_u32(&ctl->tmem_base), kConvTmemCols);
         tmem_relinquish();
     }
@@ -127,7 +130,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
     const int32_t n_tiles = p.m_blocks * p.s_tiles;
     bool ok = true;
 
-    if (warp < 4) {
+    if (warp < kProdWarps) {
         // ---------------- patch producers: -> [plane][chunk][position][8 channels] ----------------
         // Wide rows (W % 8 == 0): a TMA warp brings the raw NCHW patch of the stage ([16 channels][rows][W],
         // rows outside the image and images outside the batch zero-filled) into a shared-memory ring, so HBM
@@ -136,13 +139,13 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
         // transpose of 16-bit values in registers (byte permutes), eight 16-byte stores.  Patch positions that
         // no pixel maps to (the zero padding left and right) are zeroed once, before the first stage.
         // Other widths: gather straight from global memory with 2-byte loads.
-        const int tid = threadIdx.x;                       // 0..127
+        const int tid = threadIdx.x;                       // 0..kProdThreads-1
         const int32_t fill_pos = p.G * p.slot_pos;
         const int32_t items = p.planes * 2 * fill_pos;
         const int64_t plane_elems = (int64_t)p.H * p.W;
         const unsigned short *xs = reinterpret_cast<const unsigned short *>(p.x);
         if (p.wide) {
-            for (uint32_t off = tid * 16u; off < kSX * stage_bytes; off += 128u * 16u) sts_v4(stage0 + off, 0u, 0u, 0u, 0u);
+            for (uint32_t off = tid * 16u; off < kSX * stage_bytes; off += kProdThreads * 16u) sts_v4(stage0 + off, 0u, 0u, 0u, 0u);
         }
         Pipe px, pr;
         for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
@@ -165,7 +168,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                     const int32_t gw = p.W >> 3;
                     const int32_t units = 2 * p.G * gw * p.raw_rows;
                     const int32_t ssh = p.stride - 1;          // stride is 1 or 2: x / stride == x >> ssh, x % stride == x & ssh
-                    for (int32_t u = tid; u < units; u += 128) {
+                    for (int32_t u = tid; u < units; u += kProdThreads) {
                         // unit -> (chunk, image slot, pixel group, raw row); the row varies fastest across lanes
                         int32_t t = (int32_t)__umulhi((uint32_t)u, p.magic_rows);
                         const int32_t rr = u - t * p.raw_rows;
@@ -200,7 +203,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                     mbar_arrive(smem_u32(&ctl->raw_empty[pr.stage]));   // raw stage consumed by this thread
                     pr.advance(kRS);
                 } else {
-                    for (int32_t id = tid; id < items; id += 128) {
+                    for (int32_t id = tid; id < items; id += kProdThreads) {
                         const int32_t pos = id % fill_pos;
                         const int32_t pc = id / fill_pos;
                         const int32_t chunk = pc & 1, plane = pc >> 1;
@@ -231,7 +234,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                 px.advance(kSX);
             }
         }
-    } else if (warp == 4) {
+    } else if (warp == kMmaWarp) {
         // ---------------- MMA issuer (lane 0): 9 shifted-window MMAs per 16-channel stage ----------------
         if (lane == 0) {
             Pipe px, pa, pd;
@@ -279,7 +282,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
             }
         }
         __syncwarp();
-    } else if (warp < 9) {
+    } else if (warp < kMmaWarp + 5) {
         // ---------------- tile decode: 144 bits (16 channels x 9 taps) -> nine 128 x 16 A blocks ----------------
         const int qd = warp & 3;
         const int L = qd * 32 + lane;
@@ -330,7 +333,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                 pa.advance(2);
             }
         }
-    } else if (warp < 13) {
+    } else if (warp < kMmaWarp + 9) {
         // ---------------- epilogue: thread = output channel, 32 patch positions per TMEM load ----------------
         const int qd = warp & 3;
         const int L = qd * 32 + lane;
@@ -428,7 +431,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
             pd.advance(2);
         }
     } else {
-        // ---------------- TMA loader (warp 13): raw input patches into the shared-memory ring ----------------
+        // ---------------- TMA loader (last warp): raw input patches into the shared-memory ring ----------------
         if (p.wide) {
             Pipe pr;
             uint32_t issued_mask = 0, issued_phase = 0;
@@ -462,7 +465,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
     }
 
     // ---------------- teardown ----------------
-    if (warp == 4 && *abort_flag) {
+    if (warp == kMmaWarp && *abort_flag) {
         if (lane == 0) tc_commit(smem_u32(&ctl->x_empty[0]));
         __syncwarp();
         drain_wait(smem_u32(&ctl->x_empty[0]), 0);
@@ -470,7 +473,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == kMmaWarp) {
         tc_fence_after();
         tmem_dealloc(tmem_base, kConvTmemCols);
     }
