@@ -169,11 +169,12 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                     const int32_t units = 2 * p.G * gw * p.raw_rows;
                     const int32_t ssh = p.stride - 1;          // stride is 1 or 2: x / stride == x >> ssh, x % stride == x & ssh
                     for (int32_t u = tid; u < units; u += kProdThreads) {
-                        // unit -> (chunk, image slot, pixel group, raw row); the row varies fastest across lanes
-                        int32_t t = (int32_t)__umulhi((uint32_t)u, p.magic_rows);
-                        const int32_t rr = u - t * p.raw_rows;
-                        const int32_t t2 = gw == 1 ? t : (int32_t)__umulhi((uint32_t)t, p.magic_gw);
-                        const int32_t gx = t - t2 * gw;
+                        // unit -> (chunk, image slot, raw row, pixel group); the pixel group varies fastest across
+                        // lanes, so a warp reads 512 contiguous bytes of the raw patch per load (no bank conflicts)
+                        int32_t t = gw == 1 ? u : (int32_t)__umulhi((uint32_t)u, p.magic_gw);
+                        const int32_t gx = u - t * gw;
+                        const int32_t t2 = (int32_t)__umulhi((uint32_t)t, p.magic_rows);
+                        const int32_t rr = t - t2 * p.raw_rows;
                         const int32_t chunk = t2 >= p.G ? 1 : 0;
                         const int32_t g = t2 - chunk * p.G;
                         const uint32_t src = raw_addr + (uint32_t)(((g * 16 + chunk * 8) * p.raw_rows + rr) * p.W + gx * 8) * 2u;
@@ -244,6 +245,9 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
             // distance between the two 8-channel chunks, version 1
             const uint32_t desc_hi = 8u | (1u << 14);
             const uint32_t lbo = (uint32_t)p.buf_pos << 16;
+            uint32_t tap_disp[kTaps];                   // start of tap t's window inside a stage, in 16-byte units
+#pragma unroll
+            for (int t = 0; t < kTaps; ++t) tap_disp[t] = (uint32_t)(p.tap_plane[t] * 2 * p.buf_pos + p.tap_off[t]);
             for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
                 ok = wait_one(smem_u32(&ctl->d_empty[pd.stage]), pd.phase ^ 1u, abort_flag, p.status,
                               (2 << 24) | (bid & 0xffff));
@@ -266,7 +270,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                     na.advance(2);
 #pragma unroll
                     for (int t = 0; t < kTaps; ++t) {
-                        const uint32_t b_lo = (b_base + (uint32_t)(p.tap_plane[t] * 2 * p.buf_pos + p.tap_off[t])) | lbo;
+                        const uint32_t b_lo = (b_base + tap_disp[t]) | lbo;
                         tc_mma_ts(d_addr, a_addr + t * 8, b_lo, desc_hi, idesc, t > 0 ? 1u : (uint32_t)(ks > 0));
                         if (t == 4)
                             ready = mbar_try_wait(smem_u32(&ctl->x_full[nx.stage]), nx.phase) &&
@@ -541,7 +545,8 @@ bool plan_conv(const LayerArgs &a, ConvParams &p)
     const int max_off = range * p.PW + range;
     int need = p.n_pos + max_off;
     if (need < p.G * p.slot_pos) need = p.G * p.slot_pos;
-    p.buf_pos = (need + 7) / 8 * 8;
+    p.buf_pos = (need + 7) / 8 * 8 + 2;     // = 2 mod 8: the (plane, chunk) buffers start 32 bytes apart modulo 128,
+                                            // which spreads the producers' 16-byte stores over the banks
     for (int u = 0; u < 3; ++u)
         for (int v = 0; v < 3; ++v) {
             p.tap_plane[u * 3 + v] = py[u] * s + py[v];
