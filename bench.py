@@ -154,6 +154,7 @@ def main():
     ap.add_argument("--tokens", type=int, default=16384, help="development override of the batch size")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true")
     ap.add_argument("--ks", default="", help="development override: comma-separated subset of k values")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -172,6 +173,86 @@ def main():
 
     run_ours(args, rank, world, local_rank)
 
+
+
+def measure_other_configs(B, torch, dev, peaks):
+    """Device-time measurements of the other benchmark configurations (context for the headline line):
+    the small single layer, the 3-layer MLP, the tiled 3x3 convolutions, the ViT-B block's four tiled
+    linears and the small-batch end of the large linear sweep.  Inputs are seeded device-side normals /
+    uniforms of the configured shapes (timing does not depend on the values; parity on the seeded inputs
+    of each configuration is covered by the test-suite).  Each entry is the mean over CUDA-graph replays, so
+    the host's launch latency is excluded; 'l2' says whether the operands stay L2-resident between replays."""
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(1234)
+    hbm = peaks["hbm_gbs"] * 1e9
+    tens = peaks["bf16_tflops_sustained"] * 1e12
+
+    def graph_us(fn, reps=10, iters=5):
+        fn()
+        torch.cuda.synchronize()
+        stream = torch.cuda.Stream()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            fn()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g, stream=stream):
+            for _ in range(reps):
+                fn()
+        g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / (iters * reps)
+
+    def rand_tile(q):
+        return torch.randint(-2 ** 31, 2 ** 31 - 1, (B.tbn_tile_words(q),), device=dev, dtype=torch.int32, generator=gen)
+
+    def linear_entry(T, n, m, k, x_dtype=torch.bfloat16, act=B.ACT_NONE):
+        x = torch.randn(T, n, device=dev, generator=gen).to(x_dtype)
+        y = torch.empty(T, m, device=dev, dtype=x_dtype)
+        tile, alpha = rand_tile(n * m // k), torch.rand(k, device=dev, generator=gen) * 0.02
+        xd = B.BF16 if x_dtype == torch.bfloat16 else B.F32
+        ws = torch.empty(max(B.tbn_linear_workspace_bytes(T, n, m, k, xd), 16), dtype=torch.uint8, device=dev)
+        us = graph_us(lambda: B.tbn_linear_fwd(x, m, tile, k, alpha, B.ALPHA_PER_TILE, act=act, y=y, workspace=ws))
+        r = m // k
+        flops, nbytes = 2.0 * T * r * n, (T * n + T * m) * x.element_size() + n * m // k / 8 + 4 * k
+        bound_us = max(flops / tens, nbytes / hbm) * 1e6
+        return dict(us=us, path=B.tbn_linear_select_path(T, n, m, k, xd), alg_tflops=flops / us / 1e6,
+                    alg_gbs=nbytes / us / 1e3, bound="tensor" if flops / tens > nbytes / hbm else "hbm",
+                    frac_of_binding_roofline=bound_us / us, l2="resident" if nbytes < 100e6 else "exceeds L2")
+
+    out = {}
+    out["single_fc_512x512_k4_T64_f32"] = linear_entry(64, 512, 512, 4, torch.float32)
+    T, dims, ks = 4096, [1024, 2048, 2048, 10], [8, 8, 1]
+    x = torch.randn(T, dims[0], device=dev, generator=gen).to(torch.bfloat16)
+    tiles = [rand_tile(dims[l] * dims[l + 1] // ks[l]) for l in range(3)]
+    alphas = [torch.rand(ks[l], device=dev, generator=gen) * 0.02 for l in range(3)]
+    ws = torch.empty(B.tbn_mlp_workspace_bytes(T, dims, ks, B.BF16), dtype=torch.uint8, device=dev)
+    y = torch.empty(T, dims[-1], device=dev, dtype=torch.bfloat16)
+    us = graph_us(lambda: B.tbn_mlp_fwd(x, dims, tiles, ks, alphas, [1, 1, 1], workspace=ws, y=y))
+    out["mlp_1024_2048_2048_10_T4096"] = dict(us=us, samples_per_s=T / us * 1e6, variant="unfused chain, bf16 hidden in HBM",
+                                              bound_us_unfused_hbm=75.7e6 / hbm * 1e6)
+    for name, (Cin, H, Cout, stride) in {"conv_64_128_s2_32x32": (64, 32, 128, 2), "conv_128_256_s2_16x16": (128, 16, 256, 2),
+                                         "conv_64_128_s1_32x32": (64, 32, 128, 1)}.items():
+        xc = torch.rand(256, Cin, H, H, device=dev, generator=gen).to(torch.bfloat16)
+        tile, alpha = rand_tile(Cout * Cin * 9 // 4), torch.rand(4, device=dev, generator=gen) * 0.05
+        us = graph_us(lambda: B.tbn_conv2d_fwd(xc, Cout, 3, 3, stride, 1, tile, 4, alpha, B.ALPHA_PER_TILE, act=B.ACT_RELU),
+                      reps=3, iters=3)
+        Ho = (H + 2 - 3) // stride + 1
+        nbytes = xc.numel() * 2 + 256 * Cout * Ho * Ho * 2
+        out[name] = dict(us=us, alg_gbs=nbytes / us / 1e3, images_per_s=256 / us * 1e6, bound="hbm",
+                         frac_of_binding_roofline=nbytes / hbm * 1e6 / us)
+    for name, (n, m) in {"vit_qkv_768_2304": (768, 2304), "vit_out_768_768": (768, 768), "vit_fc1_768_3072": (768, 3072),
+                         "vit_fc2_3072_768": (3072, 768)}.items():
+        out[name] = linear_entry(25216, n, m, 8)
+    for T in (1, 16, 256, 4096):
+        for k in (2, 16):
+            out[f"large_linear_T{T}_k{k}"] = linear_entry(T, N_FEAT, N_FEAT, k)
+    return out
 
 
 def run_ours(args, rank: int, world: int, local_rank: int):
@@ -303,6 +384,11 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                           f"dense fp64 product ({2.0 * n * N_FEAT * N_FEAT / dt / 1e9:.2f} dense GFLOP/s), value "
                           f"counts algorithmic flops")
 
+    others = None
+    if rank == 0 and world == 1 and not args.no_other_configs:
+        xh = yh = hws = None
+        others = measure_other_configs(B, torch, dev, peaks)
+
     if rank == 0:
         line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                     ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
@@ -311,7 +397,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                                 step="one forward per k (4 launches)", l2="inputs larger than L2 (x and y 268 MB each)",
                                 multi_gpu="replicas only (no exchange step in the path)"),
                     clocks=clocks, e2e=e2e, gpu_launches=args.steps * len(KS), roofline=roofline,
-                    cpu_baseline=cpu, per_k=per_k)
+                    cpu_baseline=cpu, per_k=per_k, other_configs=others)
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
