@@ -91,9 +91,14 @@ int run_layer(LayerArgs a, int path, void *workspace, size_t workspace_bytes, cu
     case TBN_PATH_TENSOR: {
         if (a.is_conv ? !tensor_conv_supported(a) : !tensor_path_supported(a)) return TBN_ERR_UNSUPPORTED;
         const int64_t x_count = a.is_conv ? (int64_t)a.Nb * a.Cin * a.H * a.Wd : a.T * (int64_t)a.n;
+        // workspace layout: [bf16 copy of fp32 activations][split-K scratch of the linear kernel]
+        char *rest = static_cast<char *>(workspace);
+        size_t rest_bytes = workspace ? workspace_bytes : 0;
         if (a.x_dtype == TBN_F32) {
             const size_t need = round_up((size_t)x_count * 2, 256);
             if (!workspace || workspace_bytes < need || !aligned16(workspace)) return TBN_ERR_WORKSPACE;
+            rest += need;
+            rest_bytes -= need;
             e = launch_f32_to_bf16(static_cast<const float *>(a.x), static_cast<__nv_bfloat16 *>(workspace),
                                    x_count, s);
             if (e != cudaSuccess) return TBN_ERR_CUDA;
@@ -102,7 +107,8 @@ int run_layer(LayerArgs a, int path, void *workspace, size_t workspace_bytes, cu
         }
         int *st = device_status_ptr();
         if (!st) return TBN_ERR_CUDA;
-        return a.is_conv ? launch_tensor_conv(a, st, s) : launch_tensor_linear(a, st, s);
+        if (rest_bytes == 0 || !aligned16(rest)) { rest = nullptr; rest_bytes = 0; }
+        return a.is_conv ? launch_tensor_conv(a, st, s) : launch_tensor_linear(a, st, rest, rest_bytes, s);
     }
     default:
         return TBN_ERR_INVALID_ARG;
@@ -222,9 +228,13 @@ int tbn_expand_tile(const uint32_t *tile_bits, int64_t N, int32_t k, const float
 
 size_t tbn_linear_workspace_bytes(int64_t T, int32_t in_f, int32_t out_f, int32_t k, int x_dtype)
 {
-    (void)out_f; (void)k;
-    if (T <= 0 || in_f <= 0) return 0;
-    return tensor_scratch_bytes(T, in_f, x_dtype);
+    if (T <= 0 || in_f <= 0 || out_f <= 0 || k <= 0 || ((int64_t)in_f * out_f) % k != 0) return 0;
+    LayerArgs a;
+    std::memset(&a, 0, sizeof(a));
+    a.T = T; a.n = in_f; a.m = out_f; a.k = k; a.q = (int64_t)in_f * out_f / k;
+    a.x_dtype = TBN_BF16; a.y_dtype = TBN_BF16;
+    // bf16 copy of fp32 activations + the tensor-core kernel's split-K scratch (partial tiles and counters)
+    return tensor_scratch_bytes(T, in_f, x_dtype) + round_up(tensor_linear_scratch_bytes(a), 256);
 }
 
 int tbn_linear_select_path(int64_t T, int32_t in_f, int32_t out_f, int32_t k, int x_dtype)
@@ -350,7 +360,12 @@ size_t tbn_mlp_workspace_bytes(int64_t T, int32_t L, const int32_t *dims, const 
     int32_t widest = 0;
     for (int32_t l = 1; l < L; ++l) widest = dims[l] > widest ? dims[l] : widest;
     const size_t hidden = round_up((size_t)T * widest * 2, 256);
-    return 2 * hidden + tbn_linear_workspace_bytes(T, dims[0], dims[1], ks[0], x_dtype);
+    size_t scratch = 0;
+    for (int32_t l = 0; l < L; ++l) {
+        const size_t b = tbn_linear_workspace_bytes(T, dims[l], dims[l + 1], ks[l], l == 0 ? x_dtype : TBN_BF16);
+        scratch = b > scratch ? b : scratch;
+    }
+    return 2 * hidden + scratch;
 }
 
 int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t *dims,
@@ -381,7 +396,7 @@ int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t 
         void *out = last ? y : buf[l & 1];
         rc = tbn_linear_fwd(cur, cur_dtype, T, dims[l], dims[l + 1], tiles[l], ks[l], alphas[l],
                             alpha_modes[l], nullptr, last ? TBN_ACT_NONE : hidden_act, out,
-                            last ? y_dtype : TBN_BF16, scratch, l == 0 ? scratch_bytes : 0, stream);
+                            last ? y_dtype : TBN_BF16, scratch, scratch_bytes, stream);
         if (rc != TBN_OK) return rc;
         cur = out;
         cur_dtype = TBN_BF16;

@@ -67,7 +67,8 @@ cudaError_t launch_small_batch(const LayerArgs &a, cudaStream_t s);
 
 // The tensor-core path reports through a tbn_status because it also uses the driver API.
 bool tensor_path_supported(const LayerArgs &a);
-int launch_tensor_linear(const LayerArgs &a, int *device_status, cudaStream_t s);
+size_t tensor_linear_scratch_bytes(const LayerArgs &a);   // split-K partial tiles + arrival counters
+int launch_tensor_linear(const LayerArgs &a, int *device_status, void *scratch, size_t scratch_bytes, cudaStream_t s);
 bool tensor_conv_supported(const LayerArgs &a);
 int launch_tensor_conv(const LayerArgs &a, int *device_status, cudaStream_t s);
 

@@ -70,6 +70,9 @@ struct TcParams {
     int32_t n, m, r, k;
     int32_t k_stages;    // ceil(n / 64)
     int32_t w_tiles, t_tiles;
+    int32_t splits;      // split-K factor: CTAs that share one output tile, each walking 1/splits of the contraction
+    float *partial;      // splits > 1: fp32 partial tiles [out tile][split][NA][128 rows][NTOK tokens]
+    unsigned int *tickets;   // splits > 1: arrival counters [out tile][4 lane quadrants], zeroed before the launch
     int per_tile, act, y_bf16;
 };
 
@@ -128,7 +131,9 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
-    const int32_t n_tiles = p.w_tiles * p.t_tiles;
+    // A tile index enumerates (token tile, row block, K split) with the split fastest, so the CTAs that share an
+    // output tile run at the same time.  Split s walks stages [s*k_stages/S, (s+1)*k_stages/S).
+    const int32_t n_tiles = p.w_tiles * p.t_tiles * p.splits;
     bool ok = true;
 
     if (warp == 0) {
@@ -136,8 +141,11 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
         Pipe px;
         uint32_t issued_mask = 0, issued_phase = 0;
         for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
-            const int32_t tok0 = (tile / p.w_tiles) * NTOK;
-            for (int32_t ks = 0; ks < p.k_stages && ok; ++ks) {
+            const int32_t split = tile % p.splits, out_tile = tile / p.splits;
+            const int32_t tok0 = (out_tile / p.w_tiles) * NTOK;
+            const int32_t ks0 = (int32_t)((int64_t)split * p.k_stages / p.splits);
+            const int32_t ks1 = (int32_t)((int64_t)(split + 1) * p.k_stages / p.splits);
+            for (int32_t ks = ks0; ks < ks1 && ok; ++ks) {
                 ok = wait_bar(smem_u32(&ctl->x_empty[px.stage]), px.phase ^ 1u, abort_flag, p.status,
                               (1 << 24) | (px.stage << 16) | (bid & 0xffff));
                 if (!ok) break;
@@ -178,7 +186,10 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_addr = tmem_base + pd.stage * kDCols;
-                for (int32_t ks = 0; ks < p.k_stages; ++ks) {
+                const int32_t split = tile % p.splits;
+                const int32_t ks0 = (int32_t)((int64_t)split * p.k_stages / p.splits);
+                const int32_t ks1 = (int32_t)((int64_t)(split + 1) * p.k_stages / p.splits);
+                for (int32_t ks = ks0; ks < ks1; ++ks) {
                     if (!ready) {
                         ok = wait_one(smem_u32(&ctl->x_full[px.stage]), px.phase, abort_flag, p.status,
                                       (3 << 24) | (px.stage << 16) | (bid & 0xffff)) &&
@@ -202,7 +213,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                             for (int a = 0; a < NA; ++a)
                                 tc_mma_ts(d_addr + a * NTOK, a_addr + (a * KA + at) * 32 + kk * 8,
                                           b_lo + at * (kAtomBytes >> 4) + kk * 2, kDescHi, kIdesc,
-                                          st > 0 ? 1u : (uint32_t)(ks > 0));
+                                          st > 0 ? 1u : (uint32_t)(ks > ks0));
                             if (st == kSteps / 2 - 1)
                                 ready = mbar_try_wait(smem_u32(&ctl->x_full[nx.stage]), nx.phase) &&
                                         mbar_try_wait(smem_u32(&ctl->a_full[na.stage]), na.phase);
@@ -215,13 +226,13 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                             for (int a = 0; a < NA; ++a)
                                 tc_mma_ts(d_addr + a * NTOK, a_addr + (a * KA + at) * 32 + kk * 8,
                                           b_lo + at * (kAtomBytes >> 4) + kk * 2, kDescHi, kIdesc,
-                                          (ks > 0 || st > 0) ? 1u : 0u);
+                                          (ks > ks0 || st > 0) ? 1u : 0u);
                         }
                         ready = false;
                     }
                     tc_commit(smem_u32(&ctl->x_empty[px.stage]));
                     tc_commit(smem_u32(&ctl->a_empty[pa.stage]));
-                    if (ks == p.k_stages - 1) tc_commit(smem_u32(&ctl->d_full[pd.stage]));
+                    if (ks == ks1 - 1) tc_commit(smem_u32(&ctl->d_full[pd.stage]));
                     px = nx;
                     pa = na;
                 }
@@ -241,18 +252,21 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
         const int64_t last_word = p.n_words - 1;
         Pipe pa;
         for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
-            const int32_t row_base = (tile % p.w_tiles) * (NA * 128) + L;
+            const int32_t split = tile % p.splits, out_tile = tile / p.splits;
+            const int32_t ks0 = (int32_t)((int64_t)split * p.k_stages / p.splits);
+            const int32_t ks1 = (int32_t)((int64_t)(split + 1) * p.k_stages / p.splits);
+            const int32_t row_base = (out_tile % p.w_tiles) * (NA * 128) + L;
             int64_t bitoff[NA];
             uint32_t w[NA][kW + 1];
 #pragma unroll
             for (int a = 0; a < NA; ++a) {
                 const int32_t row = min(row_base + a * 128, p.r - 1);   // rows past the end are never stored
                 bitoff[a] = (int64_t)row * p.n;
-                const int64_t wi = bitoff[a] >> 5;
+                const int64_t wi = (bitoff[a] + (int64_t)ks0 * kStageK) >> 5;
 #pragma unroll
                 for (int i = 0; i <= kW; ++i) w[a][i] = __ldg(p.tile + min(wi + i, last_word));
             }
-            for (int32_t ks = 0; ks < p.k_stages && ok; ++ks) {
+            for (int32_t ks = ks0; ks < ks1 && ok; ++ks) {
                 uint32_t b[NA][kW];
 #pragma unroll
                 for (int a = 0; a < NA; ++a) {
@@ -260,7 +274,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
 #pragma unroll
                     for (int i = 0; i < kW; ++i) b[a][i] = __funnelshift_r(w[a][i], w[a][i + 1], sh);
                     w[a][0] = w[a][kW];
-                    if (ks + 1 < p.k_stages) {
+                    if (ks + 1 < ks1) {
                         const int64_t wi = (bitoff[a] + (int64_t)(ks + 1) * kStageK) >> 5;
 #pragma unroll
                         for (int i = 1; i <= kW; ++i) w[a][i] = __ldg(p.tile + min(wi + i, last_word));
@@ -298,24 +312,76 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
         const bool vec_ok = (p.m % 8 == 0) && (p.r % 8 == 0);       // 16-byte aligned rows of 32 features
         const bool wide_ok = (p.m % 16 == 0) && (p.r % 16 == 0);    // 32-byte aligned: 256-bit stores
         for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
-            const int64_t tok0 = (int64_t)(tile / p.w_tiles) * NTOK;
+            const int32_t split = tile % p.splits, out_tile = tile / p.splits;
+            const int64_t tok0 = (int64_t)(out_tile / p.w_tiles) * NTOK;
             ok = wait_bar(smem_u32(&ctl->d_full[pd.stage]), pd.phase, abort_flag, p.status, (6 << 24) | (bid & 0xffff));
             if (!ok) break;
             tc_fence_after();
             const int n_chunks = (int)min((int64_t)(NTOK / 32), (p.T - tok0 + 31) / 32);
+            // fp32 partial tile of (out_tile, split): [NA][128 rows][NTOK tokens]; this thread owns one row per block
+            float *part_row = nullptr;
+            if (p.splits > 1) {
+                constexpr int64_t kTileFloats = (int64_t)NA * 128 * NTOK;
+                part_row = p.partial + ((int64_t)out_tile * p.splits + split) * kTileFloats + (int64_t)(qd * 32 + lane) * NTOK;
+                // pass 1: dump this CTA's partial sums (128 contiguous bytes per thread and chunk)
+#pragma unroll 1
+                for (int a = 0; a < NA; ++a) {
+#pragma unroll 1
+                    for (int ch = 0; ch < n_chunks; ++ch) {
+                        __syncwarp();
+                        uint32_t v[32];
+                        tmem_ld_32x32(tmem_base + lane_base + pd.stage * kDCols + a * NTOK + ch * 32, v);
+                        tc_wait_ld();
+                        uint4 *dst = reinterpret_cast<uint4 *>(part_row + (int64_t)a * 128 * NTOK + ch * 32);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) __stcg(dst + i, make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]));
+                    }
+                }
+                tc_fence_before();
+                mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));           // accumulator fully read
+                // the warp that arrives last for this (output tile, lane quadrant) adds the partials and stores
+                __threadfence();
+                __syncwarp();
+                unsigned int old = 0;
+                if (lane == 0) old = atomicAdd(p.tickets + (int64_t)out_tile * 4 + qd, 1u);
+                old = __shfl_sync(0xffffffffu, old, 0);
+                if (old != (unsigned int)(p.splits - 1)) { pd.advance(DB); continue; }
+                __threadfence();
+                part_row -= (int64_t)split * kTileFloats;                  // row of split 0
+            }
 #pragma unroll 1
             for (int a = 0; a < NA; ++a) {
-                const int32_t row0 = (tile % p.w_tiles) * (NA * 128) + a * 128 + qd * 32;
+                const int32_t row0 = (out_tile % p.w_tiles) * (NA * 128) + a * 128 + qd * 32;
                 const int rows_valid = max(0, min(32, p.r - row0));
 #pragma unroll 1
                 for (int ch = 0; ch < n_chunks; ++ch) {
                     __syncwarp();                                 // reconverge before the warp-wide TMEM load
                     uint32_t v[32];
-                    tmem_ld_32x32(tmem_base + lane_base + pd.stage * kDCols + a * NTOK + ch * 32, v);
-                    tc_wait_ld();
-                    if (a == NA - 1 && ch == n_chunks - 1) {      // accumulator fully read: hand it back early
-                        tc_fence_before();
-                        mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));
+                    if (p.splits > 1) {
+                        // sum of the splits in a fixed order (split 0, 1, ...): the result does not depend on
+                        // which CTA arrived last
+                        constexpr int64_t kTileFloats = (int64_t)NA * 128 * NTOK;
+                        float acc[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
+                        for (int32_t sp = 0; sp < p.splits; ++sp) {
+                            const float4 *src = reinterpret_cast<const float4 *>(part_row + (int64_t)sp * kTileFloats +
+                                                                                 (int64_t)a * 128 * NTOK + ch * 32);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                const float4 q4 = __ldcg(src + i);
+                                acc[4 * i] += q4.x; acc[4 * i + 1] += q4.y; acc[4 * i + 2] += q4.z; acc[4 * i + 3] += q4.w;
+                            }
+                        }
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(acc[i]);
+                    } else {
+                        tmem_ld_32x32(tmem_base + lane_base + pd.stage * kDCols + a * NTOK + ch * 32, v);
+                        tc_wait_ld();
+                        if (a == NA - 1 && ch == n_chunks - 1) {  // accumulator fully read: hand it back early
+                            tc_fence_before();
+                            mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));
+                        }
                     }
 #pragma unroll
                     for (int i = 0; i < 32; ++i) tbuf[i * 33 + lane] = v[i];
@@ -398,7 +464,7 @@ int sm_count()
 }
 
 template <int NTOK, int NA, int KA, int SX, int DB>
-int launch_config(const LayerArgs &a, TcParams p, int *device_status, cudaStream_t s)
+int launch_config(const LayerArgs &a, TcParams p, int splits, void *scratch, cudaStream_t s)
 {
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return TBN_ERR_CUDA;
@@ -415,17 +481,76 @@ int launch_config(const LayerArgs &a, TcParams p, int *device_status, cudaStream
     p.w_tiles = (p.r + NA * 128 - 1) / (NA * 128);
     p.t_tiles = (int32_t)((a.T + NTOK - 1) / NTOK);
     p.k_stages = (a.n + KA * kAtomK - 1) / (KA * kAtomK);
-    p.status = device_status;
+    p.splits = splits;
+    const int64_t out_tiles = (int64_t)p.w_tiles * p.t_tiles;
+    if (splits > 1) {
+        // scratch: [tickets: out_tiles x 4 counters, padded to 256 bytes][partials]
+        const size_t ticket_bytes = ((size_t)out_tiles * 4 * sizeof(unsigned int) + 255) / 256 * 256;
+        p.tickets = static_cast<unsigned int *>(scratch);
+        p.partial = reinterpret_cast<float *>(static_cast<char *>(scratch) + ticket_bytes);
+        if (cudaMemsetAsync(scratch, 0, ticket_bytes, s) != cudaSuccess) return TBN_ERR_CUDA;
+    } else {
+        p.tickets = nullptr;
+        p.partial = nullptr;
+    }
     const size_t smem = (size_t)SX * KA * NTOK * 128 + sizeof(Control<SX>) + 1024;
     auto kern = tc_linear_kernel<NTOK, NA, KA, SX, DB>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return TBN_ERR_CUDA;
     const int sms = sm_count();
     if (sms <= 0) return TBN_ERR_CUDA;
-    const int64_t tiles = (int64_t)p.w_tiles * p.t_tiles;
+    const int64_t tiles = out_tiles * splits;
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
     kern<<<grid, kThreads, smem, s>>>(map, p);
     return cudaGetLastError() == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+}
+
+// Tile shape and split-K factor for one call.  Cost model in nanoseconds per CTA, fitted to measurements on
+// B200 (T = 16384, n = 8192): one MMA of N tokens takes about 0.45*N + 14 ns, a pipeline stage adds about 150 ns
+// of hand-offs, the epilogue costs about 2 ns per instruction of one warp (100 per 32 x 32 block + 52 per
+// repetition).  With two accumulator buffers the epilogue hides behind the next tile's main loop except once.
+// When the output has fewer tiles than the GPU has SMs, the contraction is split over several CTAs per tile
+// (each dumps an fp32 partial tile; the last to arrive adds them in a fixed order and stores).
+struct Cand { int ntok, na, ka, db; };
+constexpr Cand kCands[] = {{256, 1, 2, 1}, {192, 1, 2, 2}, {128, 2, 2, 1}, {128, 1, 2, 2}, {64, 1, 2, 2}, {32, 1, 2, 2}};
+constexpr int kNumCands = 6;
+
+struct Plan { int cand, splits; size_t scratch_bytes; };
+
+Plan plan_linear(const LayerArgs &a)
+{
+    const int sms = sm_count() > 0 ? sm_count() : 148;
+    const int32_t r = (int32_t)(a.q / a.n);
+    const double atoms = (double)((a.n + kAtomK - 1) / kAtomK);
+    Plan best = {0, 1, 0};
+    double best_cost = 1e300;
+    for (int i = 0; i < kNumCands; ++i) {
+        const Cand &c = kCands[i];
+        const int64_t wt = (r + c.na * 128 - 1) / (c.na * 128);
+        const int64_t tt = (a.T + c.ntok - 1) / c.ntok;
+        const int64_t out_tiles = wt * tt;
+        const int k_stages = (a.n + c.ka * kAtomK - 1) / (c.ka * kAtomK);
+        const double stage = c.na * c.ka * 4 * (0.45 * c.ntok + 14.0) + 150.0;
+        const double epi = c.na * (c.ntok / 32.0) * (100.0 + 52.0 * a.k) * 2.0;
+        const double dump = c.na * (c.ntok / 32.0) * 60.0 * 2.0;
+        for (int sp = 1; sp <= 16; sp *= 2) {
+            if (sp > 1 && (k_stages < 2 * sp || out_tiles * sp > sms)) break;   // >= 2 stages per split, one wave
+            const int64_t waves = (out_tiles * sp + sms - 1) / sms;
+            const double mainloop = atoms / c.ka / sp * stage;
+            double cost;
+            if (sp == 1) cost = c.db == 2 ? waves * (mainloop > epi ? mainloop : epi) + epi : waves * (mainloop + epi);
+            else cost = mainloop + dump + epi + 1500.0;                         // + ticket / partial round trip
+            if (cost < best_cost) {
+                best_cost = cost;
+                best.cand = i;
+                best.splits = sp;
+                best.scratch_bytes = sp == 1 ? 0
+                    : ((size_t)out_tiles * 4 * sizeof(unsigned int) + 255) / 256 * 256 +
+                      (size_t)out_tiles * sp * c.na * 128 * c.ntok * sizeof(float);
+            }
+        }
+    }
+    return best;
 }
 
 }  // namespace
@@ -439,7 +564,12 @@ bool tensor_path_supported(const LayerArgs &a)
     return true;
 }
 
-int launch_tensor_linear(const LayerArgs &a, int *device_status, cudaStream_t s)
+size_t tensor_linear_scratch_bytes(const LayerArgs &a)
+{
+    return tensor_path_supported(a) ? plan_linear(a).scratch_bytes : 0;
+}
+
+int launch_tensor_linear(const LayerArgs &a, int *device_status, void *scratch, size_t scratch_bytes, cudaStream_t s)
 {
     if (a.x_dtype != TBN_BF16) return TBN_ERR_UNSUPPORTED;
     TcParams p;
@@ -447,40 +577,32 @@ int launch_tensor_linear(const LayerArgs &a, int *device_status, cudaStream_t s)
     p.T = a.T; p.n_words = tbn_tile_words(a.q);
     p.n = a.n; p.m = a.m; p.r = (int32_t)(a.q / a.n); p.k = a.k;
     p.k_stages = 0;
-    p.w_tiles = 0; p.t_tiles = 0;
+    p.w_tiles = 0; p.t_tiles = 0; p.splits = 1; p.partial = nullptr; p.tickets = nullptr;
     p.per_tile = a.alpha_mode == TBN_ALPHA_PER_TILE; p.act = a.act; p.y_bf16 = a.y_dtype == TBN_BF16;
 
-    // Tile shape.  Cost model in nanoseconds per CTA, fitted to measurements on B200 at T = 16384, n = 8192:
-    // one MMA of N tokens takes about 0.45*N + 14 ns, a pipeline stage adds about 150 ns of hand-offs, the
-    // epilogue costs about 2 ns per instruction of one warp (100 per 32 x 32 block + 52 per repetition).
-    // With two accumulator buffers the epilogue hides behind the next tile's main loop except once.
-    const int sms = sm_count() > 0 ? sm_count() : 148;
-    struct Cand { int ntok, na, ka, db; };
-    const Cand cands[] = {{256, 1, 2, 1}, {192, 1, 2, 2}, {128, 2, 2, 1}, {128, 1, 2, 2}, {64, 1, 2, 2}, {32, 1, 2, 2}};
-    const int n_cands = 6;
-    int best = 0;
-    double best_cost = 1e300;
-    const char *force = getenv("TBN_TC_CONFIG");     // tuning aid: force a candidate by index
-    const double atoms = (double)((a.n + kAtomK - 1) / kAtomK);
-    for (int i = 0; i < n_cands; ++i) {
-        const Cand &c = cands[i];
-        const int64_t wt = (p.r + c.na * 128 - 1) / (c.na * 128);
-        const int64_t tt = (a.T + c.ntok - 1) / c.ntok;
-        const int64_t waves = (wt * tt + sms - 1) / sms;
-        const double stage = c.na * c.ka * 4 * (0.45 * c.ntok + 14.0) + 150.0;
-        const double mainloop = atoms / c.ka * stage;
-        const double epi = c.na * (c.ntok / 32.0) * (100.0 + 52.0 * a.k) * 2.0;
-        const double cost = c.db == 2 ? waves * (mainloop > epi ? mainloop : epi) + epi : waves * (mainloop + epi);
-        if (cost < best_cost) { best_cost = cost; best = i; }
+    Plan plan = plan_linear(a);
+    const char *force = getenv("TBN_TC_CONFIG");     // tuning aid: "<candidate>" or "<candidate>,<splits>"
+    if (force && force[0] >= '0' && force[0] < '0' + kNumCands) {
+        plan.cand = force[0] - '0';
+        plan.splits = (force[1] == ',' && atoi(force + 2) >= 1) ? atoi(force + 2) : 1;
+        const Cand &c = kCands[plan.cand];
+        const int64_t out_tiles = (int64_t)((p.r + c.na * 128 - 1) / (c.na * 128)) * ((a.T + c.ntok - 1) / c.ntok);
+        const int k_stages = (a.n + c.ka * kAtomK - 1) / (c.ka * kAtomK);
+        if (plan.splits > k_stages) plan.splits = k_stages;
+        plan.scratch_bytes = plan.splits == 1 ? 0
+            : ((size_t)out_tiles * 4 * sizeof(unsigned int) + 255) / 256 * 256 +
+              (size_t)out_tiles * plan.splits * c.na * 128 * c.ntok * sizeof(float);
     }
-    if (force && force[0] >= '0' && force[0] < '0' + n_cands && force[1] == 0) best = force[0] - '0';
-    switch (best) {
-    case 0: return launch_config<256, 1, 2, 3, 1>(a, p, device_status, s);
-    case 1: return launch_config<192, 1, 2, 4, 2>(a, p, device_status, s);
-    case 2: return launch_config<128, 2, 2, 5, 1>(a, p, device_status, s);
-    case 3: return launch_config<128, 1, 2, 6, 2>(a, p, device_status, s);
-    case 4: return launch_config<64, 1, 2, 8, 2>(a, p, device_status, s);
-    default: return launch_config<32, 1, 2, 8, 2>(a, p, device_status, s);
+    if (plan.splits > 1 && (!scratch || scratch_bytes < plan.scratch_bytes)) {
+        plan.splits = 1;                              // not enough scratch: run unsplit (same result, slower)
+    }
+    switch (plan.cand) {
+    case 0: return launch_config<256, 1, 2, 3, 1>(a, p, plan.splits, scratch, s);
+    case 1: return launch_config<192, 1, 2, 4, 2>(a, p, plan.splits, scratch, s);
+    case 2: return launch_config<128, 2, 2, 5, 1>(a, p, plan.splits, scratch, s);
+    case 3: return launch_config<128, 1, 2, 6, 2>(a, p, plan.splits, scratch, s);
+    case 4: return launch_config<64, 1, 2, 8, 2>(a, p, plan.splits, scratch, s);
+    default: return launch_config<32, 1, 2, 8, 2>(a, p, plan.splits, scratch, s);
     }
 }
 
