@@ -364,13 +364,21 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                         float acc[32];
 #pragma unroll
                         for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
-                        for (int32_t sp = 0; sp < p.splits; ++sp) {
-                            const float4 *src = reinterpret_cast<const float4 *>(part_row + (int64_t)sp * kTileFloats +
-                                                                                 (int64_t)a * 128 * NTOK + ch * 32);
+                        // two splits per round (splits is a power of two): 16 independent 16-byte loads in flight
+                        for (int32_t sp = 0; sp < p.splits; sp += 2) {
+                            const float4 *src0 = reinterpret_cast<const float4 *>(part_row + (int64_t)sp * kTileFloats +
+                                                                                  (int64_t)a * 128 * NTOK + ch * 32);
+                            const float4 *src1 = src0 + kTileFloats / 4;
+                            float4 q0[8], q1[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) { q0[i] = __ldcg(src0 + i); q1[i] = __ldcg(src1 + i); }
 #pragma unroll
                             for (int i = 0; i < 8; ++i) {
-                                const float4 q4 = __ldcg(src + i);
-                                acc[4 * i] += q4.x; acc[4 * i + 1] += q4.y; acc[4 * i + 2] += q4.z; acc[4 * i + 3] += q4.w;
+                                acc[4 * i] += q0[i].x; acc[4 * i + 1] += q0[i].y; acc[4 * i + 2] += q0[i].z; acc[4 * i + 3] += q0[i].w;
+                            }
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                acc[4 * i] += q1[i].x; acc[4 * i + 1] += q1[i].y; acc[4 * i + 2] += q1[i].z; acc[4 * i + 3] += q1[i].w;
                             }
                         }
 #pragma unroll
@@ -539,7 +547,8 @@ Plan plan_linear(const LayerArgs &a)
             const double mainloop = atoms / c.ka / sp * stage;
             double cost;
             if (sp == 1) cost = c.db == 2 ? waves * (mainloop > epi ? mainloop : epi) + epi : waves * (mainloop + epi);
-            else cost = mainloop + dump + epi + 1500.0;                         // + ticket / partial round trip
+            else cost = mainloop + dump + epi + 1500.0 +                        // ticket / partial round trip
+                        c.na * (c.ntok < a.T ? c.ntok : (double)a.T) / 32.0 * (sp / 2) * 1000.0;   // reduction: one L2 round per two splits and 32 tokens
             if (cost < best_cost) {
                 best_cost = cost;
                 best.cand = i;

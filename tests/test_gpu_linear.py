@@ -147,3 +147,24 @@ def test_tensor_path_many_tiles_sampled_rows(k):
     gen = run(B.PATH_GENERIC, x, words, al, True, m, k)
     assert_close(got, gen, "tensor vs generic")
     assert B.tbn_last_device_status() == (0, 0)
+
+
+@pytest.mark.parametrize("T,m,n,k", [(1, 8192, 8192, 2), (16, 8192, 8192, 16), (40, 4096, 4096, 4), (256, 2048, 8192, 8),
+                                     (3, 512, 2056, 2)])
+def test_tensor_path_split_k_matches_oracle_and_is_deterministic(T, m, n, k):
+    # few output tiles, long contraction: the kernel splits K over several CTAs and adds the partial tiles in a
+    # fixed order; sampled output columns through the oracle, and run-to-run bit equality
+    x, W, words, al = make_linear_case(21, T, m, n, k, True, True)
+    assert B.tbn_linear_workspace_bytes(T, n, m, k, B.BF16) > 0          # split-K scratch is requested
+    xd, td, ad = to_dev(x), to_dev(words), to_dev(al)
+    y1 = B.tbn_linear_fwd(xd, m, td, k, ad, 1, act=B.ACT_RELU, path=B.PATH_TENSOR)
+    y2 = B.tbn_linear_fwd(xd, m, td, k, ad, 1, act=B.ACT_RELU, path=B.PATH_TENSOR)
+    torch.cuda.synchronize()
+    assert torch.equal(y1, y2)
+    ref = O.linear(x, words, k, al, True, m, n, act=O.ACT_RELU)
+    assert_close(to_np64(y1), ref, f"split-K T={T} {m}x{n} k={k}")
+    # without scratch the kernel runs unsplit and must agree to fp32 reassociation
+    y3 = B.tbn_linear_fwd(xd, m, td, k, ad, 1, act=B.ACT_RELU, path=B.PATH_TENSOR,
+                          workspace=torch.empty(16, dtype=torch.uint8, device=DEV))
+    assert_close(to_np64(y3), ref, "unsplit")
+    assert B.tbn_last_device_status() == (0, 0)
