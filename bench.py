@@ -49,6 +49,24 @@ def algorithmic_bytes(T: int, k: int) -> float:
     return 2.0 * T * N_FEAT * 2 + (N_FEAT * N_FEAT // k) / 8 + 4 * k
 
 
+# DRAM traffic of the dominant launch (k = 2) from the ncu capture summarised in
+# profiles/tc_linear_k2_T8192_ncu_full.md: 236.0 MB at T = 8192; traffic is proportional to T.  The figure is
+# only valid for the kernel source it was taken from: the hash below covers tc_linear.cu and tc_common.cuh.
+TRAFFIC_BYTES_AT_T8192 = 138.769408e6 + 97.274112e6
+TRAFFIC_SOURCE_HASH = "871e18df3dabc52d"
+
+
+def measured_traffic(T: int):
+    import hashlib
+    h = hashlib.sha256()
+    for f in ("tc_linear.cu", "tc_common.cuh"):
+        with open(os.path.join(ROOT, "paper_2407_12075_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    if h.hexdigest()[:16] != TRAFFIC_SOURCE_HASH:
+        return None                      # the kernel changed since the counters were taken
+    return TRAFFIC_BYTES_AT_T8192 * T / 8192.0
+
+
 def read_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -346,7 +364,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         per_k[str(k)] = dict(ms=per_k_ms[k], alg_tflops=tf, dense_equiv_tflops=tf * k, alg_gbs=gbs,
                              frac_of_binding_roofline=t_bound / (per_k_ms[k] * 1e-3))
     roofline = dict(bound="tensor", achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak,
-                    traffic=None, peak_source=f"{peaks['source']} (sustained bf16 GEMM)", kernel_path=path)
+                    traffic=measured_traffic(T), traffic_note="bytes per k = 2 launch, scaled from an ncu capture at T = 8192",
+                    peak_source=f"{peaks['source']} (sustained bf16 GEMM)", kernel_path=path)
 
     # ---- end to end: host buffers through the C-ABI, copies inside the timed region -------------
     e2e = None
