@@ -67,6 +67,23 @@ def measured_traffic(T: int):
     return TRAFFIC_BYTES_AT_T8192 * T / 8192.0
 
 
+def max_over_ranks(value: float, device=None) -> float:
+    """Multi-rank timing rule: every rank times its own replica on its own device, the job's time is the
+    maximum over ranks.  A no-op without an initialised process group."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(flops_per_rank_step: float, world: int, ms_per_step: float) -> float:
+    """Aggregate algorithmic TFLOP/s of `world` independent replicas (weak scaling)."""
+    return world * flops_per_rank_step / (ms_per_step * 1e-3) / 1e12
+
+
 def read_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -341,16 +358,12 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     t_end.record()
     barrier()
     clocks = sampler.stop()
-    total_ms = t_beg.elapsed_time(t_end)
-    if world > 1:
-        tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    total_ms = max_over_ranks(t_beg.elapsed_time(t_end), dev)
     ms_per_step = total_ms / args.steps
     per_k_ms = {k: float(np.mean([ev[s][i][0].elapsed_time(ev[s][i][1]) for s in range(args.steps)]))
                 for i, k in enumerate(KS)}
     flops_step = sum(algorithmic_flops(T, k) for k in KS)
-    value = world * flops_step / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_value(flops_step, world, ms_per_step)
 
     # ---- roofline of the dominant kernel (the forward kernel, averaged over the four k) --------
     kern_ms = float(np.mean(list(per_k_ms.values())))
@@ -385,10 +398,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             host_step()
         torch.cuda.synchronize()
         dt = (time.perf_counter() - t0) / args.e2e_steps
-        if world > 1:
-            tt = torch.tensor([dt], device=dev, dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            dt = float(tt.item())
+        dt = max_over_ranks(dt, dev)
         nbytes = T * N_FEAT * 2 * len(KS)
         e2e = dict(value=world * flops_step / dt / 1e12, unit=UNIT, h2d_bytes_per_step=nbytes,
                    d2h_bytes_per_step=nbytes, ms_per_step=dt * 1e3, steps=args.e2e_steps)
