@@ -35,6 +35,7 @@ struct LayerArgs {
     const void *x;
     void *y;
     const uint32_t *tile;
+    const void *dense_a;   // tensor-core linear only: bf16 weight rows [q/n][n] used instead of the tile (MLP chain)
     const float *alpha;
     const float *bias;
     int64_t T;       // rows of the contraction: tokens, or Nb*Ho*Wo output pixels
@@ -58,6 +59,8 @@ cudaError_t launch_aggregate_static(const float *W, const float *A, int64_t N, i
 cudaError_t launch_pack(const float *src, int64_t q, uint32_t *tile_bits, cudaStream_t s);
 cudaError_t launch_expand(const uint32_t *tile_bits, int64_t N, int32_t k, const float *alpha,
                           int per_tile, float *B_hat, cudaStream_t s);
+cudaError_t launch_fold(const uint32_t *tile_next, int32_t rows, int32_t n_next, const float *alpha_prev, int per_tile_prev,
+                        int32_t k_prev, int32_t r_prev, __nv_bfloat16 *w_eff, cudaStream_t s);
 cudaError_t launch_f32_to_bf16(const float *src, __nv_bfloat16 *dst, int64_t count, cudaStream_t s);
 
 cudaError_t launch_generic(const LayerArgs &a, cudaStream_t s);

@@ -61,6 +61,7 @@ struct Control {
 
 struct TcParams {
     const uint32_t *tile;
+    const __nv_bfloat16 *dense_a;   // non-null: full-precision weight rows [r][n] instead of tile bits
     const float *alpha;
     const float *bias;
     void *y;
@@ -251,6 +252,48 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
         const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
         const int64_t last_word = p.n_words - 1;
         Pipe pa;
+        if (p.dense_a != nullptr) {
+            // Full-precision rows instead of tile bits (weights folded with the previous layer's alphas, see
+            // the MLP chain): row L of each block is n bf16 values, 64*KA of them per stage, copied as they are.
+            const uint4 *rows = reinterpret_cast<const uint4 *>(p.dense_a);
+            const int32_t row_vecs = p.n >> 3;                       // 16-byte vectors per row (n % 8 == 0)
+            for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
+                const int32_t split = tile % p.splits, out_tile = tile / p.splits;
+                const int32_t ks0 = (int32_t)((int64_t)split * p.k_stages / p.splits);
+                const int32_t ks1 = (int32_t)((int64_t)(split + 1) * p.k_stages / p.splits);
+                const int32_t row_base = (out_tile % p.w_tiles) * (NA * 128) + L;
+                for (int32_t ks = ks0; ks < ks1 && ok; ++ks) {
+                    uint32_t v[NA][KA][32];
+#pragma unroll
+                    for (int a = 0; a < NA; ++a) {
+                        const int32_t row = min(row_base + a * 128, p.r - 1);
+                        const uint4 *src = rows + (int64_t)row * row_vecs;
+                        const int32_t v0 = ks * (kStageK >> 3);
+#pragma unroll
+                        for (int at = 0; at < KA; ++at)
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                const int32_t vi = v0 + at * 8 + i;
+                                const uint4 q4 = vi < row_vecs ? __ldg(src + vi) : make_uint4(0u, 0u, 0u, 0u);
+                                v[a][at][4 * i] = q4.x; v[a][at][4 * i + 1] = q4.y; v[a][at][4 * i + 2] = q4.z; v[a][at][4 * i + 3] = q4.w;
+                            }
+                    }
+                    ok = wait_bar(smem_u32(&ctl->a_empty[pa.stage]), pa.phase ^ 1u, abort_flag, p.status,
+                                  (5 << 24) | (pa.stage << 16) | (bid & 0xffff));
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int a = 0; a < NA; ++a)
+#pragma unroll
+                        for (int at = 0; at < KA; ++at)
+                            tmem_st_32x32(tmem_base + lane_base + kABase + pa.stage * kACols + (a * KA + at) * 32, v[a][at]);
+                    tc_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(&ctl->a_full[pa.stage]));
+                    pa.advance(kAStages);
+                }
+            }
+        } else
         for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
             const int32_t split = tile % p.splits, out_tile = tile / p.splits;
             const int32_t ks0 = (int32_t)((int64_t)split * p.k_stages / p.splits);
@@ -582,8 +625,8 @@ int launch_tensor_linear(const LayerArgs &a, int *device_status, void *scratch, 
 {
     if (a.x_dtype != TBN_BF16) return TBN_ERR_UNSUPPORTED;
     TcParams p;
-    p.tile = a.tile; p.alpha = a.alpha; p.bias = a.bias; p.y = a.y; p.status = device_status;
-    p.T = a.T; p.n_words = tbn_tile_words(a.q);
+    p.tile = a.tile; p.dense_a = static_cast<const __nv_bfloat16 *>(a.dense_a); p.alpha = a.alpha; p.bias = a.bias; p.y = a.y; p.status = device_status;
+    p.T = a.T; p.n_words = a.dense_a ? 1 : tbn_tile_words(a.q);
     p.n = a.n; p.m = a.m; p.r = (int32_t)(a.q / a.n); p.k = a.k;
     p.k_stages = 0;
     p.w_tiles = 0; p.t_tiles = 0; p.splits = 1; p.partial = nullptr; p.tickets = nullptr;
