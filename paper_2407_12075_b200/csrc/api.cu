@@ -1,6 +1,7 @@
 // C entry points of libtbn: argument validation, path selection, workspace carving.
 // Every step of the computation runs in the kernels of the other translation units; nothing here
 // touches the data on the host, and there is no CPU fallback.
+#include <cstdlib>
 #include <cstring>
 
 #include "common.cuh"
@@ -133,6 +134,30 @@ int fill_linear(LayerArgs &a, const void *x, int x_dtype, int64_t T, int32_t in_
     return TBN_OK;
 }
 
+__device__ float g_device_one = 1.0f;       // alpha of the compact (unscaled) hidden tensors of the MLP chain
+
+const float *device_one_ptr()
+{
+    static float *cache[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!cache[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_device_one) != cudaSuccess) return nullptr;
+        cache[dev] = static_cast<float *>(p);
+    }
+    return cache[dev];
+}
+
+// Workspace layout of the compact MLP chain; false when the shapes do not allow it (every layer's tile must span
+// whole rows and the compact widths must keep 16-byte row pitches).
+constexpr int kMaxChainLayers = 64;
+struct MlpChainPlan {
+    size_t g_off[2], weff_off[kMaxChainLayers], xconv_off, scratch_off, scratch_bytes, total_bytes;
+};
+
+bool plan_mlp_chain(int64_t T, int32_t L, const int32_t *dims, const int32_t *ks, int x_dtype, MlpChainPlan &plan);
+
 int check_mlp(int64_t T, int32_t L, const int32_t *dims, const int32_t *ks)
 {
     if (T < 0 || L <= 0 || !dims || !ks) return TBN_ERR_INVALID_ARG;
@@ -143,6 +168,45 @@ int check_mlp(int64_t T, int32_t L, const int32_t *dims, const int32_t *ks)
         if (((int64_t)dims[l] * dims[l + 1]) % ks[l] != 0) return TBN_ERR_SHAPE;
     }
     return TBN_OK;
+}
+
+bool plan_mlp_chain(int64_t T, int32_t L, const int32_t *dims, const int32_t *ks, int x_dtype, MlpChainPlan &plan)
+{
+    if (L < 2 || L > kMaxChainLayers || dims[0] % 8 != 0) return false;
+    int32_t r_max = 0;
+    for (int32_t l = 0; l < L; ++l) {
+        const int64_t N = (int64_t)dims[l] * dims[l + 1];
+        if (N % ks[l] != 0 || (N / ks[l]) % dims[l] != 0) return false;          // tile spans whole rows
+        const int32_t r = dims[l + 1] / ks[l];
+        if (l < L - 1) {
+            if (r % 8 != 0) return false;                                        // TMA row pitch of the compact tensor
+            r_max = r > r_max ? r : r_max;
+        }
+    }
+    size_t off = 0;
+    const size_t g = round_up((size_t)T * r_max * 2, 256);
+    plan.g_off[0] = off; off += g;
+    plan.g_off[1] = off; off += g;
+    size_t scratch = 0;
+    int32_t n_cur = dims[0];
+    for (int32_t l = 0; l < L; ++l) {
+        const int32_t r = dims[l + 1] / ks[l];
+        plan.weff_off[l] = off;
+        if (l > 0) off += round_up((size_t)r * n_cur * 2, 256);
+        LayerArgs a;
+        std::memset(&a, 0, sizeof(a));
+        a.T = T; a.n = n_cur; a.q = (int64_t)r * n_cur; a.x_dtype = TBN_BF16; a.y_dtype = TBN_BF16;
+        a.m = l == L - 1 ? dims[l + 1] : r; a.k = l == L - 1 ? ks[l] : 1;
+        const size_t b = round_up(tensor_linear_scratch_bytes(a), 256);
+        scratch = b > scratch ? b : scratch;
+        n_cur = r;
+    }
+    plan.xconv_off = off;
+    if (x_dtype == TBN_F32) off += round_up((size_t)T * dims[0] * 2, 256);
+    plan.scratch_off = off;
+    plan.scratch_bytes = scratch;
+    plan.total_bytes = off + scratch;
+    return true;
 }
 
 }  // namespace
@@ -356,7 +420,8 @@ int tbn_conv2d_fwd(const void *x, int x_dtype, int32_t Nb, int32_t Cin, int32_t 
 size_t tbn_mlp_workspace_bytes(int64_t T, int32_t L, const int32_t *dims, const int32_t *ks, int x_dtype)
 {
     if (check_mlp(T, L, dims, ks) != TBN_OK || T == 0) return 0;
-    // two ping-pong bf16 hidden buffers sized for the widest hidden layer + the first layer's scratch
+    // (a) layer-by-layer chain: two ping-pong bf16 hidden buffers sized for the widest hidden layer + the
+    //     largest per-layer scratch
     int32_t widest = 0;
     for (int32_t l = 1; l < L; ++l) widest = dims[l] > widest ? dims[l] : widest;
     const size_t hidden = round_up((size_t)T * widest * 2, 256);
@@ -365,7 +430,11 @@ size_t tbn_mlp_workspace_bytes(int64_t T, int32_t L, const int32_t *dims, const 
         const size_t b = tbn_linear_workspace_bytes(T, dims[l], dims[l + 1], ks[l], l == 0 ? x_dtype : TBN_BF16);
         scratch = b > scratch ? b : scratch;
     }
-    return 2 * hidden + scratch;
+    const size_t unfused = 2 * hidden + scratch;
+    // (b) compact chain (see tbn_mlp_fwd): sized whenever the shapes allow it
+    MlpChainPlan plan;
+    const size_t chained = plan_mlp_chain(T, L, dims, ks, x_dtype, plan) ? plan.total_bytes : 0;
+    return unfused > chained ? unfused : chained;
 }
 
 int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t *dims,
@@ -376,18 +445,71 @@ int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t 
     int rc = check_mlp(T, L, dims, ks);
     if (rc != TBN_OK) return rc;
     if (!x || !y || !tiles || !alphas || !alpha_modes || !valid_act(hidden_act)) return TBN_ERR_INVALID_ARG;
+    if (!valid_dtype(x_dtype) || !valid_dtype(y_dtype)) return TBN_ERR_INVALID_ARG;
     for (int32_t l = 0; l < L; ++l)
         if (!tiles[l] || !alphas[l] || !valid_alpha_mode(alpha_modes[l])) return TBN_ERR_INVALID_ARG;
     if (T == 0) return TBN_OK;
     const size_t need = tbn_mlp_workspace_bytes(T, L, dims, ks, x_dtype);
     if (need > 0 && (!workspace || !aligned16(workspace) || workspace_bytes < need)) return TBN_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    char *ws = static_cast<char *>(workspace);
+
+    // Compact chain.  With a ReLU (or no) hidden activation, layer l's output is alpha_j * g[:, c] for its k
+    // repetitions j (Sec. 4.1), so only the r distinct columns g = act(Z) are written (bf16, [T, r]) and the
+    // next layer contracts g with its distinct rows folded with layer l's alphas (launch_fold): the k-fold
+    // broadcast of a hidden layer never goes to HBM and the next contraction is k times shorter.
+    MlpChainPlan plan;
+    const char *no_chain = getenv("TBN_MLP_UNFUSED");
+    if (L >= 2 && (hidden_act == TBN_ACT_RELU || hidden_act == TBN_ACT_NONE) && !(no_chain && no_chain[0] == '1') &&
+        plan_mlp_chain(T, L, dims, ks, x_dtype, plan) && aligned16(x) && aligned16(y)) {
+        int *st = device_status_ptr();
+        const float *one = device_one_ptr();
+        if (!st || !one) return TBN_ERR_CUDA;
+        const void *cur = x;
+        if (x_dtype == TBN_F32) {
+            if (launch_f32_to_bf16(static_cast<const float *>(x), reinterpret_cast<__nv_bfloat16 *>(ws + plan.xconv_off),
+                                   T * (int64_t)dims[0], s) != cudaSuccess)
+                return TBN_ERR_CUDA;
+            cur = ws + plan.xconv_off;
+        }
+        int32_t n_cur = dims[0];
+        for (int32_t l = 0; l < L; ++l) {
+            const bool last = l == L - 1;
+            const int32_t r = dims[l + 1] / ks[l];
+            LayerArgs a;
+            std::memset(&a, 0, sizeof(a));
+            a.x = cur; a.x_dtype = TBN_BF16; a.T = T; a.n = n_cur; a.tile = tiles[l];
+            if (l > 0) {
+                __nv_bfloat16 *w_eff = reinterpret_cast<__nv_bfloat16 *>(ws + plan.weff_off[l]);
+                if (launch_fold(tiles[l], r, dims[l], alphas[l - 1], alpha_modes[l - 1] == TBN_ALPHA_PER_TILE, ks[l - 1],
+                                n_cur, w_eff, s) != cudaSuccess)
+                    return TBN_ERR_CUDA;
+                a.dense_a = w_eff;
+            }
+            a.q = (int64_t)r * n_cur;
+            if (last) {
+                a.m = dims[l + 1]; a.k = ks[l]; a.alpha = alphas[l]; a.alpha_mode = alpha_modes[l];
+                a.act = TBN_ACT_NONE; a.y = y; a.y_dtype = y_dtype;
+            } else {
+                a.m = r; a.k = 1; a.alpha = one; a.alpha_mode = TBN_ALPHA_PER_LAYER;
+                a.act = hidden_act; a.y = ws + plan.g_off[l & 1]; a.y_dtype = TBN_BF16;
+            }
+            if (!tensor_path_supported(a)) return TBN_ERR_UNSUPPORTED;
+            rc = launch_tensor_linear(a, st, ws + plan.scratch_off, plan.scratch_bytes, s);
+            if (rc != TBN_OK) return rc;
+            cur = a.y;
+            n_cur = r;
+        }
+        return TBN_OK;
+    }
+
+    // Layer-by-layer chain: hidden tensors are written in full (bf16) and read back.
     int32_t widest = 0;
     for (int32_t l = 1; l < L; ++l) widest = dims[l] > widest ? dims[l] : widest;
     const size_t hidden = round_up((size_t)T * widest * 2, 256);
-    char *ws = static_cast<char *>(workspace);
     void *buf[2] = {ws, ws + hidden};
     void *scratch = ws + 2 * hidden;
-    const size_t scratch_bytes = need - 2 * hidden;
+    const size_t scratch_bytes = workspace_bytes - 2 * hidden;
 
     const void *cur = x;
     int cur_dtype = x_dtype;

@@ -197,6 +197,28 @@ f32_to_bf16_kernel(const float *__restrict__ src, __nv_bfloat16 *__restrict__ ds
         dst[count - 1] = __float2bfloat16_rn(src[count - 1]);
 }
 
+// Folding the previous layer's alphas into the next layer's distinct rows (MLP chain with ReLU or no hidden
+// activation).  The previous layer's output is h[t][j*r1 + c] = alpha1_j * g[t][c] with g = act(z) (alpha >= 0, so
+// relu(alpha z) = alpha relu(z)), hence  sum_j sum_c B2[o][j*r1 + c] h[t][j*r1 + c] = sum_c g[t][c] * W[o][c]  with
+//     W[o][c] = sum_j alpha1_j * (bit2(o*n2 + j*r1 + c) ? +1 : -1),   n2 = k1 * r1.
+// One thread per (o, c); fp32 sum in increasing j, one rounding to bf16.
+__global__ void __launch_bounds__(256)
+fold_kernel(const uint32_t *__restrict__ tile_next, int32_t rows, int32_t n_next, const float *__restrict__ alpha_prev,
+            int per_tile_prev, int32_t k_prev, int32_t r_prev, __nv_bfloat16 *__restrict__ w_eff)
+{
+    const int64_t total = (int64_t)rows * r_prev;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += stride) {
+        const int32_t o = (int32_t)(e / r_prev), c = (int32_t)(e % r_prev);
+        float acc = 0.0f;
+        for (int32_t j = 0; j < k_prev; ++j) {
+            const float al = per_tile_prev ? __ldg(alpha_prev + j) : __ldg(alpha_prev);
+            acc += tile_bit(tile_next, (int64_t)o * n_next + (int64_t)j * r_prev + c) ? al : -al;
+        }
+        w_eff[e] = __float2bfloat16_rn(acc);
+    }
+}
+
 int grid_for(int64_t work_items, int threads, int cap_blocks)
 {
     int64_t b = (work_items + threads - 1) / threads;
@@ -269,6 +291,14 @@ cudaError_t launch_expand(const uint32_t *tile_bits, int64_t N, int32_t k, const
                           int per_tile, float *B_hat, cudaStream_t s)
 {
     expand_kernel<<<grid_for(N, 256, 148 * 8), 256, 0, s>>>(tile_bits, N, N / k, alpha, per_tile, B_hat);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_fold(const uint32_t *tile_next, int32_t rows, int32_t n_next, const float *alpha_prev, int per_tile_prev,
+                        int32_t k_prev, int32_t r_prev, __nv_bfloat16 *w_eff, cudaStream_t s)
+{
+    fold_kernel<<<grid_for((int64_t)rows * r_prev, 256, 148 * 8), 256, 0, s>>>(tile_next, rows, n_next, alpha_prev,
+                                                                              per_tile_prev, k_prev, r_prev, w_eff);
     return cudaGetLastError();
 }
 
