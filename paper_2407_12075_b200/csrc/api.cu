@@ -472,6 +472,24 @@ int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t 
                 return TBN_ERR_CUDA;
             cur = ws + plan.xconv_off;
         }
+        // all folds first, kMaxFoldJobs layers per launch (they depend on the parameters only)
+        {
+            FoldJobs jobs;
+            jobs.count = 0;
+            int32_t r_prev = dims[1] / ks[0];
+            for (int32_t l = 1; l < L; ++l) {
+                FoldJob &J = jobs.job[jobs.count++];
+                J.tile_next = tiles[l]; J.alpha_prev = alphas[l - 1];
+                J.w_eff = reinterpret_cast<__nv_bfloat16 *>(ws + plan.weff_off[l]);
+                J.rows = dims[l + 1] / ks[l]; J.n_next = dims[l];
+                J.per_tile_prev = alpha_modes[l - 1] == TBN_ALPHA_PER_TILE; J.k_prev = ks[l - 1]; J.r_prev = r_prev;
+                r_prev = J.rows;
+                if (jobs.count == kMaxFoldJobs || l == L - 1) {
+                    if (launch_fold(jobs, s) != cudaSuccess) return TBN_ERR_CUDA;
+                    jobs.count = 0;
+                }
+            }
+        }
         int32_t n_cur = dims[0];
         for (int32_t l = 0; l < L; ++l) {
             const bool last = l == L - 1;
@@ -479,13 +497,7 @@ int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t 
             LayerArgs a;
             std::memset(&a, 0, sizeof(a));
             a.x = cur; a.x_dtype = TBN_BF16; a.T = T; a.n = n_cur; a.tile = tiles[l];
-            if (l > 0) {
-                __nv_bfloat16 *w_eff = reinterpret_cast<__nv_bfloat16 *>(ws + plan.weff_off[l]);
-                if (launch_fold(tiles[l], r, dims[l], alphas[l - 1], alpha_modes[l - 1] == TBN_ALPHA_PER_TILE, ks[l - 1],
-                                n_cur, w_eff, s) != cudaSuccess)
-                    return TBN_ERR_CUDA;
-                a.dense_a = w_eff;
-            }
+            if (l > 0) a.dense_a = ws + plan.weff_off[l];
             a.q = (int64_t)r * n_cur;
             if (last) {
                 a.m = dims[l + 1]; a.k = ks[l]; a.alpha = alphas[l]; a.alpha_mode = alpha_modes[l];

@@ -59,8 +59,19 @@ cudaError_t launch_aggregate_static(const float *W, const float *A, int64_t N, i
 cudaError_t launch_pack(const float *src, int64_t q, uint32_t *tile_bits, cudaStream_t s);
 cudaError_t launch_expand(const uint32_t *tile_bits, int64_t N, int32_t k, const float *alpha,
                           int per_tile, float *B_hat, cudaStream_t s);
-cudaError_t launch_fold(const uint32_t *tile_next, int32_t rows, int32_t n_next, const float *alpha_prev, int per_tile_prev,
-                        int32_t k_prev, int32_t r_prev, __nv_bfloat16 *w_eff, cudaStream_t s);
+// Folding jobs of an MLP chain (one per layer after the first), executed by one launch.
+constexpr int kMaxFoldJobs = 8;
+struct FoldJob {
+    const uint32_t *tile_next;   // tile of the layer whose rows are folded
+    const float *alpha_prev;     // alphas of the layer before it
+    __nv_bfloat16 *w_eff;        // out: rows x r_prev
+    int32_t rows, n_next, per_tile_prev, k_prev, r_prev;
+};
+struct FoldJobs {
+    FoldJob job[kMaxFoldJobs];
+    int32_t count;
+};
+cudaError_t launch_fold(const FoldJobs &jobs, cudaStream_t s);
 cudaError_t launch_f32_to_bf16(const float *src, __nv_bfloat16 *dst, int64_t count, cudaStream_t s);
 
 cudaError_t launch_generic(const LayerArgs &a, cudaStream_t s);

@@ -203,19 +203,21 @@ f32_to_bf16_kernel(const float *__restrict__ src, __nv_bfloat16 *__restrict__ ds
 //     W[o][c] = sum_j alpha1_j * (bit2(o*n2 + j*r1 + c) ? +1 : -1),   n2 = k1 * r1.
 // One thread per (o, c); fp32 sum in increasing j, one rounding to bf16.
 __global__ void __launch_bounds__(256)
-fold_kernel(const uint32_t *__restrict__ tile_next, int32_t rows, int32_t n_next, const float *__restrict__ alpha_prev,
-            int per_tile_prev, int32_t k_prev, int32_t r_prev, __nv_bfloat16 *__restrict__ w_eff)
+fold_kernel(const FoldJobs jobs)
 {
-    const int64_t total = (int64_t)rows * r_prev;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += stride) {
-        const int32_t o = (int32_t)(e / r_prev), c = (int32_t)(e % r_prev);
-        float acc = 0.0f;
-        for (int32_t j = 0; j < k_prev; ++j) {
-            const float al = per_tile_prev ? __ldg(alpha_prev + j) : __ldg(alpha_prev);
-            acc += tile_bit(tile_next, (int64_t)o * n_next + (int64_t)j * r_prev + c) ? al : -al;
+    for (int32_t jb = 0; jb < jobs.count; ++jb) {
+        const FoldJob &J = jobs.job[jb];
+        const int64_t total = (int64_t)J.rows * J.r_prev;
+        for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += stride) {
+            const int32_t o = (int32_t)(e / J.r_prev), c = (int32_t)(e % J.r_prev);
+            float acc = 0.0f;
+            for (int32_t j = 0; j < J.k_prev; ++j) {
+                const float al = J.per_tile_prev ? __ldg(J.alpha_prev + j) : __ldg(J.alpha_prev);
+                acc += tile_bit(J.tile_next, (int64_t)o * J.n_next + (int64_t)j * J.r_prev + c) ? al : -al;
+            }
+            J.w_eff[e] = __float2bfloat16_rn(acc);
         }
-        w_eff[e] = __float2bfloat16_rn(acc);
     }
 }
 
@@ -294,11 +296,14 @@ cudaError_t launch_expand(const uint32_t *tile_bits, int64_t N, int32_t k, const
     return cudaGetLastError();
 }
 
-cudaError_t launch_fold(const uint32_t *tile_next, int32_t rows, int32_t n_next, const float *alpha_prev, int per_tile_prev,
-                        int32_t k_prev, int32_t r_prev, __nv_bfloat16 *w_eff, cudaStream_t s)
+cudaError_t launch_fold(const FoldJobs &jobs, cudaStream_t s)
 {
-    fold_kernel<<<grid_for((int64_t)rows * r_prev, 256, 148 * 8), 256, 0, s>>>(tile_next, rows, n_next, alpha_prev,
-                                                                              per_tile_prev, k_prev, r_prev, w_eff);
+    int64_t most = 1;
+    for (int32_t j = 0; j < jobs.count; ++j) {
+        const int64_t t = (int64_t)jobs.job[j].rows * jobs.job[j].r_prev;
+        most = t > most ? t : most;
+    }
+    fold_kernel<<<grid_for(most, 256, 148 * 8), 256, 0, s>>>(jobs);
     return cudaGetLastError();
 }
 

@@ -139,3 +139,24 @@ def test_tensor_conv_rejects_what_it_cannot_take():
     with pytest.raises(B.TbnError) as e:
         B.tbn_conv2d_fwd(to_dev(x), 8, 3, 3, 1, 1, to_dev(words), 2, to_dev(al), 1, path=B.PATH_TENSOR)
     assert e.value.status == -3
+
+
+@pytest.mark.parametrize("T,dims,ks,act", [(200, [64, 256, 128, 24], [4, 8, 1], B.ACT_RELU),
+                                           (37, [128, 512, 512, 64], [8, 4, 2], B.ACT_NONE),
+                                           (1000, [256, 1024, 16], [16, 2], B.ACT_RELU)])
+def test_mlp_compact_chain_matches_oracle_and_layerwise_chain(T, dims, ks, act, monkeypatch):
+    # shapes whose hidden tiles span whole rows with compact widths that are multiples of 8: the hidden layers'
+    # k-fold broadcast stays out of HBM (compact chain); the layer-by-layer chain must give the same result
+    L = len(ks)
+    x = synth.to_bf16_bits(synth.normal(5, 0, T * dims[0]).reshape(T, dims[0]))
+    Ws = [synth.normal(5, 1 + l, dims[l + 1] * dims[l], 0.05).reshape(dims[l + 1], dims[l]) for l in range(L)]
+    layers, tiles, alphas = _mlp_layers(Ws, ks)
+    ref = O.mlp(x, layers, hidden_act=O.ACT_RELU if act == B.ACT_RELU else O.ACT_NONE)
+    y = B.tbn_mlp_fwd(to_dev(x), dims, tiles, ks, alphas, [1] * L, hidden_act=act)
+    torch.cuda.synchronize()
+    assert_close(to_np64(y), ref, "compact chain")
+    monkeypatch.setenv("TBN_MLP_UNFUSED", "1")
+    y2 = B.tbn_mlp_fwd(to_dev(x), dims, tiles, ks, alphas, [1] * L, hidden_act=act)
+    torch.cuda.synchronize()
+    assert_close(to_np64(y2), ref, "layer-by-layer chain")
+    assert B.tbn_last_device_status() == (0, 0)
