@@ -184,8 +184,15 @@ int tbn_conv2d_fwd_path(const void *x, int x_dtype, int32_t Nb, int32_t Cin, int
  * Chain of L fully-connected tiled layers (Sec. 5.1: an MLP with a fused ReLU):
  *     h_0 = x;  h_{l+1} = hidden_act(layer_l(h_l)) for l < L-1;  y = layer_{L-1}(h_{L-1}).
  * dims (host, L+1 ints): dims[l] -> dims[l+1] is layer l.  ks, alpha_modes: host arrays of L values.
- * tiles, alphas: HOST arrays of L DEVICE pointers.  No biases.  Hidden tensors are kept in bf16 in
- * the workspace.  x: T x dims[0];  y: T x dims[L].
+ * tiles, alphas: HOST arrays of L DEVICE pointers.  No biases.  x: T x dims[0];  y: T x dims[L].
+ * Compact chain: when the hidden activation is ReLU or none, every layer's tile spans whole rows and the
+ * numbers of distinct rows of the hidden layers are multiples of 8, a hidden layer writes only its distinct
+ * columns g = act(Z) (bf16, T x r) to the workspace -- its k repetitions are alpha_j * g (Sec. 4.1; alpha >= 0
+ * so relu(alpha z) = alpha relu(z)) -- and the next layer contracts g with its distinct rows folded with
+ * those alphas, computed on the device at every call from the tiles and alphas: the k-fold broadcast never
+ * goes to HBM and the next contraction is k times shorter.  Otherwise layers run one by one with full bf16
+ * hidden tensors in the workspace.  Both give the layer-by-layer result up to bf16 rounding of the hidden
+ * tensors / folded rows.
  */
 size_t tbn_mlp_workspace_bytes(int64_t T, int32_t L, const int32_t *dims, const int32_t *ks, int x_dtype);
 int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t *dims,
@@ -201,6 +208,9 @@ int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t 
  * Returns TBN_OK, or TBN_ERR_CUDA if the synchronisation or the copy failed.
  */
 int tbn_last_device_status(void *stream, int *code, int *detail);
+/* Testing aid: enqueue a kernel that records (code, detail) exactly as a kernel whose wait gave up would --
+ * it waits on nothing, so it cannot hang -- to exercise the status plumbing without starving a real pipeline. */
+int tbn_debug_record_status(int code, int detail, void *stream);
 
 #ifdef __cplusplus
 }

@@ -47,6 +47,7 @@ SIGNATURES = {
     "tbn_mlp_fwd": (c_int, [c_vp, c_int, c_i64, c_i32, c_vp, c_vp, c_vp, c_vp, c_vp, c_int, c_vp, c_int,
                             c_vp, c_sz, c_vp]),
     "tbn_last_device_status": (c_int, [c_vp, c_vp, c_vp]),
+    "tbn_debug_record_status": (c_int, [c_int, c_int, c_vp]),
 }
 
 _lib = None
@@ -245,3 +246,7 @@ def tbn_last_device_status():
     _check(lib().tbn_last_device_status(_stream(), ctypes.byref(code), ctypes.byref(detail)),
            "tbn_last_device_status")
     return int(code.value), int(detail.value)
+
+
+def tbn_debug_record_status(code: int, detail: int):
+    _check(lib().tbn_debug_record_status(code, detail, _stream()), "tbn_debug_record_status")

@@ -11,6 +11,11 @@ namespace tbn {
 // Device-side status record: {code, detail, reserved, reserved}.  Kernels receive its address.
 __device__ int g_device_status[4];
 
+__global__ void record_status_kernel(int *status, int code, int detail)
+{
+    if (atomicCAS(status, 0, code) == 0) status[1] = detail;
+}
+
 namespace {
 
 int *device_status_ptr()
@@ -551,6 +556,14 @@ int tbn_last_device_status(void *stream, int *code, int *detail)
     *detail = host[1];
     if (host[0] != 0 && cudaMemset(st, 0, sizeof(host)) != cudaSuccess) return TBN_ERR_CUDA;
     return TBN_OK;
+}
+
+int tbn_debug_record_status(int code, int detail, void *stream)
+{
+    int *st = device_status_ptr();
+    if (!st) return TBN_ERR_CUDA;
+    record_status_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(st, code, detail);
+    return cudaGetLastError() == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
 }
 
 }  // extern "C"

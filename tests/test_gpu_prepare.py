@@ -77,3 +77,13 @@ def test_shape_errors_surface_as_exceptions():
     W = torch.zeros(10, device=DEV)
     with pytest.raises(B.TbnError):
         B.tbn_aggregate_tile(W, 3)
+
+
+def test_device_status_word_round_trip():
+    # a wait that gives up records TBN_ERR_TIMEOUT + a detail word; the plumbing is exercised with a kernel
+    # that records the same thing without waiting on anything
+    assert B.tbn_last_device_status() == (0, 0)
+    B.tbn_debug_record_status(-6, (3 << 24) | (2 << 16) | 17)
+    B.tbn_debug_record_status(-6, 99)                       # first record wins
+    assert B.tbn_last_device_status() == (-6, (3 << 24) | (2 << 16) | 17)
+    assert B.tbn_last_device_status() == (0, 0)             # reading clears it
