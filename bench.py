@@ -287,6 +287,27 @@ def measure_other_configs(B, torch, dev, peaks):
     for T in (1, 16, 256, 4096):
         for k in (2, 16):
             out[f"large_linear_T{T}_k{k}"] = linear_entry(T, N_FEAT, N_FEAT, k)
+    # Small batch against HBM: a CUDA-graph chain of distinct layers whose tiles (4 MiB each at k = 2) add up to
+    # more than L2, so every layer's tile really comes from HBM; per-layer time and tile GB/s.
+    for T in (1, 16):
+        k, n_layers = 2, 40
+        x = torch.randn(T, N_FEAT, device=dev, generator=gen).to(torch.bfloat16)
+        ys = [torch.empty(T, N_FEAT, device=dev, dtype=torch.bfloat16) for _ in range(2)]
+        tiles = [rand_tile(N_FEAT * N_FEAT // k) for _ in range(n_layers)]
+        alpha = torch.rand(k, device=dev, generator=gen) * 0.02
+        ws = torch.empty(max(B.tbn_linear_workspace_bytes(T, N_FEAT, N_FEAT, k, B.BF16), 16), dtype=torch.uint8, device=dev)
+
+        def chain():
+            cur = x
+            for l in range(n_layers):
+                B.tbn_linear_fwd(cur, N_FEAT, tiles[l], k, alpha, B.ALPHA_PER_TILE, act=B.ACT_RELU, y=ys[l & 1], workspace=ws)
+                cur = ys[l & 1]
+
+        us = graph_us(chain, reps=1, iters=5) / n_layers
+        nbytes = N_FEAT * N_FEAT // k / 8 + 2 * T * N_FEAT * 2
+        out[f"small_batch_chain_T{T}_k{k}_{n_layers}_layers"] = dict(
+            us_per_layer=us, path=B.tbn_linear_select_path(T, N_FEAT, N_FEAT, k, B.BF16), alg_gbs=nbytes / us / 1e3,
+            bound="hbm", frac_of_binding_roofline=nbytes / hbm * 1e6 / us, l2="tiles exceed L2 (160 MiB)")
     return out
 
 
