@@ -37,6 +37,10 @@ template <> struct XVec<float> {
     }
 };
 
+// Lane l of a warp walks the row in groups of 1024 weights and owns the 32 weights [1024*I + 32*l, +32): one
+// 32-bit word of tile bits per row (128 coalesced bytes per warp) and 32 consecutive activations per token
+// (four / eight 16-byte loads, shared by the warp's RW rows).  A group's loads are all issued before its
+// arithmetic; the many resident warps per SM cover the remaining latency.
 template <typename XT, int RW, int TT>
 __global__ void __launch_bounds__(kWarps * 32)
 small_batch_kernel(const LayerArgs a, int32_t r)
@@ -48,9 +52,10 @@ small_batch_kernel(const LayerArgs a, int32_t r)
     if (row0 >= r) return;
 
     const XT *x = static_cast<const XT *>(a.x);
-    const uint8_t *bits = reinterpret_cast<const uint8_t *>(a.tile);
+    const uint8_t *bits8 = reinterpret_cast<const uint8_t *>(a.tile);
     const int32_t n = a.n;
     const int32_t row_bytes = n >> 3;
+    const bool word_rows = (n & 31) == 0;                        // every row starts on a 32-bit word
 
     float acc[RW][TT];
 #pragma unroll
@@ -58,26 +63,67 @@ small_batch_kernel(const LayerArgs a, int32_t r)
 #pragma unroll
         for (int t = 0; t < TT; ++t) acc[rr][t] = 0.0f;
 
-    for (int32_t e0 = lane * 8; e0 < n; e0 += 256) {
-        float xv[TT][8];
+    int32_t rows[RW];
 #pragma unroll
-        for (int t = 0; t < TT; ++t) {
-            if (t0 + t < a.T) {
-                XVec<XT>::load8(x + (t0 + t) * n + e0, xv[t]);
-            } else {
-#pragma unroll
-                for (int b = 0; b < 8; ++b) xv[t][b] = 0.0f;
-            }
-        }
+    for (int rr = 0; rr < RW; ++rr) rows[rr] = min(row0 + rr, r - 1);    // clamp: extra rows are not stored
+
+    for (int32_t e0 = lane * 32; e0 < n; e0 += 1024) {
+        // tile bits of this lane's 32 weights for each row (chunks past the end of the row are skipped below)
+        uint32_t nb[RW];
 #pragma unroll
         for (int rr = 0; rr < RW; ++rr) {
-            const int32_t row = min(row0 + rr, r - 1);            // clamp: extra rows are not stored
-            const uint32_t nb = ~(uint32_t)__ldg(bits + (int64_t)row * row_bytes + (e0 >> 3));
+            const int64_t byte0 = (int64_t)rows[rr] * row_bytes + (e0 >> 3);
+            uint32_t w;
+            if (word_rows) {
+                w = __ldg(reinterpret_cast<const uint32_t *>(bits8 + byte0));
+            } else {
+                w = 0;
 #pragma unroll
-            for (int b = 0; b < 8; ++b) {
-                const float sgn = __uint_as_float(0x3f800000u | ((nb << (31 - b)) & 0x80000000u));
+                for (int c = 0; c < 4; ++c)
+                    if (e0 + 8 * c < n) w |= (uint32_t)__ldg(bits8 + byte0 + c) << (8 * c);
+            }
+            nb[rr] = ~w;
+        }
+        const bool full = e0 + 32 <= n;                          // n % 8 == 0: whole chunks of 8 only
+        if (TT == 1 && full) {
+            // all activation loads of the group first, then the arithmetic
+            float xv[4][8];
 #pragma unroll
-                for (int t = 0; t < TT; ++t) acc[rr][t] = fmaf(sgn, xv[t][b], acc[rr][t]);
+            for (int c = 0; c < 4; ++c) XVec<XT>::load8(x + t0 * n + e0 + 8 * c, xv[c]);
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+                for (int rr = 0; rr < RW; ++rr)
+#pragma unroll
+                    for (int b = 0; b < 8; ++b) {
+                        // bit 1 -> +1.0f, bit 0 -> -1.0f: the inverted bit goes into the sign position of 1.0f
+                        const float sgn = __uint_as_float(0x3f800000u | ((nb[rr] << (31 - 8 * c - b)) & 0x80000000u));
+                        acc[rr][0] = fmaf(sgn, xv[c][b], acc[rr][0]);
+                    }
+        } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {                        // four chunks of 8 weights
+                const int32_t e = e0 + 8 * c;
+                if (!full && e >= n) break;
+                float xv[TT][8];
+#pragma unroll
+                for (int t = 0; t < TT; ++t) {
+                    if (t0 + t < a.T) {
+                        XVec<XT>::load8(x + (t0 + t) * n + e, xv[t]);
+                    } else {
+#pragma unroll
+                        for (int b = 0; b < 8; ++b) xv[t][b] = 0.0f;
+                    }
+                }
+#pragma unroll
+                for (int rr = 0; rr < RW; ++rr) {
+#pragma unroll
+                    for (int b = 0; b < 8; ++b) {
+                        const float sgn = __uint_as_float(0x3f800000u | ((nb[rr] << (31 - 8 * c - b)) & 0x80000000u));
+#pragma unroll
+                        for (int t = 0; t < TT; ++t) acc[rr][t] = fmaf(sgn, xv[t][b], acc[rr][t]);
+                    }
+                }
             }
         }
     }
@@ -135,8 +181,9 @@ template <typename XT>
 cudaError_t launch_rw(const LayerArgs &a, int32_t r, cudaStream_t s)
 {
     // more rows per warp reuse each activation load more often, but small layers need the blocks
-    if (r >= 148 * 4 * kWarps * 4) return launch_tt<XT, 4>(a, r, s);
-    if (r >= 148 * 2 * kWarps * 2) return launch_tt<XT, 2>(a, r, s);
+    // enough warps per SM to hide load latency first (>= ~32), activation reuse second
+    if (r >= 148 * 32 * 4) return launch_tt<XT, 4>(a, r, s);
+    if (r >= 148 * 32 * 2) return launch_tt<XT, 2>(a, r, s);
     return launch_tt<XT, 1>(a, r, s);
 }
 
