@@ -162,6 +162,148 @@ small_batch_kernel(const LayerArgs a, int32_t r)
     }
 }
 
+// ---- bf16 activations, word-aligned rows: warp-level tensor-core form --------------------------------------
+//
+// A block owns 16 distinct rows and 8*NT tokens; its warps split the contraction dimension and are summed in
+// warp order through shared memory, so the result does not depend on scheduling.  Each warp issues
+// m16n8k16 MMAs whose A fragment is decoded from tile bits in registers and whose B fragment is the
+// activations as loaded.  The contraction index may be permuted freely as long as A and B agree, which
+// removes every shuffle: within a span of 128 weights lane (g, c) (g = lane / 4, c = lane % 4) takes the
+// 32-weight chunk c, i.e. ONE 32-bit word of bits for row g and one for row g + 8, and 64 bytes of
+// activations of token g; MMA u of the span contracts weights 4u..4u+3 of all four chunks.
+__device__ __forceinline__ void mma_bf16_16x8x16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                 uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Bits 2p and 2p+1 of a 16-bit field, spread by spread16(), become the bf16 pair (+-1, +-1): bit set -> +1.
+__device__ __forceinline__ uint32_t spread16(uint32_t h)       // h < 65536: even bits stay, odd bits move up 15
+{
+    return (h | (h << 15)) & 0x55555555u;
+}
+__device__ __forceinline__ uint32_t sign_pair(uint32_t v, int p)
+{
+    return ((v << (15 - 2 * p)) & 0x80008000u) ^ 0xBF80BF80u;
+}
+
+constexpr int kMmaMaxWarps = 32;
+
+template <int NT>
+__global__ void __launch_bounds__(kMmaMaxWarps * 32)
+small_mma_kernel(const LayerArgs a, int32_t r)
+{
+    __shared__ float red[kMmaMaxWarps / NT][NT][16][8];          // [warp][token tile][row][token]: <= 16 KB
+
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int nw = blockDim.x >> 5;
+    const int g = lane >> 2, c = lane & 3;
+    const int32_t row0 = blockIdx.x * 16;
+    const int64_t t0 = (int64_t)blockIdx.y * (8 * NT);
+    const int32_t n = a.n;
+    const int32_t n_chunks = n >> 5;                             // n % 32 == 0
+    const int32_t n_spans = (n_chunks + 3) >> 2;
+
+    const uint32_t *bits = a.tile;
+    const int32_t row_words = n >> 5;
+    const uint32_t *bits_lo = bits + (int64_t)min(row0 + g, r - 1) * row_words;       // clamped rows are not stored
+    const uint32_t *bits_hi = bits + (int64_t)min(row0 + g + 8, r - 1) * row_words;
+    const __nv_bfloat16 *x = static_cast<const __nv_bfloat16 *>(a.x);
+
+    float acc[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[nt][i] = 0.0f;
+
+    for (int32_t span = warp; span < n_spans; span += nw) {
+        const int32_t chunk = span * 4 + c;
+        const bool live = chunk < n_chunks;                      // ragged last span: activations read as zero
+        const int32_t ch = live ? chunk : 0;
+        const uint32_t w_lo = __ldg(bits_lo + ch);
+        const uint32_t w_hi = __ldg(bits_hi + ch);
+        uint4 xb[NT][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            const int64_t t = t0 + nt * 8 + g;
+            if (live && t < a.T) {
+                const uint4 *px = reinterpret_cast<const uint4 *>(x + t * n + (int64_t)ch * 32);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) xb[nt][i] = __ldg(px + i);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) xb[nt][i] = make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {                   // 16 bits of each row word at a time
+            const uint32_t v_lo = spread16(half ? w_lo >> 16 : w_lo & 0xffffu);
+            const uint32_t v_hi = spread16(half ? w_hi >> 16 : w_hi & 0xffffu);
+#pragma unroll
+            for (int uu = 0; uu < 4; ++uu) {                     // MMA u = 4 * half + uu: weights 4u..4u+3 of the chunk
+                const uint32_t a0 = sign_pair(v_lo, 2 * uu), a2 = sign_pair(v_lo, 2 * uu + 1);
+                const uint32_t a1 = sign_pair(v_hi, 2 * uu), a3 = sign_pair(v_hi, 2 * uu + 1);
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const uint4 q = xb[nt][half * 2 + (uu >> 1)];
+                    const uint32_t b0 = (uu & 1) ? q.z : q.x, b1 = (uu & 1) ? q.w : q.y;
+                    mma_bf16_16x8x16(acc[nt], a0, a1, a2, a3, b0, b1);
+                }
+            }
+        }
+    }
+
+    // accumulator fragment: [0],[1] = row g, tokens 2c, 2c+1; [2],[3] = row g + 8
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        *reinterpret_cast<float2 *>(&red[warp][nt][g][2 * c]) = make_float2(acc[nt][0], acc[nt][1]);
+        *reinterpret_cast<float2 *>(&red[warp][nt][g + 8][2 * c]) = make_float2(acc[nt][2], acc[nt][3]);
+    }
+    __syncthreads();
+
+    const bool per_tile = a.alpha_mode == TBN_ALPHA_PER_TILE;
+    for (int e = threadIdx.x; e < NT * 8 * 16; e += blockDim.x) {
+        const int row = e & 15, tok = e >> 4;                    // rows fastest: 16 neighbouring outputs per token
+        const int32_t grow = row0 + row;
+        const int64_t t = t0 + tok;
+        if (grow >= r || t >= a.T) continue;
+        float z = 0.0f;
+        for (int w = 0; w < nw; ++w) z += red[w][tok >> 3][row][tok & 7];
+        for (int32_t j = 0; j < a.k; ++j) {
+            const int32_t o = j * r + grow;
+            const float al = per_tile ? __ldg(a.alpha + j) : __ldg(a.alpha);
+            const float v = apply_act(fmaf(al, z, a.bias ? __ldg(a.bias + o) : 0.0f), a.act);
+            const int64_t yi = t * a.m + o;
+            if (a.y_dtype == TBN_BF16) store_from_float(static_cast<__nv_bfloat16 *>(a.y), yi, v);
+            else store_from_float(static_cast<float *>(a.y), yi, v);
+        }
+    }
+}
+
+bool small_mma_supported(const LayerArgs &a)
+{
+    return a.x_dtype == TBN_BF16 && (a.n & 31) == 0 && (reinterpret_cast<uintptr_t>(a.x) & 15) == 0;
+}
+
+cudaError_t launch_small_mma(const LayerArgs &a, int32_t r, cudaStream_t s)
+{
+    const int nt = a.T <= 8 ? 1 : a.T <= 16 ? 2 : 4;
+    const int64_t row_blocks = (r + 15) / 16;
+    const int64_t tok_blocks = (a.T + 8 * nt - 1) / (8 * nt);
+    const int32_t n_spans = (a.n / 32 + 3) / 4;
+    // about 16 warps per SM in total, at least one span per warp, and the reduction buffer bounds warps x NT
+    int nw = 1;
+    while (nw < kMmaMaxWarps / nt && nw < n_spans && row_blocks * tok_blocks * nw < 148 * 16) nw *= 2;
+    const dim3 grid((unsigned)row_blocks, (unsigned)tok_blocks);
+    if (nt == 1) small_mma_kernel<1><<<grid, nw * 32, 0, s>>>(a, r);
+    else if (nt == 2) small_mma_kernel<2><<<grid, nw * 32, 0, s>>>(a, r);
+    else small_mma_kernel<4><<<grid, nw * 32, 0, s>>>(a, r);
+    return cudaGetLastError();
+}
+
 template <typename XT, int RW>
 cudaError_t launch_tt(const LayerArgs &a, int32_t r, cudaStream_t s)
 {
@@ -201,6 +343,7 @@ bool small_batch_supported(const LayerArgs &a)
 cudaError_t launch_small_batch(const LayerArgs &a, cudaStream_t s)
 {
     const int32_t r = (int32_t)(a.q / a.n);
+    if (small_mma_supported(a)) return launch_small_mma(a, r, s);
     return a.x_dtype == TBN_BF16 ? launch_rw<__nv_bfloat16>(a, r, s) : launch_rw<float>(a, r, s);
 }
 
