@@ -37,10 +37,6 @@ template <> struct XVec<float> {
     }
 };
 
-// Lane l of a warp walks the row in groups of 1024 weights and owns the 32 weights [1024*I + 32*l, +32): one
-// 32-bit word of tile bits per row (128 coalesced bytes per warp) and 32 consecutive activations per token
-// (four / eight 16-byte loads, shared by the warp's RW rows).  A group's loads are all issued before its
-// arithmetic; the many resident warps per SM cover the remaining latency.
 template <typename XT, int RW, int TT>
 __global__ void __launch_bounds__(kWarps * 32)
 small_batch_kernel(const LayerArgs a, int32_t r)
@@ -52,10 +48,9 @@ small_batch_kernel(const LayerArgs a, int32_t r)
     if (row0 >= r) return;
 
     const XT *x = static_cast<const XT *>(a.x);
-    const uint8_t *bits8 = reinterpret_cast<const uint8_t *>(a.tile);
+    const uint8_t *bits = reinterpret_cast<const uint8_t *>(a.tile);
     const int32_t n = a.n;
     const int32_t row_bytes = n >> 3;
-    const bool word_rows = (n & 31) == 0;                        // every row starts on a 32-bit word
 
     float acc[RW][TT];
 #pragma unroll
@@ -63,67 +58,26 @@ small_batch_kernel(const LayerArgs a, int32_t r)
 #pragma unroll
         for (int t = 0; t < TT; ++t) acc[rr][t] = 0.0f;
 
-    int32_t rows[RW];
+    for (int32_t e0 = lane * 8; e0 < n; e0 += 256) {
+        float xv[TT][8];
 #pragma unroll
-    for (int rr = 0; rr < RW; ++rr) rows[rr] = min(row0 + rr, r - 1);    // clamp: extra rows are not stored
-
-    for (int32_t e0 = lane * 32; e0 < n; e0 += 1024) {
-        // tile bits of this lane's 32 weights for each row (chunks past the end of the row are skipped below)
-        uint32_t nb[RW];
+        for (int t = 0; t < TT; ++t) {
+            if (t0 + t < a.T) {
+                XVec<XT>::load8(x + (t0 + t) * n + e0, xv[t]);
+            } else {
+#pragma unroll
+                for (int b = 0; b < 8; ++b) xv[t][b] = 0.0f;
+            }
+        }
 #pragma unroll
         for (int rr = 0; rr < RW; ++rr) {
-            const int64_t byte0 = (int64_t)rows[rr] * row_bytes + (e0 >> 3);
-            uint32_t w;
-            if (word_rows) {
-                w = __ldg(reinterpret_cast<const uint32_t *>(bits8 + byte0));
-            } else {
-                w = 0;
+            const int32_t row = min(row0 + rr, r - 1);            // clamp: extra rows are not stored
+            const uint32_t nb = ~(uint32_t)__ldg(bits + (int64_t)row * row_bytes + (e0 >> 3));
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if (e0 + 8 * c < n) w |= (uint32_t)__ldg(bits8 + byte0 + c) << (8 * c);
-            }
-            nb[rr] = ~w;
-        }
-        const bool full = e0 + 32 <= n;                          // n % 8 == 0: whole chunks of 8 only
-        if (TT == 1 && full) {
-            // all activation loads of the group first, then the arithmetic
-            float xv[4][8];
+            for (int b = 0; b < 8; ++b) {
+                const float sgn = __uint_as_float(0x3f800000u | ((nb << (31 - b)) & 0x80000000u));
 #pragma unroll
-            for (int c = 0; c < 4; ++c) XVec<XT>::load8(x + t0 * n + e0 + 8 * c, xv[c]);
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-#pragma unroll
-                for (int rr = 0; rr < RW; ++rr)
-#pragma unroll
-                    for (int b = 0; b < 8; ++b) {
-                        // bit 1 -> +1.0f, bit 0 -> -1.0f: the inverted bit goes into the sign position of 1.0f
-                        const float sgn = __uint_as_float(0x3f800000u | ((nb[rr] << (31 - 8 * c - b)) & 0x80000000u));
-                        acc[rr][0] = fmaf(sgn, xv[c][b], acc[rr][0]);
-                    }
-        } else {
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {                        // four chunks of 8 weights
-                const int32_t e = e0 + 8 * c;
-                if (!full && e >= n) break;
-                float xv[TT][8];
-#pragma unroll
-                for (int t = 0; t < TT; ++t) {
-                    if (t0 + t < a.T) {
-                        XVec<XT>::load8(x + (t0 + t) * n + e, xv[t]);
-                    } else {
-#pragma unroll
-                        for (int b = 0; b < 8; ++b) xv[t][b] = 0.0f;
-                    }
-                }
-#pragma unroll
-                for (int rr = 0; rr < RW; ++rr) {
-#pragma unroll
-                    for (int b = 0; b < 8; ++b) {
-                        const float sgn = __uint_as_float(0x3f800000u | ((nb[rr] << (31 - 8 * c - b)) & 0x80000000u));
-#pragma unroll
-                        for (int t = 0; t < TT; ++t) acc[rr][t] = fmaf(sgn, xv[t][b], acc[rr][t]);
-                    }
-                }
+                for (int t = 0; t < TT; ++t) acc[rr][t] = fmaf(sgn, xv[t][b], acc[rr][t]);
             }
         }
     }
@@ -191,11 +145,63 @@ __device__ __forceinline__ uint32_t sign_pair(uint32_t v, int p)
 
 constexpr int kMmaMaxWarps = 32;
 
+// What lane (g, c) holds of one span: a word of bits for rows g and g + 8, and 32 activations per token tile.
+template <int NT> struct SpanRegs {
+    uint32_t w_lo, w_hi;
+    uint4 xb[NT][4];
+};
+
 template <int NT>
-__global__ void __launch_bounds__(kMmaMaxWarps * 32)
+__device__ __forceinline__ void load_span(SpanRegs<NT> &sr, const uint32_t *bits_lo, const uint32_t *bits_hi,
+                                          const __nv_bfloat16 *x, int32_t n, int32_t n_chunks, int32_t span,
+                                          int c, int g, int64_t t0, int64_t T)
+{
+    const int32_t chunk = span * 4 + c;
+    const bool live = chunk < n_chunks;                          // ragged last span: activations read as zero
+    const int32_t ch = live ? chunk : 0;
+    sr.w_lo = __ldg(bits_lo + ch);
+    sr.w_hi = __ldg(bits_hi + ch);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        const int64_t t = t0 + nt * 8 + g;
+        if (live && t < T) {
+            const uint4 *px = reinterpret_cast<const uint4 *>(x + t * n + (int64_t)ch * 32);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) sr.xb[nt][i] = __ldg(px + i);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) sr.xb[nt][i] = make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+}
+
+template <int NT>
+__device__ __forceinline__ void contract_span(const SpanRegs<NT> &sr, float (&acc)[NT][4])
+{
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {                       // 16 bits of each row word at a time
+        const uint32_t v_lo = spread16(half ? sr.w_lo >> 16 : sr.w_lo & 0xffffu);
+        const uint32_t v_hi = spread16(half ? sr.w_hi >> 16 : sr.w_hi & 0xffffu);
+#pragma unroll
+        for (int uu = 0; uu < 4; ++uu) {                         // MMA u = 4 * half + uu: weights 4u..4u+3 of the chunk
+            const uint32_t a0 = sign_pair(v_lo, 2 * uu), a2 = sign_pair(v_lo, 2 * uu + 1);
+            const uint32_t a1 = sign_pair(v_hi, 2 * uu), a3 = sign_pair(v_hi, 2 * uu + 1);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                const uint4 q = sr.xb[nt][half * 2 + (uu >> 1)];
+                const uint32_t b0 = (uu & 1) ? q.z : q.x, b1 = (uu & 1) ? q.w : q.y;
+                mma_bf16_16x8x16(acc[nt], a0, a1, a2, a3, b0, b1);
+            }
+        }
+    }
+}
+
+template <int NT>
+__global__ void __launch_bounds__(kMmaMaxWarps / NT * 32, 1)
 small_mma_kernel(const LayerArgs a, int32_t r)
 {
-    __shared__ float red[kMmaMaxWarps / NT][NT][16][8];          // [warp][token tile][row][token]: <= 16 KB
+    __shared__ float red[kMmaMaxWarps / NT][NT][16][8];          // [warp][token tile][row][token]: 16 KB
+    __shared__ float alpha_s[64];
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -206,11 +212,14 @@ small_mma_kernel(const LayerArgs a, int32_t r)
     const int32_t n = a.n;
     const int32_t n_chunks = n >> 5;                             // n % 32 == 0
     const int32_t n_spans = (n_chunks + 3) >> 2;
+    const bool per_tile = a.alpha_mode == TBN_ALPHA_PER_TILE;
 
-    const uint32_t *bits = a.tile;
+    // the scales are needed only at the very end: fetch them now, off the critical path
+    if ((int)threadIdx.x < min(a.k, 64)) alpha_s[threadIdx.x] = __ldg(a.alpha + (per_tile ? threadIdx.x : 0));
+
     const int32_t row_words = n >> 5;
-    const uint32_t *bits_lo = bits + (int64_t)min(row0 + g, r - 1) * row_words;       // clamped rows are not stored
-    const uint32_t *bits_hi = bits + (int64_t)min(row0 + g + 8, r - 1) * row_words;
+    const uint32_t *bits_lo = a.tile + (int64_t)min(row0 + g, r - 1) * row_words;     // clamped rows are not stored
+    const uint32_t *bits_hi = a.tile + (int64_t)min(row0 + g + 8, r - 1) * row_words;
     const __nv_bfloat16 *x = static_cast<const __nv_bfloat16 *>(a.x);
 
     float acc[NT][4];
@@ -219,41 +228,19 @@ small_mma_kernel(const LayerArgs a, int32_t r)
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[nt][i] = 0.0f;
 
-    for (int32_t span = warp; span < n_spans; span += nw) {
-        const int32_t chunk = span * 4 + c;
-        const bool live = chunk < n_chunks;                      // ragged last span: activations read as zero
-        const int32_t ch = live ? chunk : 0;
-        const uint32_t w_lo = __ldg(bits_lo + ch);
-        const uint32_t w_hi = __ldg(bits_hi + ch);
-        uint4 xb[NT][4];
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            const int64_t t = t0 + nt * 8 + g;
-            if (live && t < a.T) {
-                const uint4 *px = reinterpret_cast<const uint4 *>(x + t * n + (int64_t)ch * 32);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) xb[nt][i] = __ldg(px + i);
-            } else {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) xb[nt][i] = make_uint4(0u, 0u, 0u, 0u);
-            }
-        }
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {                   // 16 bits of each row word at a time
-            const uint32_t v_lo = spread16(half ? w_lo >> 16 : w_lo & 0xffffu);
-            const uint32_t v_hi = spread16(half ? w_hi >> 16 : w_hi & 0xffffu);
-#pragma unroll
-            for (int uu = 0; uu < 4; ++uu) {                     // MMA u = 4 * half + uu: weights 4u..4u+3 of the chunk
-                const uint32_t a0 = sign_pair(v_lo, 2 * uu), a2 = sign_pair(v_lo, 2 * uu + 1);
-                const uint32_t a1 = sign_pair(v_hi, 2 * uu), a3 = sign_pair(v_hi, 2 * uu + 1);
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    const uint4 q = xb[nt][half * 2 + (uu >> 1)];
-                    const uint32_t b0 = (uu & 1) ? q.z : q.x, b1 = (uu & 1) ? q.w : q.y;
-                    mma_bf16_16x8x16(acc[nt], a0, a1, a2, a3, b0, b1);
-                }
-            }
-        }
+    // two spans in flight: the loads of both are issued before either is contracted
+    int32_t span = warp;
+    for (; span + nw < n_spans; span += 2 * nw) {
+        SpanRegs<NT> s0, s1;
+        load_span<NT>(s0, bits_lo, bits_hi, x, n, n_chunks, span, c, g, t0, a.T);
+        load_span<NT>(s1, bits_lo, bits_hi, x, n, n_chunks, span + nw, c, g, t0, a.T);
+        contract_span<NT>(s0, acc);
+        contract_span<NT>(s1, acc);
+    }
+    if (span < n_spans) {
+        SpanRegs<NT> s0;
+        load_span<NT>(s0, bits_lo, bits_hi, x, n, n_chunks, span, c, g, t0, a.T);
+        contract_span<NT>(s0, acc);
     }
 
     // accumulator fragment: [0],[1] = row g, tokens 2c, 2c+1; [2],[3] = row g + 8
@@ -264,17 +251,17 @@ small_mma_kernel(const LayerArgs a, int32_t r)
     }
     __syncthreads();
 
-    const bool per_tile = a.alpha_mode == TBN_ALPHA_PER_TILE;
     for (int e = threadIdx.x; e < NT * 8 * 16; e += blockDim.x) {
         const int row = e & 15, tok = e >> 4;                    // rows fastest: 16 neighbouring outputs per token
         const int32_t grow = row0 + row;
         const int64_t t = t0 + tok;
         if (grow >= r || t >= a.T) continue;
-        float z = 0.0f;
+        float z = 0.0f;                                          // warps are summed in warp order: deterministic
+#pragma unroll 8
         for (int w = 0; w < nw; ++w) z += red[w][tok >> 3][row][tok & 7];
         for (int32_t j = 0; j < a.k; ++j) {
             const int32_t o = j * r + grow;
-            const float al = per_tile ? __ldg(a.alpha + j) : __ldg(a.alpha);
+            const float al = j < 64 ? alpha_s[j] : __ldg(a.alpha + (per_tile ? j : 0));
             const float v = apply_act(fmaf(al, z, a.bias ? __ldg(a.bias + o) : 0.0f), a.act);
             const int64_t yi = t * a.m + o;
             if (a.y_dtype == TBN_BF16) store_from_float(static_cast<__nv_bfloat16 *>(a.y), yi, v);
@@ -323,9 +310,8 @@ template <typename XT>
 cudaError_t launch_rw(const LayerArgs &a, int32_t r, cudaStream_t s)
 {
     // more rows per warp reuse each activation load more often, but small layers need the blocks
-    // enough warps per SM to hide load latency first (>= ~32), activation reuse second
-    if (r >= 148 * 32 * 4) return launch_tt<XT, 4>(a, r, s);
-    if (r >= 148 * 32 * 2) return launch_tt<XT, 2>(a, r, s);
+    if (r >= 148 * 4 * kWarps * 4) return launch_tt<XT, 4>(a, r, s);
+    if (r >= 148 * 2 * kWarps * 2) return launch_tt<XT, 2>(a, r, s);
     return launch_tt<XT, 1>(a, r, s);
 }
 
