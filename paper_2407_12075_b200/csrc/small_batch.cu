@@ -197,7 +197,7 @@ __device__ __forceinline__ void contract_span(const SpanRegs<NT> &sr, float (&ac
 }
 
 template <int NT>
-__global__ void __launch_bounds__(kMmaMaxWarps / NT * 32, 1)
+__global__ void __launch_bounds__(kMmaMaxWarps / NT * 32, NT)
 small_mma_kernel(const LayerArgs a, int32_t r)
 {
     __shared__ float red[kMmaMaxWarps / NT][NT][16][8];          // [warp][token tile][row][token]: 16 KB
@@ -228,19 +228,10 @@ small_mma_kernel(const LayerArgs a, int32_t r)
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[nt][i] = 0.0f;
 
-    // two spans in flight: the loads of both are issued before either is contracted
-    int32_t span = warp;
-    for (; span + nw < n_spans; span += 2 * nw) {
-        SpanRegs<NT> s0, s1;
-        load_span<NT>(s0, bits_lo, bits_hi, x, n, n_chunks, span, c, g, t0, a.T);
-        load_span<NT>(s1, bits_lo, bits_hi, x, n, n_chunks, span + nw, c, g, t0, a.T);
-        contract_span<NT>(s0, acc);
-        contract_span<NT>(s1, acc);
-    }
-    if (span < n_spans) {
-        SpanRegs<NT> s0;
-        load_span<NT>(s0, bits_lo, bits_hi, x, n, n_chunks, span, c, g, t0, a.T);
-        contract_span<NT>(s0, acc);
+    for (int32_t span = warp; span < n_spans; span += nw) {
+        SpanRegs<NT> sr;
+        load_span<NT>(sr, bits_lo, bits_hi, x, n, n_chunks, span, c, g, t0, a.T);
+        contract_span<NT>(sr, acc);
     }
 
     // accumulator fragment: [0],[1] = row g, tokens 2c, 2c+1; [2],[3] = row g + 8
