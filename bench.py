@@ -50,10 +50,10 @@ def algorithmic_bytes(T: int, k: int) -> float:
 
 
 # DRAM traffic of the dominant launch (k = 2) from the ncu capture summarised in
-# profiles/tc_linear_k2_T8192_ncu_full.md: 236.0 MB at T = 8192; traffic is proportional to T.  The figure is
+# profiles/tc_linear_k2_T8192_ncu_full.md: 237.3 MB at T = 8192; traffic is proportional to T.  The figure is
 # only valid for the kernel source it was taken from: the hash below covers tc_linear.cu and tc_common.cuh.
-TRAFFIC_BYTES_AT_T8192 = 138.769408e6 + 97.274112e6
-TRAFFIC_SOURCE_HASH = "871e18df3dabc52d"
+TRAFFIC_BYTES_AT_T8192 = 138.498816e6 + 98.804480e6
+TRAFFIC_SOURCE_HASH = "e64c513cd4086e82"
 
 
 def measured_traffic(T: int):
