@@ -59,13 +59,13 @@ int select_linear_path(const LayerArgs &a)
 {
     const bool tensor = tensor_path_supported(a), small = small_batch_supported(a);
     if (tensor && small) {
-        // Measured on B200: the small-batch kernel sustains about 8.5e6 multiply-adds per microsecond on top of
-        // ~5 us; one CTA of the tensor-core kernel walks the whole contraction (about 0.65 us per 128 inputs)
-        // whatever the batch, plus ~5 us of launch, set-up and epilogue.
+        // Both estimates are fits to launch-to-launch times measured on B200.  With few tokens the tensor-core
+        // kernel is bound by decoding the tile (about 2 ns per input feature and CTA, split-K included) until
+        // the output tiles outnumber the SMs.
         const double r = (double)(a.q / a.n);
-        const double small_us = 5.0 + (double)a.T * r * (double)a.n / 8.5e6;
-        const double waves = (double)(((a.T + 255) / 256) * (((int64_t)r + 127) / 128) + 147) / 148;
-        const double tensor_us = 5.0 + (double)((int64_t)waves) * ((double)a.n / 128.0) * 0.65;
+        const double small_us = small_batch_estimate_us(a);
+        const double fill = (double)a.T * r / (64.0 * 4096.0) * 0.75;
+        const double tensor_us = 6.0 + 0.002 * (double)a.n * (fill > 1.0 ? fill : 1.0);
         return small_us < tensor_us ? TBN_PATH_SMALL : TBN_PATH_TENSOR;
     }
     if (tensor) return TBN_PATH_TENSOR;

@@ -78,6 +78,7 @@ cudaError_t launch_generic(const LayerArgs &a, cudaStream_t s);
 
 bool small_batch_supported(const LayerArgs &a);
 cudaError_t launch_small_batch(const LayerArgs &a, cudaStream_t s);
+double small_batch_estimate_us(const LayerArgs &a);
 
 // The tensor-core path reports through a tbn_status because it also uses the driver API.
 bool tensor_path_supported(const LayerArgs &a);

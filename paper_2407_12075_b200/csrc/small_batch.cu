@@ -176,7 +176,7 @@ __device__ __forceinline__ void load_span(SpanRegs<NT> &sr, const uint32_t *bits
 }
 
 template <int NT>
-__device__ __forceinline__ void contract_span(const SpanRegs<NT> &sr, float (&acc)[NT][4])
+__device__ __forceinline__ void contract_span(const SpanRegs<NT> &sr, float (&acc)[NT == 1 ? 2 : NT][4])
 {
 #pragma unroll
     for (int half = 0; half < 2; ++half) {                       // 16 bits of each row word at a time
@@ -190,14 +190,15 @@ __device__ __forceinline__ void contract_span(const SpanRegs<NT> &sr, float (&ac
             for (int nt = 0; nt < NT; ++nt) {
                 const uint4 q = sr.xb[nt][half * 2 + (uu >> 1)];
                 const uint32_t b0 = (uu & 1) ? q.z : q.x, b1 = (uu & 1) ? q.w : q.y;
-                mma_bf16_16x8x16(acc[nt], a0, a1, a2, a3, b0, b1);
+                // a single token tile alternates between two accumulators: two independent MMA chains
+                mma_bf16_16x8x16(acc[NT == 1 ? (uu & 1) : nt], a0, a1, a2, a3, b0, b1);
             }
         }
     }
 }
 
 template <int NT>
-__global__ void __launch_bounds__(kMmaMaxWarps / NT * 32, NT)
+__global__ void __launch_bounds__(kMmaMaxWarps / NT * 32, NT == 4 ? 2 : NT)
 small_mma_kernel(const LayerArgs a, int32_t r)
 {
     __shared__ float red[kMmaMaxWarps / NT][NT][16][8];          // [warp][token tile][row][token]: 16 KB
@@ -222,9 +223,9 @@ small_mma_kernel(const LayerArgs a, int32_t r)
     const uint32_t *bits_hi = a.tile + (int64_t)min(row0 + g + 8, r - 1) * row_words;
     const __nv_bfloat16 *x = static_cast<const __nv_bfloat16 *>(a.x);
 
-    float acc[NT][4];
+    float acc[NT == 1 ? 2 : NT][4];
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
+    for (int nt = 0; nt < (NT == 1 ? 2 : NT); ++nt)
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[nt][i] = 0.0f;
 
@@ -234,6 +235,10 @@ small_mma_kernel(const LayerArgs a, int32_t r)
         contract_span<NT>(sr, acc);
     }
 
+    if (NT == 1) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[0][i] += acc[1][i];
+    }
     // accumulator fragment: [0],[1] = row g, tokens 2c, 2c+1; [2],[3] = row g + 8
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
@@ -315,6 +320,21 @@ bool small_batch_supported(const LayerArgs &a)
     if (a.n % 8 != 0) return false;            // 16-byte activation vectors, byte-aligned bit rows
     if (a.T > 65535 * 4) return false;
     return true;
+}
+
+// Launch-to-launch time in microseconds, fitted to measurements on B200 (in = 768 .. 8192, k = 2 .. 16).
+double small_batch_estimate_us(const LayerArgs &a)
+{
+    const double r = (double)(a.q / a.n);
+    if (!small_mma_supported(a))                                 // FMA kernel: ~8.5e6 multiply-adds per microsecond
+        return 5.0 + (double)a.T * r * (double)a.n / 8.5e6;
+    // MMA kernel: a block (16 rows x 8*NT tokens) costs c(NT) us per 1e6 weights of a full 148-SM wave; the
+    // legacy warp-level MMA rate, not memory, sets c for NT = 4
+    const int nt = a.T <= 8 ? 1 : a.T <= 16 ? 2 : 4;
+    const double c = nt == 1 ? 0.19 : nt == 2 ? 0.33 : 0.64;
+    const double blocks = (double)((int64_t)((r + 15) / 16) * ((a.T + 8 * nt - 1) / (8 * nt)));
+    const double per_block = c * 16.0 * (double)a.n * 148.0 / 1e6;
+    return 2.5 + per_block * (blocks > 148.0 ? blocks / 148.0 : 1.0) + 0.06 * a.k;
 }
 
 cudaError_t launch_small_batch(const LayerArgs &a, cudaStream_t s)
