@@ -563,8 +563,10 @@ int launch_config(const LayerArgs &a, TcParams p, int splits, void *scratch, cud
 // When the output has fewer tiles than the GPU has SMs, the contraction is split over several CTAs per tile
 // (each dumps an fp32 partial tile; the last to arrive adds them in a fixed order and stores).
 struct Cand { int ntok, na, ka, db; };
-constexpr Cand kCands[] = {{256, 1, 2, 1}, {192, 1, 2, 2}, {128, 2, 2, 1}, {128, 1, 2, 2}, {64, 1, 2, 2}, {32, 1, 2, 2}};
-constexpr int kNumCands = 6;
+// 224 tokens: 74 token tiles at T = 16384, so 4 or 8 row blocks give an exact multiple of 148 CTAs
+constexpr Cand kCands[] = {{256, 1, 2, 1}, {192, 1, 2, 2}, {128, 2, 2, 1}, {128, 1, 2, 2}, {64, 1, 2, 2}, {32, 1, 2, 2},
+                           {224, 1, 2, 1}};
+constexpr int kNumCands = 7;
 
 struct Plan { int cand, splits; size_t scratch_bytes; };
 
@@ -654,6 +656,7 @@ int launch_tensor_linear(const LayerArgs &a, int *device_status, void *scratch, 
     case 2: return launch_config<128, 2, 2, 5, 1>(a, p, plan.splits, scratch, s);
     case 3: return launch_config<128, 1, 2, 6, 2>(a, p, plan.splits, scratch, s);
     case 4: return launch_config<64, 1, 2, 8, 2>(a, p, plan.splits, scratch, s);
+    case 6: return launch_config<224, 1, 2, 3, 1>(a, p, plan.splits, scratch, s);
     default: return launch_config<32, 1, 2, 8, 2>(a, p, plan.splits, scratch, s);
     }
 }

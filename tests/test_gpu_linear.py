@@ -39,7 +39,7 @@ ALIGNED = [(m, n, k) for (m, n, k) in ZOO if (m * n // k) % n == 0 and n % 8 == 
 
 
 @pytest.mark.parametrize("m,n,k", ALIGNED + [(2048, 1024, 8), (64, 8200, 2)])
-@pytest.mark.parametrize("T", [1, 2, 3, 5, 17])
+@pytest.mark.parametrize("T", [1, 2, 3, 5, 12, 17, 40, 70])
 def test_small_batch_path_matches_oracle(m, n, k, T):
     for per_tile in (False, True):
         for x_bf16 in (False, True):
@@ -131,6 +131,19 @@ def test_tensor_path_fp32_activations_bias_fp32_out():
     ref = O.linear(x, words, k, al, True, m, n, bias=bias.astype(np.float64), act=O.ACT_GELU)
     got = run(B.PATH_TENSOR, x, words, al, True, m, k, act=B.ACT_GELU, bias=bias, y_dtype=B.F32)
     assert_close(got, ref, "tensor fp32 in/out")
+
+
+@pytest.mark.parametrize("cand", range(7))
+def test_tensor_path_every_tile_shape(cand, monkeypatch):
+    # the planner picks one token-tile shape per call; the tuning variable pins each of them in turn on a case
+    # with several token tiles, a ragged token tail and a ragged row block
+    monkeypatch.setenv("TBN_TC_CONFIG", str(cand))
+    m, n, k, T = 1200, 1000, 4, 777
+    x, W, words, al = make_linear_case(21, T, m, n, k, True, True)
+    ref = O.linear(x, words, k, al, True, m, n)
+    got = run(B.PATH_TENSOR, x, words, al, True, m, k)
+    assert_close(got, ref, f"tensor tile shape {cand}")
+    assert B.tbn_last_device_status() == (0, 0)
 
 
 @pytest.mark.parametrize("k", [2, 16])
