@@ -154,15 +154,13 @@ template <int NT> struct SpanRegs {
 template <int NT>
 __device__ __forceinline__ void load_span(SpanRegs<NT> &sr, const uint32_t *bits_lo, const uint32_t *bits_hi,
                                           const __nv_bfloat16 *x, int32_t n, int32_t n_chunks, int32_t span,
-                                          int c, int g, int64_t t0, int64_t T, bool with_bits)
+                                          int c, int g, int64_t t0, int64_t T)
 {
     const int32_t chunk = span * 4 + c;
     const bool live = chunk < n_chunks;                          // ragged last span: activations read as zero
     const int32_t ch = live ? chunk : 0;
-    if (with_bits) {
-        sr.w_lo = __ldg(bits_lo + ch);
-        sr.w_hi = __ldg(bits_hi + ch);
-    }
+    sr.w_lo = __ldg(bits_lo + ch);
+    sr.w_hi = __ldg(bits_hi + ch);
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
         const int64_t t = t0 + nt * 8 + g;
@@ -200,7 +198,7 @@ __device__ __forceinline__ void contract_span(const SpanRegs<NT> &sr, float (&ac
 }
 
 template <int NT>
-__global__ void __launch_bounds__(kMmaMaxWarps / NT * 32, 1)
+__global__ void __launch_bounds__(kMmaMaxWarps / NT * 32, NT == 4 ? 2 : NT)
 small_mma_kernel(const LayerArgs a, int32_t r)
 {
     __shared__ float red[kMmaMaxWarps / NT][NT][16][8];          // [warp][token tile][row][token]: 16 KB
@@ -231,27 +229,10 @@ small_mma_kernel(const LayerArgs a, int32_t r)
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[nt][i] = 0.0f;
 
-    // The tile bits are the only operand that comes from HBM: the words of four spans are requested before the
-    // first is used, which keeps (nearly) the whole tile in flight across the grid.
-    for (int32_t span0 = warp; span0 < n_spans; span0 += 4 * nw) {
-        uint32_t w_lo[4], w_hi[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int32_t chunk = (span0 + j * nw) * 4 + c;
-            const int32_t ch = chunk < n_chunks ? chunk : 0;
-            w_lo[j] = __ldg(bits_lo + ch);
-            w_hi[j] = __ldg(bits_hi + ch);
-        }
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int32_t span = span0 + j * nw;
-            if (span >= n_spans) break;                          // warp-uniform
-            SpanRegs<NT> sr;
-            sr.w_lo = w_lo[j];
-            sr.w_hi = w_hi[j];
-            load_span<NT>(sr, bits_lo, bits_hi, x, n, n_chunks, span, c, g, t0, a.T, false);
-            contract_span<NT>(sr, acc);
-        }
+    for (int32_t span = warp; span < n_spans; span += nw) {
+        SpanRegs<NT> sr;
+        load_span<NT>(sr, bits_lo, bits_hi, x, n, n_chunks, span, c, g, t0, a.T);
+        contract_span<NT>(sr, acc);
     }
 
     if (NT == 1) {
