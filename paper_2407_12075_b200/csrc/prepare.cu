@@ -158,6 +158,144 @@ aggregate_kernel(const float *__restrict__ W, const float *__restrict__ A, int64
     }
 }
 
+// Streaming form for k <= kAggStreamK: a fixed grid of blocks walks the column chunks (chunk = block, block + grid,
+// ...), so the per-block cost of publishing partial sums, the fence and the ticket is paid once per block instead of
+// once per 4096 columns, and a thread keeps its |.| sums per tile in fp64 registers across chunks.  Loads are
+// issued kAggRows rows x kAggIter groups at a time (8 independent 16-byte loads per thread and source) before the
+// sequential fp32 adds that the bit rule requires.
+constexpr int kAggStreamK = 16;
+constexpr int kAggRows = 2;
+
+template <bool VEC, bool HAS_A>
+__global__ void __launch_bounds__(kAggThreads, 2)
+aggregate_stream_kernel(const float *__restrict__ W, const float *__restrict__ A, int64_t q, int32_t k,
+                        int per_tile, uint32_t *__restrict__ tile_bits, int64_t n_words,
+                        float *__restrict__ alpha, AggScratch *scratch, int64_t n_chunks)
+{
+    __shared__ double warp_part[kAggStreamK][kAggThreads / 32];
+    __shared__ double red[kAggThreads];
+    __shared__ unsigned int s_ticket;
+
+    const int tid = threadIdx.x;
+    const int lane = tid & 31, warp = tid >> 5;
+    double *partial = reinterpret_cast<double *>(scratch + 1);
+    const unsigned int blocks = gridDim.x;
+
+    double acc[kAggStreamK];
+#pragma unroll
+    for (int j = 0; j < kAggStreamK; ++j) acc[j] = 0.0;
+
+    for (int64_t chunk = blockIdx.x; chunk < n_chunks; chunk += blocks) {
+        const int64_t base = chunk * kAggCols;
+        float s[kAggIter][kAggVec];
+#pragma unroll
+        for (int it = 0; it < kAggIter; ++it)
+#pragma unroll
+            for (int e = 0; e < kAggVec; ++e) s[it][e] = 0.0f;
+
+#pragma unroll
+        for (int j0 = 0; j0 < kAggStreamK; j0 += kAggRows) {
+            if (j0 >= k) break;                           // uniform
+            float w[kAggRows][kAggIter][kAggVec];
+            float av[HAS_A ? kAggRows : 1][kAggIter][kAggVec];
+#pragma unroll
+            for (int jj = 0; jj < kAggRows; ++jj) {
+                const bool row_ok = j0 + jj < k;
+                const int64_t row = (int64_t)(row_ok ? j0 + jj : 0) * q;
+#pragma unroll
+                for (int it = 0; it < kAggIter; ++it) {
+                    const int64_t c = base + ((int64_t)it * kAggThreads + tid) * kAggVec;
+                    if (VEC) {
+                        float4 t = make_float4(0.f, 0.f, 0.f, 0.f), u = t;
+                        if (row_ok && c < q) {            // q % 4 == 0: the whole group is in range
+                            t = __ldg(reinterpret_cast<const float4 *>(W + row + c));
+                            if (HAS_A) u = __ldg(reinterpret_cast<const float4 *>(A + row + c));
+                        }
+                        w[jj][it][0] = t.x; w[jj][it][1] = t.y; w[jj][it][2] = t.z; w[jj][it][3] = t.w;
+                        if (HAS_A) { av[jj][it][0] = u.x; av[jj][it][1] = u.y; av[jj][it][2] = u.z; av[jj][it][3] = u.w; }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < kAggVec; ++e) {
+                            const bool in = row_ok && c + e < q;
+                            w[jj][it][e] = in ? __ldg(W + row + c + e) : 0.0f;
+                            if (HAS_A) av[jj][it][e] = in ? __ldg(A + row + c + e) : 0.0f;
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int jj = 0; jj < kAggRows; ++jj) {
+                if (j0 + jj >= k) break;                  // uniform; a skipped row must not enter the fp32 sum
+                float ab = 0.0f;
+#pragma unroll
+                for (int it = 0; it < kAggIter; ++it)
+#pragma unroll
+                    for (int e = 0; e < kAggVec; ++e) {
+                        s[it][e] = __fadd_rn(s[it][e], w[jj][it][e]);      // never fused, never reassociated
+                        ab += fabsf(HAS_A ? av[HAS_A ? jj : 0][it][e] : w[jj][it][e]);
+                    }
+                acc[j0 + jj] += (double)ab;
+            }
+        }
+
+        // Eq. 3 + packing: a thread holds 4 consecutive columns (a nibble), 8 lanes make one 32-bit word.
+#pragma unroll
+        for (int it = 0; it < kAggIter; ++it) {
+            uint32_t nib = 0;
+#pragma unroll
+            for (int e = 0; e < kAggVec; ++e) nib |= (s[it][e] > 0.0f ? 1u : 0u) << e;   // NaN and +-0 give 0
+            uint32_t word = nib << (4 * (lane & 7));
+            word |= __shfl_xor_sync(0xffffffffu, word, 1);
+            word |= __shfl_xor_sync(0xffffffffu, word, 2);
+            word |= __shfl_xor_sync(0xffffffffu, word, 4);
+            const int64_t c0 = base + ((int64_t)it * kAggThreads + (tid & ~7)) * kAggVec;
+            const int64_t widx = c0 >> 5;
+            if ((lane & 7) == 0 && widx < n_words) tile_bits[widx] = word;
+        }
+    }
+
+    // one block-level reduction per tile, then publish
+#pragma unroll
+    for (int j = 0; j < kAggStreamK; ++j) {
+        if (j >= k) break;
+        double d = acc[j];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
+        if (lane == 0) warp_part[j][warp] = d;
+    }
+    __syncthreads();
+    if (tid < k) {
+        double t = 0.0;
+#pragma unroll
+        for (int w = 0; w < kAggThreads / 32; ++w) t += warp_part[tid][w];
+        partial[(int64_t)tid * blocks + blockIdx.x] = t;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_ticket = atomicAdd(&scratch->ticket, 1u);
+    __syncthreads();
+    if (s_ticket != blocks - 1) return;
+    __threadfence();
+
+    // last block: add the blocks' partial sums in a fixed order
+    const volatile double *vp = partial;
+    const int32_t groups = per_tile ? k : 1;
+    for (int32_t j = 0; j < groups; ++j) {
+        double t = 0.0;
+        const int64_t lo = per_tile ? (int64_t)j * blocks : 0;
+        const int64_t cnt = per_tile ? (int64_t)blocks : (int64_t)k * blocks;
+        for (int64_t b = tid; b < cnt; b += kAggThreads) t += vp[lo + b];
+        red[tid] = t;
+        __syncthreads();
+        for (int off = kAggThreads / 2; off > 0; off >>= 1) {
+            if (tid < off) red[tid] += red[tid + off];
+            __syncthreads();
+        }
+        if (tid == 0) alpha[j] = (float)(red[0] / ((double)q * (per_tile ? 1.0 : (double)k)));
+        __syncthreads();
+    }
+}
+
 __global__ void __launch_bounds__(256)
 pack_kernel(const float *__restrict__ src, int64_t q, uint32_t *__restrict__ tile_bits, int64_t n_words)
 {
@@ -245,6 +383,19 @@ cudaError_t launch_aggregate(const float *W, const float *A, int64_t N, int32_t 
     const int64_t blocks = (q + kAggCols - 1) / kAggCols;
     cudaError_t e = cudaMemsetAsync(workspace, 0, sizeof(AggScratch), s);
     if (e != cudaSuccess) return e;
+    if (k <= kAggStreamK) {
+        // fixed grid: two blocks per SM, never more blocks than chunks (the scratch is sized for one block per chunk)
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+            return cudaErrorUnknown;
+        const int64_t grid = blocks < 2 * (int64_t)sms ? blocks : 2 * (int64_t)sms;
+        auto kern = q % kAggVec == 0 ? (A ? aggregate_stream_kernel<true, true> : aggregate_stream_kernel<true, false>)
+                                     : (A ? aggregate_stream_kernel<false, true> : aggregate_stream_kernel<false, false>);
+        kern<<<(unsigned)grid, kAggThreads, 0, s>>>(W, A, q, k, per_tile, tile_bits, tbn_tile_words(q), alpha,
+                                                   static_cast<AggScratch *>(workspace), blocks);
+        return cudaGetLastError();
+    }
     if (q % kAggVec == 0)      // every repetition then starts on a 16-byte boundary (W and A are 16-byte aligned)
         aggregate_kernel<true><<<(unsigned)blocks, kAggThreads, 0, s>>>(
             W, A, q, k, per_tile, tile_bits, tbn_tile_words(q), alpha, static_cast<AggScratch *>(workspace));

@@ -14,6 +14,7 @@ pytestmark = pytest.mark.gpu
 CASES = [  # (N, k)
     (64, 1), (64, 2), (64, 8), (100352, 4), (1280, 1), (262144, 4), (2304 * 768, 8),
     (96 * 40, 6), (7 * 33, 3), (1024 * 4, 4), (1025 * 3, 3), (4097 * 2, 2), (73728, 4), (1 << 22, 16),
+    (33 * 4100, 33), (1 << 20, 32), (17 * 9001, 17), (5000 * 4096 * 2, 2),      # k above / below the streaming kernel's limit; several chunks per block
 ]
 
 
