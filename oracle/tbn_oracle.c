@@ -144,6 +144,19 @@ int tbn_oracle_expand(const uint32_t *words, int64_t N, int32_t p, const float *
 }
 
 /*
+ * Full-precision tiled weights (Sec. 5.2, the "FP, Tiled" kernel of Table 7): the same
+ * replication and reshaping as Eq. 4-5, but the tile holds real values and is used as it is,
+ * no threshold and no scaling factor:  B[f] = t[f mod q],  q = N / p.
+ */
+int tbn_oracle_expand_fp(const float *tile, int64_t N, int32_t p, float *B)
+{
+    if (p <= 0 || N < 0 || N % p != 0) return -1;
+    const int64_t q = N / p;
+    for (int64_t f = 0; f < N; ++f) B[f] = tile[f % q];
+    return 0;
+}
+
+/*
  * Fully-connected layer with an explicit (already expanded) weight:
  *   y[b][i] = act( sum_{j<n} B_hat[i][j] * x[b][j] + bias[i] ),  j increasing, fp64.
  * x: T x n row-major, B_hat: m x n row-major (out x in), y: T x m row-major.

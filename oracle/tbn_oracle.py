@@ -159,6 +159,34 @@ def linear(x, words, p, alphas, per_tile, m, n, bias=None, act=ACT_NONE):
     return linear_dense(x, B_hat, m, n, bias, act)
 
 
+def expand_fp(tile: np.ndarray, N: int, p: int) -> np.ndarray:
+    """Full-precision tiled weights (Sec. 5.2, Table 7 "FP, Tiled"): B[f] = t[f mod q], flat fp32."""
+    tile = np.ascontiguousarray(tile, dtype=np.float32)
+    out = np.empty(N, dtype=np.float32)
+    rc = _load().tbn_oracle_expand_fp(_p(tile), ctypes.c_int64(N), ctypes.c_int32(p), _p(out))
+    if rc != 0:
+        raise ValueError("p must divide N")
+    return out
+
+
+def linear_fp(x, tile, p, m, n, bias=None, act=ACT_NONE):
+    """Fully-connected layer whose weight is a real-valued tile repeated p times: expand, then the dense product."""
+    return linear_dense(x, expand_fp(tile, m * n, p), m, n, bias, act)
+
+
+def linear_fp_alg1(x, tile, p, m, n, relu=False):
+    """The index-walk form (Algorithm 1) applied to a real-valued tile, all scaling factors 1."""
+    q = m * n // p
+    xd = widen(x).reshape(-1, n)
+    T = xd.shape[0]
+    t = np.ascontiguousarray(tile, dtype=np.float32)
+    ones = np.ones(p, dtype=np.float32)
+    y = np.empty((T, m), dtype=np.float64)
+    _load().tbn_oracle_linear_alg1(_p(xd), ctypes.c_int64(T), ctypes.c_int32(n), ctypes.c_int32(m), _p(t),
+                                   ctypes.c_int64(q), _p(ones), ctypes.c_int(1 if relu else 0), _p(y))
+    return y
+
+
 def linear_alg1(x, words, p, alphas, per_tile, m, n, relu=False):
     """Algorithm 1: the index-walk form of the same layer."""
     q = m * n // p

@@ -372,6 +372,63 @@ def test_table7_parameter_memory_ratios():
     assert t7["FullPrecision"][0] / t7["FP_Tiled4"][0] == t7["FP_Tiled4"][1]
 
 
+# ----------------------------------------------------------------------------- full-precision tiles (Sec. 5.2)
+@pytest.mark.parametrize("m,n,p", [(6, 4, 3), (8, 8, 2), (7, 33, 3), (12, 16, 4), (5, 10, 1)])
+def test_fp_tile_expand_is_numpy_tile_and_definition(m, n, p):
+    q = m * n // p
+    t = synth.normal(7, 3, q, 0.5)
+    B = O.expand_fp(t, m * n, p)
+    assert np.array_equal(B, np.tile(t, p))                       # 1_p (x) t with a library routine
+    for f in (0, 1, q - 1, q % (m * n), m * n - 1):               # B[f] = t[f mod q], the definition
+        assert B[f] == t[f % q]
+    if p > 1:
+        with pytest.raises(ValueError):
+            O.expand_fp(t, m * n + 1, p)
+
+
+@pytest.mark.parametrize("T,m,n,p", [(3, 6, 4, 3), (5, 8, 8, 2), (2, 7, 33, 3), (4, 12, 16, 4)])
+def test_fp_tile_linear_matches_numpy_matmul_brute_force_and_alg1(T, m, n, p):
+    q = m * n // p
+    t = synth.normal(8, 3, q, 0.5)
+    x = synth.normal(8, 0, T * n).reshape(T, n)
+    bias = synth.normal(8, 200, m, 0.1).astype(np.float64)
+    y = O.linear_fp(x, t, p, m, n, bias=bias)
+    Wfull = np.tile(t.astype(np.float64), p).reshape(m, n)
+    assert np.allclose(y, x.astype(np.float64) @ Wfull.T + bias, rtol=1e-12, atol=1e-12)
+    brute = np.zeros((T, m))
+    for b in range(T):                                             # the definition, index by index
+        for i in range(m):
+            brute[b, i] = sum(float(t[(i * n + j) % q]) * float(x[b, j]) for j in range(n)) + bias[i]
+    assert np.allclose(y, brute, rtol=1e-12, atol=1e-12)
+    walk = O.linear_fp_alg1(x, t, p, m, n)                         # second, independently written routine
+    assert np.allclose(y - bias, walk, rtol=1e-12, atol=1e-12)
+
+
+def test_fp_tile_p1_is_an_ordinary_dense_layer_and_rows_repeat():
+    T, m, n = 4, 16, 24
+    W = synth.normal(9, 1, m * n, 0.3)
+    x = synth.normal(9, 0, T * n).reshape(T, n)
+    ref = torch.nn.functional.linear(torch.from_numpy(x).double(), torch.from_numpy(W).double().reshape(m, n)).numpy()
+    assert np.allclose(O.linear_fp(x, W, 1, m, n), ref, rtol=1e-12, atol=1e-12)
+    # a tile spanning whole rows: output row i + r repeats output row i (Sec. 4.1), with no scaling in between
+    p = 4
+    r = m // p
+    y = O.linear_fp(x, W[: m * n // p], p, m, n, act=O.ACT_RELU)
+    for j in range(1, p):
+        assert np.array_equal(y[:, :r], y[:, j * r:(j + 1) * r])
+
+
+def test_fp_tile_with_sign_values_equals_the_binary_layer():
+    # a real-valued tile holding +-alpha is the binary tile with one scaling factor
+    T, m, n, p = 3, 12, 20, 3
+    W = synth.normal(10, 1, m * n, 0.02)
+    x = synth.normal(10, 0, T * n).reshape(T, n)
+    words, al = O.prepare(W, p, False)
+    q = m * n // p
+    t = np.where(bits_of(words, q) > 0, al[0], -al[0]).astype(np.float32)
+    assert np.allclose(O.linear_fp(x, t, p, m, n), O.linear(x, words, p, al, False, m, n), rtol=1e-12, atol=1e-12)
+
+
 # ----------------------------------------------------------------------------- generator
 def test_generator_is_counter_based_and_calibrated():
     a = synth.normal(4, 0, 10000)
