@@ -141,6 +141,25 @@ int tbn_linear_fwd_path(const void *x, int x_dtype, int64_t T, int32_t in_f, int
 /* The family TBN_PATH_AUTO resolves to for this shape (a tbn_path), or a negative tbn_status. */
 int tbn_linear_select_path(int64_t T, int32_t in_f, int32_t out_f, int32_t k, int x_dtype);
 
+/*
+ * Full-precision tiled weights (Sec. 5.2: the "FP, Tiled" kernel measured in Table 7 and Fig. 6; named as future
+ * work for large models in Sec. 7).  The layer stores a tile of q = in_f*out_f/k REAL values; the weight matrix is
+ * the tile repeated k times and reshaped row-major exactly as in Eq. 4-5, with no threshold and no scaling factor:
+ *     y[t][i] = act( sum_j tile[(i*in_f + j) mod q] * x[t][j] + bias[i] ).
+ * tile_values: device, q elements of tile_dtype (TBN_F32 or TBN_BF16), 16-byte aligned, never written.
+ * When the tile spans whole rows (q % in_f == 0, in_f % 8 == 0) its q/in_f rows feed the tensor-core kernel
+ * directly as the weight operand (an fp32 tile is first rounded to bf16 into the workspace; a bf16 tile is read in
+ * place) and every row is written k times; other shapes run on the index-walk kernel with the tile's own precision.
+ * path: TBN_PATH_AUTO, TBN_PATH_GENERIC or TBN_PATH_TENSOR (TBN_PATH_SMALL decodes bits: TBN_ERR_UNSUPPORTED).
+ * workspace: tbn_linear_fp_tile_workspace_bytes(...) bytes.  Other arguments, ownership and errors as tbn_linear_fwd.
+ */
+size_t tbn_linear_fp_tile_workspace_bytes(int64_t T, int32_t in_f, int32_t out_f, int32_t k, int x_dtype,
+                                          int tile_dtype);
+int tbn_linear_fp_tile_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, int32_t out_f,
+                           const void *tile_values, int tile_dtype, int32_t k,
+                           const float *bias, int act, void *y, int y_dtype,
+                           void *workspace, size_t workspace_bytes, void *stream, int path);
+
 /* Same layer with HOST activations: x_host and y_host are host buffers (pinned memory recommended).
  * The call copies x to the device, runs tbn_linear_fwd, copies y back and synchronises `stream`.
  * workspace (device) must hold tbn_linear_host_workspace_bytes(...) bytes: staging for x and y plus

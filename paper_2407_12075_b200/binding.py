@@ -38,6 +38,9 @@ SIGNATURES = {
     "tbn_linear_fwd": (c_int, _LINEAR_ARGS),
     "tbn_linear_fwd_path": (c_int, _LINEAR_ARGS + [c_int]),
     "tbn_linear_select_path": (c_int, [c_i64, c_i32, c_i32, c_i32, c_int]),
+    "tbn_linear_fp_tile_workspace_bytes": (c_sz, [c_i64, c_i32, c_i32, c_i32, c_int, c_int]),
+    "tbn_linear_fp_tile_fwd": (c_int, [c_vp, c_int, c_i64, c_i32, c_i32, c_vp, c_int, c_i32, c_vp, c_int, c_vp, c_int,
+                                       c_vp, c_sz, c_vp, c_int]),
     "tbn_linear_host_workspace_bytes": (c_sz, [c_i64, c_i32, c_i32, c_i32, c_int, c_int]),
     "tbn_linear_fwd_host": (c_int, _LINEAR_ARGS),
     "tbn_conv2d_workspace_bytes": (c_sz, [c_i32] * 10 + [c_int]),
@@ -177,6 +180,28 @@ def tbn_linear_fwd(x: torch.Tensor, out_f: int, tile: torch.Tensor, k: int, alph
     _check(lib().tbn_linear_fwd_path(_ptr(x), xd, T, in_f, out_f, _ptr(tile), k, _ptr(alpha), alpha_mode,
                                      _ptr(bias), act, _ptr(y), yd, _ptr(ws), ws.numel(), _stream(), path),
            "tbn_linear_fwd")
+    return y
+
+
+def tbn_linear_fp_tile_workspace_bytes(T, in_f, out_f, k, x_dtype, tile_dtype) -> int:
+    return int(lib().tbn_linear_fp_tile_workspace_bytes(T, in_f, out_f, k, x_dtype, tile_dtype))
+
+
+def tbn_linear_fp_tile_fwd(x: torch.Tensor, out_f: int, tile_values: torch.Tensor, k: int,
+                           bias: torch.Tensor | None = None, act: int = ACT_NONE, y_dtype: int | None = None,
+                           path: int = PATH_AUTO, y: torch.Tensor | None = None,
+                           workspace: torch.Tensor | None = None) -> torch.Tensor:
+    """Layer whose weight is a real-valued tile (fp32 or bf16, q values) repeated k times."""
+    T, in_f = x.shape
+    xd, td = _dtype_code(x), _dtype_code(tile_values)
+    yd = xd if y_dtype is None else y_dtype
+    if y is None:
+        y = torch.empty((T, out_f), dtype=_torch_dtype(yd), device=x.device)
+    ws = workspace if workspace is not None else _ws(tbn_linear_fp_tile_workspace_bytes(T, in_f, out_f, k, xd, td),
+                                                     x.device)
+    _check(lib().tbn_linear_fp_tile_fwd(_ptr(x), xd, T, in_f, out_f, _ptr(tile_values), td, k, _ptr(bias), act,
+                                        _ptr(y), yd, _ptr(ws), ws.numel(), _stream(), path),
+           "tbn_linear_fp_tile_fwd")
     return y
 
 

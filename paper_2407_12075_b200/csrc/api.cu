@@ -317,6 +317,66 @@ int tbn_linear_select_path(int64_t T, int32_t in_f, int32_t out_f, int32_t k, in
     return select_linear_path(a);
 }
 
+size_t tbn_linear_fp_tile_workspace_bytes(int64_t T, int32_t in_f, int32_t out_f, int32_t k, int x_dtype,
+                                          int tile_dtype)
+{
+    if (T <= 0 || in_f <= 0 || out_f <= 0 || k <= 0 || ((int64_t)in_f * out_f) % k != 0) return 0;
+    const int64_t q = (int64_t)in_f * out_f / k;
+    // bf16 copy of an fp32 tile for the tensor-core kernel, then what the binary layer of this shape needs
+    const size_t rows = tile_dtype == TBN_F32 ? round_up((size_t)q * 2, 256) : 0;
+    return rows + tbn_linear_workspace_bytes(T, in_f, out_f, k, x_dtype);
+}
+
+int tbn_linear_fp_tile_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, int32_t out_f,
+                           const void *tile_values, int tile_dtype, int32_t k,
+                           const float *bias, int act, void *y, int y_dtype,
+                           void *workspace, size_t workspace_bytes, void *stream, int path)
+{
+    if (T < 0 || in_f <= 0 || out_f <= 0 || k <= 0 || !tile_values) return TBN_ERR_INVALID_ARG;
+    if (!valid_dtype(x_dtype) || !valid_dtype(y_dtype) || !valid_dtype(tile_dtype)) return TBN_ERR_INVALID_ARG;
+    if (act != TBN_ACT_NONE && act != TBN_ACT_RELU && act != TBN_ACT_GELU) return TBN_ERR_INVALID_ARG;
+    if (T > 0 && (!x || !y)) return TBN_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(y) || !aligned16(tile_values)) return TBN_ERR_INVALID_ARG;
+    if (bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) return TBN_ERR_INVALID_ARG;
+    const int64_t N = (int64_t)in_f * out_f;
+    if (N % k != 0) return TBN_ERR_SHAPE;
+    if (T == 0) return TBN_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    LayerArgs a;
+    std::memset(&a, 0, sizeof(a));
+    a.x = x; a.y = y; a.bias = bias;
+    a.T = T; a.n = in_f; a.m = out_f; a.k = k; a.q = N / k;
+    a.x_dtype = x_dtype; a.y_dtype = y_dtype; a.alpha_mode = TBN_ALPHA_PER_LAYER; a.act = act;
+    a.alpha = device_one_ptr();                      // no scaling factors: every repetition is scaled by 1
+    if (!a.alpha) return TBN_ERR_CUDA;
+
+    if (path == TBN_PATH_AUTO) path = tensor_path_supported(a) ? TBN_PATH_TENSOR : TBN_PATH_GENERIC;
+    if (path == TBN_PATH_GENERIC) {
+        a.fp_tile = tile_values; a.fp_tile_dtype = tile_dtype;
+        return launch_generic(a, s) == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+    }
+    if (path != TBN_PATH_TENSOR) return TBN_ERR_UNSUPPORTED;   // the bit-decoding small-batch kernels do not apply
+    if (!tensor_path_supported(a)) return TBN_ERR_UNSUPPORTED;
+
+    // the tile's r = q / in_f rows are the A operand of the tensor-core kernel as they are (rounded to bf16)
+    char *rest = static_cast<char *>(workspace);
+    size_t rest_bytes = workspace ? workspace_bytes : 0;
+    if (tile_dtype == TBN_F32) {
+        const size_t need = round_up((size_t)a.q * 2, 256);
+        if (!workspace || !aligned16(workspace) || workspace_bytes < need) return TBN_ERR_WORKSPACE;
+        if (launch_f32_to_bf16(static_cast<const float *>(tile_values), reinterpret_cast<__nv_bfloat16 *>(rest), a.q, s) !=
+            cudaSuccess)
+            return TBN_ERR_CUDA;
+        a.dense_a = rest;
+        rest += need;
+        rest_bytes -= need;
+    } else {
+        a.dense_a = tile_values;
+    }
+    return run_layer(a, TBN_PATH_TENSOR, rest_bytes ? rest : nullptr, rest_bytes, s);
+}
+
 int tbn_linear_fwd_path(const void *x, int x_dtype, int64_t T, int32_t in_f, int32_t out_f,
                         const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
                         const float *bias, int act, void *y, int y_dtype,

@@ -36,6 +36,8 @@ struct LayerArgs {
     void *y;
     const uint32_t *tile;
     const void *dense_a;   // tensor-core linear only: bf16 weight rows [q/n][n] used instead of the tile (MLP chain)
+    const void *fp_tile;   // full-precision tile (Sec. 5.2): q values used as they are instead of bits and alphas
+    int fp_tile_dtype;     // TBN_F32 or TBN_BF16
     const float *alpha;
     const float *bias;
     int64_t T;       // rows of the contraction: tokens, or Nb*Ho*Wo output pixels

@@ -60,8 +60,12 @@ generic_kernel(const LayerArgs a)
     int64_t idx = f0 % a.q;
     int64_t aidx = f0 / a.q;
     const bool per_tile = a.alpha_mode == TBN_ALPHA_PER_TILE;
-    float alpha_cur = per_tile ? __ldg(a.alpha + aidx) : __ldg(a.alpha);
-    uint32_t word = __ldg(a.tile + (idx >> 5));
+    // a full-precision tile is used as it is: the weight is t[idx] and every scaling factor is 1
+    const bool fp = a.fp_tile != nullptr;
+    const float *fp32_tile = static_cast<const float *>(a.fp_tile);
+    const __nv_bfloat16 *bf16_tile = static_cast<const __nv_bfloat16 *>(a.fp_tile);
+    float alpha_cur = fp ? 1.0f : per_tile ? __ldg(a.alpha + aidx) : __ldg(a.alpha);
+    uint32_t word = fp ? 0u : __ldg(a.tile + (idx >> 5));
 
     float seg[kTok], tot[kTok];
 #pragma unroll
@@ -80,11 +84,12 @@ generic_kernel(const LayerArgs a)
         if (!active) continue;
         const int kc = min(kKC, a.n - k0);
         for (int kk = 0; kk < kc; ++kk) {
-            const float sgn = ((word >> (uint32_t)(idx & 31)) & 1u) ? 1.0f : -1.0f;
+            const float sgn = fp ? (a.fp_tile_dtype == TBN_BF16 ? load_as_float(bf16_tile, idx) : __ldg(fp32_tile + idx))
+                                 : ((word >> (uint32_t)(idx & 31)) & 1u) ? 1.0f : -1.0f;
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
                 const float4 xv = *reinterpret_cast<const float4 *>(&xs[kk][(g ^ (kk & 3)) * 4]);
-                seg[g * 4 + 0] = fmaf(sgn, xv.x, seg[g * 4 + 0]);   // +-1 * x is exact
+                seg[g * 4 + 0] = fmaf(sgn, xv.x, seg[g * 4 + 0]);   // binary tile: +-1 * x is exact
                 seg[g * 4 + 1] = fmaf(sgn, xv.y, seg[g * 4 + 1]);
                 seg[g * 4 + 2] = fmaf(sgn, xv.z, seg[g * 4 + 2]);
                 seg[g * 4 + 3] = fmaf(sgn, xv.w, seg[g * 4 + 3]);
@@ -95,9 +100,9 @@ generic_kernel(const LayerArgs a)
                 for (int t = 0; t < kTok; ++t) { tot[t] = fmaf(alpha_cur, seg[t], tot[t]); seg[t] = 0.0f; }
                 idx = 0;
                 ++aidx;
-                if (per_tile && aidx < a.k) alpha_cur = __ldg(a.alpha + aidx);
-                word = __ldg(a.tile);
-            } else if ((idx & 31) == 0) {
+                if (!fp && per_tile && aidx < a.k) alpha_cur = __ldg(a.alpha + aidx);
+                if (!fp) word = __ldg(a.tile);
+            } else if (!fp && (idx & 31) == 0) {
                 word = __ldg(a.tile + (idx >> 5));
             }
         }
