@@ -150,6 +150,8 @@ int tbn_linear_select_path(int64_t T, int32_t in_f, int32_t out_f, int32_t k, in
  * When the tile spans whole rows (q % in_f == 0, in_f % 8 == 0) its q/in_f rows feed the tensor-core kernel
  * directly as the weight operand (an fp32 tile is first rounded to bf16 into the workspace; a bf16 tile is read in
  * place) and every row is written k times; other shapes run on the index-walk kernel with the tile's own precision.
+ * Rounding an fp32 tile to bf16 costs a relative weight error of 2^-9, i.e. about 1e-3 of the output's scale;
+ * TBN_PATH_GENERIC keeps fp32 weights exactly.
  * path: TBN_PATH_AUTO, TBN_PATH_GENERIC or TBN_PATH_TENSOR (TBN_PATH_SMALL decodes bits: TBN_ERR_UNSUPPORTED).
  * workspace: tbn_linear_fp_tile_workspace_bytes(...) bytes.  Other arguments, ownership and errors as tbn_linear_fwd.
  */

@@ -12,9 +12,12 @@ from tests.util import DEV, assert_close, to_dev, to_np64
 pytestmark = pytest.mark.gpu
 
 
-def case(seed, T, m, n, k, x_bf16=True, sigma=0.05):
+def case(seed, T, m, n, k, x_bf16=True, sigma=None):
+    # tile values ~ N(0, 1/n): outputs of unit scale, as with the fan-in scaled initialisation the paper trains with.
+    # The tensor-core kernel rounds an fp32 tile to bf16 (relative weight error 2^-9); with unit-scale outputs that
+    # adds about 2^-9 / sqrt(3) = 1e-3 rms to the output error, inside the layer tolerance.
     q = m * n // k
-    t = synth.normal(seed, 1, q, sigma)
+    t = synth.normal(seed, 1, q, sigma if sigma is not None else n ** -0.5)
     x = synth.normal(seed, 0, T * n).reshape(T, n)
     if x_bf16:
         x = synth.to_bf16_bits(x)
