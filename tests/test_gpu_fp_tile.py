@@ -85,7 +85,7 @@ def test_misaligned_tile_auto_falls_back_and_errors():
     with pytest.raises(B.TbnError):
         B.tbn_linear_fp_tile_fwd(to_dev(x), m, to_dev(t), k, path=B.PATH_SMALL)
     with pytest.raises(B.TbnError):
-        B.tbn_linear_fp_tile_fwd(to_dev(x), 8, to_dev(t), 3)              # k does not divide the weight count
+        B.tbn_linear_fp_tile_fwd(to_dev(x), 8, to_dev(t), 5)              # k does not divide the weight count
     empty = B.tbn_linear_fp_tile_fwd(torch.empty((0, n), dtype=torch.bfloat16, device=DEV), m, to_dev(t), k)
     assert empty.shape == (0, m)
 
