@@ -284,6 +284,30 @@ def measure_other_configs(B, torch, dev, peaks):
     for name, (n, m) in {"vit_qkv_768_2304": (768, 2304), "vit_out_768_768": (768, 768), "vit_fc1_768_3072": (768, 3072),
                          "vit_fc2_3072_768": (3072, 768)}.items():
         out[name] = linear_entry(25216, n, m, 8)
+    # derived: images/s over the tiled layers only (LayerNorm, attention and residual adds of the block, and the
+    # full-precision first convolution / classifier of the conv stack, are not tiled layers and are not run)
+    vit_us = sum(out[n]["us"] for n in ("vit_qkv_768_2304", "vit_out_768_768", "vit_fc1_768_3072", "vit_fc2_3072_768"))
+    out["vit_block_tiled_linears_only"] = dict(us=vit_us, images_per_s=128 / vit_us * 1e6, includes="qkv + out-proj + fc1 + fc2")
+    conv_us = out["conv_64_128_s2_32x32"]["us"] + out["conv_128_256_s2_16x16"]["us"]
+    out["conv_stack_tiled_convs_only"] = dict(us=conv_us, images_per_s=256 / conv_us * 1e6, includes="64->128 s2 + 128->256 s2")
+    # prepare step (once per layer, outside the forward): W fp32 read once, packed tile written
+    Wagg = torch.randn(N_FEAT * N_FEAT, device=dev, generator=gen) * 0.02
+    for k in (2, 16):
+        us = graph_us(lambda: B.tbn_aggregate_tile(Wagg, k, B.ALPHA_PER_TILE), reps=3, iters=3)
+        nbytes = 4.0 * Wagg.numel() + Wagg.numel() / k / 8
+        out[f"aggregate_8192x8192_k{k}"] = dict(us=us, alg_gbs=nbytes / us / 1e3, bound="hbm", frac_of_binding_roofline=nbytes / hbm * 1e6 / us)
+    del Wagg
+    # full-precision tiled weights (Sec. 5.2): ViT fc1-shaped layer, k = 4, bf16 tile read in place
+    T, n, m, k = 25216, 768, 3072, 4
+    x = torch.randn(T, n, device=dev, generator=gen).to(torch.bfloat16)
+    y = torch.empty(T, m, device=dev, dtype=torch.bfloat16)
+    tv = (torch.randn(n * m // k, device=dev, generator=gen) * 0.02).to(torch.bfloat16)
+    ws = torch.empty(max(B.tbn_linear_fp_tile_workspace_bytes(T, n, m, k, B.BF16, B.BF16), 16), dtype=torch.uint8, device=dev)
+    us = graph_us(lambda: B.tbn_linear_fp_tile_fwd(x, m, tv, k, act=B.ACT_GELU, y=y, workspace=ws))
+    flops, nbytes = 2.0 * T * (m // k) * n, (T * n + T * m) * 2 + tv.numel() * 2
+    out["fp_tile_vit_fc1_768_3072_k4"] = dict(us=us, alg_tflops=flops / us / 1e6, alg_gbs=nbytes / us / 1e3,
+                                              bound="tensor" if flops / tens > nbytes / hbm else "hbm",
+                                              frac_of_binding_roofline=max(flops / tens, nbytes / hbm) * 1e6 / us)
     for T in (1, 16, 256, 4096):
         for k in (2, 16):
             out[f"large_linear_T{T}_k{k}"] = linear_entry(T, N_FEAT, N_FEAT, k)
