@@ -454,22 +454,40 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                                                        : (p.per_tile ? __ldg(p.alpha + j) : __ldg(p.alpha));
                         const int64_t o0 = (int64_t)j * p.r + row0;
                         const int64_t yi = tok * p.m + o0;
-                        if (rows_valid == 32 && vec_ok && plain && p.y_bf16) {
-                            uint32_t pk[16];
+                        if (rows_valid == 32 && vec_ok) {
+                            // 32 consecutive output features of one token: scale (+ bias, activation), convert, and
+                            // store as 64 (bf16) or 128 (fp32) contiguous bytes
+                            float v[32];
+                            if (plain) {
 #pragma unroll
-                            for (int e = 0; e < 16; ++e) {
-                                const __nv_bfloat162 h = __floats2bfloat162_rn(al * z[2 * e], al * z[2 * e + 1]);
-                                pk[e] = *reinterpret_cast<const uint32_t *>(&h);
-                            }
-                            __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.y) + yi;
-                            if (wide_ok) {          // two full 32-byte sectors per thread
-                                st_global_v8(dst, pk);
-                                st_global_v8(dst + 16, pk + 8);
+                                for (int i = 0; i < 32; ++i) v[i] = al * z[i];
                             } else {
 #pragma unroll
-                                for (int g = 0; g < 4; ++g)
-                                    reinterpret_cast<uint4 *>(dst)[g] =
-                                        make_uint4(pk[4 * g], pk[4 * g + 1], pk[4 * g + 2], pk[4 * g + 3]);
+                                for (int i = 0; i < 32; ++i)
+                                    v[i] = apply_act(fmaf(al, z[i], p.bias ? __ldg(p.bias + o0 + i) : 0.0f), p.act);
+                            }
+                            if (p.y_bf16) {
+                                uint32_t pk[16];
+#pragma unroll
+                                for (int e = 0; e < 16; ++e) {
+                                    const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+                                    pk[e] = *reinterpret_cast<const uint32_t *>(&h);
+                                }
+                                __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.y) + yi;
+                                if (wide_ok) {          // two full 32-byte sectors per thread
+                                    st_global_v8(dst, pk);
+                                    st_global_v8(dst + 16, pk + 8);
+                                } else {
+#pragma unroll
+                                    for (int g = 0; g < 4; ++g)
+                                        reinterpret_cast<uint4 *>(dst)[g] =
+                                            make_uint4(pk[4 * g], pk[4 * g + 1], pk[4 * g + 2], pk[4 * g + 3]);
+                                }
+                            } else {
+                                float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(p.y) + yi);
+#pragma unroll
+                                for (int g = 0; g < 8; ++g)
+                                    dst[g] = make_float4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
                             }
                         } else {
                             for (int i = 0; i < rows_valid; ++i) {
