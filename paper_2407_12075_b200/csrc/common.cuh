@@ -19,9 +19,26 @@ __device__ __forceinline__ void store_from_float(__nv_bfloat16 *p, int64_t i, fl
     p[i] = __float2bfloat16_rn(v);
 }
 
+// GELU in its erf form, v * Phi(v) with Phi(v) = (1 + erf(v / sqrt 2)) / 2.  erfc(u), u >= 0, is evaluated branch-free
+// with the rational approximation 7.1.26 of Abramowitz & Stegun (absolute error below 1.5e-7, i.e. fp32 round-off):
+// erfc(u) = (a1 t + ... + a5 t^5) exp(-u^2), t = 1 / (1 + p u); Phi(v) = erfc(u)/2 for v < 0 and 1 - erfc(u)/2
+// otherwise, so the negative tail keeps its relative accuracy.  About a dozen instructions, two of them on the
+// special-function unit, against a divergent library erff: the activation runs in the epilogue warps of the
+// tensor-core kernels, where it would otherwise cost several times the contraction itself.
+__device__ __forceinline__ float gelu_erf(float v) {
+    const float u = fabsf(v) * 0.70710678118654752440f;
+    const float t = __fdividef(1.0f, fmaf(0.3275911f, u, 1.0f));
+    float poly = fmaf(1.061405429f, t, -1.453152027f);
+    poly = fmaf(poly, t, 1.421413741f);
+    poly = fmaf(poly, t, -0.284496736f);
+    poly = fmaf(poly, t, 0.254829592f);
+    const float half_erfc = 0.5f * poly * t * __expf(-u * u);
+    return v * (v < 0.0f ? half_erfc : 1.0f - half_erfc);
+}
+
 __device__ __forceinline__ float apply_act(float v, int act) {
     if (act == TBN_ACT_RELU) return fmaxf(v, 0.0f);
-    if (act == TBN_ACT_GELU) return 0.5f * v * (1.0f + erff(v * 0.70710678118654752440f));
+    if (act == TBN_ACT_GELU) return gelu_erf(v);
     return v;
 }
 

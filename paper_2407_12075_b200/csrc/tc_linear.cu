@@ -354,6 +354,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
         Pipe pd;                                          // accumulator buffer (stage) and its phase
         const bool vec_ok = (p.m % 8 == 0) && (p.r % 8 == 0);       // 16-byte aligned rows of 32 features
         const bool wide_ok = (p.m % 16 == 0) && (p.r % 16 == 0);    // 32-byte aligned: 256-bit stores
+        const bool bias_vec = (reinterpret_cast<uintptr_t>(p.bias) & 15) == 0;
         for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
             const int32_t split = tile % p.splits, out_tile = tile / p.splits;
             const int64_t tok0 = (int64_t)(out_tile / p.w_tiles) * NTOK;
@@ -462,9 +463,19 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
 #pragma unroll
                                 for (int i = 0; i < 32; ++i) v[i] = al * z[i];
                             } else {
+                                float b[32];
+                                if (p.bias != nullptr && bias_vec) {          // o0 is a multiple of 8 here
 #pragma unroll
-                                for (int i = 0; i < 32; ++i)
-                                    v[i] = apply_act(fmaf(al, z[i], p.bias ? __ldg(p.bias + o0 + i) : 0.0f), p.act);
+                                    for (int g = 0; g < 8; ++g) {
+                                        const float4 t = __ldg(reinterpret_cast<const float4 *>(p.bias + o0) + g);
+                                        b[4 * g] = t.x; b[4 * g + 1] = t.y; b[4 * g + 2] = t.z; b[4 * g + 3] = t.w;
+                                    }
+                                } else {
+#pragma unroll
+                                    for (int i = 0; i < 32; ++i) b[i] = p.bias ? __ldg(p.bias + o0 + i) : 0.0f;
+                                }
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) v[i] = apply_act(fmaf(al, z[i], b[i]), p.act);
                             }
                             if (p.y_bf16) {
                                 uint32_t pk[16];
