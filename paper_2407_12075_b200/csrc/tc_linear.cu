@@ -47,6 +47,17 @@ __device__ __forceinline__ void decode64(uint32_t b0, uint32_t b1, uint32_t (&v)
     decode16(b1 >> 16, v + 24);
 }
 
+constexpr int kXPitch = 132;             // floats per token row of the epilogue exchange buffer (128 + 4: 16-byte rows)
+
+// Named barrier 1 belongs to the four epilogue warps.
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// Same barrier, returning how many of the 128 threads passed `pred`.
+__device__ __forceinline__ int epi_bar_count(bool pred) {
+    int n;
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %1, 0;\nbar.red.popc.u32 %0, 1, 128, p;\n}" : "=r"(n) : "r"((int)pred) : "memory");
+    return n;
+}
+
 // ---- shared-memory control block -----------------------------------------------------------------
 template <int SX>
 struct Control {
@@ -56,7 +67,8 @@ struct Control {
     uint32_t tmem_base;
     int abort_flag;
     float alpha[kMaxAlpha];
-    uint32_t transpose[4][32 * 33];      // one padded 32 x 32 block per epilogue warp
+    unsigned int ticket;                 // split-K: this CTA's arrival number, broadcast to the epilogue warps
+    float exchange[32 * kXPitch];        // epilogue: one 32-token x 128-row block, [token][row], padded rows
 };
 
 struct TcParams {
@@ -343,23 +355,29 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
             }
         }
     } else {
-        // ---------------- epilogue: TMEM -> transpose -> alpha / bias / activation -> k replicated stores ------
-        // tcgen05.ld hands thread (quadrant qd, lane) one weight row and 32 consecutive tokens.  The output is
-        // row-major [token][feature], so each 32 x 32 block goes through a private padded shared-memory buffer
-        // and comes back with thread = token holding 32 consecutive output features: every repetition j is then
-        // one multiply per element (fp32), a pack to bf16 and four 16-byte stores per thread.
-        const int qd = warp & 3;
+        // ---------------- epilogue: TMEM -> exchange -> alpha / bias / activation -> k replicated stores ------
+        // tcgen05.ld hands thread (quadrant qd, lane) one weight row and 32 consecutive tokens, but the output is
+        // row-major [token][feature]: a store instruction whose lanes are 32 different tokens touches 32 separate
+        // lines and the load/store unit, not HBM, then bounds the epilogue.  So the four warps exchange each
+        // 128-row x 32-token block through one shared buffer [token][row] and come back with lane = 8 consecutive
+        // features of a token: a warp store covers 2 tokens x 256 contiguous bytes (bf16).  Every repetition j is
+        // then one multiply per element (fp32), a pack to bf16 and one 16-byte store per token.
+        const int qd = warp & 3;                          // tensor-memory lane quadrant this warp may read
+        const int ew = warp - 6;                          // this warp stores tokens 8*ew .. 8*ew+7 of each 32-token block
         const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
-        uint32_t *tbuf = ctl->transpose[warp - 6];
+        float (*xbuf)[kXPitch] = reinterpret_cast<float (*)[kXPitch]>(ctl->exchange);
         Pipe pd;                                          // accumulator buffer (stage) and its phase
-        const bool vec_ok = (p.m % 8 == 0) && (p.r % 8 == 0);       // 16-byte aligned rows of 32 features
-        const bool wide_ok = (p.m % 16 == 0) && (p.r % 16 == 0);    // 32-byte aligned: 256-bit stores
+        const bool vec_ok = (p.m % 8 == 0) && (p.r % 8 == 0);       // 16-byte aligned groups of 8 features
         const bool bias_vec = (reinterpret_cast<uintptr_t>(p.bias) & 15) == 0;
-        for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
+        const int f0 = 8 * (lane & 15);                   // first of this lane's 8 rows inside the 128-row block
+        const int tsub = lane >> 4;                       // this lane's tokens: 8*ew + tsub + 2*i, i < 4
+        const bool plain = p.bias == nullptr && (p.act == TBN_ACT_NONE || p.act == TBN_ACT_RELU);
+        for (int32_t tile = bid; tile < n_tiles; tile += gridDim.x) {
             const int32_t split = tile % p.splits, out_tile = tile / p.splits;
             const int64_t tok0 = (int64_t)(out_tile / p.w_tiles) * NTOK;
             ok = wait_bar(smem_u32(&ctl->d_full[pd.stage]), pd.phase, abort_flag, p.status, (6 << 24) | (bid & 0xffff));
-            if (!ok) break;
+            // the four warps go on together or not at all (they share named barrier 1 below)
+            if (epi_bar_count(ok) != 128) { ok = false; break; }
             tc_fence_after();
             const int n_chunks = (int)min((int64_t)(NTOK / 32), (p.T - tok0 + 31) / 32);
             // fp32 partial tile of (out_tile, split): [NA][128 rows][NTOK tokens]; this thread owns one row per block
@@ -383,20 +401,20 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                 }
                 tc_fence_before();
                 mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));           // accumulator fully read
-                // the warp that arrives last for this (output tile, lane quadrant) adds the partials and stores
+                // the CTA that arrives last for this output tile adds the partials and stores
                 __threadfence();
-                __syncwarp();
-                unsigned int old = 0;
-                if (lane == 0) old = atomicAdd(p.tickets + (int64_t)out_tile * 4 + qd, 1u);
-                old = __shfl_sync(0xffffffffu, old, 0);
+                epi_bar();
+                if (warp == 6 && lane == 0) ctl->ticket = atomicAdd(p.tickets + (int64_t)out_tile * 4, 1u);
+                epi_bar();
+                const unsigned int old = ctl->ticket;
                 if (old != (unsigned int)(p.splits - 1)) { pd.advance(DB); continue; }
                 __threadfence();
                 part_row -= (int64_t)split * kTileFloats;                  // row of split 0
             }
 #pragma unroll 1
             for (int a = 0; a < NA; ++a) {
-                const int32_t row0 = (out_tile % p.w_tiles) * (NA * 128) + a * 128 + qd * 32;
-                const int rows_valid = max(0, min(32, p.r - row0));
+                const int32_t blk0 = (out_tile % p.w_tiles) * (NA * 128) + a * 128;   // first distinct row of the block
+                const int rows_valid = max(0, min(128, p.r - blk0));
 #pragma unroll 1
                 for (int ch = 0; ch < n_chunks; ++ch) {
                     __syncwarp();                                 // reconverge before the warp-wide TMEM load
@@ -435,79 +453,84 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                             mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));
                         }
                     }
+                    epi_bar();                                    // the previous block has been read by everyone
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) tbuf[i * 33 + lane] = v[i];
-                    __syncwarp();
-                    float z[32];
+                    for (int i = 0; i < 32; ++i) xbuf[i][qd * 32 + lane] = __uint_as_float(v[i]);
+                    epi_bar();
+                    float z[4][8];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) z[i] = __uint_as_float(tbuf[lane * 33 + i]);
-                    __syncwarp();
-                    const int64_t tok = tok0 + ch * 32 + lane;
-                    if (tok >= p.T || rows_valid == 0) continue;
+                    for (int i = 0; i < 4; ++i) {
+                        const float4 lo = *reinterpret_cast<const float4 *>(&xbuf[8 * ew + tsub + 2 * i][f0]);
+                        const float4 hi = *reinterpret_cast<const float4 *>(&xbuf[8 * ew + tsub + 2 * i][f0 + 4]);
+                        z[i][0] = lo.x; z[i][1] = lo.y; z[i][2] = lo.z; z[i][3] = lo.w;
+                        z[i][4] = hi.x; z[i][5] = hi.y; z[i][6] = hi.z; z[i][7] = hi.w;
+                    }
+                    const int nvalid = rows_valid - f0;           // this lane's rows that exist
+                    if (nvalid <= 0) continue;
                     if (p.act == TBN_ACT_RELU && p.bias == nullptr) {
                         // alpha >= 0, so relu(alpha * z) = alpha * relu(z): clamp once, outside the k loop
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) z[i] = fmaxf(z[i], 0.0f);
+                        for (int i = 0; i < 4; ++i)
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) z[i][e] = fmaxf(z[i][e], 0.0f);
                     }
-                    const bool plain = p.bias == nullptr && (p.act == TBN_ACT_NONE || p.act == TBN_ACT_RELU);
+                    const int64_t tok_first = tok0 + ch * 32 + 8 * ew + tsub;
                     for (int32_t j = 0; j < p.k; ++j) {
                         const float al = j < kMaxAlpha ? ctl->alpha[j]
                                                        : (p.per_tile ? __ldg(p.alpha + j) : __ldg(p.alpha));
-                        const int64_t o0 = (int64_t)j * p.r + row0;
-                        const int64_t yi = tok * p.m + o0;
-                        if (rows_valid == 32 && vec_ok) {
-                            // 32 consecutive output features of one token: scale (+ bias, activation), convert, and
-                            // store as 64 (bf16) or 128 (fp32) contiguous bytes
-                            float v[32];
-                            if (plain) {
-#pragma unroll
-                                for (int i = 0; i < 32; ++i) v[i] = al * z[i];
-                            } else {
-                                float b[32];
+                        const int64_t o0 = (int64_t)j * p.r + blk0 + f0;
+                        if (vec_ok && nvalid >= 8) {
+                            float b[8];
+                            if (!plain) {
                                 if (p.bias != nullptr && bias_vec) {          // o0 is a multiple of 8 here
-#pragma unroll
-                                    for (int g = 0; g < 8; ++g) {
-                                        const float4 t = __ldg(reinterpret_cast<const float4 *>(p.bias + o0) + g);
-                                        b[4 * g] = t.x; b[4 * g + 1] = t.y; b[4 * g + 2] = t.z; b[4 * g + 3] = t.w;
-                                    }
+                                    const float4 t0 = __ldg(reinterpret_cast<const float4 *>(p.bias + o0));
+                                    const float4 t1 = __ldg(reinterpret_cast<const float4 *>(p.bias + o0) + 1);
+                                    b[0] = t0.x; b[1] = t0.y; b[2] = t0.z; b[3] = t0.w;
+                                    b[4] = t1.x; b[5] = t1.y; b[6] = t1.z; b[7] = t1.w;
                                 } else {
 #pragma unroll
-                                    for (int i = 0; i < 32; ++i) b[i] = p.bias ? __ldg(p.bias + o0 + i) : 0.0f;
+                                    for (int e = 0; e < 8; ++e) b[e] = p.bias ? __ldg(p.bias + o0 + e) : 0.0f;
                                 }
-#pragma unroll
-                                for (int i = 0; i < 32; ++i) v[i] = apply_act(fmaf(al, z[i], b[i]), p.act);
                             }
-                            if (p.y_bf16) {
-                                uint32_t pk[16];
 #pragma unroll
-                                for (int e = 0; e < 16; ++e) {
-                                    const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
-                                    pk[e] = *reinterpret_cast<const uint32_t *>(&h);
-                                }
-                                __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.y) + yi;
-                                if (wide_ok) {          // two full 32-byte sectors per thread
-                                    st_global_v8(dst, pk);
-                                    st_global_v8(dst + 16, pk + 8);
+                            for (int i = 0; i < 4; ++i) {
+                                const int64_t tok = tok_first + 2 * i;
+                                if (tok >= p.T) continue;
+                                float o[8];
+#pragma unroll
+                                for (int e = 0; e < 8; ++e)
+                                    o[e] = plain ? al * z[i][e] : apply_act(fmaf(al, z[i][e], b[e]), p.act);
+                                const int64_t yi = tok * p.m + o0;
+                                if (p.y_bf16) {
+                                    uint32_t pk[4];
+#pragma unroll
+                                    for (int e = 0; e < 4; ++e) {
+                                        const __nv_bfloat162 h = __floats2bfloat162_rn(o[2 * e], o[2 * e + 1]);
+                                        pk[e] = *reinterpret_cast<const uint32_t *>(&h);
+                                    }
+                                    *reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(p.y) + yi) =
+                                        make_uint4(pk[0], pk[1], pk[2], pk[3]);
                                 } else {
-#pragma unroll
-                                    for (int g = 0; g < 4; ++g)
-                                        reinterpret_cast<uint4 *>(dst)[g] =
-                                            make_uint4(pk[4 * g], pk[4 * g + 1], pk[4 * g + 2], pk[4 * g + 3]);
+                                    float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(p.y) + yi);
+                                    dst[0] = make_float4(o[0], o[1], o[2], o[3]);
+                                    dst[1] = make_float4(o[4], o[5], o[6], o[7]);
                                 }
-                            } else {
-                                float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(p.y) + yi);
-#pragma unroll
-                                for (int g = 0; g < 8; ++g)
-                                    dst[g] = make_float4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
                             }
                         } else {
-                            for (int i = 0; i < rows_valid; ++i) {
-                                // general path: own column of the transpose buffer (unclamped accumulator)
-                                const float zz = __uint_as_float(tbuf[lane * 33 + i]);
-                                const float b = p.bias ? __ldg(p.bias + o0 + i) : 0.0f;
-                                const float val = apply_act(fmaf(al, zz, b), p.act);
-                                if (p.y_bf16) static_cast<__nv_bfloat16 *>(p.y)[yi + i] = __float2bfloat16_rn(val);
-                                else static_cast<float *>(p.y)[yi + i] = val;
+                            // ragged or unaligned rows: element by element
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const int64_t tok = tok_first + 2 * i;
+                                if (tok >= p.T) continue;
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) {
+                                    if (e >= nvalid) break;
+                                    const float bb = p.bias ? __ldg(p.bias + o0 + e) : 0.0f;
+                                    const float val = apply_act(fmaf(al, z[i][e], bb), p.act);
+                                    const int64_t yi = tok * p.m + o0 + e;
+                                    if (p.y_bf16) static_cast<__nv_bfloat16 *>(p.y)[yi] = __float2bfloat16_rn(val);
+                                    else static_cast<float *>(p.y)[yi] = val;
+                                }
                             }
                         }
                     }
