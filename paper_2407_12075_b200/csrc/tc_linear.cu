@@ -18,6 +18,7 @@
 // bounded by a wall-clock limit, after which the CTA records TBN_ERR_TIMEOUT, drains and returns.
 #include <cstdlib>
 
+#include <cstddef>
 #include "tc_common.cuh"
 
 namespace tbn {
@@ -68,8 +69,10 @@ struct Control {
     int abort_flag;
     float alpha[kMaxAlpha];
     unsigned int ticket;                 // split-K: this CTA's arrival number, broadcast to the epilogue warps
-    float exchange[32 * kXPitch];        // epilogue: one 32-token x 128-row block, [token][row], padded rows
+    alignas(16) float exchange[32 * kXPitch];   // epilogue (read with 16-byte loads): one 32-token x 128-row block, [token][row], padded rows
 };
+
+static_assert(offsetof(Control<3>, exchange) % 16 == 0 && offsetof(Control<8>, exchange) % 16 == 0, "16-byte loads");
 
 struct TcParams {
     const uint32_t *tile;
