@@ -338,19 +338,22 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                         for (int i = 1; i <= kW; ++i) w[a][i] = __ldg(p.tile + min(wi + i, last_word));
                     }
                 }
+                // decode into registers BEFORE waiting for the tensor-memory stage: the ALU work then overlaps the
+                // MMAs that still read that stage, and only the stores sit between "stage free" and "stage full"
+                uint32_t v[NA][KA][32];
+#pragma unroll
+                for (int a = 0; a < NA; ++a)
+#pragma unroll
+                    for (int at = 0; at < KA; ++at) decode64(b[a][2 * at], b[a][2 * at + 1], v[a][at]);
                 ok = wait_bar(smem_u32(&ctl->a_empty[pa.stage]), pa.phase ^ 1u, abort_flag, p.status,
                               (5 << 24) | (pa.stage << 16) | (bid & 0xffff));
                 if (!ok) break;
                 tc_fence_after();
 #pragma unroll
-                for (int a = 0; a < NA; ++a) {
+                for (int a = 0; a < NA; ++a)
 #pragma unroll
-                    for (int at = 0; at < KA; ++at) {
-                        uint32_t v[32];
-                        decode64(b[a][2 * at], b[a][2 * at + 1], v);
-                        tmem_st_32x32(tmem_base + lane_base + kABase + pa.stage * kACols + (a * KA + at) * 32, v);
-                    }
-                }
+                    for (int at = 0; at < KA; ++at)
+                        tmem_st_32x32(tmem_base + lane_base + kABase + pa.stage * kACols + (a * KA + at) * 32, v[a][at]);
                 tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(smem_u32(&ctl->a_full[pa.stage]));
