@@ -273,8 +273,8 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                         const uint32_t b_lo = (b_base + tap_disp[t]) | lbo;
                         tc_mma_ts(d_addr, a_addr + t * 8, b_lo, desc_hi, idesc, t > 0 ? 1u : (uint32_t)(ks > 0));
                         if (t == 4)
-                            ready = mbar_try_wait(smem_u32(&ctl->x_full[nx.stage]), nx.phase) &&
-                                    mbar_try_wait(smem_u32(&ctl->a_full[na.stage]), na.phase);
+                            ready = mbar_test_wait(smem_u32(&ctl->x_full[nx.stage]), nx.phase) &&
+                                    mbar_test_wait(smem_u32(&ctl->a_full[na.stage]), na.phase);
                     }
                     tc_commit(smem_u32(&ctl->x_empty[px.stage]));
                     tc_commit(smem_u32(&ctl->a_empty[pa.stage]));

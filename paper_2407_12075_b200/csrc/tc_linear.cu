@@ -231,8 +231,8 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                                           b_lo + at * (kAtomBytes >> 4) + kk * 2, kDescHi, kIdesc,
                                           st > 0 ? 1u : (uint32_t)(ks > ks0));
                             if (st == kSteps / 2 - 1)
-                                ready = mbar_try_wait(smem_u32(&ctl->x_full[nx.stage]), nx.phase) &&
-                                        mbar_try_wait(smem_u32(&ctl->a_full[na.stage]), na.phase);
+                                ready = mbar_test_wait(smem_u32(&ctl->x_full[nx.stage]), nx.phase) &&
+                                        mbar_test_wait(smem_u32(&ctl->a_full[na.stage]), na.phase);
                         }
                     } else {                              // ragged last stage: only the K steps that hold data
                         const int steps = (rem + 15) >> 4;
