@@ -29,7 +29,7 @@ using namespace tc;
 
 constexpr int kThreads = 320;
 constexpr int kAtomK = 64;             // contraction elements per 128-byte swizzle row (one TMA box, 4 MMA K steps)
-constexpr int kAStages = 2;            // decoded-weight stages in tensor memory
+constexpr int kMaxAStages = 4;         // decoded-weight stages in tensor memory: 2, or 4 where the columns allow
 constexpr int kMaxAlpha = 64;          // alphas cached in shared memory
 
 // 16 tile bits (low half of h, upper half zero) -> 8 registers of two bf16 each: bit 2j in the low half,
@@ -63,7 +63,7 @@ __device__ __forceinline__ int epi_bar_count(bool pred) {
 template <int SX>
 struct Control {
     uint64_t x_full[SX], x_empty[SX];
-    uint64_t a_full[kAStages], a_empty[kAStages];
+    uint64_t a_full[kMaxAStages], a_empty[kMaxAStages];
     uint64_t d_full[2], d_empty[2];
     uint32_t tmem_base;
     int abort_flag;
@@ -100,7 +100,7 @@ constexpr uint64_t kBDescHi = (64ull << 32) | (1ull << 46) | (2ull << 61);
 
 // NTOK tokens x (NA x 128) weight rows per CTA tile; KA 64-element K atoms per pipeline stage; SX activation
 // stages in shared memory; DB accumulator buffers (2 = the epilogue of one tile overlaps the main loop of the
-// next).  Tensor memory: DB x NA accumulators of NTOK columns, then kAStages decoded-weight stages of
+// next).  Tensor memory: DB x NA accumulators of NTOK columns, then 2 or 4 decoded-weight stages of
 // NA x KA x 32 columns.
 template <int NTOK, int NA, int KA, int SX, int DB>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -113,6 +113,9 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
     constexpr uint32_t kDCols = NA * NTOK;
     constexpr uint32_t kACols = NA * KA * 32;
     constexpr uint32_t kABase = DB * kDCols;             // first column of the decoded-weight stages
+    // four decoded-weight stages when they fit the 512 columns next to the accumulators (the decode warps then run
+    // two stages further ahead of the MMAs and their hand-off latency no longer shows), else two
+    constexpr int kAStages = (kABase + 4 * kACols <= 512) ? 4 : 2;
     constexpr uint32_t kTmemCols = next_pow2_cols(kABase + kAStages * kACols);
     static_assert(kTmemCols <= 512, "tensor memory budget");
     // instruction descriptor: D fp32, A and B bf16, both K-major, N = NTOK, M = 128
