@@ -489,7 +489,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                                                        : (p.per_tile ? __ldg(p.alpha + j) : __ldg(p.alpha));
                         const int64_t o0 = (int64_t)j * p.r + blk0 + f0;
                         if (vec_ok && nvalid >= 8) {
-                            float b[8];
+                            float b[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
                             if (!plain) {
                                 if (p.bias != nullptr && bias_vec) {          // o0 is a multiple of 8 here
                                     const float4 t0 = __ldg(reinterpret_cast<const float4 *>(p.bias + o0));
@@ -501,28 +501,47 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                                     for (int e = 0; e < 8; ++e) b[e] = p.bias ? __ldg(p.bias + o0 + e) : 0.0f;
                                 }
                             }
+                            // all 32 outputs first (the activation's instruction streams interleave), then the stores
+                            float o[4][8];
+                            if (plain) {
+#pragma unroll
+                                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) o[i][e] = al * z[i][e];
+                            } else if (p.act == TBN_ACT_GELU) {
+#pragma unroll
+                                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) o[i][e] = gelu_erf(fmaf(al, z[i][e], b[e]));
+                            } else if (p.act == TBN_ACT_RELU) {
+#pragma unroll
+                                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) o[i][e] = fmaxf(fmaf(al, z[i][e], b[e]), 0.0f);
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) o[i][e] = fmaf(al, z[i][e], b[e]);
+                            }
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
                                 const int64_t tok = tok_first + 2 * i;
                                 if (tok >= p.T) continue;
-                                float o[8];
-#pragma unroll
-                                for (int e = 0; e < 8; ++e)
-                                    o[e] = plain ? al * z[i][e] : apply_act(fmaf(al, z[i][e], b[e]), p.act);
                                 const int64_t yi = tok * p.m + o0;
                                 if (p.y_bf16) {
                                     uint32_t pk[4];
 #pragma unroll
                                     for (int e = 0; e < 4; ++e) {
-                                        const __nv_bfloat162 h = __floats2bfloat162_rn(o[2 * e], o[2 * e + 1]);
+                                        const __nv_bfloat162 h = __floats2bfloat162_rn(o[i][2 * e], o[i][2 * e + 1]);
                                         pk[e] = *reinterpret_cast<const uint32_t *>(&h);
                                     }
                                     *reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(p.y) + yi) =
                                         make_uint4(pk[0], pk[1], pk[2], pk[3]);
                                 } else {
                                     float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(p.y) + yi);
-                                    dst[0] = make_float4(o[0], o[1], o[2], o[3]);
-                                    dst[1] = make_float4(o[4], o[5], o[6], o[7]);
+                                    dst[0] = make_float4(o[i][0], o[i][1], o[i][2], o[i][3]);
+                                    dst[1] = make_float4(o[i][4], o[i][5], o[i][6], o[i][7]);
                                 }
                             }
                         } else {
