@@ -12,9 +12,10 @@
 // memory.  Each decoded 128 x 64 block is reused for all NTOK tokens of the CTA tile, and each
 // activation stage is reused by NA blocks of 128 weight rows.
 //
-// Warp roles (10 warps): 0 = TMA producer (activation stages, 128-byte swizzle), 1 = MMA issuer and
+// Warp roles (14 warps): 0 = TMA producer (activation stages, 128-byte swizzle), 1 = MMA issuer and
 // TMEM owner, 2-5 = tile decode (bits -> +-1 bf16 pairs -> tcgen05.st), 6-9 = epilogue (tcgen05.ld ->
-// alpha/bias/activation -> k-fold replicated stores).  All hand-offs are mbarriers; every wait is
+// alpha/bias/activation -> k-fold replicated stores), 10-13 = epilogue helpers (half of the arithmetic
+// and stores; they never touch tensor memory).  All hand-offs are mbarriers; every wait is
 // bounded by a wall-clock limit, after which the CTA records TBN_ERR_TIMEOUT, drains and returns.
 #include <cstdlib>
 
@@ -27,7 +28,7 @@ namespace {
 
 using namespace tc;
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 448;
 constexpr int kAtomK = 64;             // contraction elements per 128-byte swizzle row (one TMA box, 4 MMA K steps)
 constexpr int kMaxAStages = 4;         // decoded-weight stages in tensor memory: 2, or 4 where the columns allow
 constexpr int kMaxAlpha = 64;          // alphas cached in shared memory
@@ -50,12 +51,12 @@ __device__ __forceinline__ void decode64(uint32_t b0, uint32_t b1, uint32_t (&v)
 
 constexpr int kXPitch = 132;             // floats per token row of the epilogue exchange buffer (128 + 4: 16-byte rows)
 
-// Named barrier 1 belongs to the four epilogue warps.
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-// Same barrier, returning how many of the 128 threads passed `pred`.
+// Named barrier 1 belongs to the eight epilogue warps.
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// Same barrier, returning how many of the 256 threads passed `pred`.
 __device__ __forceinline__ int epi_bar_count(bool pred) {
     int n;
-    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %1, 0;\nbar.red.popc.u32 %0, 1, 128, p;\n}" : "=r"(n) : "r"((int)pred) : "memory");
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %1, 0;\nbar.red.popc.u32 %0, 1, 256, p;\n}" : "=r"(n) : "r"((int)pred) : "memory");
     return n;
 }
 
@@ -371,22 +372,27 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
         // 128-row x 32-token block through one shared buffer [token][row] and come back with lane = 8 consecutive
         // features of a token: a warp store covers 2 tokens x 256 contiguous bytes (bf16).  Every repetition j is
         // then one multiply per element (fp32), a pack to bf16 and one 16-byte store per token.
-        const int qd = warp & 3;                          // tensor-memory lane quadrant this warp may read
-        const int ew = warp - 6;                          // this warp stores tokens 8*ew .. 8*ew+7 of each 32-token block
+        // Warps 6-9 read tensor memory (and do the split-K traffic); warps 10-13 only help with the arithmetic and
+        // the stores: of a lane's four tokens per block, the readers take the first two and the helpers the last two.
+        const bool reader = warp < 10;
+        const int qd = warp & 3;                          // tensor-memory lane quadrant a reader warp may read
+        const int ew = (warp - 6) & 3;                    // this warp stores tokens 8*ew .. 8*ew+7 of each 32-token block
+        const int iset = (warp - 6) >> 2;                 // token slots 2*iset, 2*iset+1 of the lane's four
         const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
         float (*xbuf)[kXPitch] = reinterpret_cast<float (*)[kXPitch]>(ctl->exchange);
         Pipe pd;                                          // accumulator buffer (stage) and its phase
         const bool vec_ok = (p.m % 8 == 0) && (p.r % 8 == 0);       // 16-byte aligned groups of 8 features
         const bool bias_vec = (reinterpret_cast<uintptr_t>(p.bias) & 15) == 0;
         const int f0 = 8 * (lane & 15);                   // first of this lane's 8 rows inside the 128-row block
-        const int tsub = lane >> 4;                       // this lane's tokens: 8*ew + tsub + 2*i, i < 4
+        const int tsub = lane >> 4;                       // this lane's tokens: 8*ew + tsub + 2*i, i = 2*iset, 2*iset+1
         const bool plain = p.bias == nullptr && (p.act == TBN_ACT_NONE || p.act == TBN_ACT_RELU);
         for (int32_t tile = bid; tile < n_tiles; tile += gridDim.x) {
             const int32_t split = tile % p.splits, out_tile = tile / p.splits;
             const int64_t tok0 = (int64_t)(out_tile / p.w_tiles) * NTOK;
-            ok = wait_bar(smem_u32(&ctl->d_full[pd.stage]), pd.phase, abort_flag, p.status, (6 << 24) | (bid & 0xffff));
-            // the four warps go on together or not at all (they share named barrier 1 below)
-            if (epi_bar_count(ok) != 128) { ok = false; break; }
+            ok = reader ? wait_bar(smem_u32(&ctl->d_full[pd.stage]), pd.phase, abort_flag, p.status, (6 << 24) | (bid & 0xffff))
+                        : (*abort_flag == 0);
+            // the eight warps go on together or not at all (they share named barrier 1 below)
+            if (epi_bar_count(ok) != 256) { ok = false; break; }
             tc_fence_after();
             const int n_chunks = (int)min((int64_t)(NTOK / 32), (p.T - tok0 + 31) / 32);
             // fp32 partial tile of (out_tile, split): [NA][128 rows][NTOK tokens]; this thread owns one row per block
@@ -396,7 +402,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                 part_row = p.partial + ((int64_t)out_tile * p.splits + split) * kTileFloats + (int64_t)(qd * 32 + lane) * NTOK;
                 // pass 1: dump this CTA's partial sums (128 contiguous bytes per thread and chunk)
 #pragma unroll 1
-                for (int a = 0; a < NA; ++a) {
+                for (int a = 0; a < (reader ? NA : 0); ++a) {
 #pragma unroll 1
                     for (int ch = 0; ch < n_chunks; ++ch) {
                         __syncwarp();
@@ -408,8 +414,10 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                         for (int i = 0; i < 8; ++i) __stcg(dst + i, make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]));
                     }
                 }
-                tc_fence_before();
-                mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));           // accumulator fully read
+                if (reader) {
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));       // accumulator fully read
+                }
                 // the CTA that arrives last for this output tile adds the partials and stores
                 __threadfence();
                 epi_bar();
@@ -428,7 +436,9 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                 for (int ch = 0; ch < n_chunks; ++ch) {
                     __syncwarp();                                 // reconverge before the warp-wide TMEM load
                     uint32_t v[32];
-                    if (p.splits > 1) {
+                    if (!reader) {
+                        // helpers wait at the barriers below for the readers' block
+                    } else if (p.splits > 1) {
                         // sum of the splits in a fixed order (split 0, 1, ...): the result does not depend on
                         // which CTA arrived last
                         constexpr int64_t kTileFloats = (int64_t)NA * 128 * NTOK;
@@ -463,14 +473,16 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                         }
                     }
                     epi_bar();                                    // the previous block has been read by everyone
+                    if (reader) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) xbuf[i][qd * 32 + lane] = __uint_as_float(v[i]);
+                        for (int i = 0; i < 32; ++i) xbuf[i][qd * 32 + lane] = __uint_as_float(v[i]);
+                    }
                     epi_bar();
-                    float z[4][8];
+                    float z[2][8];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const float4 lo = *reinterpret_cast<const float4 *>(&xbuf[8 * ew + tsub + 2 * i][f0]);
-                        const float4 hi = *reinterpret_cast<const float4 *>(&xbuf[8 * ew + tsub + 2 * i][f0 + 4]);
+                    for (int i = 0; i < 2; ++i) {
+                        const float4 lo = *reinterpret_cast<const float4 *>(&xbuf[8 * ew + tsub + 4 * iset + 2 * i][f0]);
+                        const float4 hi = *reinterpret_cast<const float4 *>(&xbuf[8 * ew + tsub + 4 * iset + 2 * i][f0 + 4]);
                         z[i][0] = lo.x; z[i][1] = lo.y; z[i][2] = lo.z; z[i][3] = lo.w;
                         z[i][4] = hi.x; z[i][5] = hi.y; z[i][6] = hi.z; z[i][7] = hi.w;
                     }
@@ -479,11 +491,11 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                     if (p.act == TBN_ACT_RELU && p.bias == nullptr) {
                         // alpha >= 0, so relu(alpha * z) = alpha * relu(z): clamp once, outside the k loop
 #pragma unroll
-                        for (int i = 0; i < 4; ++i)
+                        for (int i = 0; i < 2; ++i)
 #pragma unroll
                             for (int e = 0; e < 8; ++e) z[i][e] = fmaxf(z[i][e], 0.0f);
                     }
-                    const int64_t tok_first = tok0 + ch * 32 + 8 * ew + tsub;
+                    const int64_t tok_first = tok0 + ch * 32 + 8 * ew + tsub + 4 * iset;
                     for (int32_t j = 0; j < p.k; ++j) {
                         const float al = j < kMaxAlpha ? ctl->alpha[j]
                                                        : (p.per_tile ? __ldg(p.alpha + j) : __ldg(p.alpha));
@@ -501,31 +513,31 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                                     for (int e = 0; e < 8; ++e) b[e] = p.bias ? __ldg(p.bias + o0 + e) : 0.0f;
                                 }
                             }
-                            // all 32 outputs first (the activation's instruction streams interleave), then the stores
-                            float o[4][8];
+                            // all 16 outputs first (the activation's instruction streams interleave), then the stores
+                            float o[2][8];
                             if (plain) {
 #pragma unroll
-                                for (int i = 0; i < 4; ++i)
+                                for (int i = 0; i < 2; ++i)
 #pragma unroll
                                     for (int e = 0; e < 8; ++e) o[i][e] = al * z[i][e];
                             } else if (p.act == TBN_ACT_GELU) {
 #pragma unroll
-                                for (int i = 0; i < 4; ++i)
+                                for (int i = 0; i < 2; ++i)
 #pragma unroll
                                     for (int e = 0; e < 8; ++e) o[i][e] = gelu_erf(fmaf(al, z[i][e], b[e]));
                             } else if (p.act == TBN_ACT_RELU) {
 #pragma unroll
-                                for (int i = 0; i < 4; ++i)
+                                for (int i = 0; i < 2; ++i)
 #pragma unroll
                                     for (int e = 0; e < 8; ++e) o[i][e] = fmaxf(fmaf(al, z[i][e], b[e]), 0.0f);
                             } else {
 #pragma unroll
-                                for (int i = 0; i < 4; ++i)
+                                for (int i = 0; i < 2; ++i)
 #pragma unroll
                                     for (int e = 0; e < 8; ++e) o[i][e] = fmaf(al, z[i][e], b[e]);
                             }
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
+                            for (int i = 0; i < 2; ++i) {
                                 const int64_t tok = tok_first + 2 * i;
                                 if (tok >= p.T) continue;
                                 const int64_t yi = tok * p.m + o0;
@@ -547,7 +559,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                         } else {
                             // ragged or unaligned rows: element by element
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
+                            for (int i = 0; i < 2; ++i) {
                                 const int64_t tok = tok_first + 2 * i;
                                 if (tok >= p.T) continue;
 #pragma unroll
