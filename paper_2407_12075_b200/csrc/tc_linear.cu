@@ -28,7 +28,7 @@ namespace {
 
 using namespace tc;
 
-constexpr int kThreads = 448;
+constexpr int kBaseThreads = 192;      // TMA, MMA and the four decode warps; the epilogue warps follow
 constexpr int kAtomK = 64;             // contraction elements per 128-byte swizzle row (one TMA box, 4 MMA K steps)
 constexpr int kMaxAStages = 4;         // decoded-weight stages in tensor memory: 2, or 4 where the columns allow
 constexpr int kMaxAlpha = 64;          // alphas cached in shared memory
@@ -51,12 +51,15 @@ __device__ __forceinline__ void decode64(uint32_t b0, uint32_t b1, uint32_t (&v)
 
 constexpr int kXPitch = 132;             // floats per token row of the epilogue exchange buffer (128 + 4: 16-byte rows)
 
-// Named barrier 1 belongs to the eight epilogue warps.
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-// Same barrier, returning how many of the 256 threads passed `pred`.
+// Named barrier 1 belongs to the epilogue warps (THREADS of them in all).
+template <int THREADS>
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, %0;" ::"n"(THREADS) : "memory"); }
+// Same barrier, returning how many of its threads passed `pred`.
+template <int THREADS>
 __device__ __forceinline__ int epi_bar_count(bool pred) {
     int n;
-    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %1, 0;\nbar.red.popc.u32 %0, 1, 256, p;\n}" : "=r"(n) : "r"((int)pred) : "memory");
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %1, 0;\nbar.red.popc.u32 %0, 1, %2, p;\n}"
+                 : "=r"(n) : "r"((int)pred), "n"(THREADS) : "memory");
     return n;
 }
 
@@ -103,11 +106,14 @@ constexpr uint64_t kBDescHi = (64ull << 32) | (1ull << 46) | (2ull << 61);
 // stages in shared memory; DB accumulator buffers (2 = the epilogue of one tile overlaps the main loop of the
 // next).  Tensor memory: DB x NA accumulators of NTOK columns, then 2 or 4 decoded-weight stages of
 // NA x KA x 32 columns.
-template <int NTOK, int NA, int KA, int SX, int DB>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int NTOK, int NA, int KA, int SX, int DB, int EPI>
+__global__ void __launch_bounds__(kBaseThreads + 32 * EPI, 1)
 tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
 {
     static_assert(NTOK % 32 == 0 && NTOK >= 32 && NTOK <= 256, "token tile");
+    static_assert(EPI == 4 || EPI == 8, "epilogue warps: the four tensor-memory readers, optionally four helpers");
+    constexpr int kEpiThreads = 32 * EPI;
+    constexpr int kSlots = EPI == 8 ? 2 : 4;             // token slots (of a lane's four per block) handled by one warp set
     constexpr uint32_t kAtomBytes = NTOK * 128;
     constexpr uint32_t kStageBytes = KA * kAtomBytes;
     constexpr int kStageK = KA * kAtomK;
@@ -372,12 +378,13 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
         // 128-row x 32-token block through one shared buffer [token][row] and come back with lane = 8 consecutive
         // features of a token: a warp store covers 2 tokens x 256 contiguous bytes (bf16).  Every repetition j is
         // then one multiply per element (fp32), a pack to bf16 and one 16-byte store per token.
-        // Warps 6-9 read tensor memory (and do the split-K traffic); warps 10-13 only help with the arithmetic and
-        // the stores: of a lane's four tokens per block, the readers take the first two and the helpers the last two.
+        // Warps 6-9 read tensor memory (and do the split-K traffic).  With EPI == 8, warps 10-13 help with the
+        // arithmetic and the stores: of a lane's four tokens per block, the readers take the first two and the
+        // helpers the last two (worth it when the activation is expensive; a plain epilogue is bound by the stores).
         const bool reader = warp < 10;
         const int qd = warp & 3;                          // tensor-memory lane quadrant a reader warp may read
         const int ew = (warp - 6) & 3;                    // this warp stores tokens 8*ew .. 8*ew+7 of each 32-token block
-        const int iset = (warp - 6) >> 2;                 // token slots 2*iset, 2*iset+1 of the lane's four
+        const int iset = (warp - 6) >> 2;                 // token slots kSlots*iset .. of the lane's four
         const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
         float (*xbuf)[kXPitch] = reinterpret_cast<float (*)[kXPitch]>(ctl->exchange);
         Pipe pd;                                          // accumulator buffer (stage) and its phase
@@ -392,7 +399,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
             ok = reader ? wait_bar(smem_u32(&ctl->d_full[pd.stage]), pd.phase, abort_flag, p.status, (6 << 24) | (bid & 0xffff))
                         : (*abort_flag == 0);
             // the eight warps go on together or not at all (they share named barrier 1 below)
-            if (epi_bar_count(ok) != 256) { ok = false; break; }
+            if (epi_bar_count<kEpiThreads>(ok) != kEpiThreads) { ok = false; break; }
             tc_fence_after();
             const int n_chunks = (int)min((int64_t)(NTOK / 32), (p.T - tok0 + 31) / 32);
             // fp32 partial tile of (out_tile, split): [NA][128 rows][NTOK tokens]; this thread owns one row per block
@@ -420,9 +427,9 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                 }
                 // the CTA that arrives last for this output tile adds the partials and stores
                 __threadfence();
-                epi_bar();
+                epi_bar<kEpiThreads>();
                 if (warp == 6 && lane == 0) ctl->ticket = atomicAdd(p.tickets + (int64_t)out_tile * 4, 1u);
-                epi_bar();
+                epi_bar<kEpiThreads>();
                 const unsigned int old = ctl->ticket;
                 if (old != (unsigned int)(p.splits - 1)) { pd.advance(DB); continue; }
                 __threadfence();
@@ -472,17 +479,17 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                             mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));
                         }
                     }
-                    epi_bar();                                    // the previous block has been read by everyone
+                    epi_bar<kEpiThreads>();                                    // the previous block has been read by everyone
                     if (reader) {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) xbuf[i][qd * 32 + lane] = __uint_as_float(v[i]);
                     }
-                    epi_bar();
-                    float z[2][8];
+                    epi_bar<kEpiThreads>();
+                    float z[kSlots][8];
 #pragma unroll
-                    for (int i = 0; i < 2; ++i) {
-                        const float4 lo = *reinterpret_cast<const float4 *>(&xbuf[8 * ew + tsub + 4 * iset + 2 * i][f0]);
-                        const float4 hi = *reinterpret_cast<const float4 *>(&xbuf[8 * ew + tsub + 4 * iset + 2 * i][f0 + 4]);
+                    for (int i = 0; i < kSlots; ++i) {
+                        const float4 lo = *reinterpret_cast<const float4 *>(&xbuf[8 * ew + tsub + 2 * (kSlots * iset + i)][f0]);
+                        const float4 hi = *reinterpret_cast<const float4 *>(&xbuf[8 * ew + tsub + 2 * (kSlots * iset + i)][f0 + 4]);
                         z[i][0] = lo.x; z[i][1] = lo.y; z[i][2] = lo.z; z[i][3] = lo.w;
                         z[i][4] = hi.x; z[i][5] = hi.y; z[i][6] = hi.z; z[i][7] = hi.w;
                     }
@@ -491,11 +498,11 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                     if (p.act == TBN_ACT_RELU && p.bias == nullptr) {
                         // alpha >= 0, so relu(alpha * z) = alpha * relu(z): clamp once, outside the k loop
 #pragma unroll
-                        for (int i = 0; i < 2; ++i)
+                        for (int i = 0; i < kSlots; ++i)
 #pragma unroll
                             for (int e = 0; e < 8; ++e) z[i][e] = fmaxf(z[i][e], 0.0f);
                     }
-                    const int64_t tok_first = tok0 + ch * 32 + 8 * ew + tsub + 4 * iset;
+                    const int64_t tok_first = tok0 + ch * 32 + 8 * ew + tsub + 2 * kSlots * iset;
                     for (int32_t j = 0; j < p.k; ++j) {
                         const float al = j < kMaxAlpha ? ctl->alpha[j]
                                                        : (p.per_tile ? __ldg(p.alpha + j) : __ldg(p.alpha));
@@ -513,31 +520,31 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                                     for (int e = 0; e < 8; ++e) b[e] = p.bias ? __ldg(p.bias + o0 + e) : 0.0f;
                                 }
                             }
-                            // all 16 outputs first (the activation's instruction streams interleave), then the stores
-                            float o[2][8];
+                            // all outputs first (the activation's instruction streams interleave), then the stores
+                            float o[kSlots][8];
                             if (plain) {
 #pragma unroll
-                                for (int i = 0; i < 2; ++i)
+                                for (int i = 0; i < kSlots; ++i)
 #pragma unroll
                                     for (int e = 0; e < 8; ++e) o[i][e] = al * z[i][e];
                             } else if (p.act == TBN_ACT_GELU) {
 #pragma unroll
-                                for (int i = 0; i < 2; ++i)
+                                for (int i = 0; i < kSlots; ++i)
 #pragma unroll
                                     for (int e = 0; e < 8; ++e) o[i][e] = gelu_erf(fmaf(al, z[i][e], b[e]));
                             } else if (p.act == TBN_ACT_RELU) {
 #pragma unroll
-                                for (int i = 0; i < 2; ++i)
+                                for (int i = 0; i < kSlots; ++i)
 #pragma unroll
                                     for (int e = 0; e < 8; ++e) o[i][e] = fmaxf(fmaf(al, z[i][e], b[e]), 0.0f);
                             } else {
 #pragma unroll
-                                for (int i = 0; i < 2; ++i)
+                                for (int i = 0; i < kSlots; ++i)
 #pragma unroll
                                     for (int e = 0; e < 8; ++e) o[i][e] = fmaf(al, z[i][e], b[e]);
                             }
 #pragma unroll
-                            for (int i = 0; i < 2; ++i) {
+                            for (int i = 0; i < kSlots; ++i) {
                                 const int64_t tok = tok_first + 2 * i;
                                 if (tok >= p.T) continue;
                                 const int64_t yi = tok * p.m + o0;
@@ -559,7 +566,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                         } else {
                             // ragged or unaligned rows: element by element
 #pragma unroll
-                            for (int i = 0; i < 2; ++i) {
+                            for (int i = 0; i < kSlots; ++i) {
                                 const int64_t tok = tok_first + 2 * i;
                                 if (tok >= p.T) continue;
 #pragma unroll
@@ -637,14 +644,16 @@ int launch_config(const LayerArgs &a, TcParams p, int splits, void *scratch, cud
         p.partial = nullptr;
     }
     const size_t smem = (size_t)SX * KA * NTOK * 128 + sizeof(Control<SX>) + 1024;
-    auto kern = tc_linear_kernel<NTOK, NA, KA, SX, DB>;
+    // four helper warps for the epilogue when its arithmetic is heavy (GELU); a plain epilogue is bound by its stores
+    const bool helpers = a.act == TBN_ACT_GELU;
+    auto kern = helpers ? tc_linear_kernel<NTOK, NA, KA, SX, DB, 8> : tc_linear_kernel<NTOK, NA, KA, SX, DB, 4>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return TBN_ERR_CUDA;
     const int sms = sm_count();
     if (sms <= 0) return TBN_ERR_CUDA;
     const int64_t tiles = out_tiles * splits;
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
-    kern<<<grid, kThreads, smem, s>>>(map, p);
+    kern<<<grid, kBaseThreads + (helpers ? 256 : 128), smem, s>>>(map, p);
     return cudaGetLastError() == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
 }
 
