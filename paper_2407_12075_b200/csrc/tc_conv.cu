@@ -313,24 +313,27 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
 #pragma unroll
                     for (int i = 0; i < 6; ++i) w[i] = __ldg(p.tile + min(wi + i, last_word));
                 }
-                ok = wait_bar(smem_u32(&ctl->a_empty[pa.stage]), pa.phase ^ 1u, abort_flag, p.status,
-                              (5 << 24) | (pa.stage << 16) | (bid & 0xffff));
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t a_addr = tmem_base + lane_base + kABase + pa.stage * kACols;
+                // decode into registers first: the ALU work overlaps the MMAs that still read the stage's slot, and only
+                // the nine stores sit between "slot free" and "slot full"
+                uint32_t v[kTaps][8];
 #pragma unroll
                 for (int t = 0; t < kTaps; ++t) {
-                    uint32_t v[8];
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         // channels 2i and 2i+1 of the stage at tap t: bits (2i)*9 + t and (2i+1)*9 + t
                         const int pe = (2 * i) * kTaps + t, po = pe + kTaps;
                         const uint32_t be = (b[pe >> 5] >> (pe & 31)) & 1u;
                         const uint32_t bo = (b[po >> 5] >> (po & 31)) & 1u;
-                        v[i] = ((be << 15) | (bo << 31)) ^ 0xBF80BF80u;       // bit 1 -> +1.0, bit 0 -> -1.0
+                        v[t][i] = ((be << 15) | (bo << 31)) ^ 0xBF80BF80u;    // bit 1 -> +1.0, bit 0 -> -1.0
                     }
-                    tmem_st_32x8(a_addr + t * 8, v);
                 }
+                ok = wait_bar(smem_u32(&ctl->a_empty[pa.stage]), pa.phase ^ 1u, abort_flag, p.status,
+                              (5 << 24) | (pa.stage << 16) | (bid & 0xffff));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_addr = tmem_base + lane_base + kABase + pa.stage * kACols;
+#pragma unroll
+                for (int t = 0; t < kTaps; ++t) tmem_st_32x8(a_addr + t * 8, v[t]);
                 tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(smem_u32(&ctl->a_full[pa.stage]));
