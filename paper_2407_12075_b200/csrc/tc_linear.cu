@@ -657,10 +657,11 @@ int launch_config(const LayerArgs &a, TcParams p, int splits, void *scratch, cud
     return cudaGetLastError() == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
 }
 
-// Tile shape and split-K factor for one call.  Cost model in nanoseconds per CTA, fitted to measurements on
-// B200 (T = 16384, n = 8192): one MMA of N tokens takes about 0.45*N + 14 ns, a pipeline stage adds about 150 ns
-// of hand-offs, the epilogue costs about 2 ns per instruction of one warp (100 per 32 x 32 block + 52 per
-// repetition).  With two accumulator buffers the epilogue hides behind the next tile's main loop except once.
+// Tile shape and split-K factor for one call.  Cost model in nanoseconds per CTA, fitted to timelines and sweeps on
+// B200 (n = 8192; T = 64 .. 16384): the issuing thread needs about 77 ns per MMA whatever the token tile, plus 0.09 ns
+// per token; a configuration with only two decoded-weight slots pays about 100 ns of hand-off per stage; the epilogue
+// is bound by its stores (about 30 bytes per ns and SM, i.e. 8.5 ns per token and repetition for 128 rows) plus 250 ns
+// per 32-token block.  With two accumulator buffers the epilogue hides behind the next tile's main loop except once.
 // When the output has fewer tiles than the GPU has SMs, the contraction is split over several CTAs per tile
 // (each dumps an fp32 partial tile; the last to arrive adds them in a fixed order and stores).
 struct Cand { int ntok, na, ka, db; };
@@ -684,8 +685,9 @@ Plan plan_linear(const LayerArgs &a)
         const int64_t tt = (a.T + c.ntok - 1) / c.ntok;
         const int64_t out_tiles = wt * tt;
         const int k_stages = (a.n + c.ka * kAtomK - 1) / (c.ka * kAtomK);
-        const double stage = c.na * c.ka * 4 * (0.45 * c.ntok + 14.0) + 150.0;
-        const double epi = c.na * (c.ntok / 32.0) * (100.0 + 52.0 * a.k) * 2.0;
+        const bool four_slots = c.db * c.na * c.ntok + 4 * c.na * c.ka * 32 <= 512;    // decoded-weight slots in tensor memory
+        const double stage = c.na * c.ka * 4 * (0.09 * c.ntok + 77.0) + (four_slots ? 0.0 : 100.0);
+        const double epi = c.na * (double)c.ntok * a.k * 8.5 + c.na * (c.ntok / 32.0) * 250.0;
         const double dump = c.na * (c.ntok / 32.0) * 60.0 * 2.0;
         for (int sp = 1; sp <= 16; sp *= 2) {
             if (sp > 1 && (k_stages < 2 * sp || out_tiles * sp > sms)) break;   // >= 2 stages per split, one wave
