@@ -660,8 +660,9 @@ int launch_config(const LayerArgs &a, TcParams p, int splits, void *scratch, cud
 // Tile shape and split-K factor for one call.  Cost model in nanoseconds per CTA, fitted to timelines and sweeps on
 // B200 (n = 8192; T = 64 .. 16384): the issuing thread needs about 77 ns per MMA whatever the token tile, plus 0.09 ns
 // per token; a configuration with only two decoded-weight slots pays about 100 ns of hand-off per stage; the epilogue
-// is bound by its stores (about 30 bytes per ns and SM, i.e. 8.5 ns per token and repetition for 128 rows) plus 250 ns
-// per 32-token block.  With two accumulator buffers the epilogue hides behind the next tile's main loop except once.
+// is bound by its stores (about 34 bytes per ns and SM, i.e. 7.5 ns per token and repetition for 128 rows) plus 250 ns
+// per 32-token block; every tile costs about 1.5 us of hand-over.  With two accumulator buffers the epilogue hides
+// behind the next tile's main loop except for the last tile.
 // When the output has fewer tiles than the GPU has SMs, the contraction is split over several CTAs per tile
 // (each dumps an fp32 partial tile; the last to arrive adds them in a fixed order and stores).
 struct Cand { int ntok, na, ka, db; };
@@ -687,14 +688,16 @@ Plan plan_linear(const LayerArgs &a)
         const int k_stages = (a.n + c.ka * kAtomK - 1) / (c.ka * kAtomK);
         const bool four_slots = c.db * c.na * c.ntok + 4 * c.na * c.ka * 32 <= 512;    // decoded-weight slots in tensor memory
         const double stage = c.na * c.ka * 4 * (0.09 * c.ntok + 77.0) + (four_slots ? 0.0 : 100.0);
-        const double epi = c.na * (double)c.ntok * a.k * 8.5 + c.na * (c.ntok / 32.0) * 250.0;
+        const double epi = c.na * (double)c.ntok * a.k * 7.5 + c.na * (c.ntok / 32.0) * 250.0;
+        const double per_tile = 1500.0;                 // tile hand-over: first bit words, barrier round trips
         const double dump = c.na * (c.ntok / 32.0) * 60.0 * 2.0;
         for (int sp = 1; sp <= 16; sp *= 2) {
             if (sp > 1 && (k_stages < 2 * sp || out_tiles * sp > sms)) break;   // >= 2 stages per split, one wave
             const int64_t waves = (out_tiles * sp + sms - 1) / sms;
             const double mainloop = atoms / c.ka / sp * stage;
             double cost;
-            if (sp == 1) cost = c.db == 2 ? waves * (mainloop > epi ? mainloop : epi) + epi : waves * (mainloop + epi);
+            if (sp == 1) cost = c.db == 2 ? mainloop + (waves - 1) * ((mainloop > epi ? mainloop : epi) + per_tile) + epi + per_tile
+                                          : waves * (mainloop + epi + per_tile);
             else cost = mainloop + dump + epi + 1500.0 +                        // ticket / partial round trip
                         c.na * (c.ntok < a.T ? c.ntok : (double)a.T) / 32.0 * (sp / 2) * 1000.0;   // reduction: one L2 round per two splits and 32 tokens
             if (cost < best_cost) {
