@@ -284,10 +284,11 @@ def measure_other_configs(B, torch, dev, peaks):
     for name, (n, m) in {"vit_qkv_768_2304": (768, 2304), "vit_out_768_768": (768, 768), "vit_fc1_768_3072": (768, 3072),
                          "vit_fc2_3072_768": (3072, 768)}.items():
         out[name] = linear_entry(25216, n, m, 8)
+    out["vit_fc1_768_3072_gelu"] = linear_entry(25216, 768, 3072, 8, act=B.ACT_GELU)
     # derived: images/s over the tiled layers only (LayerNorm, attention and residual adds of the block, and the
     # full-precision first convolution / classifier of the conv stack, are not tiled layers and are not run)
-    vit_us = sum(out[n]["us"] for n in ("vit_qkv_768_2304", "vit_out_768_768", "vit_fc1_768_3072", "vit_fc2_3072_768"))
-    out["vit_block_tiled_linears_only"] = dict(us=vit_us, images_per_s=128 / vit_us * 1e6, includes="qkv + out-proj + fc1 + fc2")
+    vit_us = sum(out[n]["us"] for n in ("vit_qkv_768_2304", "vit_out_768_768", "vit_fc1_768_3072_gelu", "vit_fc2_3072_768"))
+    out["vit_block_tiled_linears_only"] = dict(us=vit_us, images_per_s=128 / vit_us * 1e6, includes="qkv + out-proj + fc1 with fused GELU + fc2")
     conv_us = out["conv_64_128_s2_32x32"]["us"] + out["conv_128_256_s2_16x16"]["us"]
     out["conv_stack_tiled_convs_only"] = dict(us=conv_us, images_per_s=256 / conv_us * 1e6, includes="64->128 s2 + 128->256 s2")
     # prepare step (once per layer, outside the forward): W fp32 read once, packed tile written
