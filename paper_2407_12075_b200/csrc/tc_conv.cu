@@ -367,67 +367,48 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                 // pieces that share a 32-byte sector go out as one 32-byte store).  All loops are warp-uniform.
                 const int32_t rows_here = min(p.R, p.Ho - oh0);
                 const int32_t pieces = p.Wo >> 3;
-                const int32_t pairs = (pieces + 1) >> 1;             // 16-pixel items per output row
-                const int32_t imgs = min(p.G, p.Nb - img0);
-                const int32_t n_items = imgs * rows_here * pairs;
-                __nv_bfloat16 *ch_dst = static_cast<__nv_bfloat16 *>(p.y) +
-                                        ((int64_t)img0 * p.m + (ch_valid ? o : 0)) * out_plane + (int64_t)oh0 * p.Wo;
-                // two items per trip: both tensor-memory loads are in flight before either is consumed
-                for (int32_t it = 0; it < n_items; it += 2) {
-                    uint32_t v[2][16];
-                    int64_t off[2];                                  // element offset of the item from the channel's first output
-                    bool two[2];
-                    __syncwarp();
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const int32_t item = min(it + u, n_items - 1);   // an odd tail repeats the last item (not stored)
-                        const int32_t pr = item % pairs, row = item / pairs;
-                        const int32_t oh = row % rows_here, g = row / rows_here;
-                        const int32_t pc = pr * 2;
-                        two[u] = pc + 1 < pieces;
-                        off[u] = (int64_t)g * p.m * out_plane + oh * p.Wo + pc * 8;
-                        const uint32_t col = tmem_base + lane_base + pd.stage * kNMax + g * p.slot_pos + oh * p.PW + pc * 8;
-                        if (two[u]) {
-                            tmem_ld_32x16(col, v[u]);
-                        } else {
-                            uint32_t v8[8];
-                            tmem_ld_32x8(col, v8);
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) { v[u][i] = v8[i]; v[u][i + 8] = 0u; }
-                        }
-                    }
-                    tc_wait_ld();
-                    if (it + 2 >= n_items) {                         // accumulator fully read: hand it back early
-                        tc_fence_before();
-                        mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));
-                    }
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        if (it + u >= n_items) break;
-                        uint32_t pk[8];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            float v0 = fmaf(al, __uint_as_float(v[u][2 * i]), bs), v1 = fmaf(al, __uint_as_float(v[u][2 * i + 1]), bs);
-                            if (p.act == TBN_ACT_RELU) { v0 = fmaxf(v0, 0.0f); v1 = fmaxf(v1, 0.0f); }
-                            else if (p.act == TBN_ACT_GELU) { v0 = apply_act(v0, TBN_ACT_GELU); v1 = apply_act(v1, TBN_ACT_GELU); }
-                            const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
-                            pk[i] = *reinterpret_cast<const uint32_t *>(&h);
-                        }
-                        if (ch_valid) {
-                            __nv_bfloat16 *dst = ch_dst + off[u];
-                            if (two[u] && (((uintptr_t)dst) & 31u) == 0) {
-                                st_global_v8(dst, pk);
+                for (int32_t g = 0; g < p.G && img0 + g < p.Nb; ++g) {
+                    __nv_bfloat16 *img_dst = static_cast<__nv_bfloat16 *>(p.y) +
+                                             ((int64_t)(img0 + g) * p.m + (ch_valid ? o : 0)) * out_plane + (int64_t)oh0 * p.Wo;
+                    for (int32_t oh = 0; oh < rows_here; ++oh) {
+                        const uint32_t col0 = tmem_base + lane_base + pd.stage * kNMax + g * p.slot_pos + oh * p.PW;
+                        __nv_bfloat16 *row_dst = img_dst + oh * p.Wo;
+                        for (int32_t pc = 0; pc < pieces; pc += 2) {
+                            uint32_t v[16];
+                            const bool two = pc + 1 < pieces;
+                            __syncwarp();
+                            if (two) {
+                                tmem_ld_32x16(col0 + pc * 8, v);
                             } else {
-                                *reinterpret_cast<uint4 *>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                                if (two[u]) *reinterpret_cast<uint4 *>(dst + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                                uint32_t v8[8];
+                                tmem_ld_32x8(col0 + pc * 8, v8);
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) { v[i] = v8[i]; v[i + 8] = 0u; }
+                            }
+                            tc_wait_ld();
+                            uint32_t pk[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                float v0 = fmaf(al, __uint_as_float(v[2 * i]), bs), v1 = fmaf(al, __uint_as_float(v[2 * i + 1]), bs);
+                                if (p.act == TBN_ACT_RELU) { v0 = fmaxf(v0, 0.0f); v1 = fmaxf(v1, 0.0f); }
+                                else if (p.act == TBN_ACT_GELU) { v0 = apply_act(v0, TBN_ACT_GELU); v1 = apply_act(v1, TBN_ACT_GELU); }
+                                const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+                                pk[i] = *reinterpret_cast<const uint32_t *>(&h);
+                            }
+                            if (ch_valid) {
+                                __nv_bfloat16 *dst = row_dst + pc * 8;
+                                if (two && (((uintptr_t)dst) & 31u) == 0) {
+                                    st_global_v8(dst, pk);
+                                } else {
+                                    *reinterpret_cast<uint4 *>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                                    if (two) *reinterpret_cast<uint4 *>(dst + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                                }
                             }
                         }
                     }
                 }
-                if (n_items <= 0) {
-                    tc_fence_before();
-                    mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));
-                }
+                tc_fence_before();
+                mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));      // accumulator fully read
                 pd.advance(2);
                 continue;
             }
