@@ -370,48 +370,38 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                 for (int32_t g = 0; g < p.G && img0 + g < p.Nb; ++g) {
                     __nv_bfloat16 *img_dst = static_cast<__nv_bfloat16 *>(p.y) +
                                              ((int64_t)(img0 + g) * p.m + (ch_valid ? o : 0)) * out_plane + (int64_t)oh0 * p.Wo;
-                    // two output rows per trip: both tensor-memory loads are in flight before either is consumed
-                    for (int32_t oh = 0; oh < rows_here; oh += 2) {
-                        const bool second = oh + 1 < rows_here;
+                    for (int32_t oh = 0; oh < rows_here; ++oh) {
                         const uint32_t col0 = tmem_base + lane_base + pd.stage * kNMax + g * p.slot_pos + oh * p.PW;
                         __nv_bfloat16 *row_dst = img_dst + oh * p.Wo;
                         for (int32_t pc = 0; pc < pieces; pc += 2) {
-                            uint32_t v[2][16];
+                            uint32_t v[16];
                             const bool two = pc + 1 < pieces;
                             __syncwarp();
+                            if (two) {
+                                tmem_ld_32x16(col0 + pc * 8, v);
+                            } else {
+                                uint32_t v8[8];
+                                tmem_ld_32x8(col0 + pc * 8, v8);
 #pragma unroll
-                            for (int u = 0; u < 2; ++u) {
-                                const uint32_t col = col0 + (u && second ? p.PW : 0) + pc * 8;   // no second row: reload the first
-                                if (two) {
-                                    tmem_ld_32x16(col, v[u]);
-                                } else {
-                                    uint32_t v8[8];
-                                    tmem_ld_32x8(col, v8);
-#pragma unroll
-                                    for (int i = 0; i < 8; ++i) { v[u][i] = v8[i]; v[u][i + 8] = 0u; }
-                                }
+                                for (int i = 0; i < 8; ++i) { v[i] = v8[i]; v[i + 8] = 0u; }
                             }
                             tc_wait_ld();
+                            uint32_t pk[8];
 #pragma unroll
-                            for (int u = 0; u < 2; ++u) {
-                                if (u && !second) break;
-                                uint32_t pk[8];
-#pragma unroll
-                                for (int i = 0; i < 8; ++i) {
-                                    float v0 = fmaf(al, __uint_as_float(v[u][2 * i]), bs), v1 = fmaf(al, __uint_as_float(v[u][2 * i + 1]), bs);
-                                    if (p.act == TBN_ACT_RELU) { v0 = fmaxf(v0, 0.0f); v1 = fmaxf(v1, 0.0f); }
-                                    else if (p.act == TBN_ACT_GELU) { v0 = apply_act(v0, TBN_ACT_GELU); v1 = apply_act(v1, TBN_ACT_GELU); }
-                                    const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
-                                    pk[i] = *reinterpret_cast<const uint32_t *>(&h);
-                                }
-                                if (ch_valid) {
-                                    __nv_bfloat16 *dst = row_dst + u * p.Wo + pc * 8;
-                                    if (two && (((uintptr_t)dst) & 31u) == 0) {
-                                        st_global_v8(dst, pk);
-                                    } else {
-                                        *reinterpret_cast<uint4 *>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                                        if (two) *reinterpret_cast<uint4 *>(dst + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-                                    }
+                            for (int i = 0; i < 8; ++i) {
+                                float v0 = fmaf(al, __uint_as_float(v[2 * i]), bs), v1 = fmaf(al, __uint_as_float(v[2 * i + 1]), bs);
+                                if (p.act == TBN_ACT_RELU) { v0 = fmaxf(v0, 0.0f); v1 = fmaxf(v1, 0.0f); }
+                                else if (p.act == TBN_ACT_GELU) { v0 = apply_act(v0, TBN_ACT_GELU); v1 = apply_act(v1, TBN_ACT_GELU); }
+                                const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+                                pk[i] = *reinterpret_cast<const uint32_t *>(&h);
+                            }
+                            if (ch_valid) {
+                                __nv_bfloat16 *dst = row_dst + pc * 8;
+                                if (two && (((uintptr_t)dst) & 31u) == 0) {
+                                    st_global_v8(dst, pk);
+                                } else {
+                                    *reinterpret_cast<uint4 *>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                                    if (two) *reinterpret_cast<uint4 *>(dst + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
                                 }
                             }
                         }
