@@ -11,7 +11,7 @@ from tests.util import DEV, assert_close, make_linear_case, to_dev, to_np64
 
 pytestmark = pytest.mark.gpu
 
-# (m, n, k): the survey's shape zoo -- aligned, misaligned, several tiles per row, nothing divides
+# (m, n, k): a shape zoo -- aligned, misaligned, several tiles per row, nothing divides
 ZOO = [(8, 8, 1), (8, 8, 2), (8, 8, 8), (128, 784, 4), (10, 128, 1), (512, 512, 4), (2304, 768, 8),
        (96, 40, 6), (6, 64, 4), (4, 64, 8), (7, 33, 3)]
 TOKENS = [1, 2, 3, 17, 64, 129]
