@@ -571,9 +571,13 @@ int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t 
                 a.m = r; a.k = 1; a.alpha = one; a.alpha_mode = TBN_ALPHA_PER_LAYER;
                 a.act = hidden_act; a.y = ws + plan.g_off[l & 1]; a.y_dtype = TBN_BF16;
             }
-            if (!tensor_path_supported(a)) return TBN_ERR_UNSUPPORTED;
-            rc = launch_tensor_linear(a, st, ws + plan.scratch_off, plan.scratch_bytes, s);
-            if (rc != TBN_OK) return rc;
+            if (thin_dense_supported(a)) {              // a few output rows: not worth a tensor-core launch
+                if (launch_thin_dense(a, s) != cudaSuccess) return TBN_ERR_CUDA;
+            } else {
+                if (!tensor_path_supported(a)) return TBN_ERR_UNSUPPORTED;
+                rc = launch_tensor_linear(a, st, ws + plan.scratch_off, plan.scratch_bytes, s);
+                if (rc != TBN_OK) return rc;
+            }
             cur = a.y;
             n_cur = r;
         }

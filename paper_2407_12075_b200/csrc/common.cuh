@@ -98,6 +98,9 @@ cudaError_t launch_generic(const LayerArgs &a, cudaStream_t s);
 bool small_batch_supported(const LayerArgs &a);
 cudaError_t launch_small_batch(const LayerArgs &a, cudaStream_t s);
 double small_batch_estimate_us(const LayerArgs &a);
+// Thin layer (at most 16 distinct rows) with full-precision rows in dense_a: the head of a compact MLP chain.
+bool thin_dense_supported(const LayerArgs &a);
+cudaError_t launch_thin_dense(const LayerArgs &a, cudaStream_t s);
 
 // The tensor-core path reports through a tbn_status because it also uses the driver API.
 bool tensor_path_supported(const LayerArgs &a);

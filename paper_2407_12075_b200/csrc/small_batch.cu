@@ -311,6 +311,68 @@ cudaError_t launch_rw(const LayerArgs &a, int32_t r, cudaStream_t s)
     return launch_tt<XT, 1>(a, r, s);
 }
 
+// ---- thin layer with full-precision rows (the last layer of a compact MLP chain) -------------------------------
+//
+// y[t][j*r + c] = act(alpha_j * sum_i x[t][i] * W[c][i] + bias) for r <= 16 bf16 rows W (a classifier head).  The
+// whole weight block sits in shared memory as fp32; a warp owns a token, lane l takes inputs [256 g + 8 l, +8) of
+// every 256-input group, and the r sums are combined with warp shuffles.  A launch of the tensor-core kernel costs
+// several microseconds of fixed set-up, far more than this layer's arithmetic.
+constexpr int kThinRows = 16;
+constexpr int kThinMaxWeights = 8192;      // r * n fp32 values in shared memory (32 KB)
+
+__global__ void __launch_bounds__(256)
+thin_dense_kernel(const LayerArgs a, int32_t r)
+{
+    __shared__ __align__(16) float w_s[kThinMaxWeights];
+    const int32_t n = a.n;
+    const __nv_bfloat16 *W = static_cast<const __nv_bfloat16 *>(a.dense_a);
+    for (int32_t i = threadIdx.x; i < r * n; i += blockDim.x) w_s[i] = __bfloat162float(W[i]);
+    __syncthreads();
+
+    const int lane = threadIdx.x & 31;
+    const int warps = (gridDim.x * blockDim.x) >> 5;
+    const __nv_bfloat16 *x = static_cast<const __nv_bfloat16 *>(a.x);
+    const bool per_tile = a.alpha_mode == TBN_ALPHA_PER_TILE;
+    for (int64_t t = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; t < a.T; t += warps) {
+        float acc[kThinRows];
+#pragma unroll
+        for (int c = 0; c < kThinRows; ++c) acc[c] = 0.0f;
+        for (int32_t i0 = lane * 8; i0 < n; i0 += 256) {             // n % 8 == 0
+            float xv[8];
+            XVec<__nv_bfloat16>::load8(x + t * n + i0, xv);
+#pragma unroll
+            for (int c = 0; c < kThinRows; ++c) {
+                if (c >= r) break;
+                const float4 w0 = *reinterpret_cast<const float4 *>(w_s + c * n + i0);
+                const float4 w1 = *reinterpret_cast<const float4 *>(w_s + c * n + i0 + 4);
+                acc[c] = fmaf(xv[0], w0.x, acc[c]); acc[c] = fmaf(xv[1], w0.y, acc[c]);
+                acc[c] = fmaf(xv[2], w0.z, acc[c]); acc[c] = fmaf(xv[3], w0.w, acc[c]);
+                acc[c] = fmaf(xv[4], w1.x, acc[c]); acc[c] = fmaf(xv[5], w1.y, acc[c]);
+                acc[c] = fmaf(xv[6], w1.z, acc[c]); acc[c] = fmaf(xv[7], w1.w, acc[c]);
+            }
+        }
+        float mine = 0.0f;                                          // lane c ends up with the sum of row c
+#pragma unroll
+        for (int c = 0; c < kThinRows; ++c) {
+            if (c >= r) break;
+            float v = acc[c];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+            if (lane == c) mine = v;
+        }
+        if (lane < r) {
+            for (int32_t j = 0; j < a.k; ++j) {
+                const int32_t o = j * r + lane;
+                const float al = per_tile ? __ldg(a.alpha + j) : __ldg(a.alpha);
+                const float v = apply_act(fmaf(al, mine, a.bias ? __ldg(a.bias + o) : 0.0f), a.act);
+                const int64_t yi = t * a.m + o;
+                if (a.y_dtype == TBN_BF16) store_from_float(static_cast<__nv_bfloat16 *>(a.y), yi, v);
+                else store_from_float(static_cast<float *>(a.y), yi, v);
+            }
+        }
+    }
+}
+
 }  // namespace
 
 bool small_batch_supported(const LayerArgs &a)
@@ -335,6 +397,22 @@ double small_batch_estimate_us(const LayerArgs &a)
     const double blocks = (double)((int64_t)((r + 15) / 16) * ((a.T + 8 * nt - 1) / (8 * nt)));
     const double per_block = c * 16.0 * (double)a.n * 148.0 / 1e6;
     return 2.5 + per_block * (blocks > 148.0 ? blocks / 148.0 : 1.0) + 0.06 * a.k;
+}
+
+bool thin_dense_supported(const LayerArgs &a)
+{
+    if (a.is_conv || a.dense_a == nullptr || a.x_dtype != TBN_BF16 || a.q % a.n != 0 || a.n % 8 != 0) return false;
+    const int64_t r = a.q / a.n;
+    return r <= kThinRows && r * a.n <= kThinMaxWeights && (reinterpret_cast<uintptr_t>(a.x) & 15) == 0;
+}
+
+cudaError_t launch_thin_dense(const LayerArgs &a, cudaStream_t s)
+{
+    const int32_t r = (int32_t)(a.q / a.n);
+    const int64_t blocks_needed = (a.T + 7) / 8;                    // 8 warps (tokens) per block
+    const unsigned grid = (unsigned)(blocks_needed < 2 * 148 ? (blocks_needed > 0 ? blocks_needed : 1) : 2 * 148);
+    thin_dense_kernel<<<grid, 256, 0, s>>>(a, r);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_small_batch(const LayerArgs &a, cudaStream_t s)
