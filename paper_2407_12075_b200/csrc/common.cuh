@@ -47,6 +47,27 @@ __device__ __forceinline__ uint32_t tile_bit(const uint32_t *__restrict__ words,
     return (__ldg(words + (i >> 5)) >> (uint32_t)(i & 31)) & 1u;
 }
 
+// ---- programmatic dependent launch ----------------------------------------------------------------
+// A kernel launched with launch_pdl() may be scheduled while the previous kernel of the stream is still draining:
+// it calls pdl_launch_dependents() first thing (so that ITS successor may be scheduled early too) and pdl_wait()
+// before it reads or writes any global memory another kernel may touch; pdl_wait() returns once every earlier
+// kernel of the stream has completed and its writes are visible.  In a kernel launched the ordinary way both are
+// no-ops.  Only the launch latency is hidden; nothing runs out of order.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- description of one layer call, filled by the C entry points --------------------------------
 struct LayerArgs {
     const void *x;

@@ -203,6 +203,8 @@ small_mma_kernel(const LayerArgs a, int32_t r)
 {
     __shared__ float red[kMmaMaxWarps / NT][NT][16][8];          // [warp][token tile][row][token]: 16 KB
     __shared__ float alpha_s[64];
+    pdl_launch_dependents();
+    pdl_wait();                                                  // the activations may come from the previous kernel
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -281,10 +283,9 @@ cudaError_t launch_small_mma(const LayerArgs &a, int32_t r, cudaStream_t s)
     int nw = 1;
     while (nw < kMmaMaxWarps / nt && nw < n_spans && row_blocks * tok_blocks * nw < 148 * 16) nw *= 2;
     const dim3 grid((unsigned)row_blocks, (unsigned)tok_blocks);
-    if (nt == 1) small_mma_kernel<1><<<grid, nw * 32, 0, s>>>(a, r);
-    else if (nt == 2) small_mma_kernel<2><<<grid, nw * 32, 0, s>>>(a, r);
-    else small_mma_kernel<4><<<grid, nw * 32, 0, s>>>(a, r);
-    return cudaGetLastError();
+    if (nt == 1) return launch_pdl(small_mma_kernel<1>, grid, dim3(nw * 32), 0, s, a, r);
+    if (nt == 2) return launch_pdl(small_mma_kernel<2>, grid, dim3(nw * 32), 0, s, a, r);
+    return launch_pdl(small_mma_kernel<4>, grid, dim3(nw * 32), 0, s, a, r);
 }
 
 template <typename XT, int RW>
