@@ -361,6 +361,82 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
             ok = wait_bar(smem_u32(&ctl->d_full[pd.stage]), pd.phase, abort_flag, p.status, (6 << 24) | (bid & 0xffff));
             if (!ok) break;
             tc_fence_after();
+            if (rows_direct && (p.Wo & 15) == 0) {
+                // Rows made of whole 16-pixel items (32 bytes of bf16): software-pipelined.  The tensor-memory load of
+                // item i+1 is issued before item i is scaled, converted and stored, so its latency is off the path;
+                // the accumulator goes back to the MMA warp right after the last load.  Items are walked with
+                // counters (image, row, item in row): no divisions in this single-warp instruction stream.
+                const int32_t rows_here = min(p.R, p.Ho - oh0);
+                const int32_t per_row = p.Wo >> 4;
+                const int32_t imgs = min(p.G, p.Nb - img0);
+                const int32_t n_items = imgs * rows_here * per_row;
+                const int64_t img_pitch = (int64_t)p.m * out_plane;
+                __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.y) +
+                                     ((int64_t)img0 * p.m + (ch_valid ? o : 0)) * out_plane + (int64_t)oh0 * p.Wo;
+                uint32_t col = tmem_base + lane_base + pd.stage * kNMax;     // column of the item being loaded
+                int32_t ld_pc = 0, ld_oh = 0, ld_g = 0;                      // its coordinates
+                int32_t st_pc = 0, st_oh = 0;                                // coordinates of the item being stored
+                uint32_t cur[16], nxt[16];
+                __syncwarp();
+                if (n_items > 0) tmem_ld_32x16(col, cur);
+                tc_wait_ld();
+                for (int32_t it = 0; it < n_items; ++it) {
+                    const bool more = it + 1 < n_items;
+                    if (more) {                                            // advance the load cursor and issue the next load
+                        if (++ld_pc == per_row) {
+                            ld_pc = 0;
+                            if (++ld_oh == rows_here) { ld_oh = 0; ++ld_g; }
+                        }
+                        col = tmem_base + lane_base + pd.stage * kNMax + ld_g * p.slot_pos + ld_oh * p.PW + ld_pc * 16;
+                        __syncwarp();
+                        tmem_ld_32x16(col, nxt);
+                    } else {                                               // everything is in registers: hand the accumulator back
+                        tc_fence_before();
+                        mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));
+                    }
+                    uint32_t pk[8];
+                    if (p.act == TBN_ACT_RELU) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const float v0 = fmaxf(fmaf(al, __uint_as_float(cur[2 * i]), bs), 0.0f);
+                            const float v1 = fmaxf(fmaf(al, __uint_as_float(cur[2 * i + 1]), bs), 0.0f);
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+                            pk[i] = *reinterpret_cast<const uint32_t *>(&h);
+                        }
+                    } else if (p.act == TBN_ACT_GELU) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const float v0 = gelu_erf(fmaf(al, __uint_as_float(cur[2 * i]), bs));
+                            const float v1 = gelu_erf(fmaf(al, __uint_as_float(cur[2 * i + 1]), bs));
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+                            pk[i] = *reinterpret_cast<const uint32_t *>(&h);
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(fmaf(al, __uint_as_float(cur[2 * i]), bs),
+                                                                           fmaf(al, __uint_as_float(cur[2 * i + 1]), bs));
+                            pk[i] = *reinterpret_cast<const uint32_t *>(&h);
+                        }
+                    }
+                    if (ch_valid) st_global_v8(dst + st_oh * p.Wo + st_pc * 16, pk);   // 32-byte aligned: Wo % 16 == 0
+                    if (++st_pc == per_row) {
+                        st_pc = 0;
+                        if (++st_oh == rows_here) { st_oh = 0; dst += img_pitch; }
+                    }
+                    if (more) {
+                        tc_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) cur[i] = nxt[i];
+                    }
+                }
+                if (n_items <= 0) {
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));
+                }
+                pd.advance(2);
+                continue;
+            }
             if (rows_direct) {
                 // One TMEM load per output row piece: 8 consecutive accumulator columns starting at the row's first
                 // position are 8 consecutive output pixels of this thread's channel -> one 16-byte store (two
