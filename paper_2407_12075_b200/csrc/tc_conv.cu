@@ -35,6 +35,13 @@ namespace tbn {
 
 namespace {
 
+// (lo, hi) -> bf16x2 with round-to-nearest-even and negative values replaced by +0: ReLU for free.
+__device__ __forceinline__ uint32_t pack_bf16x2_relu(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
 using namespace tc;
 
 constexpr int kProdWarps = 6;           // patch producers
@@ -361,13 +368,19 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
             ok = wait_bar(smem_u32(&ctl->d_full[pd.stage]), pd.phase, abort_flag, p.status, (6 << 24) | (bid & 0xffff));
             if (!ok) break;
             tc_fence_after();
-            if (rows_direct && (p.Wo & 15) == 0) {
+            if (rows_direct && ((p.Wo & 15) == 0 || p.Wo == 8)) {
                 // Rows made of whole 16-pixel items (32 bytes of bf16): software-pipelined.  The tensor-memory load of
                 // item i+1 is issued before item i is scaled, converted and stored, so its latency is off the path;
                 // the accumulator goes back to the MMA warp right after the last load.  Items are walked with
                 // counters (image, row, item in row): no divisions in this single-warp instruction stream.
-                const int32_t rows_here = min(p.R, p.Ho - oh0);
-                const int32_t per_row = p.Wo >> 4;
+                // With 8-pixel rows an item is two consecutive rows (contiguous in NCHW); the unit "row" below is then
+                // a row pair and a pair without a second row is stored as 16 bytes.
+                const bool pair_rows = p.Wo == 8;
+                const int32_t real_rows = min(p.R, p.Ho - oh0);
+                const int32_t rows_here = pair_rows ? (real_rows + 1) >> 1 : real_rows;
+                const int32_t per_row = pair_rows ? 1 : p.Wo >> 4;
+                const int32_t row_cols = pair_rows ? 2 * p.PW : p.PW;       // accumulator columns per unit row
+                const int32_t row_elems = pair_rows ? 16 : p.Wo;            // output elements per unit row
                 const int32_t imgs = min(p.G, p.Nb - img0);
                 const int32_t n_items = imgs * rows_here * per_row;
                 const int64_t img_pitch = (int64_t)p.m * out_plane;
@@ -377,8 +390,20 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                 int32_t ld_pc = 0, ld_oh = 0, ld_g = 0;                      // its coordinates
                 int32_t st_pc = 0, st_oh = 0;                                // coordinates of the item being stored
                 uint32_t cur[16], nxt[16];
+                auto load_item = [&](uint32_t c, int32_t unit_row, uint32_t (&dstv)[16]) {
+                    if (!pair_rows) {
+                        tmem_ld_32x16(c, dstv);
+                    } else {
+                        uint32_t lo[8], hi[8];
+                        tmem_ld_32x8(c, lo);
+                        // a missing second row re-reads the first (in range); it is not stored
+                        tmem_ld_32x8(c + (2 * unit_row + 1 < real_rows ? (uint32_t)p.PW : 0u), hi);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) { dstv[i] = lo[i]; dstv[i + 8] = hi[i]; }
+                    }
+                };
                 __syncwarp();
-                if (n_items > 0) tmem_ld_32x16(col, cur);
+                if (n_items > 0) load_item(col, 0, cur);
                 tc_wait_ld();
                 for (int32_t it = 0; it < n_items; ++it) {
                     const bool more = it + 1 < n_items;
@@ -387,9 +412,9 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                             ld_pc = 0;
                             if (++ld_oh == rows_here) { ld_oh = 0; ++ld_g; }
                         }
-                        col = tmem_base + lane_base + pd.stage * kNMax + ld_g * p.slot_pos + ld_oh * p.PW + ld_pc * 16;
+                        col = tmem_base + lane_base + pd.stage * kNMax + ld_g * p.slot_pos + ld_oh * row_cols + ld_pc * 16;
                         __syncwarp();
-                        tmem_ld_32x16(col, nxt);
+                        load_item(col, ld_oh, nxt);
                     } else {                                               // everything is in registers: hand the accumulator back
                         tc_fence_before();
                         mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));
@@ -397,12 +422,9 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                     uint32_t pk[8];
                     if (p.act == TBN_ACT_RELU) {
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const float v0 = fmaxf(fmaf(al, __uint_as_float(cur[2 * i]), bs), 0.0f);
-                            const float v1 = fmaxf(fmaf(al, __uint_as_float(cur[2 * i + 1]), bs), 0.0f);
-                            const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
-                            pk[i] = *reinterpret_cast<const uint32_t *>(&h);
-                        }
+                        for (int i = 0; i < 8; ++i)     // the conversion clamps negative values to zero: no separate max
+                            pk[i] = pack_bf16x2_relu(fmaf(al, __uint_as_float(cur[2 * i]), bs),
+                                                     fmaf(al, __uint_as_float(cur[2 * i + 1]), bs));
                     } else if (p.act == TBN_ACT_GELU) {
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
@@ -419,7 +441,16 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                             pk[i] = *reinterpret_cast<const uint32_t *>(&h);
                         }
                     }
-                    if (ch_valid) st_global_v8(dst + st_oh * p.Wo + st_pc * 16, pk);   // 32-byte aligned: Wo % 16 == 0
+                    if (ch_valid) {
+                        __nv_bfloat16 *q = dst + st_oh * row_elems + st_pc * 16;
+                        const bool both = !pair_rows || 2 * st_oh + 1 < real_rows;
+                        if (both && (reinterpret_cast<uintptr_t>(q) & 31u) == 0) {
+                            st_global_v8(q, pk);
+                        } else {                                           // odd image height: 16-byte aligned only
+                            *reinterpret_cast<uint4 *>(q) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                            if (both) *reinterpret_cast<uint4 *>(q + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                        }
+                    }
                     if (++st_pc == per_row) {
                         st_pc = 0;
                         if (++st_oh == rows_here) { st_oh = 0; dst += img_pitch; }

@@ -104,6 +104,9 @@ TENSOR_CONVS = [
     (3, 32, 16, 2, 2, 0, 11, 13),      # stride 2 without padding
     (2, 64, 48, 1, 2, 2, 9, 9),        # padding 2, k = 1
     (1, 16, 16, 16, 1, 1, 40, 170),    # widest row that still fits, one distinct filter
+    (3, 32, 16, 2, 2, 1, 13, 16),      # 8-pixel output rows stored in pairs, odd output height (7 x 8)
+    (2, 32, 16, 2, 1, 1, 9, 16),       # 16-pixel rows, odd height
+    (1, 32, 16, 2, 1, 1, 6, 48),       # three 16-pixel items per row
 ]
 
 
@@ -118,6 +121,19 @@ def test_tensor_conv_matches_oracle(Nb, Cout, Cin, k, stride, pad, H, W):
         torch.cuda.synchronize()
         assert_close(to_np64(y), ref, f"tensor conv {Cout}x{Cin} s{stride} p{pad} {H}x{W}")
     assert B.tbn_last_device_status() == (0, 0)
+
+
+@pytest.mark.parametrize("act", [B.ACT_NONE, B.ACT_GELU])
+def test_tensor_conv_other_activations_and_bias(act):
+    # the ReLU epilogue clamps inside the bf16 conversion; the other activations take their own branches
+    x, Wt = synth.conv_layer(9, 3, 32, 16, 16, 64, 3, 3)
+    words, al = O.prepare(Wt, 4, True)
+    bias = synth.normal(9, 300, 64, 0.3)
+    ref = O.conv2d(x, words, 4, al, True, 64, 32, 3, 3, 1, 1, bias=bias.astype(np.float64), act=act)
+    y = B.tbn_conv2d_fwd(to_dev(x), 64, 3, 3, 1, 1, to_dev(words), 4, to_dev(al), 1, bias=to_dev(bias), act=act,
+                         path=B.PATH_TENSOR)
+    torch.cuda.synchronize()
+    assert_close(to_np64(y), ref, f"tensor conv act {act}")
 
 
 def test_tensor_conv_fp32_bias_and_agrees_with_generic():
