@@ -503,6 +503,35 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                             for (int e = 0; e < 8; ++e) z[i][e] = fmaxf(z[i][e], 0.0f);
                     }
                     const int64_t tok_first = tok0 + ch * 32 + 8 * ew + tsub + 2 * kSlots * iset;
+                    if (plain && p.y_bf16 && vec_ok && nvalid >= 8) {
+                        // The common case, with everything that does not depend on j hoisted out of the k loop: per
+                        // repetition 8 multiplies, 4 packs and one 16-byte store per token, nothing else.
+                        __nv_bfloat16 *yb[kSlots];
+                        bool tv[kSlots];
+#pragma unroll
+                        for (int i = 0; i < kSlots; ++i) {
+                            const int64_t tok = tok_first + 2 * i;
+                            tv[i] = tok < p.T;
+                            yb[i] = static_cast<__nv_bfloat16 *>(p.y) + tok * p.m + blk0 + f0;
+                        }
+                        const int32_t kk = p.k, rr = p.r;
+                        for (int32_t j = 0; j < kk; ++j) {
+                            const float al = j < kMaxAlpha ? ctl->alpha[j]
+                                                           : (p.per_tile ? __ldg(p.alpha + j) : __ldg(p.alpha));
+#pragma unroll
+                            for (int i = 0; i < kSlots; ++i) {
+                                uint32_t pk[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const __nv_bfloat162 h = __floats2bfloat162_rn(al * z[i][2 * e], al * z[i][2 * e + 1]);
+                                    pk[e] = *reinterpret_cast<const uint32_t *>(&h);
+                                }
+                                if (tv[i]) *reinterpret_cast<uint4 *>(yb[i]) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                                yb[i] += rr;
+                            }
+                        }
+                        continue;
+                    }
                     for (int32_t j = 0; j < p.k; ++j) {
                         const float al = j < kMaxAlpha ? ctl->alpha[j]
                                                        : (p.per_tile ? __ldg(p.alpha + j) : __ldg(p.alpha));
