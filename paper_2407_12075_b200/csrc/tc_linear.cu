@@ -63,19 +63,6 @@ __device__ __forceinline__ int epi_bar_count(bool pred) {
     return n;
 }
 
-// (al * lo, al * hi) -> bf16x2, round to nearest even: one packed fp32 multiply (two lanes per instruction on sm_100)
-// and one conversion.
-__device__ __forceinline__ uint32_t scale_pack_bf16x2(float al, float lo, float hi) {
-    uint32_t d;
-    asm("{\n.reg .b64 a, b, c;\n.reg .f32 x, y;\n"
-        "mov.b64 a, {%1, %2};\nmov.b64 b, {%3, %3};\n"
-        "mul.rn.f32x2 c, a, b;\n"
-        "mov.b64 {x, y}, c;\n"
-        "cvt.rn.bf16x2.f32 %0, y, x;\n}"
-        : "=r"(d) : "f"(lo), "f"(hi), "f"(al));
-    return d;
-}
-
 // ---- shared-memory control block -----------------------------------------------------------------
 template <int SX>
 struct Control {
@@ -535,7 +522,10 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                             for (int i = 0; i < kSlots; ++i) {
                                 uint32_t pk[4];
 #pragma unroll
-                                for (int e = 0; e < 4; ++e) pk[e] = scale_pack_bf16x2(al, z[i][2 * e], z[i][2 * e + 1]);
+                                for (int e = 0; e < 4; ++e) {
+                                    const __nv_bfloat162 h = __floats2bfloat162_rn(al * z[i][2 * e], al * z[i][2 * e + 1]);
+                                    pk[e] = *reinterpret_cast<const uint32_t *>(&h);
+                                }
                                 if (tv[i]) *reinterpret_cast<uint4 *>(yb[i]) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                                 yb[i] += rr;
                             }
@@ -699,7 +689,7 @@ int launch_config(const LayerArgs &a, TcParams p, int splits, void *scratch, cud
 // Tile shape and split-K factor for one call.  Cost model in nanoseconds per CTA, fitted to timelines and sweeps on
 // B200 (n = 8192; T = 64 .. 16384): the issuing thread needs about 77 ns per MMA whatever the token tile, plus 0.09 ns
 // per token; a configuration with only two decoded-weight slots pays about 100 ns of hand-off per stage; the epilogue
-// is bound by its stores (about 38 bytes per ns and SM, i.e. 6.7 ns per token and repetition for 128 rows) plus 250 ns
+// is bound by its stores (about 34 bytes per ns and SM, i.e. 7.5 ns per token and repetition for 128 rows) plus 250 ns
 // per 32-token block; every tile costs about 1.5 us of hand-over.  With two accumulator buffers the epilogue hides
 // behind the next tile's main loop except for the last tile.
 // When the output has fewer tiles than the GPU has SMs, the contraction is split over several CTAs per tile
@@ -727,7 +717,7 @@ Plan plan_linear(const LayerArgs &a)
         const int k_stages = (a.n + c.ka * kAtomK - 1) / (c.ka * kAtomK);
         const bool four_slots = c.db * c.na * c.ntok + 4 * c.na * c.ka * 32 <= 512;    // decoded-weight slots in tensor memory
         const double stage = c.na * c.ka * 4 * (0.09 * c.ntok + 77.0) + (four_slots ? 0.0 : 100.0);
-        const double epi = c.na * (double)c.ntok * a.k * 6.7 + c.na * (c.ntok / 32.0) * 250.0;
+        const double epi = c.na * (double)c.ntok * a.k * 7.5 + c.na * (c.ntok / 32.0) * 250.0;
         const double per_tile = 1500.0;                 // tile hand-over: first bit words, barrier round trips
         const double dump = c.na * (c.ntok / 32.0) * 60.0 * 2.0;
         for (int sp = 1; sp <= 16; sp *= 2) {
