@@ -689,7 +689,7 @@ int launch_config(const LayerArgs &a, TcParams p, int splits, void *scratch, cud
 // Tile shape and split-K factor for one call.  Cost model in nanoseconds per CTA, fitted to timelines and sweeps on
 // B200 (n = 8192; T = 64 .. 16384): the issuing thread needs about 77 ns per MMA whatever the token tile, plus 0.09 ns
 // per token; a configuration with only two decoded-weight slots pays about 100 ns of hand-off per stage; the epilogue
-// is bound by its stores (about 34 bytes per ns and SM, i.e. 7.5 ns per token and repetition for 128 rows) plus 250 ns
+// is bound by its stores (about 38 bytes per ns and SM, i.e. 6.7 ns per token and repetition for 128 rows) plus 250 ns
 // per 32-token block; every tile costs about 1.5 us of hand-over.  With two accumulator buffers the epilogue hides
 // behind the next tile's main loop except for the last tile.
 // When the output has fewer tiles than the GPU has SMs, the contraction is split over several CTAs per tile
@@ -717,7 +717,7 @@ Plan plan_linear(const LayerArgs &a)
         const int k_stages = (a.n + c.ka * kAtomK - 1) / (c.ka * kAtomK);
         const bool four_slots = c.db * c.na * c.ntok + 4 * c.na * c.ka * 32 <= 512;    // decoded-weight slots in tensor memory
         const double stage = c.na * c.ka * 4 * (0.09 * c.ntok + 77.0) + (four_slots ? 0.0 : 100.0);
-        const double epi = c.na * (double)c.ntok * a.k * 7.5 + c.na * (c.ntok / 32.0) * 250.0;
+        const double epi = c.na * (double)c.ntok * a.k * 6.7 + c.na * (c.ntok / 32.0) * 250.0;
         const double per_tile = 1500.0;                 // tile hand-over: first bit words, barrier round trips
         const double dump = c.na * (c.ntok / 32.0) * 60.0 * 2.0;
         for (int sp = 1; sp <= 16; sp *= 2) {
