@@ -50,10 +50,10 @@ def algorithmic_bytes(T: int, k: int) -> float:
 
 
 # DRAM traffic of the dominant launch (k = 2) from the ncu capture summarised in
-# profiles/tc_linear_k2_T8192_ncu_full.md: 236.2 MB at T = 8192; traffic is proportional to T.  The figure is
+# profiles/tc_linear_k2_T8192_ncu_full.md: 234.7 MB at T = 8192; traffic is proportional to T.  The figure is
 # only valid for the kernel source it was taken from: the hash below covers tc_linear.cu and tc_common.cuh.
-TRAFFIC_BYTES_AT_T8192 = 138.547456e6 + 97.607424e6
-TRAFFIC_SOURCE_HASH = "12f54ce62be84da5"
+TRAFFIC_BYTES_AT_T8192 = 138.608128e6 + 96.077312e6
+TRAFFIC_SOURCE_HASH = "8e21c2b5d0c26150"
 
 
 def measured_traffic(T: int):
