@@ -12,10 +12,10 @@
 // memory.  Each decoded 128 x 64 block is reused for all NTOK tokens of the CTA tile, and each
 // activation stage is reused by NA blocks of 128 weight rows.
 //
-// Warp roles (14 warps): 0 = TMA producer (activation stages, 128-byte swizzle), 1 = MMA issuer and
+// Warp roles (10 warps, 14 with EPI == 8): 0 = TMA producer (activation stages, 128-byte swizzle), 1 = MMA issuer and
 // TMEM owner, 2-5 = tile decode (bits -> +-1 bf16 pairs -> tcgen05.st), 6-9 = epilogue (tcgen05.ld ->
-// alpha/bias/activation -> k-fold replicated stores), 10-13 = epilogue helpers (half of the arithmetic
-// and stores; they never touch tensor memory).  All hand-offs are mbarriers; every wait is
+// alpha/bias/activation -> k-fold replicated stores), 10-13 = optional epilogue helpers (half of the
+// arithmetic and stores when the activation is expensive; they never touch tensor memory).  All hand-offs are mbarriers; every wait is
 // bounded by a wall-clock limit, after which the CTA records TBN_ERR_TIMEOUT, drains and returns.
 #include <cstdlib>
 
