@@ -325,8 +325,6 @@ expand_kernel(const uint32_t *__restrict__ tile_bits, int64_t N, int64_t q, cons
 __global__ void __launch_bounds__(256)
 f32_to_bf16_kernel(const float *__restrict__ src, __nv_bfloat16 *__restrict__ dst, int64_t count)
 {
-    pdl_launch_dependents();
-    pdl_wait();
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     const int64_t pairs = count >> 1;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < pairs; i += stride) {
@@ -345,8 +343,6 @@ f32_to_bf16_kernel(const float *__restrict__ src, __nv_bfloat16 *__restrict__ ds
 __global__ void __launch_bounds__(256)
 fold_kernel(const FoldJobs jobs)
 {
-    pdl_launch_dependents();
-    pdl_wait();
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int32_t jb = 0; jb < jobs.count; ++jb) {
         const FoldJob &J = jobs.job[jb];
@@ -458,12 +454,14 @@ cudaError_t launch_fold(const FoldJobs &jobs, cudaStream_t s)
         const int64_t t = (int64_t)jobs.job[j].rows * jobs.job[j].r_prev;
         most = t > most ? t : most;
     }
-    return launch_pdl(fold_kernel, dim3(grid_for(most, 256, 148 * 8)), dim3(256), 0, s, jobs);
+    fold_kernel<<<grid_for(most, 256, 148 * 8), 256, 0, s>>>(jobs);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_f32_to_bf16(const float *src, __nv_bfloat16 *dst, int64_t count, cudaStream_t s)
 {
-    return launch_pdl(f32_to_bf16_kernel, dim3(grid_for(count / 2 + 1, 256, 148 * 8)), dim3(256), 0, s, src, dst, count);
+    f32_to_bf16_kernel<<<grid_for(count / 2 + 1, 256, 148 * 8), 256, 0, s>>>(src, dst, count);
+    return cudaGetLastError();
 }
 
 }  // namespace tbn

@@ -325,8 +325,6 @@ __global__ void __launch_bounds__(256)
 thin_dense_kernel(const LayerArgs a, int32_t r)
 {
     __shared__ __align__(16) float w_s[kThinMaxWeights];
-    pdl_launch_dependents();
-    pdl_wait();                                                  // weights and activations come from earlier kernels
     const int32_t n = a.n;
     const __nv_bfloat16 *W = static_cast<const __nv_bfloat16 *>(a.dense_a);
     // 16-byte loads (n % 8 == 0, the rows are 16-byte aligned), all of a thread's loads in flight together
@@ -423,7 +421,8 @@ cudaError_t launch_thin_dense(const LayerArgs &a, cudaStream_t s)
     const int32_t r = (int32_t)(a.q / a.n);
     const int64_t blocks_needed = (a.T + 7) / 8;                    // 8 warps (tokens) per block
     const unsigned grid = (unsigned)(blocks_needed < 2 * 148 ? (blocks_needed > 0 ? blocks_needed : 1) : 2 * 148);
-    return launch_pdl(thin_dense_kernel, dim3(grid), dim3(256), 0, s, a, r);
+    thin_dense_kernel<<<grid, 256, 0, s>>>(a, r);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_small_batch(const LayerArgs &a, cudaStream_t s)

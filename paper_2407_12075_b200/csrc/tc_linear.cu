@@ -128,8 +128,6 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
     // instruction descriptor: D fp32, A and B bf16, both K-major, N = NTOK, M = 128
     constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NTOK >> 3) << 17) | (8u << 24);
 
-    pdl_launch_dependents();      // the next kernel of the stream may be scheduled while this one runs ...
-    pdl_wait();                   // ... and this one touches memory only once its predecessors have completed
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     uint8_t *smem = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
@@ -684,7 +682,8 @@ int launch_config(const LayerArgs &a, TcParams p, int splits, void *scratch, cud
     if (sms <= 0) return TBN_ERR_CUDA;
     const int64_t tiles = out_tiles * splits;
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
-    return launch_pdl(kern, dim3(grid), dim3(kBaseThreads + (helpers ? 256 : 128)), smem, s, map, p) == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+    kern<<<grid, kBaseThreads + (helpers ? 256 : 128), smem, s>>>(map, p);
+    return cudaGetLastError() == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
 }
 
 // Tile shape and split-K factor for one call.  Cost model in nanoseconds per CTA, fitted to timelines and sweeps on
