@@ -461,7 +461,9 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     # ---- the oracle on the host cores, rank 0 at N = 1 only ---------------------------------------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        rows = 96
+        # a short probe sizes the sample to roughly 12 s of CPU work on whatever host this is
+        probe_dt, probe_n, _ = oracle_sample(x_np, W_np, 4, 32)
+        rows = int(min(max(32 * 12.0 / max(probe_dt, 1e-3), 96), 4096))
         dt, n, cores = oracle_sample(x_np, W_np, 4, rows)
         cpu = dict(value=algorithmic_flops(n, 4) / dt / 1e12, unit=UNIT, cores=cores, kind="oracle",
                    sample=f"{n} seeded token rows of {T} x all 8192 outputs at k=4, {dt:.1f} s; the oracle does the "
