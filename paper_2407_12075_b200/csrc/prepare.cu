@@ -161,8 +161,7 @@ aggregate_kernel(const float *__restrict__ W, const float *__restrict__ A, int64
 // Streaming form for k <= kAggStreamK: a fixed grid of blocks walks the column chunks (chunk = block, block + grid,
 // ...), so the per-block cost of publishing partial sums, the fence and the ticket is paid once per block instead of
 // once per 4096 columns, and a thread keeps its |.| sums per tile in fp64 registers across chunks.  Loads are
-// issued 4 rows (2 when a separate alpha source is read too) x kAggIter groups at a time, i.e. 16 independent
-// 16-byte loads per thread, before the
+// issued kAggRows rows x kAggIter groups at a time (8 independent 16-byte loads per thread and source) before the
 // sequential fp32 adds that the bit rule requires.
 constexpr int kAggStreamK = 16;
 constexpr int kAggRows = 2;
@@ -173,7 +172,6 @@ aggregate_stream_kernel(const float *__restrict__ W, const float *__restrict__ A
                         int per_tile, uint32_t *__restrict__ tile_bits, int64_t n_words,
                         float *__restrict__ alpha, AggScratch *scratch, int64_t n_chunks)
 {
-    constexpr int kRowsNow = HAS_A ? kAggRows : 2 * kAggRows;   // rows loaded together (two sources halve it)
     __shared__ double warp_part[kAggStreamK][kAggThreads / 32];
     __shared__ double red[kAggThreads];
     __shared__ unsigned int s_ticket;
@@ -196,12 +194,12 @@ aggregate_stream_kernel(const float *__restrict__ W, const float *__restrict__ A
             for (int e = 0; e < kAggVec; ++e) s[it][e] = 0.0f;
 
 #pragma unroll
-        for (int j0 = 0; j0 < kAggStreamK; j0 += kRowsNow) {
+        for (int j0 = 0; j0 < kAggStreamK; j0 += kAggRows) {
             if (j0 >= k) break;                           // uniform
-            float w[kRowsNow][kAggIter][kAggVec];
-            float av[HAS_A ? kRowsNow : 1][kAggIter][kAggVec];
+            float w[kAggRows][kAggIter][kAggVec];
+            float av[HAS_A ? kAggRows : 1][kAggIter][kAggVec];
 #pragma unroll
-            for (int jj = 0; jj < kRowsNow; ++jj) {
+            for (int jj = 0; jj < kAggRows; ++jj) {
                 const bool row_ok = j0 + jj < k;
                 const int64_t row = (int64_t)(row_ok ? j0 + jj : 0) * q;
 #pragma unroll
@@ -226,7 +224,7 @@ aggregate_stream_kernel(const float *__restrict__ W, const float *__restrict__ A
                 }
             }
 #pragma unroll
-            for (int jj = 0; jj < kRowsNow; ++jj) {
+            for (int jj = 0; jj < kAggRows; ++jj) {
                 if (j0 + jj >= k) break;                  // uniform; a skipped row must not enter the fp32 sum
                 float ab = 0.0f;
 #pragma unroll
