@@ -151,26 +151,26 @@ template <int NT> struct SpanRegs {
     uint4 xb[NT][4];
 };
 
+// Loads of one span.  xrow[nt] points at this lane's token row (null when the lane has no token in that tile: its
+// registers were zeroed once and stay zero); `live` is false only for chunks past the end of a ragged last span.
 template <int NT>
 __device__ __forceinline__ void load_span(SpanRegs<NT> &sr, const uint32_t *bits_lo, const uint32_t *bits_hi,
-                                          const __nv_bfloat16 *x, int32_t n, int32_t n_chunks, int32_t span,
-                                          int c, int g, int64_t t0, int64_t T)
+                                          const __nv_bfloat16 *const (&xrow)[NT], int32_t chunk, bool live)
 {
-    const int32_t chunk = span * 4 + c;
-    const bool live = chunk < n_chunks;                          // ragged last span: activations read as zero
     const int32_t ch = live ? chunk : 0;
     sr.w_lo = __ldg(bits_lo + ch);
     sr.w_hi = __ldg(bits_hi + ch);
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-        const int64_t t = t0 + nt * 8 + g;
-        if (live && t < T) {
-            const uint4 *px = reinterpret_cast<const uint4 *>(x + t * n + (int64_t)ch * 32);
+        if (xrow[nt] != nullptr) {
+            if (live) {
+                const uint4 *px = reinterpret_cast<const uint4 *>(xrow[nt] + ch * 32);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) sr.xb[nt][i] = __ldg(px + i);
-        } else {
+                for (int i = 0; i < 4; ++i) sr.xb[nt][i] = __ldg(px + i);
+            } else {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) sr.xb[nt][i] = make_uint4(0u, 0u, 0u, 0u);
+                for (int i = 0; i < 4; ++i) sr.xb[nt][i] = make_uint4(0u, 0u, 0u, 0u);
+            }
         }
     }
 }
@@ -231,9 +231,23 @@ small_mma_kernel(const LayerArgs a, int32_t r)
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[nt][i] = 0.0f;
 
-    for (int32_t span = warp; span < n_spans; span += nw) {
-        SpanRegs<NT> sr;
-        load_span<NT>(sr, bits_lo, bits_hi, x, n, n_chunks, span, c, g, t0, a.T);
+    const __nv_bfloat16 *xrow[NT];                               // this lane's token row per tile, or null
+    SpanRegs<NT> sr;
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        const int64_t t = t0 + nt * 8 + g;
+        xrow[nt] = t < a.T ? x + t * n : nullptr;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) sr.xb[nt][i] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    const int32_t full_spans = n_chunks >> 2;                    // spans whose four chunks all exist
+    int32_t span = warp;
+    for (; span < full_spans; span += nw) {
+        load_span<NT>(sr, bits_lo, bits_hi, xrow, span * 4 + c, true);
+        contract_span<NT>(sr, acc);
+    }
+    if (span < n_spans) {                                        // the ragged last span, if this warp owns it
+        load_span<NT>(sr, bits_lo, bits_hi, xrow, span * 4 + c, span * 4 + c < n_chunks);
         contract_span<NT>(sr, acc);
     }
 
