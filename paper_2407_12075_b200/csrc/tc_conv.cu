@@ -428,8 +428,8 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                     } else if (p.act == TBN_ACT_GELU) {
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
-                            const float v0 = gelu_erf(fmaf(al, __uint_as_float(cur[2 * i]), bs));
-                            const float v1 = gelu_erf(fmaf(al, __uint_as_float(cur[2 * i + 1]), bs));
+                            const float v0 = gelu_tanh_bf16(fmaf(al, __uint_as_float(cur[2 * i]), bs));
+                            const float v1 = gelu_tanh_bf16(fmaf(al, __uint_as_float(cur[2 * i + 1]), bs));
                             const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
                             pk[i] = *reinterpret_cast<const uint32_t *>(&h);
                         }
@@ -498,7 +498,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                             for (int i = 0; i < 8; ++i) {
                                 float v0 = fmaf(al, __uint_as_float(v[2 * i]), bs), v1 = fmaf(al, __uint_as_float(v[2 * i + 1]), bs);
                                 if (p.act == TBN_ACT_RELU) { v0 = fmaxf(v0, 0.0f); v1 = fmaxf(v1, 0.0f); }
-                                else if (p.act == TBN_ACT_GELU) { v0 = apply_act(v0, TBN_ACT_GELU); v1 = apply_act(v1, TBN_ACT_GELU); }
+                                else if (p.act == TBN_ACT_GELU) { v0 = gelu_tanh_bf16(v0); v1 = gelu_tanh_bf16(v1); }
                                 const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
                                 pk[i] = *reinterpret_cast<const uint32_t *>(&h);
                             }

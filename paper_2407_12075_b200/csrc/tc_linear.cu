@@ -556,6 +556,11 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                                 for (int i = 0; i < kSlots; ++i)
 #pragma unroll
                                     for (int e = 0; e < 8; ++e) o[i][e] = al * z[i][e];
+                            } else if (p.act == TBN_ACT_GELU && p.y_bf16) {
+#pragma unroll
+                                for (int i = 0; i < kSlots; ++i)
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) o[i][e] = gelu_tanh_bf16(fmaf(al, z[i][e], b[e]));
                             } else if (p.act == TBN_ACT_GELU) {
 #pragma unroll
                                 for (int i = 0; i < kSlots; ++i)
