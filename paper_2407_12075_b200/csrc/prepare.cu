@@ -339,23 +339,43 @@ f32_to_bf16_kernel(const float *__restrict__ src, __nv_bfloat16 *__restrict__ ds
 // activation).  The previous layer's output is h[t][j*r1 + c] = alpha1_j * g[t][c] with g = act(z) (alpha >= 0, so
 // relu(alpha z) = alpha relu(z)), hence  sum_j sum_c B2[o][j*r1 + c] h[t][j*r1 + c] = sum_c g[t][c] * W[o][c]  with
 //     W[o][c] = sum_j alpha1_j * (bit2(o*n2 + j*r1 + c) ? +1 : -1),   n2 = k1 * r1.
-// One thread per (o, c); fp32 sum in increasing j, one rounding to bf16.
+// One thread per (o, c); fp32 sum in increasing j, one rounding to bf16.  The jobs of a launch run side by side
+// (blockIdx.y = job); the previous layer's alphas sit in shared memory and the k bit loads of an element are
+// independent of one another, so they are in flight together.
+constexpr int kFoldAlphas = 256;
+
 __global__ void __launch_bounds__(256)
 fold_kernel(const FoldJobs jobs)
 {
+    // the block's job, selected with compile-time indices so the parameter block is read in place
+    FoldJob J = jobs.job[0];
+#pragma unroll
+    for (int jb = 1; jb < kMaxFoldJobs; ++jb)
+        if ((int)blockIdx.y == jb) J = jobs.job[jb];
+    __shared__ float al_s[kFoldAlphas];
+    for (int j = threadIdx.x; j < J.k_prev && j < kFoldAlphas; j += blockDim.x)
+        al_s[j] = __ldg(J.alpha_prev + (J.per_tile_prev ? j : 0));
+    __syncthreads();
+
+    const int64_t total = (int64_t)J.rows * J.r_prev;
+    const bool narrow = total <= 0x7fffffff;                      // 32-bit division then
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int32_t jb = 0; jb < jobs.count; ++jb) {
-        const FoldJob &J = jobs.job[jb];
-        const int64_t total = (int64_t)J.rows * J.r_prev;
-        for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += stride) {
-            const int32_t o = (int32_t)(e / J.r_prev), c = (int32_t)(e % J.r_prev);
-            float acc = 0.0f;
-            for (int32_t j = 0; j < J.k_prev; ++j) {
-                const float al = J.per_tile_prev ? __ldg(J.alpha_prev + j) : __ldg(J.alpha_prev);
-                acc += tile_bit(J.tile_next, (int64_t)o * J.n_next + (int64_t)j * J.r_prev + c) ? al : -al;
-            }
-            J.w_eff[e] = __float2bfloat16_rn(acc);
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += stride) {
+        int64_t o, c;
+        if (narrow) {
+            const uint32_t oo = (uint32_t)e / (uint32_t)J.r_prev;
+            o = oo; c = (uint32_t)e - oo * (uint32_t)J.r_prev;
+        } else {
+            o = e / J.r_prev; c = e % J.r_prev;
         }
+        const int64_t first = o * J.n_next + c;                   // bit of repetition 0; repetition j is j * r_prev on
+        float acc = 0.0f;
+#pragma unroll 8
+        for (int32_t j = 0; j < J.k_prev; ++j) {
+            const float al = j < kFoldAlphas ? al_s[j] : __ldg(J.alpha_prev + (J.per_tile_prev ? j : 0));
+            acc += tile_bit(J.tile_next, first + (int64_t)j * J.r_prev) ? al : -al;
+        }
+        J.w_eff[e] = __float2bfloat16_rn(acc);
     }
 }
 
@@ -454,7 +474,7 @@ cudaError_t launch_fold(const FoldJobs &jobs, cudaStream_t s)
         const int64_t t = (int64_t)jobs.job[j].rows * jobs.job[j].r_prev;
         most = t > most ? t : most;
     }
-    fold_kernel<<<grid_for(most, 256, 148 * 8), 256, 0, s>>>(jobs);
+    fold_kernel<<<dim3((unsigned)grid_for(most, 256, 148 * 8), (unsigned)jobs.count), 256, 0, s>>>(jobs);
     return cudaGetLastError();
 }
 

@@ -434,7 +434,10 @@ cudaError_t launch_thin_dense(const LayerArgs &a, cudaStream_t s)
 {
     const int32_t r = (int32_t)(a.q / a.n);
     const int64_t blocks_needed = (a.T + 7) / 8;                    // 8 warps (tokens) per block
-    const unsigned grid = (unsigned)(blocks_needed < 2 * 148 ? (blocks_needed > 0 ? blocks_needed : 1) : 2 * 148);
+    // every block fills its own copy of the weight block: one token per warp while that fill is small (the layer is
+    // latency-bound: one pass of loads, sums and stores), two blocks per SM otherwise
+    const int64_t cap = (int64_t)r * a.n <= kThinMaxWeights / 2 ? 6 * 148 : 2 * 148;
+    const unsigned grid = (unsigned)(blocks_needed < cap ? (blocks_needed > 0 ? blocks_needed : 1) : cap);
     thin_dense_kernel<<<grid, 256, 0, s>>>(a, r);
     return cudaGetLastError();
 }
