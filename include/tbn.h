@@ -50,7 +50,9 @@ typedef enum {
 
 typedef enum { TBN_F32 = 0, TBN_BF16 = 1 } tbn_dtype;
 typedef enum { TBN_ALPHA_PER_LAYER = 0, TBN_ALPHA_PER_TILE = 1 } tbn_alpha_mode; /* 1 or k floats */
-typedef enum { TBN_ACT_NONE = 0, TBN_ACT_RELU = 1, TBN_ACT_GELU = 2 } tbn_act;   /* GELU: exact erf form */
+/* GELU is the erf form v * Phi(v): evaluated to 4e-7 for fp32 outputs; bf16 outputs of the tensor-core kernels use a
+ * tanh form fitted to it whose difference (<= 2.5e-5 + 2.5e-4 |v|) stays below the bf16 rounding of the result. */
+typedef enum { TBN_ACT_NONE = 0, TBN_ACT_RELU = 1, TBN_ACT_GELU = 2 } tbn_act;
 
 /* Which kernel family executes a forward call.  AUTO picks by shape. */
 typedef enum {
@@ -162,8 +164,14 @@ int tbn_linear_fp_tile_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, 
                            const float *bias, int act, void *y, int y_dtype,
                            void *workspace, size_t workspace_bytes, void *stream, int path);
 
-/* Same layer with HOST activations: x_host and y_host are host buffers (pinned memory recommended).
- * The call copies x to the device, runs tbn_linear_fwd, copies y back and synchronises `stream`.
+/* Same layer with HOST activations: x_host and y_host are host buffers (pinned memory recommended; with
+ * pageable memory the copies do not overlap anything).
+ * The call copies x to the device, runs tbn_linear_fwd, copies y back and synchronises `stream`; it returns
+ * when y_host is complete.  Token rows are independent (Algorithm 1 treats one input vector at a time), so a
+ * batch whose transfers exceed about 32 MiB goes through in up to 32 chunks of whole token rows: while one
+ * chunk is computed on `stream`, the next is copied in and the previous one copied out on two copy streams
+ * that the library creates once per device at the first such call (no device memory is allocated; calls on
+ * one device take turns on these streams).  Work queued on `stream` before the call is waited for first.
  * workspace (device) must hold tbn_linear_host_workspace_bytes(...) bytes: staging for x and y plus
  * the forward's own scratch.  tile_bits, alpha and bias stay device pointers (model state). */
 size_t tbn_linear_host_workspace_bytes(int64_t T, int32_t in_f, int32_t out_f, int32_t k,

@@ -3,6 +3,7 @@
 // touches the data on the host, and there is no CPU fallback.
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 
 #include "common.cuh"
 
@@ -38,6 +39,92 @@ inline bool valid_alpha_mode(int a) { return a == TBN_ALPHA_PER_LAYER || a == TB
 inline bool valid_act(int a) { return a == TBN_ACT_NONE || a == TBN_ACT_RELU || a == TBN_ACT_GELU; }
 inline size_t dtype_bytes(int d) { return d == TBN_BF16 ? 2 : 4; }
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ---- host-buffer forward: chunking and the per-device copy streams ------------------------------------------
+constexpr int kHostMaxChunks = 32;
+constexpr size_t kHostChunkBytes = 16u << 20;          // per direction and chunk: long enough for full link rate
+
+// Tokens per chunk of the host-buffer forward (a multiple of 256), or T when the batch goes through in one piece.
+int64_t host_chunk_tokens(int64_t T, int32_t in_f, int32_t out_f, int x_dtype, int y_dtype)
+{
+    const size_t x_row = (size_t)in_f * dtype_bytes(x_dtype), y_row = (size_t)out_f * dtype_bytes(y_dtype);
+    const size_t row = x_row > y_row ? x_row : y_row;
+    int64_t chunk = (int64_t)((kHostChunkBytes + row - 1) / row);
+    const int64_t at_most = (T + kHostMaxChunks - 1) / kHostMaxChunks;
+    if (chunk < at_most) chunk = at_most;
+    chunk = (chunk + 255) / 256 * 256;
+    return chunk * 2 > T ? T : chunk;                   // fewer than two full chunks: not worth the pipeline
+}
+
+// Scratch of the forward calls behind the host-buffer entry point: the largest need among the chunk sizes it runs.
+size_t host_inner_bytes(int64_t T, int32_t in_f, int32_t out_f, int32_t k, int x_dtype, int64_t chunk)
+{
+    if (chunk >= T) return tbn_linear_workspace_bytes(T, in_f, out_f, k, x_dtype);
+    size_t need = tbn_linear_workspace_bytes(chunk, in_f, out_f, k, x_dtype);
+    if (T % chunk != 0) {
+        const size_t tail = tbn_linear_workspace_bytes(T % chunk, in_f, out_f, k, x_dtype);
+        need = tail > need ? tail : need;
+    }
+    return need;
+}
+
+struct HostPipe {
+    std::mutex mu;
+    bool ready = false;
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t ev_in[kHostMaxChunks] = {}, ev_comp[kHostMaxChunks] = {}, ev_start = nullptr, ev_done = nullptr;
+};
+
+// The copy streams and events of the current device, created on first use (no device memory is allocated).
+HostPipe *host_pipe()
+{
+    static HostPipe pipes[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    HostPipe &hp = pipes[dev];
+    std::lock_guard<std::mutex> guard(hp.mu);
+    if (!hp.ready) {
+        bool ok = cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp.ev_start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp.ev_done, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; i < kHostMaxChunks && ok; ++i)
+            ok = cudaEventCreateWithFlags(&hp.ev_in[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&hp.ev_comp[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) return nullptr;
+        hp.ready = true;
+    }
+    return &hp;
+}
+
+// ---- MLP chain: a side stream for the folds ---------------------------------------------------------------------
+// The folds depend on the parameters only, so they can run beside the first layer.  One side stream and two events per
+// device, created at the first call that is not being captured into a graph (creating them would break the capture;
+// such a call, and any call after a failed creation, simply keeps the folds on the caller's stream).
+struct MlpFork {
+    std::mutex mu;
+    int state = 0;                                     // 0 = not created yet, 1 = ready, -1 = creation failed
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+};
+
+MlpFork *mlp_fork(cudaStream_t s)
+{
+    static MlpFork forks[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    MlpFork &f = forks[dev];
+    std::lock_guard<std::mutex> guard(f.mu);
+    if (f.state == 0) {
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(s, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return nullptr;
+        const bool ok = cudaStreamCreateWithFlags(&f.side, cudaStreamNonBlocking) == cudaSuccess &&
+                        cudaEventCreateWithFlags(&f.ev_fork, cudaEventDisableTiming) == cudaSuccess &&
+                        cudaEventCreateWithFlags(&f.ev_join, cudaEventDisableTiming) == cudaSuccess;
+        f.state = ok ? 1 : -1;
+    }
+    return f.state == 1 ? &f : nullptr;
+}
 
 // Validation shared by the fully-connected and convolution entry points.
 int check_layer_common(const void *x, int x_dtype, const uint32_t *tile, int32_t k, const float *alpha,
@@ -404,7 +491,7 @@ size_t tbn_linear_host_workspace_bytes(int64_t T, int32_t in_f, int32_t out_f, i
     if (T <= 0 || in_f <= 0 || out_f <= 0 || !valid_dtype(x_dtype) || !valid_dtype(y_dtype)) return 0;
     return round_up((size_t)T * in_f * dtype_bytes(x_dtype), 256) +
            round_up((size_t)T * out_f * dtype_bytes(y_dtype), 256) +
-           tbn_linear_workspace_bytes(T, in_f, out_f, k, x_dtype);
+           host_inner_bytes(T, in_f, out_f, k, x_dtype, host_chunk_tokens(T, in_f, out_f, x_dtype, y_dtype));
 }
 
 int tbn_linear_fwd_host(const void *x_host, int x_dtype, int64_t T, int32_t in_f, int32_t out_f,
@@ -416,23 +503,61 @@ int tbn_linear_fwd_host(const void *x_host, int x_dtype, int64_t T, int32_t in_f
         out_f <= 0)
         return TBN_ERR_INVALID_ARG;
     if (T == 0) return TBN_OK;
-    const size_t xb = round_up((size_t)T * in_f * dtype_bytes(x_dtype), 256);
-    const size_t yb = round_up((size_t)T * out_f * dtype_bytes(y_dtype), 256);
-    const size_t inner = tbn_linear_workspace_bytes(T, in_f, out_f, k, x_dtype);
+    const size_t x_row = (size_t)in_f * dtype_bytes(x_dtype), y_row = (size_t)out_f * dtype_bytes(y_dtype);
+    const size_t xb = round_up((size_t)T * x_row, 256);
+    const size_t yb = round_up((size_t)T * y_row, 256);
+    const int64_t chunk = host_chunk_tokens(T, in_f, out_f, x_dtype, y_dtype);
+    const size_t inner = host_inner_bytes(T, in_f, out_f, k, x_dtype, chunk);
     if (!workspace || !aligned16(workspace) || workspace_bytes < xb + yb + inner) return TBN_ERR_WORKSPACE;
     char *ws = static_cast<char *>(workspace);
-    void *x_dev = ws, *y_dev = ws + xb, *inner_ws = ws + xb + yb;
+    char *x_dev = ws, *y_dev = ws + xb;
+    void *inner_ws = ws + xb + yb;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (cudaMemcpyAsync(x_dev, x_host, (size_t)T * in_f * dtype_bytes(x_dtype), cudaMemcpyHostToDevice, s) !=
-        cudaSuccess)
-        return TBN_ERR_CUDA;
-    int rc = tbn_linear_fwd(x_dev, x_dtype, T, in_f, out_f, tile_bits, k, alpha, alpha_mode, bias, act, y_dev,
-                            y_dtype, inner_ws, inner, stream);
+
+    if (chunk >= T) {                     // small transfers: copy in, run, copy out on the caller's stream
+        if (cudaMemcpyAsync(x_dev, x_host, (size_t)T * x_row, cudaMemcpyHostToDevice, s) != cudaSuccess)
+            return TBN_ERR_CUDA;
+        int rc = tbn_linear_fwd(x_dev, x_dtype, T, in_f, out_f, tile_bits, k, alpha, alpha_mode, bias, act, y_dev,
+                                y_dtype, inner_ws, inner, stream);
+        if (rc != TBN_OK) return rc;
+        if (cudaMemcpyAsync(y_host, y_dev, (size_t)T * y_row, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+            return TBN_ERR_CUDA;
+        return cudaStreamSynchronize(s) == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+    }
+
+    // Token rows are independent, so the batch goes through in chunks: chunk c+1 is copied in and chunk c-1 copied
+    // out (two copy streams, both directions of the host link busy) while chunk c is computed on the caller's stream.
+    HostPipe *hp = host_pipe();
+    if (!hp) return TBN_ERR_CUDA;
+    std::lock_guard<std::mutex> guard(hp->mu);        // the copy streams and events are shared by the calls on a device
+    bool cuda_ok = cudaEventRecord(hp->ev_start, s) == cudaSuccess &&
+                   cudaStreamWaitEvent(hp->in, hp->ev_start, 0) == cudaSuccess &&
+                   cudaStreamWaitEvent(hp->out, hp->ev_start, 0) == cudaSuccess;
+    int rc = TBN_OK;
+    int c = 0;
+    for (int64_t t0 = 0; t0 < T && cuda_ok && rc == TBN_OK; t0 += chunk, ++c) {
+        const int64_t tc = T - t0 < chunk ? T - t0 : chunk;
+        cuda_ok = cudaMemcpyAsync(x_dev + t0 * x_row, static_cast<const char *>(x_host) + t0 * x_row, tc * x_row,
+                                  cudaMemcpyHostToDevice, hp->in) == cudaSuccess &&
+                  cudaEventRecord(hp->ev_in[c], hp->in) == cudaSuccess &&
+                  cudaStreamWaitEvent(s, hp->ev_in[c], 0) == cudaSuccess;
+        if (!cuda_ok) break;
+        rc = tbn_linear_fwd(x_dev + t0 * x_row, x_dtype, tc, in_f, out_f, tile_bits, k, alpha, alpha_mode, bias, act,
+                            y_dev + t0 * y_row, y_dtype, inner_ws, inner, stream);
+        if (rc != TBN_OK) break;
+        cuda_ok = cudaEventRecord(hp->ev_comp[c], s) == cudaSuccess &&
+                  cudaStreamWaitEvent(hp->out, hp->ev_comp[c], 0) == cudaSuccess &&
+                  cudaMemcpyAsync(static_cast<char *>(y_host) + t0 * y_row, y_dev + t0 * y_row, tc * y_row,
+                                  cudaMemcpyDeviceToHost, hp->out) == cudaSuccess;
+    }
+    // join: the caller's stream continues after the last copy out, then the call waits for it.  The copy streams are
+    // drained even after an error, so nothing of this call is still in flight when it returns.
+    const bool joined = cudaEventRecord(hp->ev_done, hp->out) == cudaSuccess &&
+                        cudaStreamWaitEvent(s, hp->ev_done, 0) == cudaSuccess;
+    const bool drained = cudaStreamSynchronize(hp->in) == cudaSuccess && cudaStreamSynchronize(hp->out) == cudaSuccess &&
+                         cudaStreamSynchronize(s) == cudaSuccess;
     if (rc != TBN_OK) return rc;
-    if (cudaMemcpyAsync(y_host, y_dev, (size_t)T * out_f * dtype_bytes(y_dtype), cudaMemcpyDeviceToHost, s) !=
-        cudaSuccess)
-        return TBN_ERR_CUDA;
-    return cudaStreamSynchronize(s) == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+    return cuda_ok && joined && drained ? TBN_OK : TBN_ERR_CUDA;
 }
 
 size_t tbn_conv2d_workspace_bytes(int32_t Nb, int32_t Cin, int32_t H, int32_t Wd, int32_t, int32_t, int32_t,
@@ -537,8 +662,20 @@ int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t 
                 return TBN_ERR_CUDA;
             cur = ws + plan.xconv_off;
         }
-        // all folds first, kMaxFoldJobs layers per launch (they depend on the parameters only)
+        // all folds, kMaxFoldJobs layers per launch.  They depend on the parameters only and are first needed by
+        // layer 1, so they go to the side stream (ordered after everything already queued on the caller's stream,
+        // which may still be reading this workspace) and the caller's stream joins them after launching layer 0.
+        MlpFork *fork = mlp_fork(s);
+        cudaStream_t fold_stream = s;
         {
+            std::unique_lock<std::mutex> fork_guard;
+            if (fork) {
+                fork_guard = std::unique_lock<std::mutex>(fork->mu);   // record + wait pairs of one call stay together
+                if (cudaEventRecord(fork->ev_fork, s) != cudaSuccess ||
+                    cudaStreamWaitEvent(fork->side, fork->ev_fork, 0) != cudaSuccess)
+                    return TBN_ERR_CUDA;
+                fold_stream = fork->side;
+            }
             FoldJobs jobs;
             jobs.count = 0;
             int32_t r_prev = dims[1] / ks[0];
@@ -550,10 +687,11 @@ int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t 
                 J.per_tile_prev = alpha_modes[l - 1] == TBN_ALPHA_PER_TILE; J.k_prev = ks[l - 1]; J.r_prev = r_prev;
                 r_prev = J.rows;
                 if (jobs.count == kMaxFoldJobs || l == L - 1) {
-                    if (launch_fold(jobs, s) != cudaSuccess) return TBN_ERR_CUDA;
+                    if (launch_fold(jobs, fold_stream) != cudaSuccess) return TBN_ERR_CUDA;
                     jobs.count = 0;
                 }
             }
+            if (fork && cudaEventRecord(fork->ev_join, fork->side) != cudaSuccess) return TBN_ERR_CUDA;
         }
         int32_t n_cur = dims[0];
         for (int32_t l = 0; l < L; ++l) {
@@ -571,6 +709,7 @@ int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t 
                 a.m = r; a.k = 1; a.alpha = one; a.alpha_mode = TBN_ALPHA_PER_LAYER;
                 a.act = hidden_act; a.y = ws + plan.g_off[l & 1]; a.y_dtype = TBN_BF16;
             }
+            if (l == 1 && fork && cudaStreamWaitEvent(s, fork->ev_join, 0) != cudaSuccess) return TBN_ERR_CUDA;
             if (thin_dense_supported(a)) {              // a few output rows: not worth a tensor-core launch
                 if (launch_thin_dense(a, s) != cudaSuccess) return TBN_ERR_CUDA;
             } else {

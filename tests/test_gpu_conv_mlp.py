@@ -180,3 +180,37 @@ def test_mlp_compact_chain_matches_oracle_and_layerwise_chain(T, dims, ks, act, 
     torch.cuda.synchronize()
     assert_close(to_np64(y2), ref, "layer-by-layer chain")
     assert B.tbn_last_device_status() == (0, 0)
+
+
+def test_mlp_compact_chain_replayed_from_a_graph_and_back_to_back():
+    # the compact chain runs its folds on the library's side stream (fork after the caller's queued work, join before
+    # layer 1).  Calls queued back to back share one workspace, and a captured graph must carry the fork and the join:
+    # both must reproduce the result of a single eager call bit for bit.
+    T, dims, ks = 300, [256, 512, 512, 10], [8, 8, 1]
+    x = to_dev(synth.to_bf16_bits(synth.normal(6, 0, T * dims[0]).reshape(T, dims[0])))
+    Ws = [synth.normal(6, 1 + l, dims[l + 1] * dims[l], 0.05).reshape(dims[l + 1], dims[l]) for l in range(3)]
+    layers, tiles, alphas = _mlp_layers(Ws, ks)
+    ws = torch.empty(B.tbn_mlp_workspace_bytes(T, dims, ks, B.BF16), dtype=torch.uint8, device=DEV)
+    y0 = B.tbn_mlp_fwd(x, dims, tiles, ks, alphas, [1, 1, 1], workspace=ws).clone()
+    torch.cuda.synchronize()
+    # other parameters through the same workspace in between: the second call's folds must not run early
+    Ws2 = [synth.normal(7, 1 + l, dims[l + 1] * dims[l], 0.05).reshape(dims[l + 1], dims[l]) for l in range(3)]
+    _, tiles2, alphas2 = _mlp_layers(Ws2, ks)
+    ys = []
+    for _ in range(3):
+        B.tbn_mlp_fwd(x, dims, tiles2, ks, alphas2, [1, 1, 1], workspace=ws)
+        ys.append(B.tbn_mlp_fwd(x, dims, tiles, ks, alphas, [1, 1, 1], workspace=ws).clone())
+    torch.cuda.synchronize()
+    for y in ys:
+        assert torch.equal(y, y0)
+    stream, g = torch.cuda.Stream(), torch.cuda.CUDAGraph()
+    yg = torch.empty_like(y0)
+    with torch.cuda.graph(g, stream=stream):
+        B.tbn_mlp_fwd(x, dims, tiles2, ks, alphas2, [1, 1, 1], workspace=ws, y=yg)
+        B.tbn_mlp_fwd(x, dims, tiles, ks, alphas, [1, 1, 1], workspace=ws, y=yg)
+    for _ in range(2):
+        yg.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(yg, y0)
+    assert B.tbn_last_device_status() == (0, 0)

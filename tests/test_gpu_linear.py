@@ -108,6 +108,25 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     assert_close(to_np64(yh), O.linear(x, words, k, al, True, m, n), "host entry point")
 
 
+def test_host_buffer_entry_point_chunked_pipeline():
+    # rows of 16 KB: the batch is large enough to go through in several chunks with a ragged last one (copies in,
+    # compute and copies out overlap); every token row must still come back, in its place
+    m, n, k, T = 1024, 8192, 4, 4708
+    x, W, words, al = make_linear_case(12, T, m, n, k)
+    xh = torch.from_numpy(x.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+    tile, alpha = to_dev(words), to_dev(al)
+    ws = torch.empty(B.tbn_linear_host_workspace_bytes(T, n, m, k, B.BF16, B.BF16), dtype=torch.uint8, device=DEV)
+    yd = B.tbn_linear_fwd(xh.to(DEV), m, tile, k, alpha, B.ALPHA_PER_TILE).cpu()
+    for _ in range(2):                                        # the second call reuses the copy streams and events
+        yh = torch.full((T, m), float("nan"), dtype=torch.bfloat16).pin_memory()
+        B.tbn_linear_fwd_host(xh, yh, tile, k, alpha, B.ALPHA_PER_TILE, ws)
+        assert not torch.isnan(yh).any()
+        assert_close(to_np64(yh), to_np64(yd), "chunked host entry point vs device entry point")
+    rows = np.r_[0:8, 2040:2056, 4090:4104, T - 8:T]          # chunk seams and the tail
+    assert_close(to_np64(yh)[rows], O.linear(x[rows], words, k, al, True, m, n), "chunked host entry point")
+    assert B.tbn_last_device_status() == (0, 0)
+
+
 # ------------------------------------------------------------------------------------------------
 # tensor-core (tcgen05) path
 TENSOR_SHAPES = ALIGNED + [(2048, 1024, 8), (64, 8200, 2), (256, 72, 1), (1024, 4096, 2)]
@@ -131,6 +150,24 @@ def test_tensor_path_fp32_activations_bias_fp32_out():
     ref = O.linear(x, words, k, al, True, m, n, bias=bias.astype(np.float64), act=O.ACT_GELU)
     got = run(B.PATH_TENSOR, x, words, al, True, m, k, act=B.ACT_GELU, bias=bias, y_dtype=B.F32)
     assert_close(got, ref, "tensor fp32 in/out")
+
+
+def test_tensor_path_gelu_bf16_out_wide_range():
+    # bf16 outputs take the tanh-form GELU (fitted to the erf form, special-function tanh).  Pre-activations here
+    # spread over about [-9, 9], so the fit's whole range, both tails and the cap on v^2 are exercised; beside the
+    # contract bound the error must stay within the form's own budget, 2.5e-5 + 2.5e-4 |v|, plus the bf16 rounding
+    # of the stored value.
+    m, n, k, T = 512, 256, 4, 300
+    x, W, words, al = make_linear_case(31, T, m, n, k, True, True, w_sigma=0.2)
+    bias = synth.normal(31, 200, m, 0.5)
+    pre = O.linear(x, words, k, al, True, m, n, bias=bias.astype(np.float64))
+    assert pre.min() < -6.0 and pre.max() > 6.0
+    ref = O.linear(x, words, k, al, True, m, n, bias=bias.astype(np.float64), act=O.ACT_GELU)
+    got = run(B.PATH_TENSOR, x, words, al, True, m, k, act=B.ACT_GELU, bias=bias, y_dtype=B.BF16)
+    assert_close(got, ref, "tensor gelu bf16")
+    # fp32 accumulation of 256 bf16 products moves v by ~1e-5 |v|; the stored value is rounded to bf16 (half an ulp: up to 2^-8 relative)
+    budget = 2.5e-5 + 3.0e-4 * np.abs(pre) + np.abs(ref) / 256.0 + 1e-6
+    assert float((np.abs(got - ref) / budget).max()) <= 1.0
 
 
 @pytest.mark.parametrize("cand", range(7))
