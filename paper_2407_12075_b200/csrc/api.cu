@@ -693,23 +693,35 @@ int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t 
             }
             if (fork && cudaEventRecord(fork->ev_join, fork->side) != cudaSuccess) return TBN_ERR_CUDA;
         }
-        int32_t n_cur = dims[0];
-        for (int32_t l = 0; l < L; ++l) {
-            const bool last = l == L - 1;
+        // layer l of the chain as the kernels see it: input `in` of compact width n_in
+        auto layer_args = [&](int32_t l, const void *in, int32_t n_in) {
             const int32_t r = dims[l + 1] / ks[l];
             LayerArgs a;
             std::memset(&a, 0, sizeof(a));
-            a.x = cur; a.x_dtype = TBN_BF16; a.T = T; a.n = n_cur; a.tile = tiles[l];
+            a.x = in; a.x_dtype = TBN_BF16; a.T = T; a.n = n_in; a.tile = tiles[l];
             if (l > 0) a.dense_a = ws + plan.weff_off[l];
-            a.q = (int64_t)r * n_cur;
-            if (last) {
+            a.q = (int64_t)r * n_in;
+            if (l == L - 1) {
                 a.m = dims[l + 1]; a.k = ks[l]; a.alpha = alphas[l]; a.alpha_mode = alpha_modes[l];
                 a.act = TBN_ACT_NONE; a.y = y; a.y_dtype = y_dtype;
             } else {
                 a.m = r; a.k = 1; a.alpha = one; a.alpha_mode = TBN_ALPHA_PER_LAYER;
                 a.act = hidden_act; a.y = ws + plan.g_off[l & 1]; a.y_dtype = TBN_BF16;
             }
+            return a;
+        };
+        int32_t n_cur = dims[0];
+        for (int32_t l = 0; l < L; ++l) {
+            const int32_t r = dims[l + 1] / ks[l];
+            const LayerArgs a = layer_args(l, cur, n_cur);
             if (l == 1 && fork && cudaStreamWaitEvent(s, fork->ev_join, 0) != cudaSuccess) return TBN_ERR_CUDA;
+            if (l >= 1 && l == L - 2) {                 // a narrow hidden layer and a thin last layer: one launch for both
+                const LayerArgs b = layer_args(l + 1, a.y, r);
+                if (mlp_tail_supported(a, b)) {
+                    if (launch_mlp_tail(a, b, s) != cudaSuccess) return TBN_ERR_CUDA;
+                    break;
+                }
+            }
             if (thin_dense_supported(a)) {              // a few output rows: not worth a tensor-core launch
                 if (launch_thin_dense(a, s) != cudaSuccess) return TBN_ERR_CUDA;
             } else {

@@ -138,6 +138,9 @@ double small_batch_estimate_us(const LayerArgs &a);
 // Thin layer (at most 16 distinct rows) with full-precision rows in dense_a: the head of a compact MLP chain.
 bool thin_dense_supported(const LayerArgs &a);
 cudaError_t launch_thin_dense(const LayerArgs &a, cudaStream_t s);
+// The last two layers of a compact MLP chain (folded rows; the last one thin) in one launch.
+bool mlp_tail_supported(const LayerArgs &hidden, const LayerArgs &last);
+cudaError_t launch_mlp_tail(const LayerArgs &hidden, const LayerArgs &last, cudaStream_t s);
 
 // The tensor-core path reports through a tbn_status because it also uses the driver API.
 bool tensor_path_supported(const LayerArgs &a);

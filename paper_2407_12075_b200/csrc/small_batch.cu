@@ -396,6 +396,144 @@ thin_dense_kernel(const LayerArgs a, int32_t r)
     }
 }
 
+
+// ---- the last two layers of a compact MLP chain in one launch ----------------------------------------------------
+//
+// Layer A: g2[t][o] = act(sum_i Wa[o][i] * g1[t][i]) with full-precision (folded) rows Wa [ra][na], ra <= 256;
+// layer B: y[t][j*rb + c] = alpha_j * sum_o Wb[c][o] * g2[t][o] with rb <= 16 folded rows Wb [rb][ra] (a classifier
+// head).  Both contractions are a few hundred kiloflops per token, so two launches of the 128-row tensor-memory
+// pipeline cost several times their arithmetic in fixed set-up; here a block of 8 warps owns 8*NT tokens, warp w
+// takes rows [32 w, 32 w + 32) of layer A with warp-level MMAs, the block's g2 (rounded to bf16, as the chain's
+// hidden tensors are) stays in shared memory and warps 0..NT-1 contract it with Wb.  Operand fragments are 16-byte
+// loads: within a span of 32 inputs lane (g, c) holds inputs [8c, 8c + 8) of row g / token g, and MMA u of the span
+// contracts inputs 8c + 4u .. 8c + 4u + 3 of all four c (A and B agree on the permutation, so no shuffles).
+constexpr int kTailRows = 256;          // rows of layer A at most (8 warps x 2 MMA row tiles)
+constexpr int kTailPad = 32;            // g2 row padding in shared memory: rows 16 banks apart
+
+struct TailArgs {
+    const __nv_bfloat16 *g1;            // [T][na]
+    const __nv_bfloat16 *Wa;            // [ra][na]
+    const __nv_bfloat16 *Wb;            // [rb][ra]
+    const float *alpha;                 // last layer's alphas
+    void *y;
+    int64_t T;
+    int32_t na, ra, rb, kb, mb;         // mb = kb * rb outputs
+    int per_tile, act_a, y_dtype;
+};
+
+template <int NT>
+__global__ void __launch_bounds__(256)
+mlp_tail_kernel(const TailArgs a)
+{
+    extern __shared__ __align__(16) uint8_t tail_smem[];
+    __nv_bfloat16 *g2 = reinterpret_cast<__nv_bfloat16 *>(tail_smem);          // [8 NT tokens][ra + kTailPad]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, c = lane & 3;
+    const int64_t t0 = (int64_t)blockIdx.x * (8 * NT);
+    const int32_t na = a.na, ra = a.ra;
+    const int32_t pitch = ra + kTailPad;
+
+    // ---- layer A ----
+    const int32_t m0 = warp * 32;
+    if (m0 < ra) {
+        const __nv_bfloat16 *arow[2][2];                                       // [row tile][g / g + 8], clamped
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) arow[mt][h] = a.Wa + (int64_t)min(m0 + 16 * mt + 8 * h + g, ra - 1) * na + 8 * c;
+        const __nv_bfloat16 *brow[NT];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            const int64_t t = t0 + 8 * nt + g;
+            brow[nt] = t < a.T ? a.g1 + t * na + 8 * c : nullptr;
+        }
+        float acc[2][NT][4];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[mt][nt][i] = 0.0f;
+
+        const int32_t spans = na >> 5;                                         // na % 32 == 0
+        uint4 wa[2][2][2], xb[2][NT];                                          // two register sets: [set][...]
+        auto load = [&](int set, int32_t sp) {
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) wa[set][mt][h] = __ldg(reinterpret_cast<const uint4 *>(arow[mt][h] + 32 * sp));
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+                xb[set][nt] = brow[nt] ? __ldg(reinterpret_cast<const uint4 *>(brow[nt] + 32 * sp)) : make_uint4(0u, 0u, 0u, 0u);
+        };
+        auto contract = [&](int set) {
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    mma_bf16_16x8x16(acc[mt][nt], wa[set][mt][0].x, wa[set][mt][1].x, wa[set][mt][0].y, wa[set][mt][1].y,
+                                     xb[set][nt].x, xb[set][nt].y);
+                    mma_bf16_16x8x16(acc[mt][nt], wa[set][mt][0].z, wa[set][mt][1].z, wa[set][mt][0].w, wa[set][mt][1].w,
+                                     xb[set][nt].z, xb[set][nt].w);
+                }
+        };
+        load(0, 0);
+        for (int32_t sp = 0; sp < spans; sp += 2) {                            // next span's loads before this span's MMAs
+            if (sp + 1 < spans) load(1, sp + 1);
+            contract(0);
+            if (sp + 1 >= spans) break;
+            if (sp + 2 < spans) load(0, sp + 2);
+            contract(1);
+        }
+        // accumulator fragment: [0],[1] = row g, tokens 2c, 2c+1; [2],[3] = row g + 8
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int32_t row = m0 + 16 * mt + 8 * (i >> 1) + g;
+                    const int tok = 8 * nt + 2 * c + (i & 1);
+                    float v = acc[mt][nt][i];
+                    if (a.act_a == TBN_ACT_RELU) v = fmaxf(v, 0.0f);
+                    if (row < ra) g2[tok * pitch + row] = __float2bfloat16_rn(v);
+                }
+    }
+    __syncthreads();
+
+    // ---- layer B: one 16-row MMA tile (rows >= rb are zero), warp nt takes tokens [8 nt, 8 nt + 8) ----
+    if (warp < NT) {
+        const int nt = warp;
+        float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        const bool lo_ok = g < a.rb, hi_ok = g + 8 < a.rb;
+        const __nv_bfloat16 *wlo = a.Wb + (int64_t)(lo_ok ? g : 0) * ra + 8 * c;
+        const __nv_bfloat16 *whi = a.Wb + (int64_t)(hi_ok ? g + 8 : 0) * ra + 8 * c;
+        const __nv_bfloat16 *brow = g2 + (8 * nt + g) * pitch + 8 * c;
+        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+        const int32_t spans = ra >> 5;                                         // ra % 32 == 0
+#pragma unroll 4
+        for (int32_t sp = 0; sp < spans; ++sp) {
+            const uint4 lo = lo_ok ? __ldg(reinterpret_cast<const uint4 *>(wlo + 32 * sp)) : zero;
+            const uint4 hi = hi_ok ? __ldg(reinterpret_cast<const uint4 *>(whi + 32 * sp)) : zero;
+            const uint4 b = *reinterpret_cast<const uint4 *>(brow + 32 * sp);
+            mma_bf16_16x8x16(acc, lo.x, hi.x, lo.y, hi.y, b.x, b.y);
+            mma_bf16_16x8x16(acc, lo.z, hi.z, lo.w, hi.w, b.z, b.w);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int32_t row = 8 * (i >> 1) + g;
+            const int64_t t = t0 + 8 * nt + 2 * c + (i & 1);
+            if (row >= a.rb || t >= a.T) continue;
+            for (int32_t j = 0; j < a.kb; ++j) {
+                const float al = __ldg(a.alpha + (a.per_tile ? j : 0));
+                const int64_t yi = t * a.mb + (int64_t)j * a.rb + row;
+                if (a.y_dtype == TBN_BF16) store_from_float(static_cast<__nv_bfloat16 *>(a.y), yi, al * acc[i]);
+                else store_from_float(static_cast<float *>(a.y), yi, al * acc[i]);
+            }
+        }
+    }
+}
+
 }  // namespace
 
 bool small_batch_supported(const LayerArgs &a)
@@ -439,6 +577,40 @@ cudaError_t launch_thin_dense(const LayerArgs &a, cudaStream_t s)
     const int64_t cap = (int64_t)r * a.n <= kThinMaxWeights / 2 ? 6 * 148 : 2 * 148;
     const unsigned grid = (unsigned)(blocks_needed < cap ? (blocks_needed > 0 ? blocks_needed : 1) : cap);
     thin_dense_kernel<<<grid, 256, 0, s>>>(a, r);
+    return cudaGetLastError();
+}
+
+// The fused tail takes: a hidden layer `A` with folded rows (dense_a, k = 1, scale one, ReLU or no activation, bf16
+// compact output) followed by a last layer `B` with at most 16 folded rows, no bias and no activation.
+bool mlp_tail_supported(const LayerArgs &A, const LayerArgs &B)
+{
+    if (A.is_conv || B.is_conv || !A.dense_a || !B.dense_a || A.bias || B.bias) return false;
+    if (A.x_dtype != TBN_BF16 || A.k != 1 || (A.act != TBN_ACT_RELU && A.act != TBN_ACT_NONE) || B.act != TBN_ACT_NONE)
+        return false;
+    if (A.q % A.n != 0 || B.q % B.n != 0) return false;
+    const int64_t ra = A.q / A.n, rb = B.q / B.n;
+    if (ra != A.m || ra != B.n || ra > kTailRows || ra % 32 != 0 || A.n % 32 != 0 || rb > 16 || rb < 1) return false;
+    if ((int64_t)B.k * rb != B.m) return false;
+    return (reinterpret_cast<uintptr_t>(A.x) & 15) == 0 && (reinterpret_cast<uintptr_t>(A.dense_a) & 15) == 0 &&
+           (reinterpret_cast<uintptr_t>(B.dense_a) & 15) == 0;
+}
+
+cudaError_t launch_mlp_tail(const LayerArgs &A, const LayerArgs &B, cudaStream_t s)
+{
+    TailArgs t;
+    t.g1 = static_cast<const __nv_bfloat16 *>(A.x);
+    t.Wa = static_cast<const __nv_bfloat16 *>(A.dense_a);
+    t.Wb = static_cast<const __nv_bfloat16 *>(B.dense_a);
+    t.alpha = B.alpha; t.y = B.y; t.T = A.T;
+    t.na = A.n; t.ra = A.m; t.rb = (int32_t)(B.q / B.n); t.kb = B.k; t.mb = B.m;
+    t.per_tile = B.alpha_mode == TBN_ALPHA_PER_TILE; t.act_a = A.act; t.y_dtype = B.y_dtype;
+    // 32 tokens per block while that still gives every SM a block, 16 below
+    const bool wide = A.T >= 32 * 148;
+    const int tokens = wide ? 32 : 16;
+    const size_t smem = (size_t)tokens * (t.ra + kTailPad) * sizeof(__nv_bfloat16);
+    const unsigned grid = (unsigned)((A.T + tokens - 1) / tokens);
+    if (wide) mlp_tail_kernel<4><<<grid, 256, smem, s>>>(t);
+    else mlp_tail_kernel<2><<<grid, 256, smem, s>>>(t);
     return cudaGetLastError();
 }
 

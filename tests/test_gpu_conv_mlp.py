@@ -163,7 +163,12 @@ def test_tensor_conv_rejects_what_it_cannot_take():
                                            # thin last layers (1, 16 and 10 distinct rows): the CUDA-core head kernel
                                            (513, [64, 512, 1], [8, 1], B.ACT_RELU),
                                            (64, [128, 256, 16], [4, 1], B.ACT_NONE),
-                                           (33, [256, 1024, 1024, 10], [8, 8, 1], B.ACT_RELU)])
+                                           (33, [256, 1024, 1024, 10], [8, 8, 1], B.ACT_RELU),
+                                           # narrow hidden layer + thin last layer: both in one launch (16- and
+                                           # 32-token blocks, ragged batch, 16 distinct rows written twice, 96 rows)
+                                           (4790, [64, 512, 512, 10], [8, 2, 1], B.ACT_RELU),
+                                           (70, [64, 256, 256, 32], [4, 4, 2], B.ACT_NONE),
+                                           (45, [128, 256, 192, 7], [4, 2, 1], B.ACT_RELU)])
 def test_mlp_compact_chain_matches_oracle_and_layerwise_chain(T, dims, ks, act, monkeypatch):
     # shapes whose hidden tiles span whole rows with compact widths that are multiples of 8: the hidden layers'
     # k-fold broadcast stays out of HBM (compact chain); the layer-by-layer chain must give the same result
