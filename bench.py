@@ -50,11 +50,11 @@ def algorithmic_bytes(T: int, k: int) -> float:
 
 
 # DRAM traffic of the dominant launch (k = 2) from the ncu capture summarised in
-# profiles/tc_linear_k2_T8192_ncu_full.md: 235.9 MB at T = 8192; traffic is proportional to T.  The figure is
+# profiles/tc_linear_k2_T8192_ncu_full.md: 234.0 MB at T = 8192; traffic is proportional to T.  The figure is
 # only valid for the kernel source it was taken from: the hash below covers the code (comments stripped) of
 # tc_linear.cu and tc_common.cuh.
-TRAFFIC_BYTES_AT_T8192 = 138.627584e6 + 97.303296e6
-TRAFFIC_SOURCE_HASH = "cecefe2969d56570"
+TRAFFIC_BYTES_AT_T8192 = 138.568448e6 + 95.472128e6
+TRAFFIC_SOURCE_HASH = "36fee45cc6883fa2"
 
 
 def kernel_source_hash() -> str:

@@ -52,6 +52,43 @@ __device__ __forceinline__ float gelu_tanh_bf16(float v) {
     return fmaf(hv, th, hv);
 }
 
+// Two values at once with the packed fp32 instructions of sm_100 (fma/mul .f32x2: one FMA-pipe slot for two lanes'
+// worth of arithmetic): the same formula and constants as gelu_tanh_bf16, applied to v = al * z + b.  Only the cap
+// on v^2 and the tanh itself stay scalar.
+__device__ __forceinline__ uint64_t f32x2_pack(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f32x2_unpack(uint64_t r, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(r));
+}
+__device__ __forceinline__ uint64_t f32x2_fma(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t f32x2_mul(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ void gelu_tanh_bf16_pair(float al, float z0, float z1, float b0, float b1, float &o0, float &o1) {
+    const uint64_t v = f32x2_fma(f32x2_pack(al, al), f32x2_pack(z0, z1), f32x2_pack(b0, b1));
+    float s0, s1;
+    f32x2_unpack(f32x2_mul(v, v), s0, s1);
+    const uint64_t s = f32x2_pack(fminf(s0, 50.0f), fminf(s1, 50.0f));
+    const uint64_t inner = f32x2_fma(f32x2_fma(f32x2_pack(-3.51516788e-4f, -3.51516788e-4f), s,
+                                               f32x2_pack(3.70056460e-2f, 3.70056460e-2f)),
+                                     s, f32x2_pack(7.97507884e-1f, 7.97507884e-1f));
+    float a0, a1, t0, t1;
+    f32x2_unpack(f32x2_mul(v, inner), a0, a1);
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t0) : "f"(a0));
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t1) : "f"(a1));
+    const uint64_t hv = f32x2_mul(v, f32x2_pack(0.5f, 0.5f));
+    f32x2_unpack(f32x2_fma(hv, f32x2_pack(t0, t1), hv), o0, o1);
+}
+
 __device__ __forceinline__ float apply_act(float v, int act) {
     if (act == TBN_ACT_RELU) return fmaxf(v, 0.0f);
     if (act == TBN_ACT_GELU) return gelu_erf(v);

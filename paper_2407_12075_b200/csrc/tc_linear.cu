@@ -560,7 +560,8 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
 #pragma unroll
                                 for (int i = 0; i < kSlots; ++i)
 #pragma unroll
-                                    for (int e = 0; e < 8; ++e) o[i][e] = gelu_tanh_bf16(fmaf(al, z[i][e], b[e]));
+                                    for (int e = 0; e < 8; e += 2)
+                                        gelu_tanh_bf16_pair(al, z[i][e], z[i][e + 1], b[e], b[e + 1], o[i][e], o[i][e + 1]);
                             } else if (p.act == TBN_ACT_GELU) {
 #pragma unroll
                                 for (int i = 0; i < kSlots; ++i)
