@@ -84,7 +84,8 @@ struct ConvParams {
     uint32_t magic_rows, magic_gw;   // floor(2^32 / d) + 1 for d = raw_rows, W / 8: x / d == umulhi(x, magic) for small x
     int32_t tap_plane[kTaps];  // parity plane read by tap t
     int32_t tap_off[kTaps];    // start offset (positions) of tap t inside its plane
-    int32_t m_blocks, s_tiles; // 128-channel blocks, spatial tiles
+    int32_t m_blocks, s_tiles; // 128-lane accumulator blocks, spatial tiles
+    int32_t rep;               // 128-channel output blocks written from one accumulator block (see plan_conv)
     int32_t k_stages;          // Cin / 16
     int per_tile, act, y_bf16;
 };
@@ -301,7 +302,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
         const int64_t last_word = p.n_words - 1;
         Pipe pa;
         for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
-            const int32_t o = min((tile % p.m_blocks) * 128 + L, p.m - 1);   // channels past the end are never stored
+            const int32_t o = min((tile % p.m_blocks) * p.rep * 128 + L, p.m - 1);   // channels past the end are never stored
             const int64_t row_bit = (int64_t)(o % p.r) * p.n;                  // tile row of this channel
             uint32_t w[6];
             {
@@ -361,13 +362,17 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
             const int32_t st = tile / p.m_blocks;
             const int32_t img0 = p.G > 1 ? st * p.G : st / p.bands;
             const int32_t oh0 = p.G > 1 ? 0 : (st % p.bands) * p.R;
-            const int32_t o = (tile % p.m_blocks) * 128 + L;
-            const bool ch_valid = o < p.m;
-            const float al = ch_valid ? (p.per_tile ? __ldg(p.alpha + o / p.r) : __ldg(p.alpha)) : 0.0f;
-            const float bs = (ch_valid && p.bias) ? __ldg(p.bias + o) : 0.0f;
             ok = wait_bar(smem_u32(&ctl->d_full[pd.stage]), pd.phase, abort_flag, p.status, (6 << 24) | (bid & 0xffff));
             if (!ok) break;
             tc_fence_after();
+            // one pass per channel block that shares this accumulator; the last pass hands the accumulator back
+#pragma unroll 1
+            for (int32_t rb = 0; rb < p.rep; ++rb) {
+            const bool last_pass = rb == p.rep - 1;
+            const int32_t o = ((tile % p.m_blocks) * p.rep + rb) * 128 + L;
+            const bool ch_valid = o < p.m;
+            const float al = ch_valid ? (p.per_tile ? __ldg(p.alpha + o / p.r) : __ldg(p.alpha)) : 0.0f;
+            const float bs = (ch_valid && p.bias) ? __ldg(p.bias + o) : 0.0f;
             if (rows_direct && ((p.Wo & 15) == 0 || p.Wo == 8)) {
                 // Rows made of whole 16-pixel items (32 bytes of bf16): software-pipelined.  The tensor-memory load of
                 // item i+1 is issued before item i is scaled, converted and stored, so its latency is off the path;
@@ -415,7 +420,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                         col = tmem_base + lane_base + pd.stage * kNMax + ld_g * p.slot_pos + ld_oh * row_cols + ld_pc * 16;
                         __syncwarp();
                         load_item(col, ld_oh, nxt);
-                    } else {                                               // everything is in registers: hand the accumulator back
+                    } else if (last_pass) {                                // everything is in registers: hand the accumulator back
                         tc_fence_before();
                         mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));
                     }
@@ -461,11 +466,10 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                         for (int i = 0; i < 16; ++i) cur[i] = nxt[i];
                     }
                 }
-                if (n_items <= 0) {
+                if (n_items <= 0 && last_pass) {
                     tc_fence_before();
                     mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));
                 }
-                pd.advance(2);
                 continue;
             }
             if (rows_direct) {
@@ -514,9 +518,10 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                         }
                     }
                 }
-                tc_fence_before();
-                mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));      // accumulator fully read
-                pd.advance(2);
+                if (last_pass) {
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));  // accumulator fully read
+                }
                 continue;
             }
             int32_t g = 0, oh = 0, ow = 0;                     // patch coordinates of the next position
@@ -526,7 +531,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                 uint32_t v[32];
                 tmem_ld_32x32(tmem_base + lane_base + pd.stage * kNMax + ch * 32, v);
                 tc_wait_ld();
-                if (ch == n_chunks - 1) {                        // accumulator fully read: hand it back early
+                if (ch == n_chunks - 1 && last_pass) {           // accumulator fully read: hand it back early
                     tc_fence_before();
                     mbar_arrive(smem_u32(&ctl->d_empty[pd.stage]));
                 }
@@ -542,6 +547,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
                     if (++ow == p.PW) { ow = 0; if (++oh == p.PHt) { oh = 0; ++g; } }
                 }
             }
+            }   // channel blocks of this accumulator
             pd.advance(2);
         }
     } else {
@@ -635,11 +641,34 @@ bool plan_conv(const LayerArgs &a, ConvParams &p)
     p.PW = a.Wo + range;
     if (p.PW > kNMax) return false;
     const int slot_full = (a.Ho + range) * p.PW;
+    // Lane L of channel block b holds filter (128 b + L) mod r.  When r divides 128 and the channel count is a whole
+    // number of blocks, every block has the same filters on the same lanes, hence the same accumulator: it is
+    // computed once and the epilogue writes it to all the blocks with their own alphas and biases (Sec. 4.1's
+    // replicated channels; with fewer than 128 distinct filters the tensor core has no smaller shape to offer,
+    // but it need not repeat whole blocks).
+    {
+        const int64_t r = a.q / a.n;
+        p.rep = (a.m > 128 && a.m % 128 == 0 && r <= 128 && 128 % r == 0) ? a.m / 128 : 1;
+    }
+    p.m_blocks = (a.m + 127) / 128 / p.rep;
     if ((a.Ho * p.PW) <= kNMax) {                     // whole images: possibly several per tile
         p.R = a.Ho;
         p.PHt = a.Ho + range;
-        p.G = (kNMax - p.R * p.PW) / slot_full + 1;
-        if (p.G > a.Nb) p.G = a.Nb;
+        int g_max = (kNMax - p.R * p.PW) / slot_full + 1;
+        if (g_max > a.Nb) g_max = a.Nb;
+        // Images per tile.  The main loop of a tile costs the same whatever its width (the MMA count is fixed by the
+        // input channels and an MMA takes ~112 cycles for any N <= 256) while its epilogue grows with the images it
+        // holds, so more images per tile pay only while they save a whole round of tiles over the SMs.
+        const int sms = conv_sm_count() > 0 ? conv_sm_count() : 148;
+        const double main_cycles = (double)(a.Cin / kChanPerStage) * 9.0 * 112.0 + 1500.0;
+        const double image_cycles = 350.0 * ((a.Ho * a.Wo + 15) / 16) * p.rep;
+        double best = 0.0;
+        p.G = 1;
+        for (int g = 1; g <= g_max; ++g) {
+            const int64_t tiles = (int64_t)((a.Nb + g - 1) / g) * p.m_blocks;
+            const double cost = (double)((tiles + sms - 1) / sms) * (main_cycles + g * image_cycles);
+            if (g == 1 || cost <= best) { best = cost; p.G = g; }
+        }
         p.bands = 1;
     } else {                                          // row bands of one image
         p.G = 1;
@@ -663,7 +692,6 @@ bool plan_conv(const LayerArgs &a, ConvParams &p)
             p.tap_off[u * 3 + v] = (du[u] - dmin) * p.PW + (du[v] - dmin);
         }
     p.s_tiles = p.G > 1 ? (a.Nb + p.G - 1) / p.G : a.Nb * p.bands;
-    p.m_blocks = (a.m + 127) / 128;
     p.k_stages = a.Cin / kChanPerStage;
     p.raw_rows = s * p.PHt;
     p.raw_slot_bytes = (uint32_t)(kChanPerStage * p.raw_rows * a.Wd * 2);

@@ -107,6 +107,10 @@ TENSOR_CONVS = [
     (3, 32, 16, 2, 2, 1, 13, 16),      # 8-pixel output rows stored in pairs, odd output height (7 x 8)
     (2, 32, 16, 2, 1, 1, 9, 16),       # 16-pixel rows, odd height
     (1, 32, 16, 2, 1, 1, 6, 48),       # three 16-pixel items per row
+    # 32 distinct filters on 256 / 512 channels: the channel blocks share one accumulator block, written 2 / 4 times
+    (2, 256, 16, 8, 1, 1, 6, 24),      # 8-pixel pieces (24-pixel rows)
+    (2, 512, 16, 16, 1, 1, 12, 20),    # element-wise stores (20-pixel rows)
+    (3, 384, 32, 6, 2, 1, 16, 32),     # 64 filters on three channel blocks, 16-pixel items
 ]
 
 
