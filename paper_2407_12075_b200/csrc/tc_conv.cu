@@ -362,6 +362,12 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
             const int32_t st = tile / p.m_blocks;
             const int32_t img0 = p.G > 1 ? st * p.G : st / p.bands;
             const int32_t oh0 = p.G > 1 ? 0 : (st % p.bands) * p.R;
+            // this thread's channel, scale and bias of the first pass are fetched before the wait for the accumulator,
+            // those of the next pass at the start of each pass: the loads stay off the critical path
+            int32_t o_nx = (tile % p.m_blocks) * p.rep * 128 + L;
+            bool valid_nx = o_nx < p.m;
+            float al_nx = valid_nx ? (p.per_tile ? __ldg(p.alpha + o_nx / p.r) : __ldg(p.alpha)) : 0.0f;
+            float bs_nx = (valid_nx && p.bias) ? __ldg(p.bias + o_nx) : 0.0f;
             ok = wait_bar(smem_u32(&ctl->d_full[pd.stage]), pd.phase, abort_flag, p.status, (6 << 24) | (bid & 0xffff));
             if (!ok) break;
             tc_fence_after();
@@ -369,10 +375,15 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
 #pragma unroll 1
             for (int32_t rb = 0; rb < p.rep; ++rb) {
             const bool last_pass = rb == p.rep - 1;
-            const int32_t o = ((tile % p.m_blocks) * p.rep + rb) * 128 + L;
-            const bool ch_valid = o < p.m;
-            const float al = ch_valid ? (p.per_tile ? __ldg(p.alpha + o / p.r) : __ldg(p.alpha)) : 0.0f;
-            const float bs = (ch_valid && p.bias) ? __ldg(p.bias + o) : 0.0f;
+            const int32_t o = o_nx;
+            const bool ch_valid = valid_nx;
+            const float al = al_nx, bs = bs_nx;
+            if (!last_pass) {
+                o_nx = o + 128;
+                valid_nx = o_nx < p.m;
+                al_nx = valid_nx ? (p.per_tile ? __ldg(p.alpha + o_nx / p.r) : __ldg(p.alpha)) : 0.0f;
+                bs_nx = (valid_nx && p.bias) ? __ldg(p.bias + o_nx) : 0.0f;
+            }
             if (rows_direct && ((p.Wo & 15) == 0 || p.Wo == 8)) {
                 // Rows made of whole 16-pixel items (32 bytes of bf16): software-pipelined.  The tensor-memory load of
                 // item i+1 is issued before item i is scaled, converted and stored, so its latency is off the path;
