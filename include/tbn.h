@@ -222,6 +222,11 @@ int tbn_conv2d_fwd_path(const void *x, int x_dtype, int32_t Nb, int32_t Cin, int
  * goes to HBM and the next contraction is k times shorter.  Otherwise layers run one by one with full bf16
  * hidden tensors in the workspace.  Both give the layer-by-layer result up to bf16 rounding of the hidden
  * tensors / folded rows.
+ * The folding kernels of the compact chain run on a side stream that the library creates once per device (at the
+ * first call whose `stream` is not being captured into a graph; no device memory is allocated): they start after
+ * the work already queued on `stream` and `stream` waits for them before the second layer, so the call keeps
+ * stream semantics.  When the last layer has at most 16 distinct rows and the one before it at most 256 (a
+ * multiple of 32, like its input width), the two run as one kernel.
  */
 size_t tbn_mlp_workspace_bytes(int64_t T, int32_t L, const int32_t *dims, const int32_t *ks, int x_dtype);
 int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t *dims,
