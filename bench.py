@@ -125,6 +125,19 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append([c.strip() for c in line.split(",")])
 
+    def wait_first(self, limit_s: float = 8.0):
+        """nvidia-smi can take seconds to produce its first line on a fresh box: wait for it before timing."""
+        t0 = time.time()
+        while self.proc is not None and not self.rows and time.time() - t0 < limit_s:
+            time.sleep(0.05)
+
+    def mark(self):
+        """Rows from here on belong to the timed region."""
+        self.first = len(self.rows)
+
+    def count(self) -> int:
+        return len(self.rows) - getattr(self, "first", 0)
+
     def stop(self):
         if self.proc is None:
             return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
@@ -132,7 +145,7 @@ class ClockSampler:
         self.proc.terminate()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for r in self.rows[getattr(self, "first", 0):]:
             if len(r) < 7:
                 continue
             try:
@@ -405,14 +418,26 @@ def run_ours(args, rank: int, world: int, local_rank: int):
           for _ in range(args.steps)]
     t_beg, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(local_rank)
-    barrier()
     sampler.start()
+    sampler.wait_first()
+    barrier()
+    sampler.mark()
     t_beg.record()
     for s in range(args.steps):
         step(ev[s])
     t_end.record()
+    # a short timed region can end between two samples: keep the same load running (untimed) until a few samples exist
+    extra = 0
+    torch.cuda.synchronize()
+    t_extra = time.time()
+    while sampler.proc is not None and sampler.count() < 3 and time.time() - t_extra < 3.0:
+        step()
+        torch.cuda.synchronize()
+        extra += 1
     barrier()
     clocks = sampler.stop()
+    if extra:
+        clocks["note"] = f"timed region shorter than the sampling interval: {extra} more untimed steps of the same load ran while sampling"
     total_ms = max_over_ranks(t_beg.elapsed_time(t_end), dev)
     ms_per_step = total_ms / args.steps
     per_k_ms = {k: float(np.mean([ev[s][i][0].elapsed_time(ev[s][i][1]) for s in range(args.steps)]))
