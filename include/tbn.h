@@ -81,7 +81,9 @@ const char *tbn_status_string(int status);
  * alpha     : out, 1 float (per layer) or k floats (per tile).
  * workspace : scratch of at least tbn_aggregate_workspace_bytes(N, k) bytes; contents undefined after.
  * Errors    : N % k != 0 -> TBN_ERR_SHAPE; N == 0 is TBN_ERR_INVALID_ARG.
- * The bits equal the CPU definition exactly; alpha is accumulated in fp64 in a fixed order.
+ * The bits equal the CPU definition exactly.  For alpha a thread adds the |.| of at most 16 values of one
+ * tile repetition in fp32, everything above that (per thread, per block, across blocks) is added in fp64
+ * in a fixed order, so alpha is reproducible from run to run and within 1e-6 of an fp64 sum.
  */
 size_t tbn_aggregate_workspace_bytes(int64_t N, int32_t k);
 int tbn_aggregate_tile(const float *W, const float *A, int64_t N, int32_t k, int alpha_mode,
@@ -98,7 +100,8 @@ int tbn_aggregate_tile(const float *W, const float *A, int64_t N, int32_t k, int
  *   Limit : tbn_aggregate_workspace_bytes(N, k) must not exceed 1 MiB (N up to about 500 million weights);
  *           larger layers are refused with TBN_ERR_WORKSPACE before anything is launched.
  *   Set-up: the first call on a device looks up the array's device address.  Make that first call with
- *           the device current and before any stream capture begins.
+ *           the device current and before any stream capture begins.  The look-up is not synchronised:
+ *           threads that might make the first call on a device at the same time must take turns.
  *   Sharing: every call on a device uses the same array.  The call clears the part that must start at
  *           zero, so calls that follow one another on a stream are fine; calls that may overlap on the GPU
  *           (different streams, no ordering between them) race on the array and must be serialised by the
@@ -116,12 +119,16 @@ int tbn_expand_tile(const uint32_t *tile_bits, int64_t N, int32_t k, const float
                     float *B_hat, void *stream);
 
 /* ------------------------------------------------------------------------------------------------
- * Fully-connected forward (Sec. 3 "B_hat is used for the operation on the inputs"; Algorithm 1):
+ * Fully-connected forward (Sec. 3, the paragraph after Eq. 8: the scaled tensor B_hat is what meets the
+ * inputs; Algorithm 1):
  *
  *     y[t][o] = act( sum_j B_hat[o][j] * x[t][j] + bias[o] ),   B_hat is out_f x in_f (row-major)
  *
  * x    : T x in_f, fp32 or bf16 (x_dtype).      y : T x out_f, fp32 or bf16 (y_dtype).
  * tile_bits, k, alpha, alpha_mode: as produced by tbn_aggregate_tile with N = out_f*in_f.
+ * alpha values must be non-negative, as the means of absolute values of Eq. 6-8 always are: the tensor-core
+ * kernels and the compact MLP chain use relu(alpha * z) = alpha * relu(z).  (The same holds for
+ * tbn_conv2d_fwd and tbn_mlp_fwd.)
  * bias : out_f fp32 values or NULL (the paper uses none).
  * Products are accumulated in fp32.  On the TENSOR path fp32 activations are rounded to bf16 first
  * (into the workspace); the other paths use them as given.
@@ -245,6 +252,16 @@ int tbn_last_device_status(void *stream, int *code, int *detail);
 /* Testing aid: enqueue a kernel that records (code, detail) exactly as a kernel whose wait gave up would --
  * it waits on nothing, so it cannot hang -- to exercise the status plumbing without starving a real pipeline. */
 int tbn_debug_record_status(int code, int detail, void *stream);
+/* Testing / tuning aids, process-wide, to be set while no forward call is in progress.  They replace nothing on
+ * the normal path: without them the library chooses by shape.
+ *   tbn_debug_force_linear_config: the tensor-core linear kernel runs tile shape `candidate` (an index into its
+ *     table of shapes) with the contraction split over `splits` CTAs per output tile (1, 2, 4, 8 or 16; lowered
+ *     at launch until every split has at least two stages; without enough workspace the call runs unsplit).
+ *     candidate < 0 restores the automatic choice.  TBN_ERR_INVALID_ARG for anything else.
+ *   tbn_debug_force_mlp_layerwise: non-zero makes tbn_mlp_fwd run layer by layer with full hidden tensors even
+ *     where the compact chain applies (the two must agree; tests compare them). */
+int tbn_debug_force_linear_config(int candidate, int splits);
+int tbn_debug_force_mlp_layerwise(int on);
 
 #ifdef __cplusplus
 }

@@ -51,6 +51,8 @@ SIGNATURES = {
                             c_vp, c_sz, c_vp]),
     "tbn_last_device_status": (c_int, [c_vp, c_vp, c_vp]),
     "tbn_debug_record_status": (c_int, [c_int, c_int, c_vp]),
+    "tbn_debug_force_linear_config": (c_int, [c_int, c_int]),
+    "tbn_debug_force_mlp_layerwise": (c_int, [c_int]),
 }
 
 _lib = None
@@ -275,3 +277,11 @@ def tbn_last_device_status():
 
 def tbn_debug_record_status(code: int, detail: int):
     _check(lib().tbn_debug_record_status(code, detail, _stream()), "tbn_debug_record_status")
+
+
+def tbn_debug_force_linear_config(candidate: int, splits: int = 1):
+    _check(lib().tbn_debug_force_linear_config(candidate, splits), "tbn_debug_force_linear_config")
+
+
+def tbn_debug_force_mlp_layerwise(on: bool):
+    _check(lib().tbn_debug_force_mlp_layerwise(int(bool(on))), "tbn_debug_force_mlp_layerwise")

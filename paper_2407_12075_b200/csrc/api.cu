@@ -1,7 +1,7 @@
 // C entry points of libtbn: argument validation, path selection, workspace carving.
 // Every step of the computation runs in the kernels of the other translation units; nothing here
 // touches the data on the host, and there is no CPU fallback.
-#include <cstdlib>
+#include <atomic>
 #include <cstring>
 #include <mutex>
 
@@ -225,6 +225,8 @@ int fill_linear(LayerArgs &a, const void *x, int x_dtype, int64_t T, int32_t in_
     a.is_conv = 0;
     return TBN_OK;
 }
+
+std::atomic<int> g_mlp_layerwise{0};        // testing aid: 1 = tbn_mlp_fwd runs layer by layer even where the compact chain applies
 
 __device__ float g_device_one = 1.0f;       // alpha of the compact (unscaled) hidden tensors of the MLP chain
 
@@ -649,8 +651,7 @@ int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t 
     // next layer contracts g with its distinct rows folded with layer l's alphas (launch_fold): the k-fold
     // broadcast of a hidden layer never goes to HBM and the next contraction is k times shorter.
     MlpChainPlan plan;
-    const char *no_chain = getenv("TBN_MLP_UNFUSED");
-    if (L >= 2 && (hidden_act == TBN_ACT_RELU || hidden_act == TBN_ACT_NONE) && !(no_chain && no_chain[0] == '1') &&
+    if (L >= 2 && (hidden_act == TBN_ACT_RELU || hidden_act == TBN_ACT_NONE) && g_mlp_layerwise.load() == 0 &&
         plan_mlp_chain(T, L, dims, ks, x_dtype, plan) && aligned16(x) && aligned16(y)) {
         int *st = device_status_ptr();
         const float *one = device_one_ptr();
@@ -770,6 +771,14 @@ int tbn_last_device_status(void *stream, int *code, int *detail)
     *code = host[0];
     *detail = host[1];
     if (host[0] != 0 && cudaMemset(st, 0, sizeof(host)) != cudaSuccess) return TBN_ERR_CUDA;
+    return TBN_OK;
+}
+
+int tbn_debug_force_linear_config(int candidate, int splits) { return force_linear_config(candidate, splits); }
+
+int tbn_debug_force_mlp_layerwise(int on)
+{
+    g_mlp_layerwise.store(on ? 1 : 0);
     return TBN_OK;
 }
 

@@ -183,6 +183,7 @@ cudaError_t launch_mlp_tail(const LayerArgs &hidden, const LayerArgs &last, cuda
 bool tensor_path_supported(const LayerArgs &a);
 size_t tensor_linear_scratch_bytes(const LayerArgs &a);   // split-K partial tiles + arrival counters
 int launch_tensor_linear(const LayerArgs &a, int *device_status, void *scratch, size_t scratch_bytes, cudaStream_t s);
+int force_linear_config(int candidate, int splits);          // testing / tuning aid: candidate < 0 clears
 bool tensor_conv_supported(const LayerArgs &a);
 int launch_tensor_conv(const LayerArgs &a, int *device_status, cudaStream_t s);
 

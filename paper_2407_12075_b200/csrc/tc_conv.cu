@@ -56,7 +56,6 @@ constexpr int kRS = 3;                 // raw (untransposed) patch stages in sha
 constexpr int kACols = kTaps * 8;      // 72 columns per decoded-weight stage
 constexpr int kABase = 2 * kNMax;      // first weight column
 constexpr uint32_t kConvTmemCols = 512;
-constexpr int kStageOutBytes = 0;       // (no epilogue staging in shared memory)
 
 struct ConvParams {
     const __nv_bfloat16 *x;
@@ -109,7 +108,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
     const uint32_t stage_bytes = (uint32_t)p.planes * 2u * (uint32_t)p.buf_pos * 16u;
     ConvControl *ctl = reinterpret_cast<ConvControl *>(smem + kSX * stage_bytes);
     const uint32_t stage0 = smem_u32(smem);
-    const uint32_t raw_off = (kSX * stage_bytes + kCtlBytes + kStageOutBytes + 127u) & ~127u;   // raw ring, 128-byte aligned
+    const uint32_t raw_off = (kSX * stage_bytes + kCtlBytes + 127u) & ~127u;   // raw ring, 128-byte aligned
     volatile int *abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -612,7 +611,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
 
 size_t conv_smem_bytes(const ConvParams &p)
 {
-    size_t b = (size_t)kSX * p.planes * 2 * p.buf_pos * 16 + kCtlBytes + kStageOutBytes + 128;
+    size_t b = (size_t)kSX * p.planes * 2 * p.buf_pos * 16 + kCtlBytes + 128;
     if (p.wide) b += (size_t)kRS * p.raw_stage_bytes;
     return b + 1024;
 }

@@ -17,9 +17,9 @@
 // alpha/bias/activation -> k-fold replicated stores), 10-13 = optional epilogue helpers (half of the
 // arithmetic and stores when the activation is expensive; they never touch tensor memory).  All hand-offs are mbarriers; every wait is
 // bounded by a wall-clock limit, after which the CTA records TBN_ERR_TIMEOUT, drains and returns.
-#include <cstdlib>
-
+#include <atomic>
 #include <cstddef>
+
 #include "tc_common.cuh"
 
 namespace tbn {
@@ -708,6 +708,9 @@ constexpr int kNumCands = 7;
 
 struct Plan { int cand, splits; size_t scratch_bytes; };
 
+// Forced tile shape / split factor (testing and tuning aid; -1 = the cost model decides).
+std::atomic<int> g_forced_cand{-1}, g_forced_splits{1};
+
 Plan plan_linear(const LayerArgs &a)
 {
     const int sms = sm_count() > 0 ? sm_count() : 148;
@@ -750,6 +753,17 @@ Plan plan_linear(const LayerArgs &a)
 
 }  // namespace
 
+int force_linear_config(int candidate, int splits)
+{
+    if (candidate < 0) { g_forced_cand.store(-1); g_forced_splits.store(1); return TBN_OK; }
+    // the epilogue adds the partial tiles in pairs: only powers of two up to 16 are valid split factors
+    if (candidate >= kNumCands || (splits != 1 && splits != 2 && splits != 4 && splits != 8 && splits != 16))
+        return TBN_ERR_INVALID_ARG;
+    g_forced_splits.store(splits);
+    g_forced_cand.store(candidate);
+    return TBN_OK;
+}
+
 bool tensor_path_supported(const LayerArgs &a)
 {
     if (a.is_conv) return false;
@@ -776,14 +790,14 @@ int launch_tensor_linear(const LayerArgs &a, int *device_status, void *scratch, 
     p.per_tile = a.alpha_mode == TBN_ALPHA_PER_TILE; p.act = a.act; p.y_bf16 = a.y_dtype == TBN_BF16;
 
     Plan plan = plan_linear(a);
-    const char *force = getenv("TBN_TC_CONFIG");     // tuning aid: "<candidate>" or "<candidate>,<splits>"
-    if (force && force[0] >= '0' && force[0] < '0' + kNumCands) {
-        plan.cand = force[0] - '0';
-        plan.splits = (force[1] == ',' && atoi(force + 2) >= 1) ? atoi(force + 2) : 1;
+    const int forced = g_forced_cand.load(std::memory_order_relaxed);
+    if (forced >= 0 && forced < kNumCands) {            // testing / tuning aid, see force_linear_config()
+        plan.cand = forced;
+        plan.splits = g_forced_splits.load(std::memory_order_relaxed);
         const Cand &c = kCands[plan.cand];
         const int64_t out_tiles = (int64_t)((p.r + c.na * 128 - 1) / (c.na * 128)) * ((a.T + c.ntok - 1) / c.ntok);
         const int k_stages = (a.n + c.ka * kAtomK - 1) / (c.ka * kAtomK);
-        if (plan.splits > k_stages) plan.splits = k_stages;
+        while (plan.splits > 1 && k_stages < 2 * plan.splits) plan.splits >>= 1;   // at least two stages per split
         plan.scratch_bytes = plan.splits == 1 ? 0
             : ((size_t)out_tiles * 4 * sizeof(unsigned int) + 255) / 256 * 256 +
               (size_t)out_tiles * plan.splits * c.na * 128 * c.ntok * sizeof(float);

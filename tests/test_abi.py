@@ -64,6 +64,9 @@ def test_argument_errors_are_found_on_the_host(lib):
     # the scratch-free variant refuses layers beyond its built-in 1 MiB array (it needs about N/512 bytes)
     assert lib.tbn_aggregate_tile_static(dummy, None, 1 << 31, 2, 0, dummy, dummy, None) == -4
     assert lib.tbn_aggregate_tile_static(dummy, None, 10, 3, 0, dummy, dummy, None) == -2
+    # the exact limit: q = 1 needs 16 + 8 k bytes, so k = 131071 (and the k = N = 131072 case) no longer fit
+    assert lib.tbn_aggregate_tile_static(dummy, None, 131071, 131071, 1, dummy, dummy, None) == -4
+    assert lib.tbn_aggregate_tile_static(dummy, None, 131072, 131072, 1, dummy, dummy, None) == -4
     assert lib.tbn_linear_select_path(4, 64, 64, 3, B.BF16) == -2
     conv = [dummy, B.BF16, 1, 3, 8, 8, 4, 3, 3, 1, 1, dummy, 5, dummy, 0, None, 0, dummy, B.BF16, None, 0, None]
     assert lib.tbn_conv2d_fwd(*conv) == -2                    # 108 weights, k = 5

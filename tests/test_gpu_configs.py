@@ -13,24 +13,43 @@ from tests.util import DEV, assert_close, to_dev, to_np64
 pytestmark = pytest.mark.gpu
 
 
+def sweep_sample_rows(T: int, count: int = 512) -> np.ndarray:
+    """Token rows for the oracle at the sweep's largest batch: at least one row inside every token tile of both tile
+    widths the kernel uses there (224 and 256 tokens), the first and the last row, and seeded random rows up to
+    `count` in all."""
+    rows = {0, T - 1}
+    for width in (224, 256):
+        for i in range((T + width - 1) // width):
+            rows.add(min(i * width + (i * 37 + 11) % width, T - 1))
+    rng = np.random.default_rng(4)
+    while len(rows) < count:
+        rows.add(int(rng.integers(0, T)))
+    return np.array(sorted(rows), dtype=np.int64)
+
+
 def test_large_linear_sweep_full_size_sampled_rows():
     # in = out = 8192, T = 16384 bf16 tokens, W ~ N(0, 0.02^2) aggregated on the GPU, per-tile alpha, seed 4
     c = synth.config_large_linear(16384)
     xd, Wd = to_dev(c["x"]), to_dev(c["W"])
-    rows = np.sort(np.random.default_rng(4).choice(c["T"], 6, replace=False))
-    rows[-1] = c["T"] - 1
+    rows = sweep_sample_rows(c["T"])
+    assert len(rows) >= 512
     y = torch.empty((c["T"], c["m"]), dtype=torch.bfloat16, device=DEV)
+    ws = torch.empty(max(max(B.tbn_linear_workspace_bytes(c["T"], c["n"], c["m"], k, B.BF16) for k in (2, 4, 8, 16)), 16),
+                     dtype=torch.uint8, device=DEV)
     for k in (2, 4, 8, 16):
         tile, alpha = B.tbn_aggregate_tile(Wd, k, B.ALPHA_PER_TILE)
         words, al = O.prepare(c["W"], k, True)
         assert np.array_equal(tile.cpu().numpy().view(np.uint32), words)
         assert np.allclose(alpha.cpu().numpy(), al, rtol=1e-6)
         assert B.tbn_linear_select_path(c["T"], c["n"], c["m"], k, B.BF16) == B.PATH_TENSOR
-        B.tbn_linear_fwd(xd, c["m"], tile, k, alpha, B.ALPHA_PER_TILE, y=y)
+        y.fill_(float("nan"))
+        B.tbn_linear_fwd(xd, c["m"], tile, k, alpha, B.ALPHA_PER_TILE, y=y, workspace=ws)
         torch.cuda.synchronize()
+        assert not bool(torch.isnan(y).any()), "an output element was never written"
         ref = O.linear(c["x"][rows], words, k, al, True, c["m"], c["n"])
         assert_close(to_np64(y[torch.from_numpy(rows).to(DEV)]), ref, f"large linear k={k}")
-        # the k repetitions of a distinct row differ only by alpha_j (Sec. 4.1): check it on the whole output
+        # the k repetitions of a distinct row differ only by alpha_j (Sec. 4.1): a property of the whole output that
+        # holds at any size (the sampled rows above are what is compared with the oracle)
         r = c["m"] // k
         z0 = y[:, :r].float() / alpha[0]
         zj = y[:, (k - 1) * r:].float() / alpha[k - 1]

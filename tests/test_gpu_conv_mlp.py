@@ -173,7 +173,7 @@ def test_tensor_conv_rejects_what_it_cannot_take():
                                            (4790, [64, 512, 512, 10], [8, 2, 1], B.ACT_RELU),
                                            (70, [64, 256, 256, 32], [4, 4, 2], B.ACT_NONE),
                                            (45, [128, 256, 192, 7], [4, 2, 1], B.ACT_RELU)])
-def test_mlp_compact_chain_matches_oracle_and_layerwise_chain(T, dims, ks, act, monkeypatch):
+def test_mlp_compact_chain_matches_oracle_and_layerwise_chain(T, dims, ks, act):
     # shapes whose hidden tiles span whole rows with compact widths that are multiples of 8: the hidden layers'
     # k-fold broadcast stays out of HBM (compact chain); the layer-by-layer chain must give the same result
     L = len(ks)
@@ -184,10 +184,36 @@ def test_mlp_compact_chain_matches_oracle_and_layerwise_chain(T, dims, ks, act, 
     y = B.tbn_mlp_fwd(to_dev(x), dims, tiles, ks, alphas, [1] * L, hidden_act=act)
     torch.cuda.synchronize()
     assert_close(to_np64(y), ref, "compact chain")
-    monkeypatch.setenv("TBN_MLP_UNFUSED", "1")
-    y2 = B.tbn_mlp_fwd(to_dev(x), dims, tiles, ks, alphas, [1] * L, hidden_act=act)
-    torch.cuda.synchronize()
+    B.tbn_debug_force_mlp_layerwise(True)
+    try:
+        y2 = B.tbn_mlp_fwd(to_dev(x), dims, tiles, ks, alphas, [1] * L, hidden_act=act)
+        torch.cuda.synchronize()
+    finally:
+        B.tbn_debug_force_mlp_layerwise(False)
     assert_close(to_np64(y2), ref, "layer-by-layer chain")
+    assert B.tbn_last_device_status() == (0, 0)
+
+
+@pytest.mark.parametrize("T,dims,ks,act", [(512, [512, 4096, 2048, 10], [8, 8, 1], B.ACT_RELU),
+                                           (300, [1024, 4096, 4096, 64], [4, 16, 2], B.ACT_NONE)])
+def test_mlp_compact_chain_wide_layers_fan_in_scaled(T, dims, ks, act):
+    # hidden widths of 4096 and folds over 512 / 1024 rows, weights ~N(0, 1/n) so that the hidden activations stay
+    # of order one, as they do in a trained network: the compact chain must hold the stated tolerance here too
+    L = len(ks)
+    x = synth.to_bf16_bits(synth.normal(15, 0, T * dims[0]).reshape(T, dims[0]))
+    Ws = [synth.normal(15, 1 + l, dims[l + 1] * dims[l], dims[l] ** -0.5).reshape(dims[l + 1], dims[l]) for l in range(L)]
+    layers, tiles, alphas = _mlp_layers(Ws, ks)
+    ref = O.mlp(x, layers, hidden_act=O.ACT_RELU if act == B.ACT_RELU else O.ACT_NONE)
+    y = B.tbn_mlp_fwd(to_dev(x), dims, tiles, ks, alphas, [1] * L, hidden_act=act)
+    torch.cuda.synchronize()
+    assert_close(to_np64(y), ref, "wide compact chain")
+    B.tbn_debug_force_mlp_layerwise(True)
+    try:
+        y2 = B.tbn_mlp_fwd(to_dev(x), dims, tiles, ks, alphas, [1] * L, hidden_act=act)
+        torch.cuda.synchronize()
+    finally:
+        B.tbn_debug_force_mlp_layerwise(False)
+    assert_close(to_np64(y2), ref, "wide layer-by-layer chain")
     assert B.tbn_last_device_status() == (0, 0)
 
 

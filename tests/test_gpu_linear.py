@@ -170,17 +170,45 @@ def test_tensor_path_gelu_bf16_out_wide_range():
     assert float((np.abs(got - ref) / budget).max()) <= 1.0
 
 
-@pytest.mark.parametrize("cand", range(7))
-def test_tensor_path_every_tile_shape(cand, monkeypatch):
-    # the planner picks one token-tile shape per call; the tuning variable pins each of them in turn on a case
-    # with several token tiles, a ragged token tail and a ragged row block
-    monkeypatch.setenv("TBN_TC_CONFIG", str(cand))
+@pytest.fixture
+def forced_config():
+    """Pins the tensor-core linear kernel's tile shape / split factor for one test and always restores the
+    automatic choice."""
+    yield B.tbn_debug_force_linear_config
+    B.tbn_debug_force_linear_config(-1)
+
+
+def tile_shape_count() -> int:
+    n = 0
+    while B.lib().tbn_debug_force_linear_config(n, 1) == 0:
+        n += 1
+    B.tbn_debug_force_linear_config(-1)
+    return n
+
+
+@pytest.mark.parametrize("splits", [1, 2, 4])
+def test_tensor_path_every_tile_shape(splits, forced_config):
+    # the planner picks one token-tile shape per call; the tuning hook pins each of them in turn on a case with
+    # several token tiles, a ragged token tail and a ragged row block, unsplit and with the contraction split
     m, n, k, T = 1200, 1000, 4, 777
     x, W, words, al = make_linear_case(21, T, m, n, k, True, True)
     ref = O.linear(x, words, k, al, True, m, n)
-    got = run(B.PATH_TENSOR, x, words, al, True, m, k)
-    assert_close(got, ref, f"tensor tile shape {cand}")
+    count = tile_shape_count()
+    assert count >= 7
+    ws = torch.empty(64 << 20, dtype=torch.uint8, device=DEV)
+    for cand in range(count):
+        forced_config(cand, splits)
+        y = B.tbn_linear_fwd(to_dev(x), m, to_dev(words), k, to_dev(al), 1, path=B.PATH_TENSOR, workspace=ws)
+        torch.cuda.synchronize()
+        assert_close(to_np64(y), ref, f"tensor tile shape {cand} splits {splits}")
     assert B.tbn_last_device_status() == (0, 0)
+
+
+def test_forced_config_rejects_invalid_split_factors():
+    for bad in (0, 3, 5, 6, 32, -1):
+        assert B.lib().tbn_debug_force_linear_config(0, bad) == -1
+    assert B.lib().tbn_debug_force_linear_config(10 ** 6, 1) == -1
+    B.tbn_debug_force_linear_config(-1)
 
 
 @pytest.mark.parametrize("k", [2, 16])

@@ -281,6 +281,14 @@ def test_conv_matches_torch_conv2d_on_kron_weights(Nb, Cout, Cin, kh, kw, p, str
                                      stride=stride, padding=pad).numpy()
     assert y.shape == ref.shape
     assert np.allclose(y, ref, rtol=1e-11, atol=1e-11)
+    # the bias branch (one value per output channel, added before the activation) against torch's bias argument;
+    # distinct per-channel values, so a bias indexed by anything but the channel fails
+    bias = (rng.standard_normal(Cout) * 3.0 + np.arange(Cout)).astype(np.float64)
+    for act, fn in ((O.ACT_NONE, lambda v: v), (O.ACT_RELU, torch.relu)):
+        yb = O.conv2d(x, words, p, al, True, Cout, Cin, kh, kw, stride, pad, bias=bias, act=act)
+        refb = fn(torch.nn.functional.conv2d(torch.from_numpy(x).double(), torch.from_numpy(Bk), bias=torch.from_numpy(bias),
+                                             stride=stride, padding=pad)).numpy()
+        assert np.allclose(yb, refb, rtol=1e-11, atol=1e-11)
 
 
 def test_conv_paper_example_replicated_channels():
@@ -334,6 +342,28 @@ def test_mlp_is_the_composition_of_its_layers():
         if l < 2:
             h = np.maximum(h, 0)
     assert np.allclose(O.mlp(x, layers), h, rtol=1e-11, atol=1e-11)
+
+
+def test_mlp_mirrored_mode_rounds_hidden_tensors_like_a_bf16_cast():
+    # the diagnostic mode stores every hidden tensor as bf16: composition by hand with torch's own bf16 cast
+    rng = np.random.default_rng(14)
+    dims, ks = [16, 24, 12, 5], [2, 4, 1]
+    x = rng.standard_normal((6, dims[0])).astype(np.float32)
+    layers, h = [], x.astype(np.float64)
+    for l in range(3):
+        W = rng.standard_normal(dims[l + 1] * dims[l]).astype(np.float32)
+        words, al = O.prepare(W, ks[l], True)
+        layers.append(dict(words=words, p=ks[l], alphas=al, per_tile=True, m=dims[l + 1], n=dims[l]))
+        Bk = kron_expand(bits_of(words, W.size // ks[l]), ks[l], al, True).reshape(dims[l + 1], dims[l])
+        h = h @ Bk.T
+        if l < 2:
+            h = torch.from_numpy(np.maximum(h, 0)).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+    got = O.mlp(x, layers, mirror_bf16=True)
+    assert np.allclose(got, h, rtol=1e-11, atol=1e-11)
+    assert not np.allclose(got, O.mlp(x, layers), rtol=1e-6, atol=0)      # the rounding really happens
+    # round_to_bf16 itself: ties go to even, values already representable are unchanged
+    v = np.array([1.0, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -2.5, 3.0e-5], dtype=np.float64)
+    assert np.array_equal(O.round_to_bf16(v), torch.from_numpy(v).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy())
 
 
 # ----------------------------------------------------------------------------- printed numbers

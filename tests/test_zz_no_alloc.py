@@ -8,6 +8,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import tbn_oracle as O
 from paper_2407_12075_b200 import binding as B
 from paper_2407_12075_b200 import synth
 from tests.util import to_dev
@@ -20,8 +21,8 @@ pytestmark = pytest.mark.gpu
 def test_static_scratch_entry_point_matches_ordinary_one_twice(N, k, mode):
     results = []
     for call in range(2):                       # second call sees the first call's leftovers in the array
-        W = to_dev(synth.normal(40 + call, 1, N, 0.02))
-        A = to_dev(synth.normal(40 + call, 101, N, 0.05))
+        W_np, A_np = synth.normal(40 + call, 1, N, 0.02), synth.normal(40 + call, 101, N, 0.05)
+        W, A = to_dev(W_np), to_dev(A_np)
         tile_ref, alpha_ref = B.tbn_aggregate_tile(W, k, mode, A=A)
         tile = torch.full_like(tile_ref, -1)
         alpha = torch.full_like(alpha_ref, float("nan"))
@@ -29,5 +30,29 @@ def test_static_scratch_entry_point_matches_ordinary_one_twice(N, k, mode):
         torch.cuda.synchronize()
         assert torch.equal(tile, tile_ref), f"call {call}: tile bits differ"
         assert np.allclose(alpha.cpu().numpy(), alpha_ref.cpu().numpy(), rtol=1e-6, atol=0), f"call {call}"
+        # and against the CPU definition directly, not only through the other entry point
+        words, al = O.prepare(W_np, k, mode == B.ALPHA_PER_TILE, A=A_np)
+        assert np.array_equal(tile.cpu().numpy().view(np.uint32), words), f"call {call}: tile bits differ from the oracle"
+        assert np.allclose(alpha.cpu().numpy(), al, rtol=1e-6, atol=0), f"call {call}: alpha differs from the oracle"
         results.append(tile.clone())
     assert not torch.equal(results[0], results[1])      # the two calls really had different inputs
+
+
+def test_static_scratch_limit_is_exact():
+    # one-element tiles (q = 1) need 16 + 8 k bytes of scratch: k = 131070 is the largest that fits the 1 MiB array,
+    # k = 131071 is refused before anything is launched
+    k = 131070
+    W_np = synth.normal(44, 1, k, 0.02)
+    W = to_dev(W_np)
+    tile = torch.full((B.tbn_tile_words(1),), -1, dtype=torch.int32, device=W.device)
+    alpha = torch.full((k,), float("nan"), dtype=torch.float32, device=W.device)
+    B.tbn_aggregate_tile_static(W, k, tile, alpha, B.ALPHA_PER_TILE)
+    torch.cuda.synchronize()
+    words, al = O.prepare(W_np, k, True)
+    assert np.array_equal(tile.cpu().numpy().view(np.uint32), words)
+    assert np.allclose(alpha.cpu().numpy(), al, rtol=1e-6, atol=0)
+    W1 = to_dev(synth.normal(44, 1, k + 1, 0.02))
+    alpha1 = torch.empty(k + 1, dtype=torch.float32, device=W.device)
+    with pytest.raises(B.TbnError) as e:
+        B.tbn_aggregate_tile_static(W1, k + 1, tile, alpha1, B.ALPHA_PER_TILE)
+    assert e.value.status == -4
