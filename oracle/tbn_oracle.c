@@ -243,3 +243,52 @@ void tbn_oracle_conv2d(const double *x, int32_t Nb, int32_t Cin, int32_t H, int3
         }
     }
 }
+
+/*
+ * Binary activations (Sec. 7 names tiled networks with binary weights AND binary activations as the
+ * next step; Sec. 2 recalls that such networks, XNOR-Net among them, binarise the activations with
+ * the sign function and keep a real scaling factor).  The paper fixes no formula for this case; the
+ * reading taken here, listed in the design notes, is the smallest extension of Sec. 3:
+ *   a[t][j]  = +1 if x[t][j] > 0 else -1            (the threshold rule of Eq. 3, applied to x)
+ *   beta[t]  = ||x[t][:]||_1 / n                     (the scaling of Eq. 6, applied to one input row)
+ *   y[t][i]  = act( beta[t] * sum_j B_hat[i][j] * a[t][j] + bias[i] )
+ * with B_hat the scaled tiled weight of Eq. 4-8.  Everything below is that definition written out.
+ */
+
+/* Threshold + row scale of one activation matrix.  bits[t*n + j] in {0,1}; beta nullable. */
+void tbn_oracle_binarize(const double *x, int64_t T, int32_t n, uint8_t *bits, float *beta)
+{
+    for (int64_t t = 0; t < T; ++t) {
+        double a = 0.0;
+        for (int32_t j = 0; j < n; ++j) {
+            const double v = x[t * n + j];
+            bits[t * n + j] = (v > 0.0) ? 1 : 0;           /* zero, negative zero and NaN give -1 */
+            a += fabs(v);
+        }
+        if (beta) beta[t] = (float)(a / (double)n);
+    }
+}
+
+/*
+ * The integer part of the binary-activation layer: D[t][i] = sum_j b[i][j] * a[t][j] with
+ * b[i][j] = +-1 the unscaled tiled weight (Eq. 4-5: bit (i*n + j) mod q of the tile) and a = +-1.
+ * Exact in integers.  abits: T x n values in {0,1}.
+ */
+void tbn_oracle_linear_bin_int(const uint8_t *abits, int64_t T, int32_t n, int32_t m,
+                               const uint32_t *words, int64_t q, int64_t *D)
+{
+    const int64_t total = T * (int64_t)m;
+#pragma omp parallel for schedule(static)
+    for (int64_t o = 0; o < total; ++o) {
+        const int64_t t = o / m;
+        const int32_t i = (int32_t)(o % m);
+        int64_t acc = 0;
+        for (int32_t j = 0; j < n; ++j) {
+            const int64_t f = ((int64_t)i * n + j) % q;
+            const int b = ((words[f >> 5] >> (f & 31)) & 1u) ? 1 : -1;
+            const int a = abits[t * n + j] ? 1 : -1;
+            acc += b * a;
+        }
+        D[o] = acc;
+    }
+}

@@ -204,6 +204,54 @@ def linear_alg1(x, words, p, alphas, per_tile, m, n, relu=False):
     return y
 
 
+# --------------------------------------------------------------------------- #
+# Binary activations (Sec. 7: binary weights AND binary activations)           #
+# --------------------------------------------------------------------------- #
+def row_words(n: int) -> int:
+    """Words of one packed activation row: ceil(n/32) rounded up to a multiple of 4 (16-byte rows)."""
+    return ((int(n) + 31) // 32 + 3) // 4 * 4
+
+
+def binarize(x: np.ndarray):
+    """Threshold rule of Eq. 3 applied to the activations, and the per-row scale beta_t = ||x_t||_1 / n
+    (Eq. 6 applied to one input row).  Returns (bits uint8 [T, n] in {0,1}, beta float32 [T])."""
+    xd = widen(x)
+    T, n = xd.shape
+    bits = np.empty((T, n), dtype=np.uint8)
+    beta = np.empty(T, dtype=np.float32)
+    _load().tbn_oracle_binarize(_p(np.ascontiguousarray(xd)), ctypes.c_int64(T), ctypes.c_int32(n), _p(bits), _p(beta))
+    return bits, beta
+
+
+def pack_rows(bits: np.ndarray) -> np.ndarray:
+    """[T, n] bits -> [T, row_words(n)] uint32, each row packed like a tile (LSB first, zero padding)."""
+    T, n = bits.shape
+    out = np.zeros((T, row_words(n)), dtype=np.uint32)
+    for t in range(T):
+        out[t, :tile_words(n)][: (n + 31) // 32] = pack_bits(bits[t])[: (n + 31) // 32]
+    return out
+
+
+def linear_bin_int(abits: np.ndarray, words: np.ndarray, p: int, m: int, n: int) -> np.ndarray:
+    """D[t][i] = sum_j b[i][j] a[t][j] over +-1 values: the integer accumulator of the binary-activation layer."""
+    abits = np.ascontiguousarray(abits, dtype=np.uint8)
+    T = abits.shape[0]
+    words = np.ascontiguousarray(words, dtype=np.uint32)
+    D = np.empty((T, m), dtype=np.int64)
+    _load().tbn_oracle_linear_bin_int(_p(abits), ctypes.c_int64(T), ctypes.c_int32(n), ctypes.c_int32(m), _p(words),
+                                      ctypes.c_int64(m * n // p), _p(D))
+    return D
+
+
+def linear_bin(abits, beta, words, p, alphas, per_tile, m, n, bias=None, act=ACT_NONE):
+    """y[t][i] = act(beta_t * sum_j B_hat[i][j] a[t][j] + bias[i]): the tiled layer of Eq. 4-8 applied to the
+    sign vector of the activations, each row scaled by its beta -- i.e. the dense layer on the inputs beta_t * (+-1)."""
+    a_pm = np.where(np.asarray(abits) > 0, 1.0, -1.0)
+    if beta is not None:
+        a_pm = a_pm * np.asarray(beta, dtype=np.float64)[:, None]      # exact: beta_t * (+-1)
+    return linear(a_pm, words, p, alphas, per_tile, m, n, bias=bias, act=act)
+
+
 def conv_out_hw(H, Wd, kh, kw, stride, pad):
     return (H + 2 * pad - kh) // stride + 1, (Wd + 2 * pad - kw) // stride + 1
 
