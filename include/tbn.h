@@ -48,7 +48,7 @@ typedef enum {
     TBN_ERR_TIMEOUT = -6      /* a device-side bounded wait gave up (see tbn_last_device_status) */
 } tbn_status;
 
-typedef enum { TBN_F32 = 0, TBN_BF16 = 1 } tbn_dtype;
+typedef enum { TBN_F32 = 0, TBN_BF16 = 1, TBN_I32 = 2 /* only as y_dtype of tbn_linear_bin_fwd */ } tbn_dtype;
 typedef enum { TBN_ALPHA_PER_LAYER = 0, TBN_ALPHA_PER_TILE = 1 } tbn_alpha_mode; /* 1 or k floats */
 /* GELU is the erf form v * Phi(v): evaluated to 4e-7 for fp32 outputs; bf16 outputs of the tensor-core kernels use a
  * tanh form fitted to it whose difference (<= 2.5e-5 + 2.5e-4 |v|) stays below the bf16 rounding of the result. */
@@ -189,6 +189,37 @@ int tbn_linear_fwd_host(const void *x_host, int x_dtype, int64_t T, int32_t in_f
                         void *workspace, size_t workspace_bytes, void *stream);
 
 /* ------------------------------------------------------------------------------------------------
+ * Binary activations (Sec. 7 names tiled networks with binary weights AND binary activations as the next step;
+ * Sec. 2 describes such networks: sign activations with a real scaling factor, contracted by XNOR and
+ * popcount).  The paper gives no formula for this case; this library takes the smallest extension of Sec. 3:
+ *
+ *     a[t][j] = x[t][j] > 0 ? +1 : -1             the threshold rule of Eq. 3 (zero, -0 and NaN give -1)
+ *     beta[t] = ||x[t][:]||_1 / in_f              the scale of Eq. 6 applied to one input row
+ *     D[t][o] = sum_j b[o][j] * a[t][j]           b = the unscaled +-1 tiled weight of Eq. 4-5; an integer
+ *     y[t][o] = act( beta[t] * sum_j B_hat[o][j] * a[t][j] + bias[o] )
+ *
+ * (where the tile spans whole rows: y[t][j*r + c] = act(beta[t] * alpha_j * D[t][c] + bias), D contracted once per
+ * distinct row and written k times, Sec. 4.1).  D is computed exactly: D = cnt - 2 popcount(w xor x) on the
+ * CUDA-core path, 4 popcount(w and x) - 2 popcount(w) - 2 popcount(x) + in_f with the and-popcount as an 8-bit
+ * integer tensor-core product on the tensor path.
+ *
+ * tbn_binarize_fwd: x (T x in_f, fp32 or bf16) -> x_bits: T rows of tbn_row_words(in_f) words each (row pitch a
+ *   multiple of 128 bits; bit j of a row at word j/32, position j%32; padding bits zero), and beta (T floats; may be
+ *   NULL when the caller wants no scale).  beta is accumulated in fp64 in a fixed order.
+ * tbn_linear_bin_fwd: x_bits as written by tbn_binarize_fwd; beta: T floats or NULL (= 1; must be >= 0, like alpha);
+ *   tile_bits, k, alpha, alpha_mode, bias, act as for tbn_linear_fwd.  y: T x out_f; y_dtype TBN_F32 or TBN_BF16,
+ *   or TBN_I32 for the raw integers D (alpha, beta, bias and act are then not applied).
+ *   path: TBN_PATH_AUTO; TBN_PATH_GENERIC = the popcount kernel (any shape, any alignment of the tile against the rows;
+ *   one packed activation row must fit 48 KB); TBN_PATH_TENSOR = the integer tensor-core kernel (needs
+ *   q % in_f == 0 and in_f % 32 == 0; TBN_ERR_UNSUPPORTED otherwise).  No workspace.  T == 0 is a no-op.
+ */
+int64_t tbn_row_words(int32_t in_f);
+int tbn_binarize_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, uint32_t *x_bits, float *beta, void *stream);
+int tbn_linear_bin_fwd(const uint32_t *x_bits, int64_t T, int32_t in_f, int32_t out_f,
+                       const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                       const float *beta, const float *bias, int act, void *y, int y_dtype, void *stream, int path);
+
+/* ------------------------------------------------------------------------------------------------
  * 2-D convolution forward.  The paper defines tiling for convolutional layers (Sec. 3: the tile
  * fills the whole weight tensor) but ships no convolution kernel (Sec. 6 lists it as future work).
  * The weight tensor is (Cout, Cin, kh, kw) in row-major order, N = Cout*Cin*kh*kw:
@@ -262,6 +293,8 @@ int tbn_debug_record_status(int code, int detail, void *stream);
  *     where the compact chain applies (the two must agree; tests compare them). */
 int tbn_debug_force_linear_config(int candidate, int splits);
 int tbn_debug_force_mlp_layerwise(int on);
+/* Same for the tile shape of the binary-activation tensor-core kernel (candidate < 0: automatic). */
+int tbn_debug_force_bin_config(int candidate);
 
 #ifdef __cplusplus
 }

@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libtbn.so")
 
 OK = 0
-F32, BF16 = 0, 1
+F32, BF16, I32 = 0, 1, 2
 ALPHA_PER_LAYER, ALPHA_PER_TILE = 0, 1
 ACT_NONE, ACT_RELU, ACT_GELU = 0, 1, 2
 PATH_AUTO, PATH_GENERIC, PATH_SMALL, PATH_TENSOR = 0, 1, 2, 3
@@ -53,6 +53,11 @@ SIGNATURES = {
     "tbn_debug_record_status": (c_int, [c_int, c_int, c_vp]),
     "tbn_debug_force_linear_config": (c_int, [c_int, c_int]),
     "tbn_debug_force_mlp_layerwise": (c_int, [c_int]),
+    "tbn_debug_force_bin_config": (c_int, [c_int]),
+    "tbn_row_words": (c_i64, [c_i32]),
+    "tbn_binarize_fwd": (c_int, [c_vp, c_int, c_i64, c_i32, c_vp, c_vp, c_vp]),
+    "tbn_linear_bin_fwd": (c_int, [c_vp, c_i64, c_i32, c_i32, c_vp, c_i32, c_vp, c_int, c_vp, c_vp, c_int, c_vp, c_int,
+                                   c_vp, c_int]),
 }
 
 _lib = None
@@ -108,7 +113,7 @@ def _dtype_code(t: torch.Tensor) -> int:
 
 
 def _torch_dtype(code: int):
-    return torch.bfloat16 if code == BF16 else torch.float32
+    return {BF16: torch.bfloat16, F32: torch.float32, I32: torch.int32}[code]
 
 
 def _ws(nbytes: int, device):
@@ -285,3 +290,32 @@ def tbn_debug_force_linear_config(candidate: int, splits: int = 1):
 
 def tbn_debug_force_mlp_layerwise(on: bool):
     _check(lib().tbn_debug_force_mlp_layerwise(int(bool(on))), "tbn_debug_force_mlp_layerwise")
+
+
+def tbn_row_words(n: int) -> int:
+    return int(lib().tbn_row_words(n))
+
+
+def tbn_binarize_fwd(x: torch.Tensor, with_beta: bool = True, x_bits: torch.Tensor | None = None,
+                     beta: torch.Tensor | None = None):
+    """Sign bits of the activations, packed row by row, and the per-row scale mean|x|.  Returns (x_bits, beta)."""
+    T, n = x.shape
+    if x_bits is None:
+        x_bits = torch.empty((T, tbn_row_words(n)), dtype=torch.int32, device=x.device)
+    if with_beta and beta is None:
+        beta = torch.empty(T, dtype=torch.float32, device=x.device)
+    _check(lib().tbn_binarize_fwd(_ptr(x), _dtype_code(x), T, n, _ptr(x_bits), _ptr(beta) if with_beta else None,
+                                  _stream()), "tbn_binarize_fwd")
+    return x_bits, (beta if with_beta else None)
+
+
+def tbn_linear_bin_fwd(x_bits: torch.Tensor, in_f: int, out_f: int, tile: torch.Tensor, k: int, alpha: torch.Tensor,
+                       alpha_mode: int, beta: torch.Tensor | None = None, bias: torch.Tensor | None = None,
+                       act: int = ACT_NONE, y_dtype: int = BF16, path: int = PATH_AUTO,
+                       y: torch.Tensor | None = None) -> torch.Tensor:
+    T = x_bits.shape[0]
+    if y is None:
+        y = torch.empty((T, out_f), dtype=_torch_dtype(y_dtype), device=x_bits.device)
+    _check(lib().tbn_linear_bin_fwd(_ptr(x_bits), T, in_f, out_f, _ptr(tile), k, _ptr(alpha), alpha_mode, _ptr(beta),
+                                    _ptr(bias), act, _ptr(y), y_dtype, _stream(), path), "tbn_linear_bin_fwd")
+    return y

@@ -759,6 +759,56 @@ int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t 
     return TBN_OK;
 }
 
+int64_t tbn_row_words(int32_t n) { return tbn_tile_words(n); }
+
+int tbn_binarize_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, uint32_t *x_bits, float *beta, void *stream)
+{
+    if (T < 0 || in_f <= 0 || !valid_dtype(x_dtype)) return TBN_ERR_INVALID_ARG;
+    if (T == 0) return TBN_OK;
+    if (!x || !x_bits || !aligned16(x) || !aligned16(x_bits)) return TBN_ERR_INVALID_ARG;
+    if (beta && (reinterpret_cast<uintptr_t>(beta) & 3u)) return TBN_ERR_INVALID_ARG;
+    return launch_binarize(x, x_dtype, T, in_f, x_bits, beta, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? TBN_OK : TBN_ERR_CUDA;
+}
+
+int tbn_linear_bin_fwd(const uint32_t *x_bits, int64_t T, int32_t in_f, int32_t out_f,
+                       const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                       const float *beta, const float *bias, int act, void *y, int y_dtype, void *stream, int path)
+{
+    if (T < 0 || in_f <= 0 || out_f <= 0 || k <= 0) return TBN_ERR_INVALID_ARG;
+    if (!tile_bits || !alpha || !valid_alpha_mode(alpha_mode) || !valid_act(act)) return TBN_ERR_INVALID_ARG;
+    if (!(valid_dtype(y_dtype) || y_dtype == TBN_I32)) return TBN_ERR_INVALID_ARG;
+    if (path < TBN_PATH_AUTO || path > TBN_PATH_TENSOR) return TBN_ERR_INVALID_ARG;
+    if (T > 0 && (!x_bits || !y)) return TBN_ERR_INVALID_ARG;
+    if (!aligned16(x_bits) || !aligned16(y) || !aligned16(tile_bits)) return TBN_ERR_INVALID_ARG;
+    if ((bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) || (beta && (reinterpret_cast<uintptr_t>(beta) & 3u)))
+        return TBN_ERR_INVALID_ARG;
+    const int64_t N = (int64_t)in_f * out_f;
+    if (N % k != 0) return TBN_ERR_SHAPE;
+    if (T == 0) return TBN_OK;
+    BinArgs a;
+    std::memset(&a, 0, sizeof(a));
+    a.x_bits = x_bits; a.tile = tile_bits; a.alpha = alpha; a.beta = beta; a.bias = bias; a.y = y;
+    a.T = T; a.q = N / k; a.x_row_words = (int32_t)tbn_row_words(in_f); a.n = in_f; a.m = out_f; a.k = k;
+    a.alpha_mode = alpha_mode; a.act = act; a.y_dtype = y_dtype;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (path == TBN_PATH_AUTO) {
+        // A handful of tokens is bound by reading the tile once and by launch latency: the popcount kernel.  From a
+        // few dozen tokens on the 8-bit tensor-core contraction is an order of magnitude faster than popcounts.
+        path = (bin_tensor_supported(a) && T >= 32) ? TBN_PATH_TENSOR : TBN_PATH_GENERIC;
+    }
+    if (path == TBN_PATH_TENSOR) {
+        if (!bin_tensor_supported(a)) return TBN_ERR_UNSUPPORTED;
+        int *st = device_status_ptr();
+        if (!st) return TBN_ERR_CUDA;
+        return launch_bin_tensor(a, st, s);
+    }
+    if (path != TBN_PATH_GENERIC || !bin_popc_supported(a)) return TBN_ERR_UNSUPPORTED;
+    return launch_bin_popc(a, s) == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+}
+
+int tbn_debug_force_bin_config(int candidate) { return force_bin_config(candidate); }
+
 int tbn_last_device_status(void *stream, int *code, int *detail)
 {
     if (!code || !detail) return TBN_ERR_INVALID_ARG;

@@ -142,6 +142,27 @@ struct LayerArgs {
     int32_t Nb, Cin, H, Wd, kh, kw, stride, pad, Ho, Wo;
 };
 
+// ---- binary-activation layer (bit-packed activations; see bin_act.cu) ---------------------------------
+struct BinArgs {
+    const uint32_t *x_bits;   // [T][x_row_words] packed activation signs, padding bits zero
+    const uint32_t *tile;
+    const float *alpha;
+    const float *beta;        // per-token scale, or null (= 1)
+    const float *bias;
+    void *y;
+    int64_t T;
+    int64_t q;
+    int32_t x_row_words;
+    int32_t n, m, k;
+    int alpha_mode, act, y_dtype;   // y_dtype TBN_I32: the raw integer accumulators
+};
+cudaError_t launch_binarize(const void *x, int x_dtype, int64_t T, int32_t n, uint32_t *bits, float *beta, cudaStream_t s);
+bool bin_popc_supported(const BinArgs &a);
+cudaError_t launch_bin_popc(const BinArgs &a, cudaStream_t s);
+bool bin_tensor_supported(const BinArgs &a);
+int launch_bin_tensor(const BinArgs &a, int *device_status, cudaStream_t s);
+int force_bin_config(int candidate);                           // testing / tuning aid: candidate < 0 clears
+
 // ---- launchers implemented in the other translation units ---------------------------------------
 cudaError_t launch_aggregate(const float *W, const float *A, int64_t N, int32_t k, int per_tile,
                              uint32_t *tile_bits, float *alpha, void *workspace, cudaStream_t s);
