@@ -354,6 +354,39 @@ def measure_other_configs(B, torch, dev, peaks):
     for T in (1, 16, 256, 4096):
         for k in (2, 16):
             out[f"large_linear_T{T}_k{k}"] = linear_entry(T, N_FEAT, N_FEAT, k)
+    # binary activations (Sec. 7): threshold + packing, then the XNOR / popcount layer on the sweep's shape.  Integer
+    # ops = 2*T*r*n.  Large batches run on the 8-bit integer tensor cores (peak taken as twice the measured bf16 burst
+    # peak, the nominal ratio); the popcount rate of the CUDA cores (16 popcounts of 32 bits per clock and SM) is
+    # quoted beside it as the bound a popcount kernel would have.
+    T = 16384
+    x = torch.randn(T, N_FEAT, device=dev, generator=gen).to(torch.bfloat16)
+    xb = torch.empty((T, B.tbn_row_words(N_FEAT)), dtype=torch.int32, device=dev)
+    beta = torch.empty(T, dtype=torch.float32, device=dev)
+    us = graph_us(lambda: B.tbn_binarize_fwd(x, x_bits=xb, beta=beta), reps=3, iters=3)
+    nbytes = x.numel() * 2 + xb.numel() * 4 + T * 4
+    out["binarize_T16384_8192"] = dict(us=us, alg_gbs=nbytes / us / 1e3, bound="hbm", frac_of_binding_roofline=nbytes / hbm * 1e6 / us)
+    y = torch.empty(T, N_FEAT, device=dev, dtype=torch.bfloat16)
+    int8_peak = 2.0 * tens
+    popc_peak = 148 * 16 * 32 * 2 * 1.965e9
+    for k in (2, 16):
+        tile, alpha = rand_tile(N_FEAT * N_FEAT // k), torch.rand(k, device=dev, generator=gen) * 0.02
+        us = graph_us(lambda: B.tbn_linear_bin_fwd(xb, N_FEAT, N_FEAT, tile, k, alpha, B.ALPHA_PER_TILE, beta=beta, y=y),
+                      reps=3, iters=3)
+        ops = 2.0 * T * (N_FEAT // k) * N_FEAT
+        nbytes = xb.numel() * 4 + y.numel() * 2 + N_FEAT * N_FEAT // k / 8
+        t_bound = max(ops / int8_peak, nbytes / hbm)
+        out[f"bin_linear_T{T}_k{k}"] = dict(us=us, alg_tops=ops / us / 1e6, alg_gbs=nbytes / us / 1e3,
+                                            bound="tensor (int8)" if ops / int8_peak > nbytes / hbm else "hbm",
+                                            frac_of_binding_roofline=t_bound * 1e6 / us,
+                                            popcount_alu_peak_tops=popc_peak / 1e12)
+    del x, y
+    xb16 = xb[:16].contiguous()
+    y16 = torch.empty(16, N_FEAT, device=dev, dtype=torch.bfloat16)
+    tile, alpha = rand_tile(N_FEAT * N_FEAT // 2), torch.rand(2, device=dev, generator=gen) * 0.02
+    us = graph_us(lambda: B.tbn_linear_bin_fwd(xb16, N_FEAT, N_FEAT, tile, 2, alpha, B.ALPHA_PER_TILE, beta=beta[:16], y=y16))
+    out["bin_linear_T16_k2_popcount_kernel"] = dict(us=us, alg_tops=2.0 * 16 * (N_FEAT // 2) * N_FEAT / us / 1e6,
+                                                    alg_gbs=(N_FEAT * N_FEAT // 2 / 8 + 16 * N_FEAT * 2.125) / us / 1e3,
+                                                    bound="launch / hbm", l2="resident")
     # Small batch against HBM: a CUDA-graph chain of distinct layers whose tiles (4 MiB each at k = 2) add up to
     # more than L2, so every layer's tile really comes from HBM; per-layer time and tile GB/s.
     for T in (1, 16):

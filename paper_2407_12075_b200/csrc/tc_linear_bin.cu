@@ -164,61 +164,78 @@ tc_linear_bin_kernel(const BinParams p)
         // 32-byte sector), expands them and writes the row's 128-byte line of each of the two swizzle rows: the
         // 16-byte piece c of row R goes to position c xor (R mod 8), so the 8 lanes of a quarter warp hit 8
         // different bank groups.
+        // The bits of a stage are requested two stages ahead (across tile boundaries too): a stage's loads are a
+        // round trip to L2, longer than the expansion of a stage, and nothing else would hide it.
         const int tid = threadIdx.x;
+        constexpr int H = NTOK / 128;
         Pipe px;
         uint32_t sd = 0, sd_phase = 0;
-        for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
-            const int64_t tok0 = (int64_t)(tile / p.w_tiles) * NTOK;
-            int32_t pc[NTOK / 128];
+        auto load_bits = [&](uint4 (&v)[H][2], int32_t tl, int32_t ks) {
+            const int64_t tok0 = (int64_t)(tl / p.w_tiles) * NTOK;
 #pragma unroll
-            for (int h = 0; h < NTOK / 128; ++h) pc[h] = 0;
-            for (int32_t ks = 0; ks < p.k_stages && ok; ++ks) {
-                // this stage's bits first, so that the loads overlap the wait
-                uint4 v[NTOK / 128][2];
+            for (int h = 0; h < H; ++h) {
+                const int64_t tok = tok0 + tid + 128 * h;
+                v[h][0] = v[h][1] = make_uint4(0u, 0u, 0u, 0u);
+                if (tl < n_tiles && tok < p.T) {
+                    const uint4 *src = reinterpret_cast<const uint4 *>(p.x_bits + tok * p.xw + ks * 8);
+                    if (ks * 8 < p.xw) v[h][0] = __ldg(src);
+                    if (ks * 8 + 4 < p.xw) v[h][1] = __ldg(src + 1);
+                }
+            }
+        };
+        auto next_item = [&](int32_t &tl, int32_t &ks) {
+            if (++ks == p.k_stages) { ks = 0; tl += gridDim.x; }
+        };
+        int32_t tile = bid, ks = 0;                         // the stage being expanded
+        int32_t ltile = bid, lks = 0;                       // the stage being requested
+        uint4 cur[H][2], nx1[H][2], nx2[H][2];
+        load_bits(cur, ltile, lks); next_item(ltile, lks);
+        load_bits(nx1, ltile, lks); next_item(ltile, lks);
+        int32_t pc[H];
 #pragma unroll
-                for (int h = 0; h < NTOK / 128; ++h) {
-                    const int64_t tok = tok0 + tid + 128 * h;
-                    v[h][0] = v[h][1] = make_uint4(0u, 0u, 0u, 0u);
-                    if (tok < p.T) {
-                        const uint4 *src = reinterpret_cast<const uint4 *>(p.x_bits + tok * p.xw + ks * 8);
-                        if (ks * 8 < p.xw) v[h][0] = __ldg(src);
-                        if (ks * 8 + 4 < p.xw) v[h][1] = __ldg(src + 1);
+        for (int h = 0; h < H; ++h) pc[h] = 0;
+        while (tile < n_tiles) {
+            load_bits(nx2, ltile, lks); next_item(ltile, lks);
+            ok = wait_bar(smem_u32(&ctl->x_empty[px.stage]), px.phase ^ 1u, abort_flag, p.status,
+                          (1 << 24) | (px.stage << 16) | (bid & 0xffff));
+            if (!ok) break;
+#pragma unroll
+            for (int h = 0; h < H; ++h) {
+                const int row = tid + 128 * h;
+                const uint32_t sw = (uint32_t)row & 7u;
+#pragma unroll
+                for (int at = 0; at < kBinKA; ++at) {
+                    const uint32_t w4[4] = {cur[h][at].x, cur[h][at].y, cur[h][at].z, cur[h][at].w};
+                    const uint32_t line = stage0 + px.stage * kStageBytes + at * kAtomBytes + (uint32_t)row * 128u;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        pc[h] += __popc(w4[i]);
+                        uint32_t e[8];
+                        expand_word(w4[i], e);
+                        sts_v4(line + (((uint32_t)(2 * i) ^ sw) << 4), e[0], e[1], e[2], e[3]);
+                        sts_v4(line + (((uint32_t)(2 * i + 1) ^ sw) << 4), e[4], e[5], e[6], e[7]);
                     }
                 }
-                ok = wait_bar(smem_u32(&ctl->x_empty[px.stage]), px.phase ^ 1u, abort_flag, p.status,
-                              (1 << 24) | (px.stage << 16) | (bid & 0xffff));
+            }
+            fence_proxy_async();                           // generic-proxy stores -> visible to the tensor core
+            mbar_arrive(smem_u32(&ctl->x_full[px.stage]));
+            px.advance(SX);
+            if (ks == p.k_stages - 1) {
+                // the tile's row popcounts for the epilogue
+                ok = wait_bar(smem_u32(&ctl->side_empty[sd]), sd_phase ^ 1u, abort_flag, p.status, (9 << 24) | (bid & 0xffff));
                 if (!ok) break;
 #pragma unroll
-                for (int h = 0; h < NTOK / 128; ++h) {
-                    const int row = tid + 128 * h;
-                    const uint32_t sw = (uint32_t)row & 7u;
-#pragma unroll
-                    for (int at = 0; at < kBinKA; ++at) {
-                        const uint32_t w4[4] = {v[h][at].x, v[h][at].y, v[h][at].z, v[h][at].w};
-                        const uint32_t line = stage0 + px.stage * kStageBytes + at * kAtomBytes + (uint32_t)row * 128u;
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            pc[h] += __popc(w4[i]);
-                            uint32_t e[8];
-                            expand_word(w4[i], e);
-                            sts_v4(line + (((uint32_t)(2 * i) ^ sw) << 4), e[0], e[1], e[2], e[3]);
-                            sts_v4(line + (((uint32_t)(2 * i + 1) ^ sw) << 4), e[4], e[5], e[6], e[7]);
-                        }
-                    }
-                }
-                fence_proxy_async();                       // generic-proxy stores -> visible to the tensor core
-                mbar_arrive(smem_u32(&ctl->x_full[px.stage]));
-                px.advance(SX);
+                for (int h = 0; h < H; ++h) { ctl->px[sd][tid + 128 * h] = pc[h]; pc[h] = 0; }
+                mbar_arrive(smem_u32(&ctl->side_full[sd]));
+                sd ^= 1u;
+                if (sd == 0) sd_phase ^= 1u;
             }
-            if (!ok) break;
-            // the tile's row popcounts for the epilogue
-            ok = wait_bar(smem_u32(&ctl->side_empty[sd]), sd_phase ^ 1u, abort_flag, p.status, (9 << 24) | (bid & 0xffff));
-            if (!ok) break;
+            next_item(tile, ks);
 #pragma unroll
-            for (int h = 0; h < NTOK / 128; ++h) ctl->px[sd][tid + 128 * h] = pc[h];
-            mbar_arrive(smem_u32(&ctl->side_full[sd]));
-            sd ^= 1u;
-            if (sd == 0) sd_phase ^= 1u;
+            for (int h = 0; h < H; ++h) {
+                cur[h][0] = nx1[h][0]; cur[h][1] = nx1[h][1];
+                nx1[h][0] = nx2[h][0]; nx1[h][1] = nx2[h][1];
+            }
         }
     } else if (warp == kBinMmaWarp) {
         // ---------------- MMA issuer (lane 0): 8 MMAs of K = 32 per stage ----------------
@@ -543,9 +560,12 @@ int launch_bin_tensor(const BinArgs &a, int *device_status, cudaStream_t s)
     p.w_tiles = 0; p.t_tiles = 0;
     p.per_tile = a.alpha_mode == TBN_ALPHA_PER_TILE; p.act = a.act;
     p.y_mode = a.y_dtype == TBN_I32 ? 2 : a.y_dtype == TBN_BF16 ? 1 : 0;
-    // Two accumulator buffers of 128 tokens let the k-fold store loop of one tile run under the main loop of the
-    // next; one buffer of 256 tokens halves the number of tiles.  The second pays when the epilogue is short.
-    int cand = a.T <= 128 ? 1 : (a.k >= 4 ? 1 : 0);
+    // 256-token tiles (one accumulator buffer) halve the shared-memory traffic per tile and measured faster wherever
+    // they fill the GPU; when they would leave SMs idle, 128-token tiles with two accumulator buffers (the k-fold
+    // store loop of one tile runs under the main loop of the next) give twice as many tiles.
+    const int sms = bin_sm_count() > 0 ? bin_sm_count() : 148;
+    const int64_t tiles256 = (int64_t)((p.r + 127) / 128) * ((a.T + 255) / 256);
+    int cand = tiles256 >= sms ? 0 : 1;
     const int forced = g_forced_bin.load(std::memory_order_relaxed);
     if (forced >= 0) cand = forced;
     switch (cand) {
