@@ -296,6 +296,50 @@ def mlp(x, layers, hidden_act=ACT_RELU, mirror_bf16=False):
 
 
 # --------------------------------------------------------------------------- #
+# Training-side tiling module (Sec. 3: Eq. 1-5 in the forward of a custom       #
+# differentiation module, gradients passed straight through on the way back)   #
+# --------------------------------------------------------------------------- #
+def tile_fwd(W: np.ndarray, p: int, per_tile: bool, A: np.ndarray | None = None):
+    """Training forward of the tiling module: W (and A) -> the scaled tiled weight B_hat the layer then uses
+    (Eq. 1-5, then Eq. 6 / Eq. 7-8 and the scaling paragraph).  Returns (B_hat fp32 [N], packed tile, alphas)."""
+    words, al = prepare(W, p, per_tile, A)
+    return expand(words, np.asarray(W).size, p, al, per_tile), words, al
+
+
+def tile_bwd(G: np.ndarray, words: np.ndarray, alphas: np.ndarray, per_tile: bool, W: np.ndarray, p: int,
+             A: np.ndarray | None = None):
+    """Backward of the tiling module for G = dL/dB_hat (fp64 arithmetic).
+
+    Eq. 1-5 are not differentiable; the paper passes the gradient with respect to B straight through to W
+    (the straight-through paragraph of Sec. 3):  dL/dW := dL/dB.  B_hat = alpha_j * B, so dL/dB = alpha_j * G.
+    The scaling factors are ordinary differentiable functions of S (= A, or W when no separate tensor is used):
+    alpha_j = sum_{f in segment j} |S[f]| / q (Eq. 8; one segment of N values for Eq. 6), hence
+        dL/dalpha_j = sum_{f in segment j} G[f] * B[f],      dL/dS[f] = dL/dalpha_{j(f)} * sign(S[f]) / q
+    with sign(0) = 0.  Without a separate A both contributions land on W.
+    Returns (dW [N], dA [N] or None, dalpha [1 or p])."""
+    G = np.asarray(G, dtype=np.float64).reshape(-1)
+    N = G.size
+    q = N // p
+    i = np.arange(q)
+    t = np.where((np.asarray(words, dtype=np.uint32)[i >> 5] >> (i & 31).astype(np.uint32)) & 1, 1.0, -1.0)
+    al = np.asarray(alphas, dtype=np.float64)
+    dW = np.empty(N)
+    dalpha = np.zeros(p if per_tile else 1)
+    for j in range(p):
+        seg = slice(j * q, (j + 1) * q)
+        dW[seg] = (al[j] if per_tile else al[0]) * G[seg]
+        dalpha[j if per_tile else 0] += float(np.sum(G[seg] * t))
+    S = np.asarray(W if A is None else A, dtype=np.float64).reshape(-1)
+    dS = np.empty(N)
+    for j in range(p):
+        seg = slice(j * q, (j + 1) * q)
+        dS[seg] = (dalpha[j] / q if per_tile else dalpha[0] / N) * np.sign(S[seg])
+    if A is None:
+        return dW + dS, None, dalpha
+    return dW, dS, dalpha
+
+
+# --------------------------------------------------------------------------- #
 # Storage accounting (Sec. 5.1 Table 6, Sec. 5.2 Table 7)                      #
 # --------------------------------------------------------------------------- #
 def layer_storage_bytes(N: int, p: int, n_alpha: int) -> float:
