@@ -339,6 +339,18 @@ def measure_other_configs(B, torch, dev, peaks):
         us = graph_us(lambda: B.tbn_aggregate_tile(Wagg, k, B.ALPHA_PER_TILE), reps=3, iters=3)
         nbytes = 4.0 * Wagg.numel() + Wagg.numel() / k / 8
         out[f"aggregate_8192x8192_k{k}"] = dict(us=us, alg_gbs=nbytes / us / 1e3, bound="hbm", frac_of_binding_roofline=nbytes / hbm * 1e6 / us)
+    # training-side tiling module (Sec. 3): forward = one read of W + one write of B_hat; backward = G read twice, W read
+    # once (sign for the alpha path), dW written once
+    for k in (4,):
+        us = graph_us(lambda: B.tbn_tile_fwd(Wagg, k, B.ALPHA_PER_TILE), reps=3, iters=3)
+        nbytes = 8.0 * Wagg.numel() + Wagg.numel() / k / 8
+        out[f"tile_fwd_8192x8192_k{k}"] = dict(us=us, alg_gbs=nbytes / us / 1e3, bound="hbm", frac_of_binding_roofline=nbytes / hbm * 1e6 / us)
+        _, t_bits, t_alpha = B.tbn_tile_fwd(Wagg, k, B.ALPHA_PER_TILE)
+        Gagg = torch.randn(Wagg.numel(), device=dev, generator=gen)
+        us = graph_us(lambda: B.tbn_tile_bwd(Gagg, t_bits, t_alpha, Wagg, k, B.ALPHA_PER_TILE), reps=3, iters=3)
+        nbytes = 16.0 * Wagg.numel()
+        out[f"tile_bwd_8192x8192_k{k}"] = dict(us=us, alg_gbs=nbytes / us / 1e3, bound="hbm", frac_of_binding_roofline=nbytes / hbm * 1e6 / us)
+        del Gagg
     del Wagg
     # full-precision tiled weights (Sec. 5.2): ViT fc1-shaped layer, k = 4, bf16 tile read in place
     T, n, m, k = 25216, 768, 3072, 4

@@ -110,6 +110,32 @@ int tbn_aggregate_tile(const float *W, const float *A, int64_t N, int32_t k, int
 int tbn_aggregate_tile_static(const float *W, const float *A, int64_t N, int32_t k, int alpha_mode,
                               uint32_t *tile_bits, float *alpha, void *stream);
 
+/* ------------------------------------------------------------------------------------------------
+ * Training-side tiling module (Sec. 3).  The paper trains full-precision W (and optionally A), builds the tiled
+ * weight in the forward pass of a custom differentiation module (Eq. 1-5), and passes the gradient straight
+ * through the non-differentiable steps on the way back (the paragraph after Eq. 5: dL/dW := dL/dB).
+ *
+ * tbn_tile_fwd: one read of W (and A) -> tile_bits and alpha exactly as tbn_aggregate_tile, and
+ *     B_hat[j*q + i] = alpha_j * (bit_i ? +1 : -1)        N values, fp32 or bf16 (b_dtype), row-major like W:
+ *   the weight the training forward then contracts with the inputs.  B_hat is written from the bits; W is not
+ *   read a second time.  workspace: tbn_aggregate_workspace_bytes(N, k).
+ * tbn_tile_bwd: G = dL/dB_hat (N fp32 values) ->
+ *     dalpha_j = sum_i G[j*q + i] * t_i                   (per layer: one sum over all N; fp64, fixed order)
+ *     dW[f]    = alpha_j * G[f]                           the straight-through part, one fp32 multiply
+ *     dS[f]    = dalpha_j * sign(S[f]) / q                the scaling factors are differentiated as ordinary
+ *                                                         functions of S (Eq. 6-8; sign(0) = 0; / N per layer)
+ *   With a separate tensor (A != NULL) dS is written to dA; without one (A == NULL, dA == NULL) S = W and dS is
+ *   added to dW.  dalpha (1 or k floats) may be NULL.  The paper states the straight-through rule only; taking the
+ *   gradient of the scaling factors as well is this library's reading (it is what automatic differentiation of
+ *   Eq. 6-8 gives).  workspace: tbn_tile_bwd_workspace_bytes(N, k).  Errors as tbn_aggregate_tile.
+ */
+int tbn_tile_fwd(const float *W, const float *A, int64_t N, int32_t k, int alpha_mode, void *B_hat, int b_dtype,
+                 uint32_t *tile_bits, float *alpha, void *workspace, size_t workspace_bytes, void *stream);
+size_t tbn_tile_bwd_workspace_bytes(int64_t N, int32_t k);
+int tbn_tile_bwd(const float *G, const uint32_t *tile_bits, const float *alpha, const float *W, const float *A,
+                 int64_t N, int32_t k, int alpha_mode, float *dW, float *dA, float *dalpha,
+                 void *workspace, size_t workspace_bytes, void *stream);
+
 /* Pack an existing real-valued tile (Sec. 5.1: tiles are stored one bit per element):
  * src[i] > 0 -> bit 1, else 0.  src: q fp32 values.  tile_bits: tbn_tile_words(q) words. */
 int tbn_pack_tile(const float *src, int64_t q, uint32_t *tile_bits, void *stream);

@@ -54,6 +54,9 @@ SIGNATURES = {
     "tbn_debug_force_linear_config": (c_int, [c_int, c_int]),
     "tbn_debug_force_mlp_layerwise": (c_int, [c_int]),
     "tbn_debug_force_bin_config": (c_int, [c_int]),
+    "tbn_tile_fwd": (c_int, [c_vp, c_vp, c_i64, c_i32, c_int, c_vp, c_int, c_vp, c_vp, c_vp, c_sz, c_vp]),
+    "tbn_tile_bwd_workspace_bytes": (c_sz, [c_i64, c_i32]),
+    "tbn_tile_bwd": (c_int, [c_vp, c_vp, c_vp, c_vp, c_vp, c_i64, c_i32, c_int, c_vp, c_vp, c_vp, c_vp, c_sz, c_vp]),
     "tbn_row_words": (c_i64, [c_i32]),
     "tbn_binarize_fwd": (c_int, [c_vp, c_int, c_i64, c_i32, c_vp, c_vp, c_vp]),
     "tbn_linear_bin_fwd": (c_int, [c_vp, c_i64, c_i32, c_i32, c_vp, c_i32, c_vp, c_int, c_vp, c_vp, c_int, c_vp, c_int,
@@ -319,3 +322,31 @@ def tbn_linear_bin_fwd(x_bits: torch.Tensor, in_f: int, out_f: int, tile: torch.
     _check(lib().tbn_linear_bin_fwd(_ptr(x_bits), T, in_f, out_f, _ptr(tile), k, _ptr(alpha), alpha_mode, _ptr(beta),
                                     _ptr(bias), act, _ptr(y), y_dtype, _stream(), path), "tbn_linear_bin_fwd")
     return y
+
+
+def tbn_tile_fwd(W: torch.Tensor, k: int, alpha_mode: int = ALPHA_PER_TILE, A: torch.Tensor | None = None,
+                 b_dtype: int = F32):
+    """Training forward of the tiling module.  Returns (B_hat [N], tile_bits, alpha)."""
+    N = W.numel()
+    if k <= 0 or N % k:
+        raise TbnError(-2, "tbn_tile_fwd")
+    B_hat = torch.empty(N, dtype=_torch_dtype(b_dtype), device=W.device)
+    tile = torch.empty(tbn_tile_words(N // k), dtype=torch.int32, device=W.device)
+    alpha = torch.empty(k if alpha_mode == ALPHA_PER_TILE else 1, dtype=torch.float32, device=W.device)
+    ws = _ws(lib().tbn_aggregate_workspace_bytes(N, k), W.device)
+    _check(lib().tbn_tile_fwd(_ptr(W), _ptr(A), N, k, alpha_mode, _ptr(B_hat), b_dtype, _ptr(tile), _ptr(alpha), _ptr(ws),
+                              ws.numel(), _stream()), "tbn_tile_fwd")
+    return B_hat, tile, alpha
+
+
+def tbn_tile_bwd(G: torch.Tensor, tile: torch.Tensor, alpha: torch.Tensor, W: torch.Tensor, k: int,
+                 alpha_mode: int = ALPHA_PER_TILE, A: torch.Tensor | None = None):
+    """Straight-through backward of the tiling module.  Returns (dW, dA or None, dalpha)."""
+    N = W.numel()
+    dW = torch.empty(N, dtype=torch.float32, device=W.device)
+    dA = torch.empty(N, dtype=torch.float32, device=W.device) if A is not None else None
+    dalpha = torch.empty(k if alpha_mode == ALPHA_PER_TILE else 1, dtype=torch.float32, device=W.device)
+    ws = _ws(lib().tbn_tile_bwd_workspace_bytes(N, k), W.device)
+    _check(lib().tbn_tile_bwd(_ptr(G), _ptr(tile), _ptr(alpha), _ptr(W), _ptr(A), N, k, alpha_mode, _ptr(dW), _ptr(dA),
+                              _ptr(dalpha), _ptr(ws), ws.numel(), _stream()), "tbn_tile_bwd")
+    return dW, dA, dalpha

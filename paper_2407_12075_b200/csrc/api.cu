@@ -759,6 +759,36 @@ int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t 
     return TBN_OK;
 }
 
+size_t tbn_tile_bwd_workspace_bytes(int64_t N, int32_t k)
+{
+    if (N <= 0 || k <= 0 || N % k != 0) return 0;
+    return round_up(tile_bwd_workspace_bytes(N, k), 256);
+}
+
+int tbn_tile_fwd(const float *W, const float *A, int64_t N, int32_t k, int alpha_mode, void *B_hat, int b_dtype,
+                 uint32_t *tile_bits, float *alpha, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!B_hat || !valid_dtype(b_dtype) || !aligned16(B_hat)) return TBN_ERR_INVALID_ARG;
+    int rc = tbn_aggregate_tile(W, A, N, k, alpha_mode, tile_bits, alpha, workspace, workspace_bytes, stream);
+    if (rc != TBN_OK) return rc;
+    return launch_tile_expand(tile_bits, N, k, alpha, alpha_mode == TBN_ALPHA_PER_TILE, B_hat, b_dtype,
+                              static_cast<cudaStream_t>(stream)) == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+}
+
+int tbn_tile_bwd(const float *G, const uint32_t *tile_bits, const float *alpha, const float *W, const float *A,
+                 int64_t N, int32_t k, int alpha_mode, float *dW, float *dA, float *dalpha,
+                 void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!G || !tile_bits || !alpha || !W || !dW || N <= 0 || k <= 0 || !valid_alpha_mode(alpha_mode)) return TBN_ERR_INVALID_ARG;
+    if ((A == nullptr) != (dA == nullptr)) return TBN_ERR_INVALID_ARG;       // dA goes with a separate A
+    if (N % k != 0) return TBN_ERR_SHAPE;
+    if (!aligned16(G) || !aligned16(W) || !aligned16(dW) || (A && (!aligned16(A) || !aligned16(dA))) || !aligned16(tile_bits))
+        return TBN_ERR_INVALID_ARG;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < tile_bwd_workspace_bytes(N, k)) return TBN_ERR_WORKSPACE;
+    return launch_tile_bwd(G, tile_bits, alpha, W, A, N, k, alpha_mode == TBN_ALPHA_PER_TILE, dW, dA, dalpha, workspace,
+                           static_cast<cudaStream_t>(stream)) == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+}
+
 int64_t tbn_row_words(int32_t n) { return tbn_tile_words(n); }
 
 int tbn_binarize_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, uint32_t *x_bits, float *beta, void *stream)

@@ -163,6 +163,14 @@ bool bin_tensor_supported(const BinArgs &a);
 int launch_bin_tensor(const BinArgs &a, int *device_status, cudaStream_t s);
 int force_bin_config(int candidate);                           // testing / tuning aid: candidate < 0 clears
 
+// ---- training-side tiling module (train.cu) ---------------------------------------------------------
+cudaError_t launch_tile_expand(const uint32_t *tile, int64_t N, int32_t k, const float *alpha, int per_tile, void *B_hat,
+                               int b_dtype, cudaStream_t s);
+size_t tile_bwd_workspace_bytes(int64_t N, int32_t k);
+cudaError_t launch_tile_bwd(const float *G, const uint32_t *tile, const float *alpha, const float *W, const float *A,
+                            int64_t N, int32_t k, int per_tile, float *dW, float *dA, float *dalpha_out, void *workspace,
+                            cudaStream_t s);
+
 // ---- launchers implemented in the other translation units ---------------------------------------
 cudaError_t launch_aggregate(const float *W, const float *A, int64_t N, int32_t k, int per_tile,
                              uint32_t *tile_bits, float *alpha, void *workspace, cudaStream_t s);
