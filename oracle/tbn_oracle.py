@@ -296,6 +296,63 @@ def mlp(x, layers, hidden_act=ACT_RELU, mirror_bf16=False):
 
 
 # --------------------------------------------------------------------------- #
+# Transformer encoder block with tiled linears (Sec. 4.3 trains Vision            #
+# Transformers whose Q, K, V, projection and feed-forward layers are tiled;    #
+# Sec. 5.2 profiles the kernel inside one).  The glue is the standard pre-norm  #
+# block; none of it is specific to the paper.                                   #
+# --------------------------------------------------------------------------- #
+def layernorm(x: np.ndarray, gamma=None, beta=None, eps: float = 1e-5) -> np.ndarray:
+    """Row-wise (v - mean) / sqrt(var + eps) with the biased variance, optional affine; fp64."""
+    v = widen(x)
+    mu = v.mean(axis=-1, keepdims=True)
+    var = ((v - mu) ** 2).mean(axis=-1, keepdims=True)
+    y = (v - mu) / np.sqrt(var + eps)
+    if gamma is not None:
+        y = y * np.asarray(gamma, dtype=np.float64)
+    if beta is not None:
+        y = y + np.asarray(beta, dtype=np.float64)
+    return y
+
+
+def attention(qkv: np.ndarray, Nb: int, S: int, heads: int, d_head: int) -> np.ndarray:
+    """Multi-head softmax attention.  qkv: [Nb*S, 3*heads*d_head] with columns (q | k | v), head h at
+    h*d_head inside each third.  out[b, s, h*d_head + e] = sum_t softmax_t(q_s . k_t / sqrt(d_head)) v_t[e]; fp64."""
+    v = widen(qkv).reshape(Nb, S, 3, heads, d_head)
+    out = np.empty((Nb, S, heads, d_head))
+    for b in range(Nb):
+        for h in range(heads):
+            q, k, val = v[b, :, 0, h, :], v[b, :, 1, h, :], v[b, :, 2, h, :]
+            sc = (q @ k.T) / np.sqrt(float(d_head))
+            sc = sc - sc.max(axis=1, keepdims=True)
+            pr = np.exp(sc)
+            pr = pr / pr.sum(axis=1, keepdims=True)
+            out[b, :, h, :] = pr @ val
+    return out.reshape(Nb * S, heads * d_head)
+
+
+def vit_block(x: np.ndarray, Nb: int, S: int, heads: int, layers: dict, mirror_bf16: bool = False) -> np.ndarray:
+    """Pre-norm encoder block: x1 = x + proj(attn(qkv(LN(x)))); y = x1 + fc2(gelu(fc1(LN(x1)))).
+    layers: dict with keys qkv, proj, fc1, fc2, each dict(words, p, alphas, per_tile, m, n).  LayerNorm without affine
+    parameters, eps 1e-5; GELU in its erf form.  Strict mode keeps fp64 throughout; mirror_bf16 rounds every tensor a
+    bf16 pipeline would store (diagnostic)."""
+    rnd = round_to_bf16 if mirror_bf16 else (lambda v: v)
+
+    def lin(h, name, act=ACT_NONE):
+        L = layers[name]
+        return linear(h, L["words"], L["p"], L["alphas"], L["per_tile"], L["m"], L["n"], act=act)
+
+    x0 = widen(x)
+    d = x0.shape[1]
+    h1 = rnd(layernorm(x0))
+    qkv = rnd(lin(h1, "qkv"))
+    a = rnd(attention(qkv, Nb, S, heads, d // heads))
+    x1 = rnd(x0 + lin(a, "proj"))
+    h2 = rnd(layernorm(x1))
+    f = rnd(lin(h2, "fc1", ACT_GELU))
+    return x1 + lin(f, "fc2")
+
+
+# --------------------------------------------------------------------------- #
 # Training-side tiling module (Sec. 3: Eq. 1-5 in the forward of a custom       #
 # differentiation module, gradients passed straight through on the way back)   #
 # --------------------------------------------------------------------------- #
