@@ -176,6 +176,14 @@ int tbn_linear_fwd_path(const void *x, int x_dtype, int64_t T, int32_t in_f, int
 /* The family TBN_PATH_AUTO resolves to for this shape (a tbn_path), or a negative tbn_status. */
 int tbn_linear_select_path(int64_t T, int32_t in_f, int32_t out_f, int32_t k, int x_dtype);
 
+/* Same layer with a residual input: y = act(...) + residual, where residual is a tensor shaped and typed like y (NULL:
+ * exactly tbn_linear_fwd_path).  The residual connections of a Transformer block around the tiled projection and
+ * feed-forward layers (Sec. 4.3) are the use; the paper itself writes no formula for it. */
+int tbn_linear_res_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, int32_t out_f,
+                       const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                       const float *bias, int act, const void *residual, void *y, int y_dtype,
+                       void *workspace, size_t workspace_bytes, void *stream, int path);
+
 /*
  * Full-precision tiled weights (Sec. 5.2: the "FP, Tiled" kernel measured in Table 7 and Fig. 6; named as future
  * work for large models in Sec. 7).  The layer stores a tile of q = in_f*out_f/k REAL values; the weight matrix is
@@ -297,6 +305,35 @@ int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t 
                 const uint32_t *const *tiles, const int32_t *ks, const float *const *alphas,
                 const int *alpha_modes, int hidden_act, void *y, int y_dtype,
                 void *workspace, size_t workspace_bytes, void *stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Transformer encoder block with tiled linears (Sec. 4.3 trains Vision Transformers whose Q, K, V, projection and
+ * feed-forward layers are tiled; Sec. 5.2 measures the kernel inside one).  The block is the standard pre-norm one:
+ *
+ *     x1 = x  + proj( attention( qkv( LN(x) ) ) )
+ *     y  = x1 + fc2( gelu( fc1( LN(x1) ) ) )
+ *
+ * with the four linears tiled (no biases, as in the paper), LayerNorm without affine parameters (eps 1e-5), the erf
+ * form of GELU and softmax(q k^T / sqrt(d_head)) v attention.  Everything but the four linears is ordinary glue that
+ * the paper does not define; it is here so that the block runs end to end on the device.
+ *
+ * tbn_layernorm_fwd: y[t][:] = (x[t][:] - mean) / sqrt(var + eps) * gamma + beta over the d values of a row (biased
+ *   variance, statistics in fp32); gamma, beta: d floats each or NULL.  x, y: T x d, fp32 or bf16.
+ * tbn_attention_fwd: qkv: (Nb*S) x (3*heads*d_head) bf16, columns (q | k | v), head h at h*d_head inside each third;
+ *   out: (Nb*S) x (heads*d_head) bf16.  bf16 operands, fp32 accumulation and softmax.  d_head must be 64 and
+ *   S <= 208 (TBN_ERR_UNSUPPORTED otherwise).
+ * tbn_vit_block_fwd: x, y: (Nb*S) x d bf16.  tiles / ks / alphas / alpha_modes: HOST arrays of 4 entries in the order
+ *   qkv (d -> 3d), proj (d -> d), fc1 (d -> mlp_dim), fc2 (mlp_dim -> d); tiles and alphas hold DEVICE pointers.
+ *   workspace: tbn_vit_block_workspace_bytes(...) bytes (the block's intermediate tensors in bf16 plus the linears'
+ *   scratch).  Seven launches on `stream`; intermediate tensors are stored as bf16.
+ */
+int tbn_layernorm_fwd(const void *x, int x_dtype, int64_t T, int32_t d, const float *gamma, const float *beta, float eps,
+                      void *y, int y_dtype, void *stream);
+int tbn_attention_fwd(const void *qkv, int32_t Nb, int32_t S, int32_t heads, int32_t d_head, void *out, void *stream);
+size_t tbn_vit_block_workspace_bytes(int32_t Nb, int32_t S, int32_t d, int32_t mlp_dim, const int32_t *ks);
+int tbn_vit_block_fwd(const void *x, int32_t Nb, int32_t S, int32_t d, int32_t heads, int32_t mlp_dim,
+                      const uint32_t *const *tiles, const int32_t *ks, const float *const *alphas, const int *alpha_modes,
+                      void *y, void *workspace, size_t workspace_bytes, void *stream);
 
 /* ------------------------------------------------------------------------------------------------
  * Device-side status.  Kernels that wait on hardware barriers bound every wait; when a wait gives

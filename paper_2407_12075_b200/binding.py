@@ -38,6 +38,12 @@ SIGNATURES = {
     "tbn_linear_fwd": (c_int, _LINEAR_ARGS),
     "tbn_linear_fwd_path": (c_int, _LINEAR_ARGS + [c_int]),
     "tbn_linear_select_path": (c_int, [c_i64, c_i32, c_i32, c_i32, c_int]),
+    "tbn_linear_res_fwd": (c_int, [c_vp, c_int, c_i64, c_i32, c_i32, c_vp, c_i32, c_vp, c_int, c_vp, c_int, c_vp, c_vp, c_int,
+                                   c_vp, c_sz, c_vp, c_int]),
+    "tbn_layernorm_fwd": (c_int, [c_vp, c_int, c_i64, c_i32, c_vp, c_vp, ctypes.c_float, c_vp, c_int, c_vp]),
+    "tbn_attention_fwd": (c_int, [c_vp, c_i32, c_i32, c_i32, c_i32, c_vp, c_vp]),
+    "tbn_vit_block_workspace_bytes": (c_sz, [c_i32, c_i32, c_i32, c_i32, c_vp]),
+    "tbn_vit_block_fwd": (c_int, [c_vp, c_i32, c_i32, c_i32, c_i32, c_i32, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp, c_sz, c_vp]),
     "tbn_linear_fp_tile_workspace_bytes": (c_sz, [c_i64, c_i32, c_i32, c_i32, c_int, c_int]),
     "tbn_linear_fp_tile_fwd": (c_int, [c_vp, c_int, c_i64, c_i32, c_i32, c_vp, c_int, c_i32, c_vp, c_int, c_vp, c_int,
                                        c_vp, c_sz, c_vp, c_int]),
@@ -350,3 +356,54 @@ def tbn_tile_bwd(G: torch.Tensor, tile: torch.Tensor, alpha: torch.Tensor, W: to
     _check(lib().tbn_tile_bwd(_ptr(G), _ptr(tile), _ptr(alpha), _ptr(W), _ptr(A), N, k, alpha_mode, _ptr(dW), _ptr(dA),
                               _ptr(dalpha), _ptr(ws), ws.numel(), _stream()), "tbn_tile_bwd")
     return dW, dA, dalpha
+
+
+def tbn_linear_res_fwd(x: torch.Tensor, out_f: int, tile: torch.Tensor, k: int, alpha: torch.Tensor, alpha_mode: int,
+                       residual: torch.Tensor, bias: torch.Tensor | None = None, act: int = ACT_NONE,
+                       path: int = PATH_AUTO, y: torch.Tensor | None = None, workspace: torch.Tensor | None = None):
+    """y = act(layer(x)) + residual; residual has y's shape and dtype."""
+    T, in_f = x.shape
+    xd, yd = _dtype_code(x), _dtype_code(residual)
+    if y is None:
+        y = torch.empty((T, out_f), dtype=residual.dtype, device=x.device)
+    ws = workspace if workspace is not None else _ws(tbn_linear_workspace_bytes(T, in_f, out_f, k, xd), x.device)
+    _check(lib().tbn_linear_res_fwd(_ptr(x), xd, T, in_f, out_f, _ptr(tile), k, _ptr(alpha), alpha_mode, _ptr(bias), act,
+                                    _ptr(residual), _ptr(y), yd, _ptr(ws), ws.numel(), _stream(), path), "tbn_linear_res_fwd")
+    return y
+
+
+def tbn_layernorm_fwd(x: torch.Tensor, gamma: torch.Tensor | None = None, beta: torch.Tensor | None = None,
+                      eps: float = 1e-5, y_dtype: int | None = None) -> torch.Tensor:
+    T, d = x.shape
+    yd = _dtype_code(x) if y_dtype is None else y_dtype
+    y = torch.empty((T, d), dtype=_torch_dtype(yd), device=x.device)
+    _check(lib().tbn_layernorm_fwd(_ptr(x), _dtype_code(x), T, d, _ptr(gamma), _ptr(beta), eps, _ptr(y), yd, _stream()),
+           "tbn_layernorm_fwd")
+    return y
+
+
+def tbn_attention_fwd(qkv: torch.Tensor, Nb: int, S: int, heads: int, d_head: int) -> torch.Tensor:
+    out = torch.empty((Nb * S, heads * d_head), dtype=torch.bfloat16, device=qkv.device)
+    _check(lib().tbn_attention_fwd(_ptr(qkv), Nb, S, heads, d_head, _ptr(out), _stream()), "tbn_attention_fwd")
+    return out
+
+
+def tbn_vit_block_workspace_bytes(Nb, S, d, mlp_dim, ks) -> int:
+    return int(lib().tbn_vit_block_workspace_bytes(Nb, S, d, mlp_dim, ctypes.cast(_i32_array(ks), c_vp)))
+
+
+def tbn_vit_block_fwd(x: torch.Tensor, Nb: int, S: int, heads: int, mlp_dim: int, tiles, ks, alphas, alpha_modes,
+                      workspace: torch.Tensor | None = None, y: torch.Tensor | None = None) -> torch.Tensor:
+    """Pre-norm encoder block; tiles / ks / alphas / alpha_modes in the order qkv, proj, fc1, fc2."""
+    T, d = x.shape
+    if y is None:
+        y = torch.empty_like(x)
+    ws = workspace if workspace is not None else _ws(tbn_vit_block_workspace_bytes(Nb, S, d, mlp_dim, ks), x.device)
+    k_arr = _i32_array(ks)
+    m_arr = (c_int * 4)(*[int(v) for v in alpha_modes])
+    t_arr = (c_vp * 4)(*[_ptr(t) for t in tiles])
+    a_arr = (c_vp * 4)(*[_ptr(a) for a in alphas])
+    _check(lib().tbn_vit_block_fwd(_ptr(x), Nb, S, d, heads, mlp_dim, ctypes.cast(t_arr, c_vp), ctypes.cast(k_arr, c_vp),
+                                   ctypes.cast(a_arr, c_vp), ctypes.cast(m_arr, c_vp), _ptr(y), _ptr(ws), ws.numel(),
+                                   _stream()), "tbn_vit_block_fwd")
+    return y

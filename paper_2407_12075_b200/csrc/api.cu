@@ -478,6 +478,20 @@ int tbn_linear_fwd_path(const void *x, int x_dtype, int64_t T, int32_t in_f, int
     return run_layer(a, path, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
 }
 
+int tbn_linear_res_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, int32_t out_f,
+                       const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                       const float *bias, int act, const void *residual, void *y, int y_dtype,
+                       void *workspace, size_t workspace_bytes, void *stream, int path)
+{
+    LayerArgs a;
+    int rc = fill_linear(a, x, x_dtype, T, in_f, out_f, tile_bits, k, alpha, alpha_mode, bias, act, y,
+                         y_dtype, path);
+    if (rc != TBN_OK) return rc;
+    if (residual && !aligned16(residual)) return TBN_ERR_INVALID_ARG;
+    a.residual = residual;
+    return run_layer(a, path, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
 int tbn_linear_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, int32_t out_f,
                    const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
                    const float *bias, int act, void *y, int y_dtype,
@@ -787,6 +801,88 @@ int tbn_tile_bwd(const float *G, const uint32_t *tile_bits, const float *alpha, 
     if (!workspace || !aligned16(workspace) || workspace_bytes < tile_bwd_workspace_bytes(N, k)) return TBN_ERR_WORKSPACE;
     return launch_tile_bwd(G, tile_bits, alpha, W, A, N, k, alpha_mode == TBN_ALPHA_PER_TILE, dW, dA, dalpha, workspace,
                            static_cast<cudaStream_t>(stream)) == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+}
+
+int tbn_layernorm_fwd(const void *x, int x_dtype, int64_t T, int32_t d, const float *gamma, const float *beta, float eps,
+                      void *y, int y_dtype, void *stream)
+{
+    if (T < 0 || d <= 0 || !valid_dtype(x_dtype) || !valid_dtype(y_dtype) || !(eps >= 0.0f)) return TBN_ERR_INVALID_ARG;
+    if (T == 0) return TBN_OK;
+    if (!x || !y) return TBN_ERR_INVALID_ARG;
+    return launch_layernorm(x, x_dtype, T, d, gamma, beta, eps, y, y_dtype, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? TBN_OK : TBN_ERR_CUDA;
+}
+
+int tbn_attention_fwd(const void *qkv, int32_t Nb, int32_t S, int32_t heads, int32_t d_head, void *out, void *stream)
+{
+    if (Nb < 0 || S <= 0 || heads <= 0 || d_head <= 0) return TBN_ERR_INVALID_ARG;
+    if (Nb == 0) return TBN_OK;
+    if (!qkv || !out || !aligned16(qkv) || !aligned16(out)) return TBN_ERR_INVALID_ARG;
+    if (!attention_supported(S, heads, d_head) || (int64_t)Nb * heads > 0x7fffffffLL) return TBN_ERR_UNSUPPORTED;
+    return launch_attention(qkv, Nb, S, heads, d_head, out, static_cast<cudaStream_t>(stream)) == cudaSuccess ? TBN_OK
+                                                                                                               : TBN_ERR_CUDA;
+}
+
+// workspace layout of the encoder block: [h: T x d][qkv: T x 3d][att: T x d][x1: T x d][f: T x mlp] bf16, then the
+// largest scratch of its four linears
+static size_t block_offsets(int64_t T, int32_t d, int32_t mlp, const int32_t *ks, size_t off[6])
+{
+    size_t o = 0;
+    const size_t sizes[5] = {(size_t)T * d * 2, (size_t)T * 3 * d * 2, (size_t)T * d * 2, (size_t)T * d * 2, (size_t)T * mlp * 2};
+    for (int i = 0; i < 5; ++i) { off[i] = o; o += round_up(sizes[i], 256); }
+    off[5] = o;
+    size_t scratch = 0;
+    const int32_t shapes[4][2] = {{d, 3 * d}, {d, d}, {d, mlp}, {mlp, d}};
+    for (int l = 0; l < 4; ++l) {
+        const size_t b = tbn_linear_workspace_bytes(T, shapes[l][0], shapes[l][1], ks[l], TBN_BF16);
+        scratch = b > scratch ? b : scratch;
+    }
+    return o + scratch;
+}
+
+size_t tbn_vit_block_workspace_bytes(int32_t Nb, int32_t S, int32_t d, int32_t mlp_dim, const int32_t *ks)
+{
+    if (Nb <= 0 || S <= 0 || d <= 0 || mlp_dim <= 0 || !ks) return 0;
+    size_t off[6];
+    return block_offsets((int64_t)Nb * S, d, mlp_dim, ks, off);
+}
+
+int tbn_vit_block_fwd(const void *x, int32_t Nb, int32_t S, int32_t d, int32_t heads, int32_t mlp_dim,
+                      const uint32_t *const *tiles, const int32_t *ks, const float *const *alphas, const int *alpha_modes,
+                      void *y, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (Nb < 0 || S <= 0 || d <= 0 || heads <= 0 || mlp_dim <= 0 || !tiles || !ks || !alphas || !alpha_modes)
+        return TBN_ERR_INVALID_ARG;
+    if (d % heads != 0) return TBN_ERR_SHAPE;
+    for (int l = 0; l < 4; ++l)
+        if (!tiles[l] || !alphas[l] || ks[l] <= 0 || !valid_alpha_mode(alpha_modes[l])) return TBN_ERR_INVALID_ARG;
+    if (Nb == 0) return TBN_OK;
+    if (!x || !y || !aligned16(x) || !aligned16(y)) return TBN_ERR_INVALID_ARG;
+    if (!attention_supported(S, heads, d / heads)) return TBN_ERR_UNSUPPORTED;
+    const int64_t T = (int64_t)Nb * S;
+    size_t off[6];
+    const size_t need = block_offsets(T, d, mlp_dim, ks, off);
+    if (!workspace || !aligned16(workspace) || workspace_bytes < need) return TBN_ERR_WORKSPACE;
+    char *ws = static_cast<char *>(workspace);
+    void *h = ws + off[0], *qkv = ws + off[1], *att = ws + off[2], *x1 = ws + off[3], *f = ws + off[4], *scratch = ws + off[5];
+    const size_t scratch_bytes = workspace_bytes - off[5];
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int B16 = TBN_BF16, AUTO = TBN_PATH_AUTO;
+    int rc;
+    if (launch_layernorm(x, B16, T, d, nullptr, nullptr, 1e-5f, h, B16, s) != cudaSuccess) return TBN_ERR_CUDA;
+    rc = tbn_linear_fwd_path(h, B16, T, d, 3 * d, tiles[0], ks[0], alphas[0], alpha_modes[0], nullptr, TBN_ACT_NONE, qkv, B16,
+                             scratch, scratch_bytes, stream, AUTO);
+    if (rc != TBN_OK) return rc;
+    if (launch_attention(qkv, Nb, S, heads, d / heads, att, s) != cudaSuccess) return TBN_ERR_CUDA;
+    rc = tbn_linear_res_fwd(att, B16, T, d, d, tiles[1], ks[1], alphas[1], alpha_modes[1], nullptr, TBN_ACT_NONE, x, x1, B16,
+                            scratch, scratch_bytes, stream, AUTO);
+    if (rc != TBN_OK) return rc;
+    if (launch_layernorm(x1, B16, T, d, nullptr, nullptr, 1e-5f, h, B16, s) != cudaSuccess) return TBN_ERR_CUDA;
+    rc = tbn_linear_fwd_path(h, B16, T, d, mlp_dim, tiles[2], ks[2], alphas[2], alpha_modes[2], nullptr, TBN_ACT_GELU, f, B16,
+                             scratch, scratch_bytes, stream, AUTO);
+    if (rc != TBN_OK) return rc;
+    return tbn_linear_res_fwd(f, B16, T, mlp_dim, d, tiles[3], ks[3], alphas[3], alpha_modes[3], nullptr, TBN_ACT_NONE, x1, y, B16,
+                              scratch, scratch_bytes, stream, AUTO);
 }
 
 int64_t tbn_row_words(int32_t n) { return tbn_tile_words(n); }

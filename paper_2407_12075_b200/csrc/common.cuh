@@ -131,6 +131,7 @@ struct LayerArgs {
     int fp_tile_dtype;     // TBN_F32 or TBN_BF16
     const float *alpha;
     const float *bias;
+    const void *residual;  // fully-connected only: a tensor shaped and typed like y, added after the activation (or null)
     int64_t T;       // rows of the contraction: tokens, or Nb*Ho*Wo output pixels
     int32_t n;       // contraction length: in_features or Cin*kh*kw
     int32_t m;       // output features / channels
@@ -170,6 +171,12 @@ size_t tile_bwd_workspace_bytes(int64_t N, int32_t k);
 cudaError_t launch_tile_bwd(const float *G, const uint32_t *tile, const float *alpha, const float *W, const float *A,
                             int64_t N, int32_t k, int per_tile, float *dW, float *dA, float *dalpha_out, void *workspace,
                             cudaStream_t s);
+
+// ---- encoder-block glue (block.cu) ----------------------------------------------------------------------
+cudaError_t launch_layernorm(const void *x, int x_dtype, int64_t T, int32_t d, const float *gamma, const float *beta, float eps,
+                             void *y, int y_dtype, cudaStream_t s);
+bool attention_supported(int32_t S, int32_t heads, int32_t d_head);
+cudaError_t launch_attention(const void *qkv, int32_t Nb, int32_t S, int32_t heads, int32_t d_head, void *out, cudaStream_t s);
 
 // ---- launchers implemented in the other translation units ---------------------------------------
 cudaError_t launch_aggregate(const float *W, const float *A, int64_t N, int32_t k, int per_tile,

@@ -114,7 +114,7 @@ generic_kernel(const LayerArgs a)
     for (int t = 0; t < kTok; ++t) {
         const int64_t tok = t0 + t;
         if (tok >= a.T) break;
-        const float v = apply_act(fmaf(alpha_cur, seg[t], tot[t]) + b, a.act);
+        float v = apply_act(fmaf(alpha_cur, seg[t], tot[t]) + b, a.act);
         int64_t yi;
         if (!a.is_conv) {
             yi = tok * a.m + o;
@@ -122,6 +122,9 @@ generic_kernel(const LayerArgs a)
             const int64_t hw = (int64_t)a.Ho * a.Wo;
             yi = ((tok / hw) * a.m + o) * hw + tok % hw;
         }
+        if (a.residual != nullptr)
+            v += a.y_dtype == TBN_BF16 ? load_as_float(static_cast<const __nv_bfloat16 *>(a.residual), yi)
+                                       : load_as_float(static_cast<const float *>(a.residual), yi);
         if (a.y_dtype == TBN_BF16) store_from_float(static_cast<__nv_bfloat16 *>(a.y), yi, v);
         else store_from_float(static_cast<float *>(a.y), yi, v);
     }

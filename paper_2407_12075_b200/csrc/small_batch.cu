@@ -109,8 +109,11 @@ small_batch_kernel(const LayerArgs a, int32_t r)
                 if (r2 == rr && t2 == t) z = acc[r2][t2];
         const int32_t o = j * r + row;
         const float al = per_tile ? __ldg(a.alpha + j) : __ldg(a.alpha);
-        const float v = apply_act(fmaf(al, z, a.bias ? __ldg(a.bias + o) : 0.0f), a.act);
+        float v = apply_act(fmaf(al, z, a.bias ? __ldg(a.bias + o) : 0.0f), a.act);
         const int64_t yi = (t0 + t) * a.m + o;
+        if (a.residual != nullptr)
+            v += a.y_dtype == TBN_BF16 ? load_as_float(static_cast<const __nv_bfloat16 *>(a.residual), yi)
+                                       : load_as_float(static_cast<const float *>(a.residual), yi);
         if (a.y_dtype == TBN_BF16) store_from_float(static_cast<__nv_bfloat16 *>(a.y), yi, v);
         else store_from_float(static_cast<float *>(a.y), yi, v);
     }
@@ -274,8 +277,11 @@ small_mma_kernel(const LayerArgs a, int32_t r)
         for (int32_t j = 0; j < a.k; ++j) {
             const int32_t o = j * r + grow;
             const float al = j < 64 ? alpha_s[j] : __ldg(a.alpha + (per_tile ? j : 0));
-            const float v = apply_act(fmaf(al, z, a.bias ? __ldg(a.bias + o) : 0.0f), a.act);
+            float v = apply_act(fmaf(al, z, a.bias ? __ldg(a.bias + o) : 0.0f), a.act);
             const int64_t yi = t * a.m + o;
+            if (a.residual != nullptr)
+                v += a.y_dtype == TBN_BF16 ? load_as_float(static_cast<const __nv_bfloat16 *>(a.residual), yi)
+                                           : load_as_float(static_cast<const float *>(a.residual), yi);
             if (a.y_dtype == TBN_BF16) store_from_float(static_cast<__nv_bfloat16 *>(a.y), yi, v);
             else store_from_float(static_cast<float *>(a.y), yi, v);
         }
