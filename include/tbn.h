@@ -281,6 +281,19 @@ int tbn_conv2d_fwd_path(const void *x, int x_dtype, int32_t Nb, int32_t Cin, int
                         const float *bias, int act, void *y, int y_dtype,
                         void *workspace, size_t workspace_bytes, void *stream, int path);
 
+/* The full-precision ends of a convolution stack.  Layers below the size threshold of Sec. 3 (hyperparameter lambda)
+ * are not tiled: in a ResNet-style stack the first convolution and the classifier stay full precision.
+ * tbn_conv2d_dense_fwd: the convolution above with an explicit fp32 weight (Cout, Cin, kh, kw) instead of a tile, for
+ *   short contractions (Cin*kh*kw <= 512; TBN_ERR_UNSUPPORTED beyond); x, y NCHW, fp32 or bf16; bias Cout floats or NULL.
+ * tbn_global_avgpool_fwd: y[b][c] = mean over the H*Wd positions of x[b][c]; x NCHW, y (Nb, C); fp32 accumulation.
+ * (A full-precision classifier is tbn_linear_fp_tile_fwd with k = 1.)  Neither is defined by the paper; both are
+ * ordinary layers that the stack needs to run end to end. */
+int tbn_conv2d_dense_fwd(const void *x, int x_dtype, int32_t Nb, int32_t Cin, int32_t H, int32_t Wd, int32_t Cout, int32_t kh,
+                         int32_t kw, int32_t stride, int32_t pad, const float *weight, const float *bias, int act, void *y,
+                         int y_dtype, void *stream);
+int tbn_global_avgpool_fwd(const void *x, int x_dtype, int32_t Nb, int32_t C, int32_t H, int32_t Wd, void *y, int y_dtype,
+                           void *stream);
+
 /* ------------------------------------------------------------------------------------------------
  * Chain of L fully-connected tiled layers (Sec. 5.1: an MLP with a fused ReLU):
  *     h_0 = x;  h_{l+1} = hidden_act(layer_l(h_l)) for l < L-1;  y = layer_{L-1}(h_{L-1}).

@@ -278,6 +278,19 @@ def conv2d(x, words, p, alphas, per_tile, Cout, Cin, kh, kw, stride, pad, bias=N
     return conv2d_dense(x, B_hat, Cout, Cin, kh, kw, stride, pad, bias, act)
 
 
+def conv_stack(x, W0, convs, Wfc):
+    """ResNet-style stack with full-precision ends (Sec. 3: layers below the size threshold are not tiled):
+    dense 3x3 convolution W0 (stride 1, padding 1) -> ReLU -> tiled 3x3 convolutions (each a dict words, p, alphas, per_tile,
+    Cout, Cin, stride; padding 1) with ReLU -> global average pooling -> dense classifier Wfc [classes, C].  fp64."""
+    W0 = np.asarray(W0, dtype=np.float32)
+    h = conv2d_dense(x, W0, W0.shape[0], W0.shape[1], W0.shape[2], W0.shape[3], 1, 1, act=ACT_RELU)
+    for c in convs:
+        h = conv2d(h, c["words"], c["p"], c["alphas"], c["per_tile"], c["Cout"], c["Cin"], 3, 3, c["stride"], 1, act=ACT_RELU)
+    pooled = h.mean(axis=(2, 3))
+    Wfc = np.asarray(Wfc, dtype=np.float32)
+    return linear_dense(pooled, Wfc, Wfc.shape[0], Wfc.shape[1])
+
+
 def mlp(x, layers, hidden_act=ACT_RELU, mirror_bf16=False):
     """Chain of tiled fully-connected layers (Sec. 5.1's MLP with fused ReLU).
 

@@ -52,6 +52,8 @@ SIGNATURES = {
     "tbn_conv2d_workspace_bytes": (c_sz, [c_i32] * 10 + [c_int]),
     "tbn_conv2d_fwd": (c_int, _CONV_ARGS),
     "tbn_conv2d_fwd_path": (c_int, _CONV_ARGS + [c_int]),
+    "tbn_conv2d_dense_fwd": (c_int, [c_vp, c_int] + [c_i32] * 9 + [c_vp, c_vp, c_int, c_vp, c_int, c_vp]),
+    "tbn_global_avgpool_fwd": (c_int, [c_vp, c_int, c_i32, c_i32, c_i32, c_i32, c_vp, c_int, c_vp]),
     "tbn_mlp_workspace_bytes": (c_sz, [c_i64, c_i32, c_vp, c_vp, c_int]),
     "tbn_mlp_fwd": (c_int, [c_vp, c_int, c_i64, c_i32, c_vp, c_vp, c_vp, c_vp, c_vp, c_int, c_vp, c_int,
                             c_vp, c_sz, c_vp]),
@@ -406,4 +408,27 @@ def tbn_vit_block_fwd(x: torch.Tensor, Nb: int, S: int, heads: int, mlp_dim: int
     _check(lib().tbn_vit_block_fwd(_ptr(x), Nb, S, d, heads, mlp_dim, ctypes.cast(t_arr, c_vp), ctypes.cast(k_arr, c_vp),
                                    ctypes.cast(a_arr, c_vp), ctypes.cast(m_arr, c_vp), _ptr(y), _ptr(ws), ws.numel(),
                                    _stream()), "tbn_vit_block_fwd")
+    return y
+
+
+def tbn_conv2d_dense_fwd(x: torch.Tensor, weight: torch.Tensor, stride: int, pad: int, bias=None, act=ACT_NONE,
+                         y_dtype=None) -> torch.Tensor:
+    """Convolution with an explicit fp32 weight (Cout, Cin, kh, kw): the untiled first layer of a stack."""
+    Nb, Cin, H, Wd = x.shape
+    Cout, _, kh, kw = weight.shape
+    xd = _dtype_code(x)
+    yd = xd if y_dtype is None else y_dtype
+    Ho, Wo = (H + 2 * pad - kh) // stride + 1, (Wd + 2 * pad - kw) // stride + 1
+    y = torch.empty((Nb, Cout, Ho, Wo), dtype=_torch_dtype(yd), device=x.device)
+    _check(lib().tbn_conv2d_dense_fwd(_ptr(x), xd, Nb, Cin, H, Wd, Cout, kh, kw, stride, pad, _ptr(weight), _ptr(bias), act,
+                                      _ptr(y), yd, _stream()), "tbn_conv2d_dense_fwd")
+    return y
+
+
+def tbn_global_avgpool_fwd(x: torch.Tensor, y_dtype=None) -> torch.Tensor:
+    Nb, C, H, Wd = x.shape
+    xd = _dtype_code(x)
+    yd = xd if y_dtype is None else y_dtype
+    y = torch.empty((Nb, C), dtype=_torch_dtype(yd), device=x.device)
+    _check(lib().tbn_global_avgpool_fwd(_ptr(x), xd, Nb, C, H, Wd, _ptr(y), yd, _stream()), "tbn_global_avgpool_fwd")
     return y

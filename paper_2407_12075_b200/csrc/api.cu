@@ -885,6 +885,30 @@ int tbn_vit_block_fwd(const void *x, int32_t Nb, int32_t S, int32_t d, int32_t h
                               scratch, scratch_bytes, stream, AUTO);
 }
 
+int tbn_conv2d_dense_fwd(const void *x, int x_dtype, int32_t Nb, int32_t Cin, int32_t H, int32_t Wd, int32_t Cout, int32_t kh,
+                         int32_t kw, int32_t stride, int32_t pad, const float *weight, const float *bias, int act, void *y,
+                         int y_dtype, void *stream)
+{
+    if (Nb < 0 || Cin <= 0 || H <= 0 || Wd <= 0 || Cout <= 0 || kh <= 0 || kw <= 0 || stride <= 0 || pad < 0) return TBN_ERR_INVALID_ARG;
+    if (!weight || !valid_dtype(x_dtype) || !valid_dtype(y_dtype) || !valid_act(act)) return TBN_ERR_INVALID_ARG;
+    if (H + 2 * pad < kh || Wd + 2 * pad < kw) return TBN_ERR_SHAPE;
+    if (Nb == 0) return TBN_OK;
+    if (!x || !y) return TBN_ERR_INVALID_ARG;
+    if (!dense_conv_supported(Cin, kh, kw) || Cout > 65535 * 8) return TBN_ERR_UNSUPPORTED;
+    return launch_dense_conv(x, x_dtype, weight, bias, y, y_dtype, Nb, Cin, H, Wd, Cout, kh, kw, stride, pad, act,
+                             static_cast<cudaStream_t>(stream)) == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+}
+
+int tbn_global_avgpool_fwd(const void *x, int x_dtype, int32_t Nb, int32_t C, int32_t H, int32_t Wd, void *y, int y_dtype, void *stream)
+{
+    if (Nb < 0 || C <= 0 || H <= 0 || Wd <= 0 || !valid_dtype(x_dtype) || !valid_dtype(y_dtype)) return TBN_ERR_INVALID_ARG;
+    if (Nb == 0) return TBN_OK;
+    if (!x || !y) return TBN_ERR_INVALID_ARG;
+    if ((int64_t)H * Wd > 0x7fffffffLL) return TBN_ERR_UNSUPPORTED;
+    return launch_global_avgpool(x, x_dtype, (int64_t)Nb * C, H * Wd, y, y_dtype, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? TBN_OK : TBN_ERR_CUDA;
+}
+
 int64_t tbn_row_words(int32_t n) { return tbn_tile_words(n); }
 
 int tbn_binarize_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, uint32_t *x_bits, float *beta, void *stream)

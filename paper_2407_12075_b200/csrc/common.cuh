@@ -178,6 +178,13 @@ cudaError_t launch_layernorm(const void *x, int x_dtype, int64_t T, int32_t d, c
 bool attention_supported(int32_t S, int32_t heads, int32_t d_head);
 cudaError_t launch_attention(const void *qkv, int32_t Nb, int32_t S, int32_t heads, int32_t d_head, void *out, cudaStream_t s);
 
+// ---- full-precision ends of a convolution stack (dense_ends.cu) ---------------------------------------------
+bool dense_conv_supported(int32_t Cin, int32_t kh, int32_t kw);
+cudaError_t launch_dense_conv(const void *x, int x_dtype, const float *w, const float *bias, void *y, int y_dtype, int32_t Nb,
+                              int32_t Cin, int32_t H, int32_t Wd, int32_t Cout, int32_t kh, int32_t kw, int32_t stride, int32_t pad,
+                              int act, cudaStream_t s);
+cudaError_t launch_global_avgpool(const void *x, int x_dtype, int64_t planes, int32_t hw, void *y, int y_dtype, cudaStream_t s);
+
 // ---- launchers implemented in the other translation units ---------------------------------------
 cudaError_t launch_aggregate(const float *W, const float *A, int64_t N, int32_t k, int per_tile,
                              uint32_t *tile_bits, float *alpha, void *workspace, cudaStream_t s);

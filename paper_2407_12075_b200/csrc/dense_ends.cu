@@ -1,0 +1,114 @@
+// The full-precision ends of a tiled convolution stack.  The paper tiles only layers above a size threshold (Sec. 3,
+// hyperparameter lambda): in a ResNet-style stack the first convolution (a few thousand weights) and the classifier
+// stay full precision.  These kernels run them, and the global average pooling between the last convolution and the
+// classifier, so that the stack executes end to end on the device.  All three are small, memory-bound layers.
+#include "common.cuh"
+
+namespace tbn {
+
+namespace {
+
+constexpr int kDcCo = 8;              // output channels per thread
+constexpr int kDcMaxW = 4096;         // weights of one group of kDcCo filters held in shared memory (fp32)
+
+// Direct convolution with a dense fp32 weight (Cout, Cin, kh, kw) for layers with a short contraction (Cin*kh*kw up to
+// 512): a thread owns one output pixel and kDcCo consecutive output channels; the weights of those channels sit in
+// shared memory and are read as broadcasts; consecutive threads own consecutive pixels of a row, so every store
+// instruction writes one contiguous run per channel plane.
+template <typename XT, typename YT>
+__global__ void __launch_bounds__(256)
+dense_conv_kernel(const XT *__restrict__ x, const float *__restrict__ w, const float *__restrict__ bias, YT *__restrict__ y,
+                  int32_t Nb, int32_t Cin, int32_t H, int32_t Wd, int32_t Cout, int32_t kh, int32_t kw, int32_t stride,
+                  int32_t pad, int32_t Ho, int32_t Wo, int act)
+{
+    __shared__ float ws[kDcMaxW];
+    const int32_t n = Cin * kh * kw;
+    const int32_t co0 = blockIdx.y * kDcCo;
+    for (int32_t i = threadIdx.x; i < kDcCo * n; i += blockDim.x) {
+        const int32_t c = i / n, r = i - c * n;
+        ws[i] = co0 + c < Cout ? __ldg(w + (int64_t)(co0 + c) * n + r) : 0.0f;
+    }
+    __syncthreads();
+    const int64_t pixels = (int64_t)Nb * Ho * Wo;
+    for (int64_t pix = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; pix < pixels; pix += (int64_t)gridDim.x * blockDim.x) {
+        const int32_t ow = (int32_t)(pix % Wo);
+        const int64_t t = pix / Wo;
+        const int32_t oh = (int32_t)(t % Ho);
+        const int64_t b = t / Ho;
+        float acc[kDcCo];
+#pragma unroll
+        for (int c = 0; c < kDcCo; ++c) acc[c] = 0.0f;
+        for (int32_t ci = 0; ci < Cin; ++ci)
+            for (int32_t u = 0; u < kh; ++u) {
+                const int32_t ih = oh * stride + u - pad;
+                if (ih < 0 || ih >= H) continue;
+                for (int32_t v = 0; v < kw; ++v) {
+                    const int32_t iw = ow * stride + v - pad;
+                    if (iw < 0 || iw >= Wd) continue;
+                    const float xv = load_as_float(x, ((b * Cin + ci) * H + ih) * (int64_t)Wd + iw);
+                    const int32_t r = (ci * kh + u) * kw + v;
+#pragma unroll
+                    for (int c = 0; c < kDcCo; ++c) acc[c] = fmaf(ws[c * n + r], xv, acc[c]);
+                }
+            }
+#pragma unroll
+        for (int c = 0; c < kDcCo; ++c) {
+            if (co0 + c >= Cout) break;
+            const float o = apply_act(acc[c] + (bias ? __ldg(bias + co0 + c) : 0.0f), act);
+            store_from_float(y, ((b * Cout + co0 + c) * Ho + oh) * (int64_t)Wo + ow, o);
+        }
+    }
+}
+
+// Mean over the H*W positions of every (image, channel) plane: one warp per plane, fp32 accumulation.
+template <typename XT, typename YT>
+__global__ void __launch_bounds__(256)
+global_avgpool_kernel(const XT *__restrict__ x, int64_t planes, int32_t hw, YT *__restrict__ y)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t p = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; p < planes; p += warps) {
+        float s = 0.0f;
+        for (int32_t i = lane; i < hw; i += 32) s += load_as_float(x, p * hw + i);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+        if (lane == 0) store_from_float(y, p, s / (float)hw);
+    }
+}
+
+}  // namespace
+
+bool dense_conv_supported(int32_t Cin, int32_t kh, int32_t kw) { return (int64_t)Cin * kh * kw * kDcCo <= kDcMaxW; }
+
+cudaError_t launch_dense_conv(const void *x, int x_dtype, const float *w, const float *bias, void *y, int y_dtype, int32_t Nb,
+                              int32_t Cin, int32_t H, int32_t Wd, int32_t Cout, int32_t kh, int32_t kw, int32_t stride, int32_t pad,
+                              int act, cudaStream_t s)
+{
+    const int32_t Ho = (H + 2 * pad - kh) / stride + 1, Wo = (Wd + 2 * pad - kw) / stride + 1;
+    const int64_t pixels = (int64_t)Nb * Ho * Wo;
+    const int64_t bx = (pixels + 255) / 256;
+    const dim3 grid((unsigned)(bx < 148 * 64 ? (bx > 0 ? bx : 1) : 148 * 64), (unsigned)((Cout + kDcCo - 1) / kDcCo));
+#define TBN_DC(XT, YT) dense_conv_kernel<XT, YT><<<grid, 256, 0, s>>>(static_cast<const XT *>(x), w, bias, static_cast<YT *>(y), Nb, \
+                                                                       Cin, H, Wd, Cout, kh, kw, stride, pad, Ho, Wo, act)
+    if (x_dtype == TBN_BF16 && y_dtype == TBN_BF16) TBN_DC(__nv_bfloat16, __nv_bfloat16);
+    else if (x_dtype == TBN_BF16) TBN_DC(__nv_bfloat16, float);
+    else if (y_dtype == TBN_BF16) TBN_DC(float, __nv_bfloat16);
+    else TBN_DC(float, float);
+#undef TBN_DC
+    return cudaGetLastError();
+}
+
+cudaError_t launch_global_avgpool(const void *x, int x_dtype, int64_t planes, int32_t hw, void *y, int y_dtype, cudaStream_t s)
+{
+    const int64_t bx = (planes + 7) / 8;
+    const unsigned grid = (unsigned)(bx < 148 * 16 ? (bx > 0 ? bx : 1) : 148 * 16);
+#define TBN_GAP(XT, YT) global_avgpool_kernel<XT, YT><<<grid, 256, 0, s>>>(static_cast<const XT *>(x), planes, hw, static_cast<YT *>(y))
+    if (x_dtype == TBN_BF16 && y_dtype == TBN_BF16) TBN_GAP(__nv_bfloat16, __nv_bfloat16);
+    else if (x_dtype == TBN_BF16) TBN_GAP(__nv_bfloat16, float);
+    else if (y_dtype == TBN_BF16) TBN_GAP(float, __nv_bfloat16);
+    else TBN_GAP(float, float);
+#undef TBN_GAP
+    return cudaGetLastError();
+}
+
+}  // namespace tbn

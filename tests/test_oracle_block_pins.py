@@ -66,3 +66,26 @@ def test_block_is_the_composition_and_images_are_independent():
     # the mirrored mode differs only by storage rounding
     ym = O.vit_block(x, Nb, S, heads, layers, mirror_bf16=True)
     assert 0 < np.abs(ym - y).max() < 0.05
+
+
+def test_conv_stack_is_the_composition_of_torch_layers():
+    rng = np.random.default_rng(3)
+    Nb, H = 2, 8
+    x = rng.random((Nb, 3, H, H)).astype(np.float32)
+    W0 = (rng.standard_normal((8, 3, 3, 3)) * 0.3).astype(np.float32)
+    convs, dense = [], []
+    cin = 8
+    for cout, p, stride in ((16, 4, 2), (32, 2, 2)):
+        W = (rng.standard_normal(cout * cin * 9) * (2.0 / (cin * 9)) ** 0.5).astype(np.float32)
+        words, al = O.prepare(W, p, True)
+        convs.append(dict(words=words, p=p, alphas=al, per_tile=True, Cout=cout, Cin=cin, stride=stride))
+        dense.append((torch.from_numpy(O.expand(words, W.size, p, al, True).astype(np.float64).reshape(cout, cin, 3, 3)), stride))
+        cin = cout
+    Wfc = (rng.standard_normal((5, 32)) * 0.2).astype(np.float32)
+    y = O.conv_stack(x, W0, convs, Wfc)
+    F = torch.nn.functional
+    h = F.relu(F.conv2d(torch.from_numpy(x).double(), torch.from_numpy(W0).double(), padding=1))
+    for Wd, stride in dense:
+        h = F.relu(F.conv2d(h, Wd, stride=stride, padding=1))
+    ref = (F.adaptive_avg_pool2d(h, 1).flatten(1) @ torch.from_numpy(Wfc).double().T).numpy()
+    assert y.shape == (Nb, 5) and np.allclose(y, ref, rtol=1e-11, atol=1e-11)
