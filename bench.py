@@ -327,6 +327,44 @@ def measure_other_configs(B, torch, dev, peaks):
                          "vit_fc2_3072_768": (3072, 768)}.items():
         out[name] = linear_entry(25216, n, m, 8)
     out["vit_fc1_768_3072_gelu"] = linear_entry(25216, 768, 3072, 8, act=B.ACT_GELU)
+    # the whole ViT-B shaped encoder block (LayerNorm, tiled qkv, attention, tiled projection + residual, LayerNorm,
+    # tiled fc1 + GELU, tiled fc2 + residual) and the whole convolution stack (full-precision first convolution, two
+    # tiled stride-2 convolutions, global average pooling, full-precision classifier), each run as one chain
+    Nb, S, d, heads, mlp, bks = 128, 197, 768, 12, 3072, [8, 8, 8, 8]
+    xb_ = torch.randn(Nb * S, d, device=dev, generator=gen).to(torch.bfloat16)
+    shapes = [(3 * d, d), (d, d), (mlp, d), (d, mlp)]
+    btiles = [rand_tile(m_ * n_ // 8) for (m_, n_) in shapes]
+    balphas = [torch.rand(8, device=dev, generator=gen) * 0.03 for _ in shapes]
+    bws = torch.empty(B.tbn_vit_block_workspace_bytes(Nb, S, d, mlp, bks), dtype=torch.uint8, device=dev)
+    by = torch.empty_like(xb_)
+    us = graph_us(lambda: B.tbn_vit_block_fwd(xb_, Nb, S, heads, mlp, btiles, bks, balphas, [1, 1, 1, 1], workspace=bws, y=by),
+                  reps=3, iters=3)
+    out["vit_block_whole_T25216"] = dict(us=us, images_per_s=Nb / us * 1e6, launches=7,
+                                         includes="LN + qkv + attention + proj(+res) + LN + fc1(GELU) + fc2(+res)")
+    qkv_ = torch.randn(Nb * S, 3 * d, device=dev, generator=gen).to(torch.bfloat16)
+    us = graph_us(lambda: B.tbn_attention_fwd(qkv_, Nb, S, heads, 64), reps=3, iters=3)
+    out["vit_attention_only"] = dict(us=us, dense_tflops=4.0 * Nb * heads * S * S * 64 / us / 1e6, note="warp-level MMA, not a tiled layer")
+    us = graph_us(lambda: B.tbn_layernorm_fwd(xb_), reps=3, iters=3)
+    out["vit_layernorm_only"] = dict(us=us, alg_gbs=2.0 * xb_.numel() * 2 / us / 1e3)
+    del bws, qkv_, by, xb_
+    xc0 = torch.rand(256, 3, 32, 32, device=dev, generator=gen).to(torch.bfloat16)
+    W0 = torch.randn(64, 3, 3, 3, device=dev, generator=gen) * 0.27
+    ct1, ca1 = rand_tile(128 * 64 * 9 // 4), torch.rand(4, device=dev, generator=gen) * 0.05
+    ct2, ca2 = rand_tile(256 * 128 * 9 // 4), torch.rand(4, device=dev, generator=gen) * 0.03
+    Wfc = torch.randn(10 * 256, device=dev, generator=gen) * 0.06
+
+    def stack():
+        h = B.tbn_conv2d_dense_fwd(xc0, W0, 1, 1, act=B.ACT_RELU)
+        h = B.tbn_conv2d_fwd(h, 128, 3, 3, 2, 1, ct1, 4, ca1, B.ALPHA_PER_TILE, act=B.ACT_RELU)
+        h = B.tbn_conv2d_fwd(h, 256, 3, 3, 2, 1, ct2, 4, ca2, B.ALPHA_PER_TILE, act=B.ACT_RELU)
+        return B.tbn_linear_fp_tile_fwd(B.tbn_global_avgpool_fwd(h, y_dtype=B.F32), 10, Wfc, 1, y_dtype=B.F32)
+
+    us = graph_us(stack, reps=3, iters=3)
+    out["conv_stack_whole_batch256"] = dict(us=us, images_per_s=256 / us * 1e6, launches=5,
+                                            includes="dense conv 3->64 + tiled 64->128 s2 + tiled 128->256 s2 + avg pool + dense classifier")
+    us = graph_us(lambda: B.tbn_conv2d_dense_fwd(xc0, W0, 1, 1, act=B.ACT_RELU), reps=3, iters=3)
+    out["conv_first_dense_3_64"] = dict(us=us, alg_gbs=(xc0.numel() * 2 + 256 * 64 * 1024 * 2) / us / 1e3, bound="hbm",
+                                        frac_of_binding_roofline=(xc0.numel() * 2 + 256 * 64 * 1024 * 2) / hbm * 1e6 / us)
     # derived: images/s over the tiled layers only (LayerNorm, attention and residual adds of the block, and the
     # full-precision first convolution / classifier of the conv stack, are not tiled layers and are not run)
     vit_us = sum(out[n]["us"] for n in ("vit_qkv_768_2304", "vit_out_768_768", "vit_fc1_768_3072_gelu", "vit_fc2_3072_768"))

@@ -359,6 +359,15 @@ int tbn_last_device_status(void *stream, int *code, int *detail);
 /* Testing aid: enqueue a kernel that records (code, detail) exactly as a kernel whose wait gave up would --
  * it waits on nothing, so it cannot hang -- to exercise the status plumbing without starving a real pipeline. */
 int tbn_debug_record_status(int code, int detail, void *stream);
+/* Testing aids for the bounded waits themselves.  tbn_debug_set_wait_limit_us sets the limit of every device-side
+ * wait on the current device (microseconds; 0 restores the default of 2 s; the call synchronises the device first).
+ * tbn_debug_wait_timeout_probe enqueues a one-block kernel whose threads wait, through the same bounded-wait routines
+ * the tensor-core kernels use, on a barrier that nothing arrives at: the waits run out after the limit, the kernel
+ * records TBN_ERR_TIMEOUT with `detail`, takes the abort path (one warp times out, another leaves through the block's
+ * abort flag, then the quiet drain wait) and returns normally, so the context stays usable.  Set a short limit first:
+ * with the default the probe takes 2 s. */
+int tbn_debug_set_wait_limit_us(int limit_us);
+int tbn_debug_wait_timeout_probe(int detail, void *stream);
 /* Testing / tuning aids, process-wide, to be set while no forward call is in progress.  They replace nothing on
  * the normal path: without them the library chooses by shape.
  *   tbn_debug_force_linear_config: the tensor-core linear kernel runs tile shape `candidate` (an index into its

@@ -59,6 +59,8 @@ SIGNATURES = {
                             c_vp, c_sz, c_vp]),
     "tbn_last_device_status": (c_int, [c_vp, c_vp, c_vp]),
     "tbn_debug_record_status": (c_int, [c_int, c_int, c_vp]),
+    "tbn_debug_set_wait_limit_us": (c_int, [c_int]),
+    "tbn_debug_wait_timeout_probe": (c_int, [c_int, c_vp]),
     "tbn_debug_force_linear_config": (c_int, [c_int, c_int]),
     "tbn_debug_force_mlp_layerwise": (c_int, [c_int]),
     "tbn_debug_force_bin_config": (c_int, [c_int]),
@@ -240,13 +242,14 @@ def tbn_linear_fwd_host(x_host: torch.Tensor, y_host: torch.Tensor, tile, k, alp
 
 
 def tbn_conv2d_fwd(x: torch.Tensor, Cout: int, kh: int, kw: int, stride: int, pad: int, tile, k, alpha,
-                   alpha_mode, bias=None, act=ACT_NONE, y_dtype=None, path=PATH_AUTO) -> torch.Tensor:
+                   alpha_mode, bias=None, act=ACT_NONE, y_dtype=None, path=PATH_AUTO, y=None) -> torch.Tensor:
     Nb, Cin, H, Wd = x.shape
     xd = _dtype_code(x)
     yd = xd if y_dtype is None else y_dtype
     Ho = (H + 2 * pad - kh) // stride + 1
     Wo = (Wd + 2 * pad - kw) // stride + 1
-    y = torch.empty((Nb, Cout, max(Ho, 0), max(Wo, 0)), dtype=_torch_dtype(yd), device=x.device)
+    if y is None:
+        y = torch.empty((Nb, Cout, max(Ho, 0), max(Wo, 0)), dtype=_torch_dtype(yd), device=x.device)
     need = lib().tbn_conv2d_workspace_bytes(Nb, Cin, H, Wd, Cout, kh, kw, stride, pad, k, xd)
     ws = _ws(need, x.device)
     _check(lib().tbn_conv2d_fwd_path(_ptr(x), xd, Nb, Cin, H, Wd, Cout, kh, kw, stride, pad, _ptr(tile), k,
@@ -432,3 +435,11 @@ def tbn_global_avgpool_fwd(x: torch.Tensor, y_dtype=None) -> torch.Tensor:
     y = torch.empty((Nb, C), dtype=_torch_dtype(yd), device=x.device)
     _check(lib().tbn_global_avgpool_fwd(_ptr(x), xd, Nb, C, H, Wd, _ptr(y), yd, _stream()), "tbn_global_avgpool_fwd")
     return y
+
+
+def tbn_debug_set_wait_limit_us(limit_us: int):
+    _check(lib().tbn_debug_set_wait_limit_us(limit_us), "tbn_debug_set_wait_limit_us")
+
+
+def tbn_debug_wait_timeout_probe(detail: int):
+    _check(lib().tbn_debug_wait_timeout_probe(detail, _stream()), "tbn_debug_wait_timeout_probe")

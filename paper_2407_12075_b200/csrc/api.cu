@@ -9,7 +9,7 @@
 
 namespace tbn {
 
-// Device-side status record: {code, detail, reserved, reserved}.  Kernels receive its address.
+// Device-side status record: {code, detail, wait limit in microseconds (0 = default), reserved}.  Kernels receive its address.
 __device__ int g_device_status[4];
 
 __global__ void record_status_kernel(int *status, int code, int detail)
@@ -970,8 +970,24 @@ int tbn_last_device_status(void *stream, int *code, int *detail)
     if (cudaMemcpy(host, st, sizeof(host), cudaMemcpyDeviceToHost) != cudaSuccess) return TBN_ERR_CUDA;
     *code = host[0];
     *detail = host[1];
-    if (host[0] != 0 && cudaMemset(st, 0, sizeof(host)) != cudaSuccess) return TBN_ERR_CUDA;
+    if (host[0] != 0 && cudaMemset(st, 0, 2 * sizeof(int)) != cudaSuccess) return TBN_ERR_CUDA;   // code and detail only
     return TBN_OK;
+}
+
+int tbn_debug_set_wait_limit_us(int limit_us)
+{
+    if (limit_us < 0) return TBN_ERR_INVALID_ARG;
+    int *st = device_status_ptr();
+    if (!st) return TBN_ERR_CUDA;
+    if (cudaDeviceSynchronize() != cudaSuccess) return TBN_ERR_CUDA;      // no kernel may be reading the word meanwhile
+    return cudaMemcpy(st + 2, &limit_us, sizeof(int), cudaMemcpyHostToDevice) == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+}
+
+int tbn_debug_wait_timeout_probe(int detail, void *stream)
+{
+    int *st = device_status_ptr();
+    if (!st) return TBN_ERR_CUDA;
+    return launch_wait_probe(st, detail, static_cast<cudaStream_t>(stream)) == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
 }
 
 int tbn_debug_force_linear_config(int candidate, int splits) { return force_linear_config(candidate, splits); }

@@ -227,6 +227,7 @@ bool tensor_path_supported(const LayerArgs &a);
 size_t tensor_linear_scratch_bytes(const LayerArgs &a);   // split-K partial tiles + arrival counters
 int launch_tensor_linear(const LayerArgs &a, int *device_status, void *scratch, size_t scratch_bytes, cudaStream_t s);
 int force_linear_config(int candidate, int splits);          // testing / tuning aid: candidate < 0 clears
+cudaError_t launch_wait_probe(int *status, int detail, cudaStream_t s);   // testing aid: a bounded wait that runs out
 bool tensor_conv_supported(const LayerArgs &a);
 int launch_tensor_conv(const LayerArgs &a, int *device_status, cudaStream_t s);
 

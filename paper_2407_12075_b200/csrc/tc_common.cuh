@@ -173,11 +173,14 @@ static __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, vol
     for (int i = 0; i < 64; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
+    // the host may shorten the limit (status word 2, in microseconds; 0 = the default) to test this branch
+    const int limit_us = *reinterpret_cast<volatile int *>(status + 2);
+    const uint64_t limit_ns = limit_us > 0 ? (uint64_t)limit_us * 1000ull : kWaitLimitNs;
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 63u) == 0) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
+            if (global_timer_ns() - t0 > limit_ns) {
                 *abort_flag = 1;
                 if (atomicCAS(status, 0, (int)TBN_ERR_TIMEOUT) == 0) status[1] = detail;
                 __threadfence();

@@ -773,6 +773,37 @@ Plan plan_linear(const LayerArgs &a)
 
 }  // namespace
 
+// Exercises the bounded waits themselves: a block waits on an mbarrier that nothing ever arrives at.  Warp 0 (all
+// lanes) runs out of time, records the status and raises the block's abort flag; warp 1's single waiting lane leaves
+// through the abort flag; one thread then runs the quiet drain wait.  The kernel returns normally.
+__global__ void __launch_bounds__(64, 1)
+wait_probe_kernel(int *status, int detail)
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    bool ok = true;
+    if (warp == 0) ok = wait_bar(smem_u32(&bar), 0u, &abort_flag, status, detail);
+    else if (lane == 0) ok = wait_one(smem_u32(&bar), 0u, &abort_flag, status, detail + 1);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        drain_wait(smem_u32(&bar), 0u);
+        if (ok) status[1] = -1;          // the wait must not have succeeded: nothing arrives at this barrier
+    }
+}
+
+cudaError_t launch_wait_probe(int *status, int detail, cudaStream_t s)
+{
+    wait_probe_kernel<<<1, 64, 0, s>>>(status, detail);
+    return cudaGetLastError();
+}
+
 int force_linear_config(int candidate, int splits)
 {
     if (candidate < 0) { g_forced_cand.store(-1); g_forced_splits.store(1); return TBN_OK; }
