@@ -178,7 +178,8 @@ int tbn_linear_select_path(int64_t T, int32_t in_f, int32_t out_f, int32_t k, in
 
 /* Same layer with a residual input: y = act(...) + residual, where residual is a tensor shaped and typed like y (NULL:
  * exactly tbn_linear_fwd_path).  The residual connections of a Transformer block around the tiled projection and
- * feed-forward layers (Sec. 4.3) are the use; the paper itself writes no formula for it. */
+ * feed-forward layers (Sec. 4.3) are the use; the paper itself writes no formula for it.  residual must not be y.
+ * The CUDA-core kernels add it in their epilogue; after the tensor-core kernel it is added by a pass of its own. */
 int tbn_linear_res_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, int32_t out_f,
                        const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
                        const float *bias, int act, const void *residual, void *y, int y_dtype,

@@ -201,7 +201,10 @@ int run_layer(LayerArgs a, int path, void *workspace, size_t workspace_bytes, cu
         int *st = device_status_ptr();
         if (!st) return TBN_ERR_CUDA;
         if (rest_bytes == 0 || !aligned16(rest)) { rest = nullptr; rest_bytes = 0; }
-        return a.is_conv ? launch_tensor_conv(a, st, s) : launch_tensor_linear(a, st, rest, rest_bytes, s);
+        if (a.is_conv) return launch_tensor_conv(a, st, s);
+        const int rc = launch_tensor_linear(a, st, rest, rest_bytes, s);
+        if (rc != TBN_OK || a.residual == nullptr) return rc;
+        return launch_add_inplace(a.y, a.residual, a.T * (int64_t)a.m, a.y_dtype, s) == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
     }
     default:
         return TBN_ERR_INVALID_ARG;
@@ -487,7 +490,7 @@ int tbn_linear_res_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, int3
     int rc = fill_linear(a, x, x_dtype, T, in_f, out_f, tile_bits, k, alpha, alpha_mode, bias, act, y,
                          y_dtype, path);
     if (rc != TBN_OK) return rc;
-    if (residual && !aligned16(residual)) return TBN_ERR_INVALID_ARG;
+    if (residual && (!aligned16(residual) || residual == y)) return TBN_ERR_INVALID_ARG;   // the output may not alias it
     a.residual = residual;
     return run_layer(a, path, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
 }

@@ -131,7 +131,8 @@ struct LayerArgs {
     int fp_tile_dtype;     // TBN_F32 or TBN_BF16
     const float *alpha;
     const float *bias;
-    const void *residual;  // fully-connected only: a tensor shaped and typed like y, added after the activation (or null)
+    const void *residual;  // fully-connected only: a tensor shaped and typed like y, added after the activation (or null);
+                           // the CUDA-core kernels add it in their epilogue, the tensor-core path in a pass of its own
     int64_t T;       // rows of the contraction: tokens, or Nb*Ho*Wo output pixels
     int32_t n;       // contraction length: in_features or Cin*kh*kw
     int32_t m;       // output features / channels
@@ -209,6 +210,7 @@ struct FoldJobs {
 };
 cudaError_t launch_fold(const FoldJobs &jobs, cudaStream_t s);
 cudaError_t launch_f32_to_bf16(const float *src, __nv_bfloat16 *dst, int64_t count, cudaStream_t s);
+cudaError_t launch_add_inplace(void *y, const void *res, int64_t count, int dtype, cudaStream_t s);   // y += res
 
 cudaError_t launch_generic(const LayerArgs &a, cudaStream_t s);
 

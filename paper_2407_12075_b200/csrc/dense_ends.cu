@@ -60,6 +60,65 @@ dense_conv_kernel(const XT *__restrict__ x, const float *__restrict__ w, const f
     }
 }
 
+// The stack's own first layer, 3 input channels and a 3x3 filter (27 inputs per output): the 27 inputs of a pixel are
+// loaded once into registers (zero outside the image) and contracted with kFcCo output channels, whose weights are
+// laid out [input][channel] in shared memory so that four channels come with one broadcast 16-byte load.
+constexpr int kFcN = 27;
+constexpr int kFcCo = 32;
+
+template <typename XT, typename YT>
+__global__ void __launch_bounds__(256)
+first_conv3x3_kernel(const XT *__restrict__ x, const float *__restrict__ w, const float *__restrict__ bias, YT *__restrict__ y,
+                     int32_t Nb, int32_t H, int32_t Wd, int32_t Cout, int32_t stride, int32_t pad, int32_t Ho, int32_t Wo, int act)
+{
+    __shared__ __align__(16) float ws[kFcN * kFcCo];
+    __shared__ float bs[kFcCo];
+    const int32_t co0 = blockIdx.y * kFcCo;
+    for (int32_t i = threadIdx.x; i < kFcN * kFcCo; i += blockDim.x) {
+        const int32_t r = i / kFcCo, c = i - r * kFcCo;
+        ws[i] = co0 + c < Cout ? __ldg(w + (int64_t)(co0 + c) * kFcN + r) : 0.0f;
+    }
+    if (threadIdx.x < kFcCo) bs[threadIdx.x] = (bias && co0 + (int)threadIdx.x < Cout) ? __ldg(bias + co0 + threadIdx.x) : 0.0f;
+    __syncthreads();
+    const int64_t pixels = (int64_t)Nb * Ho * Wo;
+    for (int64_t pix = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; pix < pixels; pix += (int64_t)gridDim.x * blockDim.x) {
+        const int32_t ow = (int32_t)(pix % Wo);
+        const int64_t t = pix / Wo;
+        const int32_t oh = (int32_t)(t % Ho);
+        const int64_t b = t / Ho;
+        float xin[kFcN];
+#pragma unroll
+        for (int ci = 0; ci < 3; ++ci)
+#pragma unroll
+            for (int u = 0; u < 3; ++u)
+#pragma unroll
+                for (int v = 0; v < 3; ++v) {
+                    const int32_t ih = oh * stride + u - pad, iw = ow * stride + v - pad;
+                    const bool in = ih >= 0 && ih < H && iw >= 0 && iw < Wd;
+                    xin[(ci * 3 + u) * 3 + v] = in ? load_as_float(x, ((b * 3 + ci) * H + ih) * (int64_t)Wd + iw) : 0.0f;
+                }
+        float acc[kFcCo];
+#pragma unroll
+        for (int c = 0; c < kFcCo; ++c) acc[c] = bs[c];
+#pragma unroll
+        for (int r = 0; r < kFcN; ++r) {
+#pragma unroll
+            for (int c = 0; c < kFcCo; c += 4) {
+                const float4 w4 = *reinterpret_cast<const float4 *>(&ws[r * kFcCo + c]);
+                acc[c] = fmaf(w4.x, xin[r], acc[c]);
+                acc[c + 1] = fmaf(w4.y, xin[r], acc[c + 1]);
+                acc[c + 2] = fmaf(w4.z, xin[r], acc[c + 2]);
+                acc[c + 3] = fmaf(w4.w, xin[r], acc[c + 3]);
+            }
+        }
+#pragma unroll
+        for (int c = 0; c < kFcCo; ++c) {
+            if (co0 + c >= Cout) break;
+            store_from_float(y, ((b * Cout + co0 + c) * Ho + oh) * (int64_t)Wo + ow, apply_act(acc[c], act));
+        }
+    }
+}
+
 // Mean over the H*W positions of every (image, channel) plane: one warp per plane, fp32 accumulation.
 template <typename XT, typename YT>
 __global__ void __launch_bounds__(256)
@@ -87,6 +146,17 @@ cudaError_t launch_dense_conv(const void *x, int x_dtype, const float *w, const 
     const int32_t Ho = (H + 2 * pad - kh) / stride + 1, Wo = (Wd + 2 * pad - kw) / stride + 1;
     const int64_t pixels = (int64_t)Nb * Ho * Wo;
     const int64_t bx = (pixels + 255) / 256;
+    if (Cin == 3 && kh == 3 && kw == 3) {
+        const dim3 grid((unsigned)(bx < 148 * 64 ? (bx > 0 ? bx : 1) : 148 * 64), (unsigned)((Cout + kFcCo - 1) / kFcCo));
+#define TBN_FC(XT, YT) first_conv3x3_kernel<XT, YT><<<grid, 256, 0, s>>>(static_cast<const XT *>(x), w, bias, static_cast<YT *>(y), Nb, \
+                                                                         H, Wd, Cout, stride, pad, Ho, Wo, act)
+        if (x_dtype == TBN_BF16 && y_dtype == TBN_BF16) TBN_FC(__nv_bfloat16, __nv_bfloat16);
+        else if (x_dtype == TBN_BF16) TBN_FC(__nv_bfloat16, float);
+        else if (y_dtype == TBN_BF16) TBN_FC(float, __nv_bfloat16);
+        else TBN_FC(float, float);
+#undef TBN_FC
+        return cudaGetLastError();
+    }
     const dim3 grid((unsigned)(bx < 148 * 64 ? (bx > 0 ? bx : 1) : 148 * 64), (unsigned)((Cout + kDcCo - 1) / kDcCo));
 #define TBN_DC(XT, YT) dense_conv_kernel<XT, YT><<<grid, 256, 0, s>>>(static_cast<const XT *>(x), w, bias, static_cast<YT *>(y), Nb, \
                                                                        Cin, H, Wd, Cout, kh, kw, stride, pad, Ho, Wo, act)

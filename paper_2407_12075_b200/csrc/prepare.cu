@@ -379,6 +379,30 @@ fold_kernel(const FoldJobs jobs)
     }
 }
 
+// y += res element by element (same shape and type): the residual connection after a tensor-core layer.  Fusing the
+// residual loads into that kernel's epilogue measured slower than this pass: its four epilogue warps cannot keep
+// enough loads in flight next to the k-fold replicated stores.
+template <typename YT>
+__global__ void __launch_bounds__(256)
+add_inplace_kernel(YT *__restrict__ y, const YT *__restrict__ res, int64_t count)
+{
+    constexpr int V = 16 / sizeof(YT);
+    const int64_t vecs = count / V;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < vecs; i += stride) {
+        uint4 a = reinterpret_cast<const uint4 *>(y)[i];
+        const uint4 b = __ldg(reinterpret_cast<const uint4 *>(res) + i);
+        YT *pa = reinterpret_cast<YT *>(&a);
+        const YT *pb = reinterpret_cast<const YT *>(&b);
+#pragma unroll
+        for (int e = 0; e < V; ++e) store_from_float(pa, e, load_as_float(pa, e) + load_as_float(pb, e));
+        reinterpret_cast<uint4 *>(y)[i] = a;
+    }
+    if (blockIdx.x == 0)
+        for (int64_t i = vecs * V + threadIdx.x; i < count; i += blockDim.x)
+            store_from_float(y, i, load_as_float(y, i) + load_as_float(res, i));
+}
+
 int grid_for(int64_t work_items, int threads, int cap_blocks)
 {
     int64_t b = (work_items + threads - 1) / threads;
@@ -475,6 +499,17 @@ cudaError_t launch_fold(const FoldJobs &jobs, cudaStream_t s)
         most = t > most ? t : most;
     }
     fold_kernel<<<dim3((unsigned)grid_for(most, 256, 148 * 8), (unsigned)jobs.count), 256, 0, s>>>(jobs);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_add_inplace(void *y, const void *res, int64_t count, int dtype, cudaStream_t s)
+{
+    const int v = dtype == TBN_BF16 ? 8 : 4;
+    const int grid = grid_for(count / v + 1, 256, 148 * 16);
+    if (dtype == TBN_BF16)
+        add_inplace_kernel<<<grid, 256, 0, s>>>(static_cast<__nv_bfloat16 *>(y), static_cast<const __nv_bfloat16 *>(res), count);
+    else
+        add_inplace_kernel<<<grid, 256, 0, s>>>(static_cast<float *>(y), static_cast<const float *>(res), count);
     return cudaGetLastError();
 }
 

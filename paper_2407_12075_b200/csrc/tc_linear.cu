@@ -83,7 +83,6 @@ struct TcParams {
     const __nv_bfloat16 *dense_a;   // non-null: full-precision weight rows [r][n] instead of tile bits
     const float *alpha;
     const float *bias;
-    const void *residual;    // shaped and typed like y, added after the activation (or null)
     void *y;
     int *status;
     int64_t T;
@@ -393,7 +392,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
         const bool bias_vec = (reinterpret_cast<uintptr_t>(p.bias) & 15) == 0;
         const int f0 = 8 * (lane & 15);                   // first of this lane's 8 rows inside the 128-row block
         const int tsub = lane >> 4;                       // this lane's tokens: 8*ew + tsub + 2*i, i = 2*iset, 2*iset+1
-        const bool plain = p.bias == nullptr && p.residual == nullptr && (p.act == TBN_ACT_NONE || p.act == TBN_ACT_RELU);
+        const bool plain = p.bias == nullptr && (p.act == TBN_ACT_NONE || p.act == TBN_ACT_RELU);
         for (int32_t tile = bid; tile < n_tiles; tile += gridDim.x) {
             const int32_t split = tile % p.splits, out_tile = tile / p.splits;
             const int64_t tok0 = (int64_t)(out_tile / p.w_tiles) * NTOK;
@@ -584,22 +583,6 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                                 const int64_t tok = tok_first + 2 * i;
                                 if (tok >= p.T) continue;
                                 const int64_t yi = tok * p.m + o0;
-                                if (p.residual != nullptr) {          // o0 is a multiple of 8 here: 16-byte aligned
-                                    if (p.y_bf16) {
-                                        const uint4 rv = __ldg(reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(p.residual) + yi));
-                                        const uint32_t rw[4] = {rv.x, rv.y, rv.z, rv.w};
-#pragma unroll
-                                        for (int e = 0; e < 4; ++e) {
-                                            o[i][2 * e] += __uint_as_float(rw[e] << 16);
-                                            o[i][2 * e + 1] += __uint_as_float(rw[e] & 0xffff0000u);
-                                        }
-                                    } else {
-                                        const float4 *rp = reinterpret_cast<const float4 *>(static_cast<const float *>(p.residual) + yi);
-                                        const float4 r0 = __ldg(rp), r1 = __ldg(rp + 1);
-                                        o[i][0] += r0.x; o[i][1] += r0.y; o[i][2] += r0.z; o[i][3] += r0.w;
-                                        o[i][4] += r1.x; o[i][5] += r1.y; o[i][6] += r1.z; o[i][7] += r1.w;
-                                    }
-                                }
                                 if (p.y_bf16) {
                                     uint32_t pk[4];
 #pragma unroll
@@ -625,11 +608,8 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                                 for (int e = 0; e < 8; ++e) {
                                     if (e >= nvalid) break;
                                     const float bb = p.bias ? __ldg(p.bias + o0 + e) : 0.0f;
-                                    float val = apply_act(fmaf(al, z[i][e], bb), p.act);
+                                    const float val = apply_act(fmaf(al, z[i][e], bb), p.act);
                                     const int64_t yi = tok * p.m + o0 + e;
-                                    if (p.residual != nullptr)
-                                        val += p.y_bf16 ? load_as_float(static_cast<const __nv_bfloat16 *>(p.residual), yi)
-                                                        : load_as_float(static_cast<const float *>(p.residual), yi);
                                     if (p.y_bf16) static_cast<__nv_bfloat16 *>(p.y)[yi] = __float2bfloat16_rn(val);
                                     else static_cast<float *>(p.y)[yi] = val;
                                 }
@@ -833,7 +813,7 @@ int launch_tensor_linear(const LayerArgs &a, int *device_status, void *scratch, 
 {
     if (a.x_dtype != TBN_BF16) return TBN_ERR_UNSUPPORTED;
     TcParams p;
-    p.tile = a.tile; p.dense_a = static_cast<const __nv_bfloat16 *>(a.dense_a); p.alpha = a.alpha; p.bias = a.bias; p.residual = a.residual; p.y = a.y; p.status = device_status;
+    p.tile = a.tile; p.dense_a = static_cast<const __nv_bfloat16 *>(a.dense_a); p.alpha = a.alpha; p.bias = a.bias; p.y = a.y; p.status = device_status;
     p.T = a.T; p.n_words = a.dense_a ? 1 : tbn_tile_words(a.q);
     p.n = a.n; p.m = a.m; p.r = (int32_t)(a.q / a.n); p.k = a.k;
     p.k_stages = 0;
