@@ -50,10 +50,10 @@ def algorithmic_bytes(T: int, k: int) -> float:
 
 
 # DRAM traffic of the dominant launch (k = 2) from an ncu capture of that kernel at T = 8192 (dram bytes read +
-# written: 234.0 MB); traffic is proportional to T.  The figure is only valid for the kernel source it was taken
+# written: 235.1 MB); traffic is proportional to T.  The figure is only valid for the kernel source it was taken
 # from: the hash below covers the code (comments stripped) of tc_linear.cu and tc_common.cuh.
-TRAFFIC_BYTES_AT_T8192 = 138.568448e6 + 95.472128e6
-TRAFFIC_SOURCE_HASH = "36fee45cc6883fa2"
+TRAFFIC_BYTES_AT_T8192 = 138.643200e6 + 96.431872e6
+TRAFFIC_SOURCE_HASH = "97eb7ca1eacc71f3"
 
 
 def kernel_source_hash() -> str:
