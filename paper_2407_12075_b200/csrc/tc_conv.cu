@@ -243,8 +243,11 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
             }
         }
     } else if (warp == kMmaWarp) {
-        // ---------------- MMA issuer (lane 0): 9 shifted-window MMAs per 16-channel stage ----------------
-        if (lane == 0) {
+        // ---------------- MMA issuer: 9 shifted-window MMAs per 16-channel stage ----------------
+        {
+            // all 32 lanes run the loop in lockstep, one elected lane performs each MMA and commit (see tc_mma_ts_elect)
+            const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0);
+            const uint32_t leader = elect_one();
             Pipe px, pa, pd;
             bool ready = false;
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_pos >> 3) << 17) | (8u << 24);
@@ -256,36 +259,36 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
 #pragma unroll
             for (int t = 0; t < kTaps; ++t) tap_disp[t] = (uint32_t)(p.tap_plane[t] * 2 * p.buf_pos + p.tap_off[t]);
             for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
-                ok = wait_one(smem_u32(&ctl->d_empty[pd.stage]), pd.phase ^ 1u, abort_flag, p.status,
+                ok = wait_bar(smem_u32(&ctl->d_empty[pd.stage]), pd.phase ^ 1u, abort_flag, p.status,
                               (2 << 24) | (bid & 0xffff));
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t d_addr = tmem_base + pd.stage * kNMax;
+                const uint32_t d_addr = tmem_u + pd.stage * kNMax;
                 for (int32_t ks = 0; ks < p.k_stages; ++ks) {
                     if (!ready) {
-                        ok = wait_one(smem_u32(&ctl->x_full[px.stage]), px.phase, abort_flag, p.status,
+                        ok = wait_bar(smem_u32(&ctl->x_full[px.stage]), px.phase, abort_flag, p.status,
                                       (3 << 24) | (px.stage << 16) | (bid & 0xffff)) &&
-                             wait_one(smem_u32(&ctl->a_full[pa.stage]), pa.phase, abort_flag, p.status,
+                             wait_bar(smem_u32(&ctl->a_full[pa.stage]), pa.phase, abort_flag, p.status,
                                       (4 << 24) | (pa.stage << 16) | (bid & 0xffff));
                         if (!ok) break;
                     }
                     tc_fence_after();
                     const uint32_t b_base = ((stage0 + px.stage * stage_bytes) & 0x3FFFFu) >> 4;   // 16-byte units
-                    const uint32_t a_addr = tmem_base + kABase + pa.stage * kACols;
+                    const uint32_t a_addr = tmem_u + kABase + pa.stage * kACols;
                     Pipe nx = px, na = pa;
                     nx.advance(kSX);
                     na.advance(2);
 #pragma unroll
                     for (int t = 0; t < kTaps; ++t) {
                         const uint32_t b_lo = (b_base + tap_disp[t]) | lbo;
-                        tc_mma_ts(d_addr, a_addr + t * 8, b_lo, desc_hi, idesc, t > 0 ? 1u : (uint32_t)(ks > 0));
+                        tc_mma_ts_elect(d_addr, a_addr + t * 8, b_lo, desc_hi, idesc, t > 0 ? 1u : (uint32_t)(ks > 0), leader);
                         if (t == 4)
-                            ready = mbar_test_wait(smem_u32(&ctl->x_full[nx.stage]), nx.phase) &&
-                                    mbar_test_wait(smem_u32(&ctl->a_full[na.stage]), na.phase);
+                            ready = __all_sync(0xffffffffu, mbar_test_wait(smem_u32(&ctl->x_full[nx.stage]), nx.phase) &&
+                                                                mbar_test_wait(smem_u32(&ctl->a_full[na.stage]), na.phase)) != 0;
                     }
-                    tc_commit(smem_u32(&ctl->x_empty[px.stage]));
-                    tc_commit(smem_u32(&ctl->a_empty[pa.stage]));
-                    if (ks == p.k_stages - 1) tc_commit(smem_u32(&ctl->d_full[pd.stage]));
+                    tc_commit_elect(smem_u32(&ctl->x_empty[px.stage]), leader);
+                    tc_commit_elect(smem_u32(&ctl->a_empty[pa.stage]), leader);
+                    if (ks == p.k_stages - 1) tc_commit_elect(smem_u32(&ctl->d_full[pd.stage]), leader);
                     px = nx;
                     pa = na;
                 }
@@ -596,7 +599,7 @@ tc_conv3x3_kernel(const __grid_constant__ CUtensorMap x_map, const ConvParams p)
 
     // ---------------- teardown ----------------
     if (warp == kMmaWarp && *abort_flag) {
-        if (lane == 0) tc_commit(smem_u32(&ctl->x_empty[0]));
+        tc_commit_elect(smem_u32(&ctl->x_empty[0]), elect_one());     // by the lane that issued the MMAs
         __syncwarp();
         drain_wait(smem_u32(&ctl->x_empty[0]), 0);
         drain_wait(smem_u32(&ctl->x_empty[0]), 1);

@@ -194,39 +194,41 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                 if (issued_mask & (1u << s)) drain_wait(smem_u32(&ctl->x_full[s]), (issued_phase >> s) & 1u);
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer (lane 0) ----------------
+        // ---------------- MMA issuer ----------------
         // tcgen05.mma is issued by one thread, and that thread's instructions execute back to back with no
         // other warp to hide their latency: every instruction between two MMAs is dead time for the tensor
         // cores once their small queue has drained.  So the K steps of a full stage are unrolled with all
-        // offsets immediate (two adds per MMA), the NEXT stage's barriers are polled in the middle of the
-        // current stage (if they are already complete, the common case, the next stage starts at once),
-        // and the other 31 lanes stay out of the loop.
-        if (lane == 0) {
+        // offsets immediate (two adds per MMA) and the NEXT stage's barriers are polled in the middle of the
+        // current stage (if they are already complete, the common case, the next stage starts at once).
+        {
+            // all 32 lanes run the loop in lockstep; one elected lane performs each MMA and commit (see tc_mma_ts_elect)
+            const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0);
+            const uint32_t leader = elect_one();
             Pipe px, pa, pd;
             bool ready = false;
             constexpr uint32_t kDescHi = (uint32_t)(kBDescHi >> 32);
             constexpr int kSteps = KA * 4;             // 16-element K steps per full stage
             for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
-                ok = wait_one(smem_u32(&ctl->d_empty[pd.stage]), pd.phase ^ 1u, abort_flag, p.status,
+                ok = wait_bar(smem_u32(&ctl->d_empty[pd.stage]), pd.phase ^ 1u, abort_flag, p.status,
                               (2 << 24) | (bid & 0xffff));
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t d_addr = tmem_base + pd.stage * kDCols;
+                const uint32_t d_addr = tmem_u + pd.stage * kDCols;
                 const int32_t split = tile % p.splits;
                 const int32_t ks0 = (int32_t)((int64_t)split * p.k_stages / p.splits);
                 const int32_t ks1 = (int32_t)((int64_t)(split + 1) * p.k_stages / p.splits);
                 for (int32_t ks = ks0; ks < ks1; ++ks) {
                     if (!ready) {
-                        ok = wait_one(smem_u32(&ctl->x_full[px.stage]), px.phase, abort_flag, p.status,
+                        ok = wait_bar(smem_u32(&ctl->x_full[px.stage]), px.phase, abort_flag, p.status,
                                       (3 << 24) | (px.stage << 16) | (bid & 0xffff)) &&
-                             wait_one(smem_u32(&ctl->a_full[pa.stage]), pa.phase, abort_flag, p.status,
+                             wait_bar(smem_u32(&ctl->a_full[pa.stage]), pa.phase, abort_flag, p.status,
                                       (4 << 24) | (pa.stage << 16) | (bid & 0xffff));
                         if (!ok) break;
                     }
                     tc_fence_after();
                     // descriptor low word: start address in 16-byte units | leading offset 1 << 16
                     const uint32_t b_lo = (((stage0 + px.stage * kStageBytes) & 0x3FFFFu) >> 4) | (1u << 16);
-                    const uint32_t a_addr = tmem_base + kABase + pa.stage * kACols;
+                    const uint32_t a_addr = tmem_u + kABase + pa.stage * kACols;
                     Pipe nx = px, na = pa;
                     nx.advance(SX);
                     na.advance(kAStages);
@@ -237,12 +239,12 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                             const int at = st >> 2, kk = st & 3;
 #pragma unroll
                             for (int a = 0; a < NA; ++a)
-                                tc_mma_ts(d_addr + a * NTOK, a_addr + (a * KA + at) * 32 + kk * 8,
+                                tc_mma_ts_elect(d_addr + a * NTOK, a_addr + (a * KA + at) * 32 + kk * 8,
                                           b_lo + at * (kAtomBytes >> 4) + kk * 2, kDescHi, kIdesc,
-                                          st > 0 ? 1u : (uint32_t)(ks > ks0));
+                                          st > 0 ? 1u : (uint32_t)(ks > ks0), leader);
                             if (st == kSteps / 2 - 1)
-                                ready = mbar_test_wait(smem_u32(&ctl->x_full[nx.stage]), nx.phase) &&
-                                        mbar_test_wait(smem_u32(&ctl->a_full[na.stage]), na.phase);
+                                ready = __all_sync(0xffffffffu, mbar_test_wait(smem_u32(&ctl->x_full[nx.stage]), nx.phase) &&
+                                                                    mbar_test_wait(smem_u32(&ctl->a_full[na.stage]), na.phase)) != 0;
                         }
                     } else {                              // ragged last stage: only the K steps that hold data
                         const int steps = (rem + 15) >> 4;
@@ -250,15 +252,15 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
                             const int at = st >> 2, kk = st & 3;
 #pragma unroll
                             for (int a = 0; a < NA; ++a)
-                                tc_mma_ts(d_addr + a * NTOK, a_addr + (a * KA + at) * 32 + kk * 8,
+                                tc_mma_ts_elect(d_addr + a * NTOK, a_addr + (a * KA + at) * 32 + kk * 8,
                                           b_lo + at * (kAtomBytes >> 4) + kk * 2, kDescHi, kIdesc,
-                                          (ks > ks0 || st > 0) ? 1u : 0u);
+                                          (ks > ks0 || st > 0) ? 1u : 0u, leader);
                         }
                         ready = false;
                     }
-                    tc_commit(smem_u32(&ctl->x_empty[px.stage]));
-                    tc_commit(smem_u32(&ctl->a_empty[pa.stage]));
-                    if (ks == ks1 - 1) tc_commit(smem_u32(&ctl->d_full[pd.stage]));
+                    tc_commit_elect(smem_u32(&ctl->x_empty[px.stage]), leader);
+                    tc_commit_elect(smem_u32(&ctl->a_empty[pa.stage]), leader);
+                    if (ks == ks1 - 1) tc_commit_elect(smem_u32(&ctl->d_full[pd.stage]), leader);
                     px = nx;
                     pa = na;
                 }
@@ -625,7 +627,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p)
     // ---------------- teardown ----------------
     if (warp == 1 && *abort_flag) {
         // make sure no MMA is still reading shared or tensor memory before they are released
-        if (lane == 0) tc_commit(smem_u32(&ctl->x_empty[0]));
+        tc_commit_elect(smem_u32(&ctl->x_empty[0]), elect_one());     // by the lane that issued the MMAs
         __syncwarp();
         drain_wait(smem_u32(&ctl->x_empty[0]), 0);
         drain_wait(smem_u32(&ctl->x_empty[0]), 1);

@@ -95,14 +95,16 @@ __device__ __forceinline__ int epi_bar128_count(bool pred) {
 }
 
 // D[tmem] (+)= A[tmem] * B[smem]^T, signed 8-bit x signed 8-bit -> int32, M = 128, K = 32
+// (executed by the whole converged warp, performed by the elected lane: see tc_mma_ts_elect)
 __device__ __forceinline__ void tc_mma_ts_i8(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_desc_lo, uint32_t b_desc_hi,
-                                             uint32_t idesc, uint32_t accumulate) {
+                                             uint32_t idesc, uint32_t accumulate, uint32_t leader) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 bd;\n\t"
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 bd;\n\t"
+        "setp.ne.b32 q, %6, 0;\n\t"
         "setp.ne.b32 p, %5, 0;\n\t"
         "mov.b64 bd, {%2, %3};\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], bd, %4, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "r"(b_desc_lo), "r"(b_desc_hi), "r"(idesc), "r"(accumulate) : "memory");
+        "@q tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], bd, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_desc_lo), "r"(b_desc_hi), "r"(idesc), "r"(accumulate), "r"(leader) : "memory");
 }
 
 constexpr uint64_t kBinBDescHi = (64ull << 32) | (1ull << 46) | (2ull << 61);   // as the bf16 kernel: SW128, K-major
@@ -238,29 +240,31 @@ tc_linear_bin_kernel(const BinParams p)
             }
         }
     } else if (warp == kBinMmaWarp) {
-        // ---------------- MMA issuer (lane 0): 8 MMAs of K = 32 per stage ----------------
-        if (lane == 0) {
+        // ---------------- MMA issuer: 8 MMAs of K = 32 per stage ----------------
+        {
+            const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0);
+            const uint32_t leader = elect_one();
             Pipe px, pa, pd;
             bool ready = false;
             constexpr uint32_t kDescHi = (uint32_t)(kBinBDescHi >> 32);
             constexpr int kSteps = kBinKA * 4;
             for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
-                ok = wait_one(smem_u32(&ctl->d_empty[pd.stage]), pd.phase ^ 1u, abort_flag, p.status,
+                ok = wait_bar(smem_u32(&ctl->d_empty[pd.stage]), pd.phase ^ 1u, abort_flag, p.status,
                               (2 << 24) | (bid & 0xffff));
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t d_addr = tmem_base + pd.stage * kDCols;
+                const uint32_t d_addr = tmem_u + pd.stage * kDCols;
                 for (int32_t ks = 0; ks < p.k_stages; ++ks) {
                     if (!ready) {
-                        ok = wait_one(smem_u32(&ctl->x_full[px.stage]), px.phase, abort_flag, p.status,
+                        ok = wait_bar(smem_u32(&ctl->x_full[px.stage]), px.phase, abort_flag, p.status,
                                       (3 << 24) | (px.stage << 16) | (bid & 0xffff)) &&
-                             wait_one(smem_u32(&ctl->a_full[pa.stage]), pa.phase, abort_flag, p.status,
+                             wait_bar(smem_u32(&ctl->a_full[pa.stage]), pa.phase, abort_flag, p.status,
                                       (4 << 24) | (pa.stage << 16) | (bid & 0xffff));
                         if (!ok) break;
                     }
                     tc_fence_after();
                     const uint32_t b_lo = (((stage0 + px.stage * kStageBytes) & 0x3FFFFu) >> 4) | (1u << 16);
-                    const uint32_t a_addr = tmem_base + kABase + pa.stage * kBinACols;
+                    const uint32_t a_addr = tmem_u + kABase + pa.stage * kBinACols;
                     Pipe nx = px, na = pa;
                     nx.advance(SX);
                     na.advance(kBinAStages);
@@ -269,14 +273,14 @@ tc_linear_bin_kernel(const BinParams p)
                     for (int st = 0; st < kSteps; ++st) {
                         const int at = st >> 2, kk = st & 3;
                         tc_mma_ts_i8(d_addr, a_addr + at * 32 + kk * 8, b_lo + at * (kAtomBytes >> 4) + kk * 2, kDescHi,
-                                     kIdesc, st > 0 ? 1u : (uint32_t)(ks > 0));
+                                     kIdesc, st > 0 ? 1u : (uint32_t)(ks > 0), leader);
                         if (st == kSteps / 2 - 1)
-                            ready = mbar_test_wait(smem_u32(&ctl->x_full[nx.stage]), nx.phase) &&
-                                    mbar_test_wait(smem_u32(&ctl->a_full[na.stage]), na.phase);
+                            ready = __all_sync(0xffffffffu, mbar_test_wait(smem_u32(&ctl->x_full[nx.stage]), nx.phase) &&
+                                                                mbar_test_wait(smem_u32(&ctl->a_full[na.stage]), na.phase)) != 0;
                     }
-                    tc_commit(smem_u32(&ctl->x_empty[px.stage]));
-                    tc_commit(smem_u32(&ctl->a_empty[pa.stage]));
-                    if (ks == p.k_stages - 1) tc_commit(smem_u32(&ctl->d_full[pd.stage]));
+                    tc_commit_elect(smem_u32(&ctl->x_empty[px.stage]), leader);
+                    tc_commit_elect(smem_u32(&ctl->a_empty[pa.stage]), leader);
+                    if (ks == p.k_stages - 1) tc_commit_elect(smem_u32(&ctl->d_full[pd.stage]), leader);
                     px = nx;
                     pa = na;
                 }
@@ -490,7 +494,7 @@ tc_linear_bin_kernel(const BinParams p)
     // ---------------- teardown ----------------
     if (warp == kBinMmaWarp && *abort_flag) {
         // make sure no MMA is still reading shared or tensor memory before they are released
-        if (lane == 0) tc_commit(smem_u32(&ctl->x_empty[0]));
+        tc_commit_elect(smem_u32(&ctl->x_empty[0]), elect_one());     // by the lane that issued the MMAs
         __syncwarp();
         drain_wait(smem_u32(&ctl->x_empty[0]), 0);
         drain_wait(smem_u32(&ctl->x_empty[0]), 1);
