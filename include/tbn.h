@@ -185,6 +185,24 @@ int tbn_linear_res_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, int3
                        const float *bias, int act, const void *residual, void *y, int y_dtype,
                        void *workspace, size_t workspace_bytes, void *stream, int path);
 
+/* Compact chaining of two tiled layers through any activation (Sec. 4.1: with a tile that spans whole rows the k
+ * repetitions of an output channel are the same pre-activation z scaled by different alphas).  The first layer writes
+ * only its r_z distinct pre-activations -- call tbn_linear_fwd with out_f = r_z, k = 1 and an alpha of 1.0 on the same
+ * tile (a tile of r_z rows IS a k = 1 layer of r_z outputs) -- and this call consumes them:
+ *
+ *     x[t][j*r_z + c] = act_z(alpha_z[j] * z[t][c])        j < k_z, c < r_z     (never written to memory)
+ *     y[t][o]         = act( sum_i B_hat[o][i] * x[t][i] + bias[o] )             B_hat: out_f x (r_z * k_z), tiled
+ *
+ * The activation of the first layer is evaluated while the activation operand is staged on chip, so the k_z-fold
+ * larger tensor x is neither written by the first layer nor read by the second.  (With ReLU or no activation
+ * tbn_mlp_fwd gets the same saving by folding alpha_z into the weights; this call is what covers GELU.)
+ * z: T x r_z bf16.  alpha_z: 1 or k_z floats (alpha_mode_z), k_z <= 64.  Needs r_z % 64 == 0 and a tile that spans
+ * whole rows (q % (r_z*k_z) == 0); TBN_ERR_UNSUPPORTED otherwise.  Tensor-core kernel; no workspace.  Other arguments as
+ * tbn_linear_fwd. */
+int tbn_linear_compact_fwd(const void *z, int64_t T, int32_t rz, int32_t kz, const float *alpha_z, int alpha_mode_z, int act_z,
+                           int32_t out_f, const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                           const float *bias, int act, void *y, int y_dtype, void *stream);
+
 /*
  * Full-precision tiled weights (Sec. 5.2: the "FP, Tiled" kernel measured in Table 7 and Fig. 6; named as future
  * work for large models in Sec. 7).  The layer stores a tile of q = in_f*out_f/k REAL values; the weight matrix is

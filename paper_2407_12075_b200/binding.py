@@ -40,6 +40,8 @@ SIGNATURES = {
     "tbn_linear_select_path": (c_int, [c_i64, c_i32, c_i32, c_i32, c_int]),
     "tbn_linear_res_fwd": (c_int, [c_vp, c_int, c_i64, c_i32, c_i32, c_vp, c_i32, c_vp, c_int, c_vp, c_int, c_vp, c_vp, c_int,
                                    c_vp, c_sz, c_vp, c_int]),
+    "tbn_linear_compact_fwd": (c_int, [c_vp, c_i64, c_i32, c_i32, c_vp, c_int, c_int, c_i32, c_vp, c_i32, c_vp, c_int, c_vp, c_int,
+                                       c_vp, c_int, c_vp]),
     "tbn_layernorm_fwd": (c_int, [c_vp, c_int, c_i64, c_i32, c_vp, c_vp, ctypes.c_float, c_vp, c_int, c_vp]),
     "tbn_attention_fwd": (c_int, [c_vp, c_i32, c_i32, c_i32, c_i32, c_vp, c_vp]),
     "tbn_vit_block_workspace_bytes": (c_sz, [c_i32, c_i32, c_i32, c_i32, c_vp]),
@@ -443,3 +445,17 @@ def tbn_debug_set_wait_limit_us(limit_us: int):
 
 def tbn_debug_wait_timeout_probe(detail: int):
     _check(lib().tbn_debug_wait_timeout_probe(detail, _stream()), "tbn_debug_wait_timeout_probe")
+
+
+def tbn_linear_compact_fwd(z: torch.Tensor, kz: int, alpha_z: torch.Tensor, alpha_mode_z: int, act_z: int, out_f: int,
+                           tile: torch.Tensor, k: int, alpha: torch.Tensor, alpha_mode: int, bias=None, act=ACT_NONE,
+                           y_dtype: int = BF16, y: torch.Tensor | None = None) -> torch.Tensor:
+    """Second of two tiled layers chained in compact form: z holds the first layer's distinct pre-activations
+    (T x r_z, bf16); its k_z-fold output act_z(alpha_z[j] * z) is rebuilt on chip."""
+    T, rz = z.shape
+    if y is None:
+        y = torch.empty((T, out_f), dtype=_torch_dtype(y_dtype), device=z.device)
+    _check(lib().tbn_linear_compact_fwd(_ptr(z), T, rz, kz, _ptr(alpha_z), alpha_mode_z, act_z, out_f, _ptr(tile), k,
+                                        _ptr(alpha), alpha_mode, _ptr(bias), act, _ptr(y), y_dtype, _stream()),
+           "tbn_linear_compact_fwd")
+    return y

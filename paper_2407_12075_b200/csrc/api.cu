@@ -806,6 +806,32 @@ int tbn_tile_bwd(const float *G, const uint32_t *tile_bits, const float *alpha, 
                            static_cast<cudaStream_t>(stream)) == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
 }
 
+int tbn_linear_compact_fwd(const void *z, int64_t T, int32_t rz, int32_t kz, const float *alpha_z, int alpha_mode_z, int act_z,
+                           int32_t out_f, const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                           const float *bias, int act, void *y, int y_dtype, void *stream)
+{
+    if (T < 0 || rz <= 0 || kz <= 0 || out_f <= 0 || k <= 0) return TBN_ERR_INVALID_ARG;
+    if (!alpha_z || !tile_bits || !alpha || !valid_alpha_mode(alpha_mode_z) || !valid_alpha_mode(alpha_mode) || !valid_act(act_z) ||
+        !valid_act(act) || !valid_dtype(y_dtype))
+        return TBN_ERR_INVALID_ARG;
+    if (T > 0 && (!z || !y)) return TBN_ERR_INVALID_ARG;
+    if (!aligned16(z) || !aligned16(y) || !aligned16(tile_bits)) return TBN_ERR_INVALID_ARG;
+    if (bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) return TBN_ERR_INVALID_ARG;
+    const int64_t n = (int64_t)rz * kz;
+    const int64_t N = n * out_f;
+    if (N % k != 0) return TBN_ERR_SHAPE;
+    if (T == 0) return TBN_OK;
+    CompactArgs a;
+    std::memset(&a, 0, sizeof(a));
+    a.z = z; a.alpha_z = alpha_z; a.tile = tile_bits; a.alpha = alpha; a.bias = bias; a.y = y;
+    a.T = T; a.q = N / k; a.rz = rz; a.kz = kz; a.m = out_f; a.k = k;
+    a.alpha_mode_z = alpha_mode_z; a.act_z = act_z; a.alpha_mode = alpha_mode; a.act = act; a.y_dtype = y_dtype;
+    if (!compact_linear_supported(a)) return TBN_ERR_UNSUPPORTED;
+    int *st = device_status_ptr();
+    if (!st) return TBN_ERR_CUDA;
+    return launch_compact_linear(a, st, static_cast<cudaStream_t>(stream));
+}
+
 int tbn_layernorm_fwd(const void *x, int x_dtype, int64_t T, int32_t d, const float *gamma, const float *beta, float eps,
                       void *y, int y_dtype, void *stream)
 {

@@ -186,6 +186,23 @@ cudaError_t launch_dense_conv(const void *x, int x_dtype, const float *w, const 
                               int act, cudaStream_t s);
 cudaError_t launch_global_avgpool(const void *x, int x_dtype, int64_t planes, int32_t hw, void *y, int y_dtype, cudaStream_t s);
 
+// ---- layer fed with the compact form of the previous tiled layer's output (tc_linear_compact.cu) ---------
+struct CompactArgs {
+    const void *z;            // [T][rz] bf16: distinct pre-activations of the previous layer
+    const float *alpha_z;     // its alphas (1 or kz)
+    const uint32_t *tile;
+    const float *alpha;
+    const float *bias;
+    void *y;
+    int64_t T;
+    int64_t q;                // this layer's tile length in bits
+    int32_t rz, kz;           // this layer's input width is rz * kz
+    int32_t m, k;
+    int alpha_mode_z, act_z, alpha_mode, act, y_dtype;
+};
+bool compact_linear_supported(const CompactArgs &a);
+int launch_compact_linear(const CompactArgs &a, int *device_status, cudaStream_t s);
+
 // ---- launchers implemented in the other translation units ---------------------------------------
 cudaError_t launch_aggregate(const float *W, const float *A, int64_t N, int32_t k, int per_tile,
                              uint32_t *tile_bits, float *alpha, void *workspace, cudaStream_t s);

@@ -4,7 +4,8 @@ of launches):
     python -m paper_2407_12075_b200.profile_cases <case> [--reps N]
 
 Cases: linear_k2, linear_k16 (8192 x 8192, T = 8192), bin_k2, bin_k16 (binary activations, 8192 x 8192, T = 4096),
-conv_s2 (64 -> 128, 32 x 32, batch 64), attention (64 images x 12 heads x 197 tokens), binarize, tile_bwd.
+conv_s2 (64 -> 128, 32 x 32, batch 64), attention (64 images x 12 heads x 197 tokens), binarize, tile_bwd,
+compact_gelu (second MLP layer of a ViT-B block fed the first layer's 384 distinct pre-activations, T = 25,216).
 Inputs are seeded device-side random values of the benchmark's shapes; every run checks the device status word.
 """
 from __future__ import annotations
@@ -55,6 +56,13 @@ def main():
     elif args.case == "attention":
         qkv = torch.randn(64 * 197, 3 * 768, device=dev, generator=gen).to(torch.bfloat16)
         run = lambda: B.tbn_attention_fwd(qkv, 64, 197, 12, 64)
+    elif args.case == "compact_gelu":
+        T, d, mlp, k = 128 * 197, 768, 3072, 8
+        z = torch.randn(T, mlp // k, device=dev, generator=gen).to(torch.bfloat16)
+        y = torch.empty(T, d, device=dev, dtype=torch.bfloat16)
+        tile = rand_tile(d * mlp // k)
+        a1, a2 = torch.rand(k, device=dev, generator=gen) * 0.05, torch.rand(k, device=dev, generator=gen) * 0.02
+        run = lambda: B.tbn_linear_compact_fwd(z, k, a1, B.ALPHA_PER_TILE, B.ACT_GELU, d, tile, k, a2, B.ALPHA_PER_TILE, y=y)
     elif args.case == "tile_bwd":
         N, k = 4096 * 4096, 4
         W = torch.randn(N, device=dev, generator=gen) * 0.02
