@@ -39,12 +39,15 @@ layernorm_kernel(const XT *__restrict__ x, int64_t T, int32_t d, const float *__
 }
 
 // ---- multi-head softmax attention, bf16 operands, fp32 accumulation and softmax ---------------------------------
-// One block per (image, head): Q, K (row pitch 72 elements) and V transposed (key index contiguous) sit in shared
-// memory; a warp owns 16 query rows at a time and keeps the whole score row block in registers (S <= 16 * NT16
-// keys), so the softmax is exact (no running rescale).  Both contractions are warp-level m16n8k16 MMAs; the
-// probabilities are rounded to bf16 for the second one.
+// One block per (image, head): Q, K and V sit in shared memory as they are in the input (row = token, 64 elements,
+// row pitch 72); a warp owns 16 query rows at a time and keeps the whole score row block in registers (S <= 16 * NT16
+// keys), so the softmax is exact (no running rescale).  Both contractions are warp-level m16n8k16 MMAs whose operand
+// fragments come from ldmatrix: four 8 x 8 blocks per instruction, K as stored (key-major = the "col" operand of
+// Q K^T), V through the transposing form (the contraction index of P V is the key, which is V's row).  The
+// probabilities are rounded to bf16 for the second contraction.  The score MMAs run with the contraction step
+// outermost so that consecutive MMAs write different accumulators (no dependent chains).
 constexpr int kAttD = 64;
-constexpr int kAttPitch = 72;           // 36 words: the 8 rows a fragment load touches fall on different banks
+constexpr int kAttPitch = 72;           // 36 words: the 8 rows of an 8 x 8 block fall on different banks
 constexpr int kAttWarps = 7;
 
 __device__ __forceinline__ void att_mma(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
@@ -53,6 +56,16 @@ __device__ __forceinline__ void att_mma(float (&d)[4], uint32_t a0, uint32_t a1,
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void att_ldsm4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void att_ldsm4_t(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
@@ -60,20 +73,20 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 }
 
 template <int NT16>
-__global__ void __launch_bounds__(kAttWarps * 32)
+__global__ void __launch_bounds__(kAttWarps * 32, 2)
 attention_kernel(const __nv_bfloat16 *__restrict__ qkv, int32_t S, int32_t heads, __nv_bfloat16 *__restrict__ out)
 {
     constexpr int SP = NT16 * 16;                       // padded sequence length
-    constexpr int kVtPitch = SP + 8;                    // (SP + 8) / 2 words = 12 mod 32 for SP = 208, 4 mod 32 for 64 / 128
+    constexpr int NT8 = 2 * NT16;                       // 8-key score blocks
     extern __shared__ __align__(16) uint8_t att_smem[];
     __nv_bfloat16 *Qs = reinterpret_cast<__nv_bfloat16 *>(att_smem);
     __nv_bfloat16 *Ks = Qs + SP * kAttPitch;
-    __nv_bfloat16 *Vt = Ks + SP * kAttPitch;            // [64][kVtPitch]
+    __nv_bfloat16 *Vs = Ks + SP * kAttPitch;
     const int b = blockIdx.x / heads, h = blockIdx.x % heads;
     const int64_t row_pitch = (int64_t)3 * heads * kAttD;
     const __nv_bfloat16 *base = qkv + (int64_t)b * S * row_pitch + h * kAttD;
 
-    // stage Q, K (16-byte pieces) and V transposed; rows past the sequence are zero
+    // stage Q, K, V in 16-byte pieces; rows past the sequence are zero (a zero V row keeps 0 * V finite)
     for (int idx = threadIdx.x; idx < SP * 8; idx += blockDim.x) {
         const int s = idx >> 3, c = idx & 7;
         uint4 q = make_uint4(0u, 0u, 0u, 0u), k = q, v = q;
@@ -85,44 +98,49 @@ attention_kernel(const __nv_bfloat16 *__restrict__ qkv, int32_t S, int32_t heads
         }
         *reinterpret_cast<uint4 *>(Qs + s * kAttPitch + c * 8) = q;
         *reinterpret_cast<uint4 *>(Ks + s * kAttPitch + c * 8) = k;
-        const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            reinterpret_cast<unsigned short *>(Vt)[(c * 8 + 2 * e) * kVtPitch + s] = (unsigned short)(vw[e] & 0xffffu);
-            reinterpret_cast<unsigned short *>(Vt)[(c * 8 + 2 * e + 1) * kVtPitch + s] = (unsigned short)(vw[e] >> 16);
-        }
+        *reinterpret_cast<uint4 *>(Vs + s * kAttPitch + c * 8) = v;
     }
     __syncthreads();
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, c = lane & 3;
+    const int mat = lane >> 3, l8 = lane & 7;           // ldmatrix: lanes 8 i .. 8 i + 7 give the row addresses of block i
+    const uint32_t q_s = (uint32_t)__cvta_generic_to_shared(Qs), k_s = (uint32_t)__cvta_generic_to_shared(Ks),
+                   v_s = (uint32_t)__cvta_generic_to_shared(Vs);
+    // K blocks of one instruction: keys nt * 8 + l8, columns (32 kp) + 8 mat -> b0, b1 of steps 2 kp and 2 kp + 1
+    const uint32_t k_lane = k_s + (uint32_t)(l8 * kAttPitch + mat * 8) * 2u;
+    // V blocks (transposed on load): keys 16 kk + 8 (mat & 1) + l8, columns 16 np + 8 (mat >> 1) -> b0, b1 of column
+    // blocks 2 np and 2 np + 1
+    const uint32_t v_lane = v_s + (uint32_t)(((mat & 1) * 8 + l8) * kAttPitch + (mat >> 1) * 8) * 2u;
     const float scale = 0.125f * 1.4426950408889634f;   // 1/sqrt(64) * log2(e): the softmax runs on exp2
     for (int qt = warp; qt < NT16; qt += kAttWarps) {
         if (qt * 16 >= S) break;
-        // scores of 16 query rows against all keys
+        // Q blocks: rows 16 qt + 8 (mat & 1) + l8, columns 16 kk + 8 (mat >> 1) -> a0 .. a3 of step kk
         uint32_t aq[4][4];
+        const uint32_t q_lane = q_s + (uint32_t)((qt * 16 + (mat & 1) * 8 + l8) * kAttPitch + (mat >> 1) * 8) * 2u;
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-            const __nv_bfloat16 *q0 = Qs + (qt * 16 + g) * kAttPitch + kk * 16 + 2 * c;
-            aq[kk][0] = *reinterpret_cast<const uint32_t *>(q0);
-            aq[kk][1] = *reinterpret_cast<const uint32_t *>(q0 + 8 * kAttPitch);
-            aq[kk][2] = *reinterpret_cast<const uint32_t *>(q0 + 8);
-            aq[kk][3] = *reinterpret_cast<const uint32_t *>(q0 + 8 * kAttPitch + 8);
-        }
-        float sc[2 * NT16][4];
+        for (int kk = 0; kk < 4; ++kk) att_ldsm4(q_lane + kk * 32, aq[kk][0], aq[kk][1], aq[kk][2], aq[kk][3]);
+        // scores of 16 query rows against all keys
+        float sc[NT8][4];
 #pragma unroll
-        for (int nt = 0; nt < 2 * NT16; ++nt) {
-            sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.0f;
-            const __nv_bfloat16 *k0 = Ks + (nt * 8 + g) * kAttPitch + 2 * c;
+        for (int nt = 0; nt < NT8; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.0f;
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-                att_mma(sc[nt], aq[kk][0], aq[kk][1], aq[kk][2], aq[kk][3], *reinterpret_cast<const uint32_t *>(k0 + kk * 16),
-                        *reinterpret_cast<const uint32_t *>(k0 + kk * 16 + 8));
+        for (int kp = 0; kp < 2; ++kp) {
+#pragma unroll
+            for (int nt = 0; nt < NT8; nt += 2) {
+                uint32_t b[2][4];
+                att_ldsm4(k_lane + (uint32_t)(nt * 8 * kAttPitch * 2 + kp * 64), b[0][0], b[0][1], b[0][2], b[0][3]);
+                att_ldsm4(k_lane + (uint32_t)((nt + 1) * 8 * kAttPitch * 2 + kp * 64), b[1][0], b[1][1], b[1][2], b[1][3]);
+                att_mma(sc[nt], aq[2 * kp][0], aq[2 * kp][1], aq[2 * kp][2], aq[2 * kp][3], b[0][0], b[0][1]);
+                att_mma(sc[nt + 1], aq[2 * kp][0], aq[2 * kp][1], aq[2 * kp][2], aq[2 * kp][3], b[1][0], b[1][1]);
+                att_mma(sc[nt], aq[2 * kp + 1][0], aq[2 * kp + 1][1], aq[2 * kp + 1][2], aq[2 * kp + 1][3], b[0][2], b[0][3]);
+                att_mma(sc[nt + 1], aq[2 * kp + 1][0], aq[2 * kp + 1][1], aq[2 * kp + 1][2], aq[2 * kp + 1][3], b[1][2], b[1][3]);
+            }
         }
         // mask the padded keys, row maxima (rows g and g + 8), exponentials, row sums
         float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
-        for (int nt = 0; nt < 2 * NT16; ++nt) {
+        for (int nt = 0; nt < NT8; ++nt) {
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
                 if (nt * 8 + 2 * c + e >= S) { sc[nt][e] = -INFINITY; sc[nt][2 + e] = -INFINITY; }
@@ -132,31 +150,33 @@ attention_kernel(const __nv_bfloat16 *__restrict__ qkv, int32_t S, int32_t heads
         }
         m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 1)); m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 2));
         m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 1)); m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 2));
+        // exponentials, row sums (of the unrounded values), and the bf16 pairs that are the A fragments of the second
+        // contraction: block pair (2 kk, 2 kk + 1) of the scores is exactly the a0 .. a3 layout of step kk
         float l0 = 0.0f, l1 = 0.0f;
+        uint32_t pa[NT16][4];
+        const float ms0 = m0 * scale, ms1 = m1 * scale;
 #pragma unroll
-        for (int nt = 0; nt < 2 * NT16; ++nt) {
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                sc[nt][e] = exp2f((sc[nt][e] - m0) * scale);
-                sc[nt][2 + e] = exp2f((sc[nt][2 + e] - m1) * scale);
-                l0 += sc[nt][e];
-                l1 += sc[nt][2 + e];
-            }
+        for (int nt = 0; nt < NT8; ++nt) {
+            const float e0 = exp2f(fmaf(sc[nt][0], scale, -ms0)), e1 = exp2f(fmaf(sc[nt][1], scale, -ms0));
+            const float e2 = exp2f(fmaf(sc[nt][2], scale, -ms1)), e3 = exp2f(fmaf(sc[nt][3], scale, -ms1));
+            l0 += e0 + e1;
+            l1 += e2 + e3;
+            pa[nt >> 1][(nt & 1) * 2] = pack_bf16(e0, e1);
+            pa[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(e2, e3);
         }
         l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
         l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-        // weighted sum of the values: the score fragments are the A operand of the second contraction as they are
         float o[8][4];
 #pragma unroll
         for (int nt = 0; nt < 8; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.0f;
 #pragma unroll
         for (int kk = 0; kk < NT16; ++kk) {
-            const uint32_t a0 = pack_bf16(sc[2 * kk][0], sc[2 * kk][1]), a1 = pack_bf16(sc[2 * kk][2], sc[2 * kk][3]);
-            const uint32_t a2 = pack_bf16(sc[2 * kk + 1][0], sc[2 * kk + 1][1]), a3 = pack_bf16(sc[2 * kk + 1][2], sc[2 * kk + 1][3]);
 #pragma unroll
-            for (int nt = 0; nt < 8; ++nt) {
-                const __nv_bfloat16 *v0 = Vt + (nt * 8 + g) * kVtPitch + kk * 16 + 2 * c;
-                att_mma(o[nt], a0, a1, a2, a3, *reinterpret_cast<const uint32_t *>(v0), *reinterpret_cast<const uint32_t *>(v0 + 8));
+            for (int np = 0; np < 4; ++np) {
+                uint32_t v0, v1, v2, v3;
+                att_ldsm4_t(v_lane + (uint32_t)(kk * 16 * kAttPitch * 2 + np * 32), v0, v1, v2, v3);
+                att_mma(o[2 * np], pa[kk][0], pa[kk][1], pa[kk][2], pa[kk][3], v0, v1);
+                att_mma(o[2 * np + 1], pa[kk][0], pa[kk][1], pa[kk][2], pa[kk][3], v2, v3);
             }
         }
         const float r0 = 1.0f / l0, r1 = 1.0f / l1;
@@ -175,7 +195,7 @@ template <int NT16>
 cudaError_t launch_attention_nt(const __nv_bfloat16 *qkv, int32_t Nb, int32_t S, int32_t heads, __nv_bfloat16 *out, cudaStream_t s)
 {
     constexpr int SP = NT16 * 16;
-    const size_t smem = (size_t)(2 * SP * kAttPitch + kAttD * (SP + 8)) * sizeof(__nv_bfloat16);
+    const size_t smem = (size_t)(3 * SP * kAttPitch) * sizeof(__nv_bfloat16);
     auto kern = attention_kernel<NT16>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
