@@ -903,10 +903,18 @@ int tbn_vit_block_fwd(const void *x, int32_t Nb, int32_t S, int32_t d, int32_t h
                              scratch, scratch_bytes, stream, AUTO);
     if (rc != TBN_OK) return rc;
     if (launch_attention(qkv, Nb, S, heads, d / heads, att, s) != cudaSuccess) return TBN_ERR_CUDA;
-    rc = tbn_linear_res_fwd(att, B16, T, d, d, tiles[1], ks[1], alphas[1], alpha_modes[1], nullptr, TBN_ACT_NONE, x, x1, B16,
-                            scratch, scratch_bytes, stream, AUTO);
-    if (rc != TBN_OK) return rc;
-    if (launch_layernorm(x1, B16, T, d, nullptr, nullptr, 1e-5f, h, B16, s) != cudaSuccess) return TBN_ERR_CUDA;
+    if (add_layernorm_supported(d)) {
+        // the projection writes into x1; one pass then forms x1 = x + projection and h = LayerNorm(x1)
+        rc = tbn_linear_fwd_path(att, B16, T, d, d, tiles[1], ks[1], alphas[1], alpha_modes[1], nullptr, TBN_ACT_NONE, x1, B16,
+                                 scratch, scratch_bytes, stream, AUTO);
+        if (rc != TBN_OK) return rc;
+        if (launch_add_layernorm(x, x1, x1, T, d, nullptr, nullptr, 1e-5f, h, s) != cudaSuccess) return TBN_ERR_CUDA;
+    } else {
+        rc = tbn_linear_res_fwd(att, B16, T, d, d, tiles[1], ks[1], alphas[1], alpha_modes[1], nullptr, TBN_ACT_NONE, x, x1, B16,
+                                scratch, scratch_bytes, stream, AUTO);
+        if (rc != TBN_OK) return rc;
+        if (launch_layernorm(x1, B16, T, d, nullptr, nullptr, 1e-5f, h, B16, s) != cudaSuccess) return TBN_ERR_CUDA;
+    }
     rc = tbn_linear_fwd_path(h, B16, T, d, mlp_dim, tiles[2], ks[2], alphas[2], alpha_modes[2], nullptr, TBN_ACT_GELU, f, B16,
                              scratch, scratch_bytes, stream, AUTO);
     if (rc != TBN_OK) return rc;

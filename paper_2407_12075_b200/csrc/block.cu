@@ -38,6 +38,84 @@ layernorm_kernel(const XT *__restrict__ x, int64_t T, int32_t d, const float *__
     }
 }
 
+// bf16 rows of up to 256 * NP elements (a multiple of 8), one warp per row, the row held in registers: each lane takes
+// 16-byte pieces lane, lane + 32, ...  With a second operand b the row normalised is the bf16-rounded sum a + b,
+// which is also written out (the residual stream of an encoder block: one pass instead of an addition pass followed
+// by a normalisation pass; sum_out may be b itself, every piece is read before it is written by the same thread).
+template <int NP>
+__global__ void __launch_bounds__(256)
+add_layernorm_bf16_kernel(const __nv_bfloat16 *__restrict__ a, const __nv_bfloat16 *b, __nv_bfloat16 *sum_out, int64_t T, int32_t d,
+                          const float *__restrict__ gamma, const float *__restrict__ beta, float eps, __nv_bfloat16 *__restrict__ y)
+{
+    const int lane = threadIdx.x & 31;
+    const int32_t pieces = d >> 3;
+    const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t t = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; t < T; t += warps) {
+        const int64_t row = t * d;
+        float v[NP][8];
+        float s = 0.0f;
+#pragma unroll
+        for (int i = 0; i < NP; ++i) {
+            const int32_t pc = lane + 32 * i;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) v[i][e] = 0.0f;
+            if (pc < pieces) {
+                const uint4 ua = *reinterpret_cast<const uint4 *>(a + row + pc * 8);
+                const uint32_t wa[4] = {ua.x, ua.y, ua.z, ua.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    v[i][2 * e] = __uint_as_float(wa[e] << 16);
+                    v[i][2 * e + 1] = __uint_as_float(wa[e] & 0xffff0000u);
+                }
+                if (b != nullptr) {
+                    const uint4 ub = *reinterpret_cast<const uint4 *>(b + row + pc * 8);
+                    const uint32_t wb[4] = {ub.x, ub.y, ub.z, ub.w};
+                    uint32_t ws[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const __nv_bfloat162 h2 = __floats2bfloat162_rn(v[i][2 * e] + __uint_as_float(wb[e] << 16),
+                                                                        v[i][2 * e + 1] + __uint_as_float(wb[e] & 0xffff0000u));
+                        ws[e] = *reinterpret_cast<const uint32_t *>(&h2);
+                        v[i][2 * e] = __uint_as_float(ws[e] << 16);
+                        v[i][2 * e + 1] = __uint_as_float(ws[e] & 0xffff0000u);
+                    }
+                    *reinterpret_cast<uint4 *>(sum_out + row + pc * 8) = make_uint4(ws[0], ws[1], ws[2], ws[3]);
+                }
+#pragma unroll
+                for (int e = 0; e < 8; ++e) s += v[i][e];
+            }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+        const float mu = s / (float)d;
+        float q = 0.0f;
+#pragma unroll
+        for (int i = 0; i < NP; ++i)
+            if (lane + 32 * i < pieces) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) { const float c = v[i][e] - mu; q = fmaf(c, c, q); }
+            }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) q += __shfl_xor_sync(0xffffffffu, q, off);
+        const float rstd = rsqrtf(q / (float)d + eps);
+#pragma unroll
+        for (int i = 0; i < NP; ++i) {
+            const int32_t pc = lane + 32 * i;
+            if (pc >= pieces) continue;
+            uint32_t wo[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float o0 = (v[i][2 * e] - mu) * rstd, o1 = (v[i][2 * e + 1] - mu) * rstd;
+                if (gamma) { o0 *= __ldg(gamma + pc * 8 + 2 * e); o1 *= __ldg(gamma + pc * 8 + 2 * e + 1); }
+                if (beta) { o0 += __ldg(beta + pc * 8 + 2 * e); o1 += __ldg(beta + pc * 8 + 2 * e + 1); }
+                const __nv_bfloat162 h2 = __floats2bfloat162_rn(o0, o1);
+                wo[e] = *reinterpret_cast<const uint32_t *>(&h2);
+            }
+            *reinterpret_cast<uint4 *>(y + row + pc * 8) = make_uint4(wo[0], wo[1], wo[2], wo[3]);
+        }
+    }
+}
+
 // ---- multi-head softmax attention, bf16 operands, fp32 accumulation and softmax ---------------------------------
 // One block per (image, head): Q, K and V sit in shared memory as they are in the input (row = token, 64 elements,
 // row pitch 72); a warp owns 16 query rows at a time and keeps the whole score row block in registers (S <= 16 * NT16
@@ -205,11 +283,31 @@ cudaError_t launch_attention_nt(const __nv_bfloat16 *qkv, int32_t Nb, int32_t S,
 
 }  // namespace
 
+bool add_layernorm_supported(int32_t d) { return d > 0 && d % 8 == 0 && d <= 1024; }
+
+cudaError_t launch_add_layernorm(const void *a, const void *b, void *sum_out, int64_t T, int32_t d, const float *gamma,
+                                 const float *beta, float eps, void *y, cudaStream_t s)
+{
+    if (!add_layernorm_supported(d)) return cudaErrorInvalidValue;
+    const int64_t blocks_needed = (T + 7) / 8;
+    const unsigned grid = (unsigned)(blocks_needed < 148 * 16 ? (blocks_needed > 0 ? blocks_needed : 1) : 148 * 16);
+    const __nv_bfloat16 *pa = static_cast<const __nv_bfloat16 *>(a), *pb = static_cast<const __nv_bfloat16 *>(b);
+    __nv_bfloat16 *ps = static_cast<__nv_bfloat16 *>(sum_out), *py = static_cast<__nv_bfloat16 *>(y);
+    if (d <= 256) add_layernorm_bf16_kernel<1><<<grid, 256, 0, s>>>(pa, pb, ps, T, d, gamma, beta, eps, py);
+    else if (d <= 512) add_layernorm_bf16_kernel<2><<<grid, 256, 0, s>>>(pa, pb, ps, T, d, gamma, beta, eps, py);
+    else if (d <= 768) add_layernorm_bf16_kernel<3><<<grid, 256, 0, s>>>(pa, pb, ps, T, d, gamma, beta, eps, py);
+    else add_layernorm_bf16_kernel<4><<<grid, 256, 0, s>>>(pa, pb, ps, T, d, gamma, beta, eps, py);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_layernorm(const void *x, int x_dtype, int64_t T, int32_t d, const float *gamma, const float *beta, float eps,
                              void *y, int y_dtype, cudaStream_t s)
 {
     const int64_t blocks_needed = (T + 7) / 8;
     const unsigned grid = (unsigned)(blocks_needed < 148 * 16 ? (blocks_needed > 0 ? blocks_needed : 1) : 148 * 16);
+    if (add_layernorm_supported(d) && x_dtype == TBN_BF16 && y_dtype == TBN_BF16 && !(reinterpret_cast<uintptr_t>(x) & 15u) &&
+        !(reinterpret_cast<uintptr_t>(y) & 15u))
+        return launch_add_layernorm(x, nullptr, nullptr, T, d, gamma, beta, eps, y, s);
     if (x_dtype == TBN_BF16 && y_dtype == TBN_BF16)
         layernorm_kernel<<<grid, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(x), T, d, gamma, beta, eps, static_cast<__nv_bfloat16 *>(y));
     else if (x_dtype == TBN_BF16)

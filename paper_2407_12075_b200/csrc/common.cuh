@@ -174,6 +174,11 @@ cudaError_t launch_tile_bwd(const float *G, const uint32_t *tile, const float *a
                             cudaStream_t s);
 
 // ---- encoder-block glue (block.cu) ----------------------------------------------------------------------
+bool add_layernorm_supported(int32_t d);
+// y = LayerNorm(bf16(a + b)) with the rounded sum also written to sum_out (b = nullptr: plain LayerNorm of a); bf16, 16-byte
+// aligned rows
+cudaError_t launch_add_layernorm(const void *a, const void *b, void *sum_out, int64_t T, int32_t d, const float *gamma,
+                                 const float *beta, float eps, void *y, cudaStream_t s);
 cudaError_t launch_layernorm(const void *x, int x_dtype, int64_t T, int32_t d, const float *gamma, const float *beta, float eps,
                              void *y, int y_dtype, cudaStream_t s);
 bool attention_supported(int32_t S, int32_t heads, int32_t d_head);

@@ -60,19 +60,22 @@ dense_conv_kernel(const XT *__restrict__ x, const float *__restrict__ w, const f
     }
 }
 
-// The stack's own first layer, 3 input channels and a 3x3 filter (27 inputs per output): the 27 inputs of a pixel are
-// loaded once into registers (zero outside the image) and contracted with kFcCo output channels, whose weights are
-// laid out [input][channel] in shared memory so that four channels come with one broadcast 16-byte load.
+// The stack's own first layer, 3 input channels and a 3x3 filter (27 inputs per output).  A thread owns two
+// horizontally adjacent output pixels and kFcCo output channels: the 27 inputs of each pixel are loaded once into
+// registers (zero outside the image); the weights are laid out [input][channel] in shared memory so that four channels
+// come with one broadcast 16-byte load, which then feeds both pixels; two channels share one packed fp32 FMA
+// (fma.rn.f32x2), so an output costs half an FMA-pipe instruction per input.  The pixel pair is stored as one
+// 4-byte bf16 pair where the row length allows it (a warp then writes 128 contiguous bytes per channel).
 constexpr int kFcN = 27;
 constexpr int kFcCo = 32;
 
 template <typename XT, typename YT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(128)
 first_conv3x3_kernel(const XT *__restrict__ x, const float *__restrict__ w, const float *__restrict__ bias, YT *__restrict__ y,
                      int32_t Nb, int32_t H, int32_t Wd, int32_t Cout, int32_t stride, int32_t pad, int32_t Ho, int32_t Wo, int act)
 {
     __shared__ __align__(16) float ws[kFcN * kFcCo];
-    __shared__ float bs[kFcCo];
+    __shared__ __align__(8) float bs[kFcCo];
     const int32_t co0 = blockIdx.y * kFcCo;
     for (int32_t i = threadIdx.x; i < kFcN * kFcCo; i += blockDim.x) {
         const int32_t r = i / kFcCo, c = i - r * kFcCo;
@@ -80,41 +83,61 @@ first_conv3x3_kernel(const XT *__restrict__ x, const float *__restrict__ w, cons
     }
     if (threadIdx.x < kFcCo) bs[threadIdx.x] = (bias && co0 + (int)threadIdx.x < Cout) ? __ldg(bias + co0 + threadIdx.x) : 0.0f;
     __syncthreads();
-    const int64_t pixels = (int64_t)Nb * Ho * Wo;
-    for (int64_t pix = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; pix < pixels; pix += (int64_t)gridDim.x * blockDim.x) {
-        const int32_t ow = (int32_t)(pix % Wo);
-        const int64_t t = pix / Wo;
+    const int32_t Wp = (Wo + 1) >> 1;                       // pixel pairs per output row
+    const int64_t items = (int64_t)Nb * Ho * Wp;
+    const bool pair_store = (Wo & 1) == 0;
+    // one item per thread (no grid-stride loop: the compiler would keep the loop-invariant weights in registers)
+    const int64_t it = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (it < items) {
+        const int32_t ow = (int32_t)(it % Wp) * 2;
+        const int64_t t = it / Wp;
         const int32_t oh = (int32_t)(t % Ho);
         const int64_t b = t / Ho;
-        float xin[kFcN];
+        float xin[2][kFcN];
 #pragma unroll
-        for (int ci = 0; ci < 3; ++ci)
+        for (int px = 0; px < 2; ++px)
 #pragma unroll
-            for (int u = 0; u < 3; ++u)
+            for (int ci = 0; ci < 3; ++ci)
 #pragma unroll
-                for (int v = 0; v < 3; ++v) {
-                    const int32_t ih = oh * stride + u - pad, iw = ow * stride + v - pad;
-                    const bool in = ih >= 0 && ih < H && iw >= 0 && iw < Wd;
-                    xin[(ci * 3 + u) * 3 + v] = in ? load_as_float(x, ((b * 3 + ci) * H + ih) * (int64_t)Wd + iw) : 0.0f;
-                }
-        float acc[kFcCo];
+                for (int u = 0; u < 3; ++u)
 #pragma unroll
-        for (int c = 0; c < kFcCo; ++c) acc[c] = bs[c];
+                    for (int v = 0; v < 3; ++v) {
+                        const int32_t ih = oh * stride + u - pad, iw = (ow + px) * stride + v - pad;
+                        const bool in = ow + px < Wo && ih >= 0 && ih < H && iw >= 0 && iw < Wd;
+                        xin[px][(ci * 3 + u) * 3 + v] = in ? load_as_float(x, ((b * 3 + ci) * H + ih) * (int64_t)Wd + iw) : 0.0f;
+                    }
+        uint64_t acc[2][kFcCo / 2];                         // [pixel][channel pair]
+#pragma unroll
+        for (int c = 0; c < kFcCo / 2; ++c) acc[0][c] = acc[1][c] = *reinterpret_cast<const uint64_t *>(&bs[2 * c]);
 #pragma unroll
         for (int r = 0; r < kFcN; ++r) {
+            const uint64_t x0 = f32x2_pack(xin[0][r], xin[0][r]), x1 = f32x2_pack(xin[1][r], xin[1][r]);
 #pragma unroll
-            for (int c = 0; c < kFcCo; c += 4) {
-                const float4 w4 = *reinterpret_cast<const float4 *>(&ws[r * kFcCo + c]);
-                acc[c] = fmaf(w4.x, xin[r], acc[c]);
-                acc[c + 1] = fmaf(w4.y, xin[r], acc[c + 1]);
-                acc[c + 2] = fmaf(w4.z, xin[r], acc[c + 2]);
-                acc[c + 3] = fmaf(w4.w, xin[r], acc[c + 3]);
+            for (int c = 0; c < kFcCo / 2; c += 2) {
+                const ulonglong2 w4 = *reinterpret_cast<const ulonglong2 *>(&ws[r * kFcCo + 2 * c]);
+                acc[0][c] = f32x2_fma(w4.x, x0, acc[0][c]);
+                acc[0][c + 1] = f32x2_fma(w4.y, x0, acc[0][c + 1]);
+                acc[1][c] = f32x2_fma(w4.x, x1, acc[1][c]);
+                acc[1][c + 1] = f32x2_fma(w4.y, x1, acc[1][c + 1]);
             }
         }
 #pragma unroll
         for (int c = 0; c < kFcCo; ++c) {
             if (co0 + c >= Cout) break;
-            store_from_float(y, ((b * Cout + co0 + c) * Ho + oh) * (int64_t)Wo + ow, apply_act(acc[c], act));
+            float p0lo, p0hi, p1lo, p1hi;
+            f32x2_unpack(acc[0][c >> 1], p0lo, p0hi);
+            f32x2_unpack(acc[1][c >> 1], p1lo, p1hi);
+            const float o0 = apply_act((c & 1) ? p0hi : p0lo, act), o1 = apply_act((c & 1) ? p1hi : p1lo, act);
+            const int64_t yi = ((b * Cout + co0 + c) * Ho + oh) * (int64_t)Wo + ow;
+            if constexpr (sizeof(YT) == 2) {
+                if (pair_store) {                               // yi is even: 4-byte aligned
+                    const __nv_bfloat162 h2 = __floats2bfloat162_rn(o0, o1);
+                    *reinterpret_cast<__nv_bfloat162 *>(y + yi) = h2;
+                    continue;
+                }
+            }
+            store_from_float(y, yi, o0);
+            if (ow + 1 < Wo) store_from_float(y, yi + 1, o1);
         }
     }
 }
@@ -147,8 +170,10 @@ cudaError_t launch_dense_conv(const void *x, int x_dtype, const float *w, const 
     const int64_t pixels = (int64_t)Nb * Ho * Wo;
     const int64_t bx = (pixels + 255) / 256;
     if (Cin == 3 && kh == 3 && kw == 3) {
-        const dim3 grid((unsigned)(bx < 148 * 64 ? (bx > 0 ? bx : 1) : 148 * 64), (unsigned)((Cout + kFcCo - 1) / kFcCo));
-#define TBN_FC(XT, YT) first_conv3x3_kernel<XT, YT><<<grid, 256, 0, s>>>(static_cast<const XT *>(x), w, bias, static_cast<YT *>(y), Nb, \
+        const int64_t pb = ((int64_t)Nb * Ho * ((Wo + 1) / 2) + 127) / 128;       // a thread owns two pixels
+        if (pb > 0x7fffffffLL) return cudaErrorInvalidValue;
+        const dim3 grid((unsigned)(pb > 0 ? pb : 1), (unsigned)((Cout + kFcCo - 1) / kFcCo));
+#define TBN_FC(XT, YT) first_conv3x3_kernel<XT, YT><<<grid, 128, 0, s>>>(static_cast<const XT *>(x), w, bias, static_cast<YT *>(y), Nb, \
                                                                          H, Wd, Cout, stride, pad, Ho, Wo, act)
         if (x_dtype == TBN_BF16 && y_dtype == TBN_BF16) TBN_FC(__nv_bfloat16, __nv_bfloat16);
         else if (x_dtype == TBN_BF16) TBN_FC(__nv_bfloat16, float);
