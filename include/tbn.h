@@ -265,12 +265,24 @@ int tbn_linear_fwd_host(const void *x_host, int x_dtype, int64_t T, int32_t in_f
  *   path: TBN_PATH_AUTO; TBN_PATH_GENERIC = the popcount kernel (any shape, any alignment of the tile against the rows;
  *   one packed activation row must fit 48 KB); TBN_PATH_TENSOR = the integer tensor-core kernel (needs
  *   q % in_f == 0 and in_f % 32 == 0; TBN_ERR_UNSUPPORTED otherwise).  No workspace.  T == 0 is a no-op.
+ * tbn_bin_expand_fwd / tbn_linear_bin_bytes_fwd: the tensor path with the activation signs held as bytes, which a
+ *   layer's activations are expanded to ONCE (instead of on chip by every row block of the layer): x_bytes is T rows of
+ *   in_f bytes, 0x00 for -1 and 0xFF for +1, and byte 4 s + j (s < 8, j < 4) of every group of 32 elements holds element
+ *   8 j + 7 - s of the group (the order in which the kernel expands the weight bits; any order works as long as both
+ *   operands share it); x_pop is T int32 values, the number of +1 elements of each row.  Both are written by
+ *   tbn_bin_expand_fwd from x_bits.  in_f % 32 == 0 (TBN_ERR_UNSUPPORTED otherwise); x_bytes 16-byte aligned.
+ *   tbn_linear_bin_bytes_fwd has otherwise the arguments and results of tbn_linear_bin_fwd on TBN_PATH_TENSOR: the
+ *   integers D are identical.
  */
 int64_t tbn_row_words(int32_t in_f);
 int tbn_binarize_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, uint32_t *x_bits, float *beta, void *stream);
 int tbn_linear_bin_fwd(const uint32_t *x_bits, int64_t T, int32_t in_f, int32_t out_f,
                        const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
                        const float *beta, const float *bias, int act, void *y, int y_dtype, void *stream, int path);
+int tbn_bin_expand_fwd(const uint32_t *x_bits, int64_t T, int32_t in_f, void *x_bytes, int32_t *x_pop, void *stream);
+int tbn_linear_bin_bytes_fwd(const void *x_bytes, const int32_t *x_pop, int64_t T, int32_t in_f, int32_t out_f,
+                             const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                             const float *beta, const float *bias, int act, void *y, int y_dtype, void *stream);
 
 /* ------------------------------------------------------------------------------------------------
  * 2-D convolution forward.  The paper defines tiling for convolutional layers (Sec. 3: the tile

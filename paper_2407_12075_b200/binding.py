@@ -73,6 +73,9 @@ SIGNATURES = {
     "tbn_binarize_fwd": (c_int, [c_vp, c_int, c_i64, c_i32, c_vp, c_vp, c_vp]),
     "tbn_linear_bin_fwd": (c_int, [c_vp, c_i64, c_i32, c_i32, c_vp, c_i32, c_vp, c_int, c_vp, c_vp, c_int, c_vp, c_int,
                                    c_vp, c_int]),
+    "tbn_bin_expand_fwd": (c_int, [c_vp, c_i64, c_i32, c_vp, c_vp, c_vp]),
+    "tbn_linear_bin_bytes_fwd": (c_int, [c_vp, c_vp, c_i64, c_i32, c_i32, c_vp, c_i32, c_vp, c_int, c_vp, c_vp, c_int, c_vp,
+                                         c_int, c_vp]),
 }
 
 _lib = None
@@ -334,6 +337,29 @@ def tbn_linear_bin_fwd(x_bits: torch.Tensor, in_f: int, out_f: int, tile: torch.
         y = torch.empty((T, out_f), dtype=_torch_dtype(y_dtype), device=x_bits.device)
     _check(lib().tbn_linear_bin_fwd(_ptr(x_bits), T, in_f, out_f, _ptr(tile), k, _ptr(alpha), alpha_mode, _ptr(beta),
                                     _ptr(bias), act, _ptr(y), y_dtype, _stream(), path), "tbn_linear_bin_fwd")
+    return y
+
+
+def tbn_bin_expand_fwd(x_bits: torch.Tensor, in_f: int, x_bytes: torch.Tensor | None = None, x_pop: torch.Tensor | None = None):
+    """Packed activation signs -> (one byte per element, 0x00 / 0xFF, in the tensor kernel's element order; row popcounts)."""
+    T = x_bits.shape[0]
+    if x_bytes is None:
+        x_bytes = torch.empty((T, in_f), dtype=torch.uint8, device=x_bits.device)
+    if x_pop is None:
+        x_pop = torch.empty(T, dtype=torch.int32, device=x_bits.device)
+    _check(lib().tbn_bin_expand_fwd(_ptr(x_bits), T, in_f, _ptr(x_bytes), _ptr(x_pop), _stream()), "tbn_bin_expand_fwd")
+    return x_bytes, x_pop
+
+
+def tbn_linear_bin_bytes_fwd(x_bytes: torch.Tensor, x_pop: torch.Tensor, in_f: int, out_f: int, tile: torch.Tensor, k: int,
+                             alpha: torch.Tensor, alpha_mode: int, beta: torch.Tensor | None = None,
+                             bias: torch.Tensor | None = None, act: int = ACT_NONE, y_dtype: int = BF16,
+                             y: torch.Tensor | None = None) -> torch.Tensor:
+    T = x_bytes.shape[0]
+    if y is None:
+        y = torch.empty((T, out_f), dtype=_torch_dtype(y_dtype), device=x_bytes.device)
+    _check(lib().tbn_linear_bin_bytes_fwd(_ptr(x_bytes), _ptr(x_pop), T, in_f, out_f, _ptr(tile), k, _ptr(alpha), alpha_mode,
+                                          _ptr(beta), _ptr(bias), act, _ptr(y), y_dtype, _stream()), "tbn_linear_bin_bytes_fwd")
     return y
 
 

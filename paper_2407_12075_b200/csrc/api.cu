@@ -994,6 +994,43 @@ int tbn_linear_bin_fwd(const uint32_t *x_bits, int64_t T, int32_t in_f, int32_t 
     return launch_bin_popc(a, s) == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
 }
 
+int tbn_bin_expand_fwd(const uint32_t *x_bits, int64_t T, int32_t in_f, void *x_bytes, int32_t *x_pop, void *stream)
+{
+    if (T < 0 || in_f <= 0) return TBN_ERR_INVALID_ARG;
+    if (in_f % 32 != 0) return TBN_ERR_UNSUPPORTED;
+    if (T == 0) return TBN_OK;
+    if (!x_bits || !x_bytes || !x_pop || !aligned16(x_bits) || !aligned16(x_bytes) || (reinterpret_cast<uintptr_t>(x_pop) & 3u))
+        return TBN_ERR_INVALID_ARG;
+    return launch_bin_expand(x_bits, T, in_f, (int32_t)tbn_row_words(in_f), x_bytes, x_pop, static_cast<cudaStream_t>(stream)) ==
+                   cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
+}
+
+int tbn_linear_bin_bytes_fwd(const void *x_bytes, const int32_t *x_pop, int64_t T, int32_t in_f, int32_t out_f,
+                             const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
+                             const float *beta, const float *bias, int act, void *y, int y_dtype, void *stream)
+{
+    if (T < 0 || in_f <= 0 || out_f <= 0 || k <= 0) return TBN_ERR_INVALID_ARG;
+    if (!tile_bits || !alpha || !valid_alpha_mode(alpha_mode) || !valid_act(act)) return TBN_ERR_INVALID_ARG;
+    if (!(valid_dtype(y_dtype) || y_dtype == TBN_I32)) return TBN_ERR_INVALID_ARG;
+    if (T > 0 && (!x_bytes || !x_pop || !y)) return TBN_ERR_INVALID_ARG;
+    if (!aligned16(x_bytes) || !aligned16(y) || !aligned16(tile_bits) || (reinterpret_cast<uintptr_t>(x_pop) & 3u))
+        return TBN_ERR_INVALID_ARG;
+    if ((bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) || (beta && (reinterpret_cast<uintptr_t>(beta) & 3u)))
+        return TBN_ERR_INVALID_ARG;
+    const int64_t N = (int64_t)in_f * out_f;
+    if (N % k != 0) return TBN_ERR_SHAPE;
+    if (T == 0) return TBN_OK;
+    BinArgs a;
+    std::memset(&a, 0, sizeof(a));
+    a.x_bytes = x_bytes; a.x_pop = x_pop; a.tile = tile_bits; a.alpha = alpha; a.beta = beta; a.bias = bias; a.y = y;
+    a.T = T; a.q = N / k; a.x_row_words = (int32_t)tbn_row_words(in_f); a.n = in_f; a.m = out_f; a.k = k;
+    a.alpha_mode = alpha_mode; a.act = act; a.y_dtype = y_dtype;
+    if (!bin_tensor_supported(a)) return TBN_ERR_UNSUPPORTED;
+    int *st = device_status_ptr();
+    if (!st) return TBN_ERR_CUDA;
+    return launch_bin_tensor(a, st, static_cast<cudaStream_t>(stream));
+}
+
 int tbn_debug_force_bin_config(int candidate) { return force_bin_config(candidate); }
 
 int tbn_last_device_status(void *stream, int *code, int *detail)

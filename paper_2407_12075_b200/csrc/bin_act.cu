@@ -177,7 +177,45 @@ bin_popc_kernel(const BinArgs a)
     }
 }
 
+// Packed activation signs -> one byte per element, 0x00 (bit 0) or 0xFF (bit 1), in the element order of the 8-bit
+// tensor-core kernel: byte 4 s + j of every group of 32 elements holds bit 8 j + 7 - s of the group's word (one byte
+// permute in sign mode per four elements); and the popcount of every row.  One warp per row, one word per lane and
+// step, two 16-byte stores per word.
+__global__ void __launch_bounds__(256)
+bin_expand_kernel(const uint32_t *__restrict__ bits, int64_t T, int32_t nw, int32_t row_words, uint8_t *__restrict__ bytes,
+                  int32_t *__restrict__ row_pop)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t t = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; t < T; t += warps) {
+        int32_t cnt = 0;
+        for (int32_t w = lane; w < nw; w += 32) {
+            const uint32_t v = __ldg(bits + t * row_words + w);
+            cnt += __popc(v);
+            uint32_t e[8];
+#pragma unroll
+            for (int sft = 0; sft < 8; ++sft) asm("prmt.b32 %0, %1, %1, 0xBA98;" : "=r"(e[sft]) : "r"(v << sft));
+            uint4 *dst = reinterpret_cast<uint4 *>(bytes + (t * nw + w) * 32);
+            dst[0] = make_uint4(e[0], e[1], e[2], e[3]);
+            dst[1] = make_uint4(e[4], e[5], e[6], e[7]);
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
+        if (lane == 0) row_pop[t] = cnt;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_bin_expand(const uint32_t *bits, int64_t T, int32_t n, int32_t row_words, void *bytes, int32_t *row_pop,
+                              cudaStream_t s)
+{
+    if (n % 32 != 0) return cudaErrorInvalidValue;
+    const int64_t blocks_needed = (T + 7) / 8;
+    const unsigned grid = (unsigned)(blocks_needed < 148 * 32 ? (blocks_needed > 0 ? blocks_needed : 1) : 148 * 32);
+    bin_expand_kernel<<<grid, 256, 0, s>>>(bits, T, n / 32, row_words, static_cast<uint8_t *>(bytes), row_pop);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_binarize(const void *x, int x_dtype, int64_t T, int32_t n, uint32_t *bits, float *beta, cudaStream_t s)
 {

@@ -147,6 +147,8 @@ struct LayerArgs {
 // ---- binary-activation layer (bit-packed activations; see bin_act.cu) ---------------------------------
 struct BinArgs {
     const uint32_t *x_bits;   // [T][x_row_words] packed activation signs, padding bits zero
+    const void *x_bytes;      // optional: the same signs as bytes 0x00 / 0xFF, [T][n] (tensor path only), or null
+    const int32_t *x_pop;     // with x_bytes: popcount of every row
     const uint32_t *tile;
     const float *alpha;
     const float *beta;        // per-token scale, or null (= 1)
@@ -159,6 +161,8 @@ struct BinArgs {
     int alpha_mode, act, y_dtype;   // y_dtype TBN_I32: the raw integer accumulators
 };
 cudaError_t launch_binarize(const void *x, int x_dtype, int64_t T, int32_t n, uint32_t *bits, float *beta, cudaStream_t s);
+cudaError_t launch_bin_expand(const uint32_t *bits, int64_t T, int32_t n, int32_t row_words, void *bytes, int32_t *row_pop,
+                              cudaStream_t s);
 bool bin_popc_supported(const BinArgs &a);
 cudaError_t launch_bin_popc(const BinArgs &a, cudaStream_t s);
 bool bin_tensor_supported(const BinArgs &a);

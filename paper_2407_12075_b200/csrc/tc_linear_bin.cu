@@ -19,11 +19,17 @@
 // warps with ordinary stores in the swizzled layout, since no copy engine expands bits), accumulators in tensor memory.
 // A stage is 256 contraction elements: 8 words of bits per row, 8 MMAs of K = 32.
 //
+// Byte form of the activations (template flag BYTES): when the caller has expanded the activation bits to the same
+// 0x00 / 0xFF bytes in global memory once (tbn_bin_expand_fwd, same element order), the stage is filled by TMA like the
+// bf16 kernel's and the producer warps only fetch the row popcounts (counted once, with the bytes): the shared-memory stores of the expansion, which
+// bind the bit form, disappear, at the price of an 8 times larger activation tensor in HBM.
+//
 // Warp roles (13 warps): 0-3 activation producers, 4 MMA issuer / TMEM owner, 5-8 weight decode, 9-12 epilogue
 // (tcgen05.ld -> integer combine -> exchange through shared memory -> beta_t alpha_j scaling, bias, activation ->
 // k-fold replicated stores).  All hand-offs are mbarriers; every wait is bounded (see tc_common.cuh).
 #include <atomic>
 #include <cstddef>
+#include <cstring>
 
 #include "tc_common.cuh"
 
@@ -59,6 +65,7 @@ struct BinControl {
 
 struct BinParams {
     const uint32_t *x_bits;
+    const int32_t *x_pop;    // byte form: popcount of every activation row
     const uint32_t *tile;
     const float *alpha;
     const float *beta;
@@ -109,10 +116,14 @@ __device__ __forceinline__ void tc_mma_ts_i8(uint32_t d_tmem, uint32_t a_tmem, u
 
 constexpr uint64_t kBinBDescHi = (64ull << 32) | (1ull << 46) | (2ull << 61);   // as the bf16 kernel: SW128, K-major
 
-template <int NTOK, int SX, int DB>
+template <int NTOK, int SX, int DB, bool BYTES>
 __global__ void __launch_bounds__(kBinThreads, 1)
-tc_linear_bin_kernel(const BinParams p)
+tc_linear_bin_kernel(const __grid_constant__ CUtensorMap xb_map, const BinParams p)
 {
+    // BYTES: the activation bytes exist in global memory (tbn_bin_expand_fwd) and TMA stages them; warp 0 issues the
+    // copies, warps 1-3 fetch the tile's row popcounts
+    constexpr uint32_t kXFullCount = BYTES ? 1u : (uint32_t)kBinProd;
+    constexpr uint32_t kSideProd = BYTES ? 96u : (uint32_t)kBinProd;
     static_assert(NTOK == 128 || NTOK == 256, "token tile");
     constexpr uint32_t kAtomBytes = NTOK * 128;
     constexpr uint32_t kStageBytes = kBinKA * kAtomBytes;
@@ -134,11 +145,11 @@ tc_linear_bin_kernel(const BinParams p)
     const int bid = blockIdx.x;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < SX; ++s) { mbar_init(smem_u32(&ctl->x_full[s]), kBinProd); mbar_init(smem_u32(&ctl->x_empty[s]), 1); }
+        for (int s = 0; s < SX; ++s) { mbar_init(smem_u32(&ctl->x_full[s]), kXFullCount); mbar_init(smem_u32(&ctl->x_empty[s]), 1); }
         for (int s = 0; s < kBinAStages; ++s) { mbar_init(smem_u32(&ctl->a_full[s]), 128); mbar_init(smem_u32(&ctl->a_empty[s]), 1); }
         for (int s = 0; s < 2; ++s) {
             mbar_init(smem_u32(&ctl->d_full[s]), 1); mbar_init(smem_u32(&ctl->d_empty[s]), 128);
-            mbar_init(smem_u32(&ctl->side_full[s]), kBinProd + 128); mbar_init(smem_u32(&ctl->side_empty[s]), 128);
+            mbar_init(smem_u32(&ctl->side_full[s]), kSideProd + 128); mbar_init(smem_u32(&ctl->side_empty[s]), 128);
         }
         ctl->abort_flag = 0;
         fence_barrier_init();
@@ -160,7 +171,52 @@ tc_linear_bin_kernel(const BinParams p)
     const int32_t n_tiles = p.w_tiles * p.t_tiles;
     bool ok = true;
 
-    if (warp < kBinMmaWarp) {
+    if (BYTES && warp == 0) {
+        // ---------------- loader: activation bytes -> swizzled shared-memory stage by TMA ----------------
+        // Rows past T and columns past n arrive as zeros (and still count their bytes on the barrier).
+        Pipe px;
+        uint32_t issued_mask = 0, issued_phase = 0;
+        for (int32_t tile = bid; tile < n_tiles && ok; tile += gridDim.x) {
+            const int32_t tok0 = (tile / p.w_tiles) * NTOK;
+            for (int32_t ks = 0; ks < p.k_stages; ++ks) {
+                ok = wait_bar(smem_u32(&ctl->x_empty[px.stage]), px.phase ^ 1u, abort_flag, p.status,
+                              (1 << 24) | (px.stage << 16) | (bid & 0xffff));
+                if (!ok) break;
+                if (lane == 0) {
+                    const uint32_t bar = smem_u32(&ctl->x_full[px.stage]);
+                    mbar_arrive_expect_tx(bar, kStageBytes);
+#pragma unroll
+                    for (int at = 0; at < kBinKA; ++at)
+                        tma_load_2d(stage0 + px.stage * kStageBytes + at * kAtomBytes, &xb_map, ks * kBinStageK + at * kBinAtomK,
+                                    tok0, bar);
+                }
+                issued_mask |= 1u << px.stage;
+                issued_phase = (issued_phase & ~(1u << px.stage)) | (px.phase << px.stage);
+                __syncwarp();
+                px.advance(SX);
+            }
+        }
+        if (!ok) {   // let copies in flight land before the block's shared memory goes away
+            for (int s = 0; s < SX; ++s)
+                if (issued_mask & (1u << s)) drain_wait(smem_u32(&ctl->x_full[s]), (issued_phase >> s) & 1u);
+        }
+    } else if (BYTES && warp < kBinMmaWarp) {
+        // ---------------- row popcounts of the tile's tokens, counted once when the bytes were written (warps 1-3) ----------------
+        uint32_t sd = 0, sd_phase = 0;
+        for (int32_t tile = bid; tile < n_tiles; tile += gridDim.x) {
+            ok = wait_bar(smem_u32(&ctl->side_empty[sd]), sd_phase ^ 1u, abort_flag, p.status, (9 << 24) | (bid & 0xffff));
+            if (!ok) break;
+            const int64_t tok0 = (int64_t)(tile / p.w_tiles) * NTOK;
+            for (int row = (warp - 1) * 32 + lane; row < NTOK; row += 96) {
+                const int64_t tok = tok0 + row;
+                ctl->px[sd][row] = tok < p.T ? __ldg(p.x_pop + tok) : 0;
+            }
+            __syncwarp();
+            mbar_arrive(smem_u32(&ctl->side_full[sd]));
+            sd ^= 1u;
+            if (sd == 0) sd_phase ^= 1u;
+        }
+    } else if (warp < kBinMmaWarp) {
         // ---------------- activation producers: bits -> bytes -> swizzled shared-memory stage ----------------
         // Thread tid owns token rows tid, tid + 128 (, ...) of the tile: per stage it reads the row's 8 words (one
         // 32-byte sector), expands them and writes the row's 128-byte line of each of the two swizzle rows: the
@@ -517,19 +573,33 @@ int bin_sm_count()
 }
 
 template <int NTOK, int SX, int DB>
-int launch_bin_config(BinParams p, cudaStream_t s)
+int launch_bin_config(BinParams p, const void *x_bytes, cudaStream_t s)
 {
     p.w_tiles = (p.r + 127) / 128;
     p.t_tiles = (int32_t)((p.T + NTOK - 1) / NTOK);
     const size_t smem = (size_t)SX * kBinKA * NTOK * 128 + sizeof(BinControl<SX>) + 1024;
-    auto kern = tc_linear_bin_kernel<NTOK, SX, DB>;
+    CUtensorMap map;
+    std::memset(&map, 0, sizeof(map));
+    if (x_bytes) {                                         // T rows of n bytes; a box is one swizzle row of a stage
+        EncodeTiledFn encode = encode_tiled_fn();
+        if (!encode) return TBN_ERR_CUDA;
+        const cuuint64_t dims[2] = {(cuuint64_t)p.n, (cuuint64_t)p.T};
+        const cuuint64_t strides[1] = {(cuuint64_t)p.n};
+        const cuuint32_t box[2] = {(cuuint32_t)kBinAtomK, (cuuint32_t)NTOK};
+        const cuuint32_t estr[2] = {1, 1};
+        if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(x_bytes), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return TBN_ERR_CUDA;
+    }
+    auto kern = x_bytes ? tc_linear_bin_kernel<NTOK, SX, DB, true> : tc_linear_bin_kernel<NTOK, SX, DB, false>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return TBN_ERR_CUDA;
     const int sms = bin_sm_count();
     if (sms <= 0) return TBN_ERR_CUDA;
     const int64_t tiles = (int64_t)p.w_tiles * p.t_tiles;
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
-    kern<<<grid, kBinThreads, smem, s>>>(p);
+    kern<<<grid, kBinThreads, smem, s>>>(map, p);
     return cudaGetLastError() == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
 }
 
@@ -550,6 +620,7 @@ bool bin_tensor_supported(const BinArgs &a)
     if (a.q % a.n != 0) return false;                 // the tile must span whole rows
     if (a.n % 32 != 0) return false;                  // rows of weight bits start on word boundaries
     if (a.T >= ((int64_t)1 << 31) - 256) return false;
+    if (a.x_bytes && (a.n % 16 != 0 || !a.x_pop)) return false;       // row pitch of the byte form (implied by n % 32 == 0)
     return true;
 }
 
@@ -557,7 +628,7 @@ int launch_bin_tensor(const BinArgs &a, int *device_status, cudaStream_t s)
 {
     if (!bin_tensor_supported(a)) return TBN_ERR_UNSUPPORTED;
     BinParams p;
-    p.x_bits = a.x_bits; p.tile = a.tile; p.alpha = a.alpha; p.beta = a.beta; p.bias = a.bias; p.y = a.y;
+    p.x_bits = a.x_bits; p.x_pop = a.x_pop; p.tile = a.tile; p.alpha = a.alpha; p.beta = a.beta; p.bias = a.bias; p.y = a.y;
     p.status = device_status;
     p.T = a.T; p.xw = a.x_row_words; p.n = a.n; p.m = a.m; p.r = (int32_t)(a.q / a.n); p.k = a.k;
     p.nw = a.n / 32; p.k_stages = (a.n + kBinStageK - 1) / kBinStageK;
@@ -573,9 +644,9 @@ int launch_bin_tensor(const BinArgs &a, int *device_status, cudaStream_t s)
     const int forced = g_forced_bin.load(std::memory_order_relaxed);
     if (forced >= 0) cand = forced;
     switch (cand) {
-    case 0: return launch_bin_config<256, 3, 1>(p, s);
-    case 1: return launch_bin_config<128, 5, 2>(p, s);
-    default: return launch_bin_config<128, 5, 1>(p, s);
+    case 0: return launch_bin_config<256, 3, 1>(p, a.x_bytes, s);
+    case 1: return launch_bin_config<128, 5, 2>(p, a.x_bytes, s);
+    default: return launch_bin_config<128, 5, 1>(p, a.x_bytes, s);
     }
 }
 

@@ -135,6 +135,83 @@ def test_large_sweep_shape_sampled_rows_integers_exact():
     assert B.tbn_last_device_status() == (0, 0)
 
 
+def expand_reference(bits_rows: np.ndarray, n: int) -> np.ndarray:
+    """The documented byte form written out element by element: byte 4 s + j of each group of 32 elements is 0xFF when
+    element 8 j + 7 - s of the group is +1, else 0x00."""
+    T = bits_rows.shape[0]
+    out = np.zeros((T, n), dtype=np.uint8)
+    for g in range(n // 32):
+        for sft in range(8):
+            for j in range(4):
+                out[:, 32 * g + 4 * sft + j] = np.where(bits_rows[:, 32 * g + 8 * j + 7 - sft] != 0, 0xFF, 0x00)
+    return out
+
+
+@pytest.mark.parametrize("T,n", [(1, 32), (5, 96), (130, 768), (33, 4096)])
+def test_expand_to_bytes_matches_the_documented_order(T, n):
+    x = synth.to_bf16_bits(synth.normal(70 + n, 0, T * n).reshape(T, n))
+    abits, _ = O.binarize(x)
+    xb = to_dev(O.pack_rows(abits))
+    got, pop = B.tbn_bin_expand_fwd(xb, n)
+    torch.cuda.synchronize()
+    assert got.shape == (T, n) and got.dtype == torch.uint8
+    assert np.array_equal(got.cpu().numpy(), expand_reference(np.asarray(abits), n))
+    assert np.array_equal(pop.cpu().numpy(), np.asarray(abits, dtype=np.int64).sum(axis=1))
+    with pytest.raises(B.TbnError) as e:
+        B.tbn_bin_expand_fwd(torch.zeros((2, 4), dtype=torch.int32, device=DEV), 40)      # not a multiple of 32
+    assert e.value.status == -3
+
+
+@pytest.mark.parametrize("T,m,n,k", TENSOR)
+def test_byte_form_integers_exact_every_tile_shape(T, m, n, k):
+    x, words, al, abits, beta = _case(64, T, m, n, k, True)
+    xb, td, ad = to_dev(O.pack_rows(abits)), to_dev(words), to_dev(al)
+    xbytes, xpop = B.tbn_bin_expand_fwd(xb, n)
+    want = O.linear_bin_int(abits, words, k, m, n)
+    cand = 0
+    try:
+        while B.lib().tbn_debug_force_bin_config(cand) == 0:
+            D = B.tbn_linear_bin_bytes_fwd(xbytes, xpop, n, m, td, k, ad, 1, y_dtype=B.I32)
+            torch.cuda.synchronize()
+            assert np.array_equal(D.cpu().numpy().astype(np.int64), want), f"tile shape {cand}"
+            cand += 1
+    finally:
+        B.lib().tbn_debug_force_bin_config(-1)
+    assert cand >= 2
+    assert B.tbn_last_device_status() == (0, 0)
+
+
+@pytest.mark.parametrize("act,y_dtype,with_bias", [(B.ACT_RELU, B.BF16, False), (B.ACT_GELU, B.BF16, True), (B.ACT_NONE, B.F32, True)])
+def test_byte_form_scaled_outputs(act, y_dtype, with_bias):
+    T, m, n, k = 777, 1200, 992, 4
+    x, words, al, abits, beta = _case(65, T, m, n, k, True)
+    xb, td, ad = to_dev(O.pack_rows(abits)), to_dev(words), to_dev(al)
+    bias = synth.normal(65, 200, m, 0.2) if with_bias else None
+    ref = O.linear_bin(abits, beta, words, k, al, True, m, n, bias=None if bias is None else bias.astype(np.float64), act=act)
+    y = B.tbn_linear_bin_bytes_fwd(*B.tbn_bin_expand_fwd(xb, n), n, m, td, k, ad, 1, beta=to_dev(beta),
+                                   bias=None if bias is None else to_dev(bias), act=act, y_dtype=y_dtype)
+    torch.cuda.synchronize()
+    assert_close(to_np64(y), ref, "byte form")
+    assert B.tbn_last_device_status() == (0, 0)
+
+
+def test_byte_form_large_sweep_shape_sampled_rows_integers_exact():
+    T, m, n = 4096, 8192, 8192
+    x = synth.to_bf16_bits(synth.normal(4, 0, T * n).reshape(T, n))
+    W = synth.normal(4, 1, m * n, 0.02)
+    xb, bt = B.tbn_binarize_fwd(to_dev(x))
+    xbytes, xpop = B.tbn_bin_expand_fwd(xb, n)
+    rows = np.unique(np.concatenate([np.arange(0, T, 128) + np.arange(T // 128) % 128, [0, T - 1]]))
+    abits, beta = O.binarize(x[rows])
+    for k in (2, 16):
+        words, al = O.prepare(W, k, True)
+        D = B.tbn_linear_bin_bytes_fwd(xbytes, xpop, n, m, to_dev(words), k, to_dev(al), 1, y_dtype=B.I32)
+        torch.cuda.synchronize()
+        assert np.array_equal(D[torch.from_numpy(rows).to(DEV)].cpu().numpy().astype(np.int64),
+                              O.linear_bin_int(abits, words, k, m, n))
+    assert B.tbn_last_device_status() == (0, 0)
+
+
 def test_argument_errors():
     xb = torch.zeros((4, 4), dtype=torch.int32, device=DEV)
     t = torch.zeros(8, dtype=torch.int32, device=DEV)
