@@ -429,7 +429,27 @@ def measure_other_configs(B, torch, dev, peaks):
                                             bound="tensor (int8)" if ops / int8_peak > nbytes / hbm else "hbm",
                                             frac_of_binding_roofline=t_bound * 1e6 / us,
                                             popcount_alu_peak_tops=popc_peak / 1e12)
-    del x, y
+    # the same layer with the activation signs expanded to bytes once (one pass over the bits) and staged by TMA
+    xbytes = torch.empty((T, N_FEAT), dtype=torch.uint8, device=dev)
+    xpop = torch.empty(T, dtype=torch.int32, device=dev)
+    us = graph_us(lambda: B.tbn_bin_expand_fwd(xb, N_FEAT, x_bytes=xbytes, x_pop=xpop), reps=3, iters=3)
+    nbytes = xb.numel() * 4 + xbytes.numel() + T * 4
+    out["bin_expand_T16384_8192"] = dict(us=us, alg_gbs=nbytes / us / 1e3, bound="hbm", frac_of_binding_roofline=nbytes / hbm * 1e6 / us)
+    us = graph_us(lambda: B.tbn_binarize_bytes_fwd(x), reps=3, iters=3)
+    nbytes = x.numel() * 2 + xb.numel() * 4 + xbytes.numel() + T * 8
+    out["binarize_with_bytes_T16384_8192"] = dict(us=us, alg_gbs=nbytes / us / 1e3, bound="hbm", frac_of_binding_roofline=nbytes / hbm * 1e6 / us,
+                                                  note="threshold, packing, row scale, sign bytes and row popcounts in one pass")
+    for k in (2, 16):
+        tile, alpha = rand_tile(N_FEAT * N_FEAT // k), torch.rand(k, device=dev, generator=gen) * 0.02
+        us = graph_us(lambda: B.tbn_linear_bin_bytes_fwd(xbytes, xpop, N_FEAT, N_FEAT, tile, k, alpha, B.ALPHA_PER_TILE, beta=beta,
+                                                         y=y), reps=3, iters=3)
+        ops = 2.0 * T * (N_FEAT // k) * N_FEAT
+        nbytes = xbytes.numel() + y.numel() * 2 + N_FEAT * N_FEAT // k / 8
+        t_bound = max(ops / int8_peak, nbytes / hbm)
+        out[f"bin_linear_bytes_T{T}_k{k}"] = dict(us=us, alg_tops=ops / us / 1e6, alg_gbs=nbytes / us / 1e3,
+                                                  bound="tensor (int8)" if ops / int8_peak > nbytes / hbm else "hbm",
+                                                  frac_of_binding_roofline=t_bound * 1e6 / us)
+    del x, y, xbytes
     xb16 = xb[:16].contiguous()
     y16 = torch.empty(16, N_FEAT, device=dev, dtype=torch.bfloat16)
     tile, alpha = rand_tile(N_FEAT * N_FEAT // 2), torch.rand(2, device=dev, generator=gen) * 0.02

@@ -273,6 +273,8 @@ int tbn_linear_fwd_host(const void *x_host, int x_dtype, int64_t T, int32_t in_f
  *   tbn_bin_expand_fwd from x_bits.  in_f % 32 == 0 (TBN_ERR_UNSUPPORTED otherwise); x_bytes 16-byte aligned.
  *   tbn_linear_bin_bytes_fwd has otherwise the arguments and results of tbn_linear_bin_fwd on TBN_PATH_TENSOR: the
  *   integers D are identical.
+ * tbn_binarize_bytes_fwd: tbn_binarize_fwd and tbn_bin_expand_fwd in one pass over x (x_bits, beta, x_bytes and x_pop as
+ *   above, bit for bit the same; in_f % 32 == 0).
  */
 int64_t tbn_row_words(int32_t in_f);
 int tbn_binarize_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, uint32_t *x_bits, float *beta, void *stream);
@@ -280,6 +282,8 @@ int tbn_linear_bin_fwd(const uint32_t *x_bits, int64_t T, int32_t in_f, int32_t 
                        const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
                        const float *beta, const float *bias, int act, void *y, int y_dtype, void *stream, int path);
 int tbn_bin_expand_fwd(const uint32_t *x_bits, int64_t T, int32_t in_f, void *x_bytes, int32_t *x_pop, void *stream);
+int tbn_binarize_bytes_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, uint32_t *x_bits, float *beta, void *x_bytes,
+                           int32_t *x_pop, void *stream);
 int tbn_linear_bin_bytes_fwd(const void *x_bytes, const int32_t *x_pop, int64_t T, int32_t in_f, int32_t out_f,
                              const uint32_t *tile_bits, int32_t k, const float *alpha, int alpha_mode,
                              const float *beta, const float *bias, int act, void *y, int y_dtype, void *stream);

@@ -74,6 +74,7 @@ SIGNATURES = {
     "tbn_linear_bin_fwd": (c_int, [c_vp, c_i64, c_i32, c_i32, c_vp, c_i32, c_vp, c_int, c_vp, c_vp, c_int, c_vp, c_int,
                                    c_vp, c_int]),
     "tbn_bin_expand_fwd": (c_int, [c_vp, c_i64, c_i32, c_vp, c_vp, c_vp]),
+    "tbn_binarize_bytes_fwd": (c_int, [c_vp, c_int, c_i64, c_i32, c_vp, c_vp, c_vp, c_vp, c_vp]),
     "tbn_linear_bin_bytes_fwd": (c_int, [c_vp, c_vp, c_i64, c_i32, c_i32, c_vp, c_i32, c_vp, c_int, c_vp, c_vp, c_int, c_vp,
                                          c_int, c_vp]),
 }
@@ -349,6 +350,18 @@ def tbn_bin_expand_fwd(x_bits: torch.Tensor, in_f: int, x_bytes: torch.Tensor | 
         x_pop = torch.empty(T, dtype=torch.int32, device=x_bits.device)
     _check(lib().tbn_bin_expand_fwd(_ptr(x_bits), T, in_f, _ptr(x_bytes), _ptr(x_pop), _stream()), "tbn_bin_expand_fwd")
     return x_bytes, x_pop
+
+
+def tbn_binarize_bytes_fwd(x: torch.Tensor):
+    """Threshold, packing, row scale, sign bytes and row popcounts in one pass.  Returns (x_bits, beta, x_bytes, x_pop)."""
+    T, n = x.shape
+    x_bits = torch.empty((T, tbn_row_words(n)), dtype=torch.int32, device=x.device)
+    beta = torch.empty(T, dtype=torch.float32, device=x.device)
+    x_bytes = torch.empty((T, n), dtype=torch.uint8, device=x.device)
+    x_pop = torch.empty(T, dtype=torch.int32, device=x.device)
+    _check(lib().tbn_binarize_bytes_fwd(_ptr(x), _dtype_code(x), T, n, _ptr(x_bits), _ptr(beta), _ptr(x_bytes), _ptr(x_pop),
+                                        _stream()), "tbn_binarize_bytes_fwd")
+    return x_bits, beta, x_bytes, x_pop
 
 
 def tbn_linear_bin_bytes_fwd(x_bytes: torch.Tensor, x_pop: torch.Tensor, in_f: int, out_f: int, tile: torch.Tensor, k: int,

@@ -954,7 +954,19 @@ int tbn_binarize_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, uint32
     if (T == 0) return TBN_OK;
     if (!x || !x_bits || !aligned16(x) || !aligned16(x_bits)) return TBN_ERR_INVALID_ARG;
     if (beta && (reinterpret_cast<uintptr_t>(beta) & 3u)) return TBN_ERR_INVALID_ARG;
-    return launch_binarize(x, x_dtype, T, in_f, x_bits, beta, static_cast<cudaStream_t>(stream)) == cudaSuccess
+    return launch_binarize(x, x_dtype, T, in_f, x_bits, beta, nullptr, nullptr, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? TBN_OK : TBN_ERR_CUDA;
+}
+
+int tbn_binarize_bytes_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, uint32_t *x_bits, float *beta, void *x_bytes,
+                           int32_t *x_pop, void *stream)
+{
+    if (T < 0 || in_f <= 0 || !valid_dtype(x_dtype)) return TBN_ERR_INVALID_ARG;
+    if (in_f % 32 != 0) return TBN_ERR_UNSUPPORTED;
+    if (T == 0) return TBN_OK;
+    if (!x || !x_bits || !x_bytes || !x_pop || !aligned16(x) || !aligned16(x_bits) || !aligned16(x_bytes)) return TBN_ERR_INVALID_ARG;
+    if ((beta && (reinterpret_cast<uintptr_t>(beta) & 3u)) || (reinterpret_cast<uintptr_t>(x_pop) & 3u)) return TBN_ERR_INVALID_ARG;
+    return launch_binarize(x, x_dtype, T, in_f, x_bits, beta, x_bytes, x_pop, static_cast<cudaStream_t>(stream)) == cudaSuccess
                ? TBN_OK : TBN_ERR_CUDA;
 }
 

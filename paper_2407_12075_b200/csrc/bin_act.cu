@@ -42,14 +42,17 @@ __device__ __forceinline__ void load8f<float>(const float *p, float (&v)[8]) {
 template <typename XT, bool VEC>
 __global__ void __launch_bounds__(256)
 binarize_kernel(const XT *__restrict__ x, int64_t T, int32_t n, int32_t row_words, uint32_t *__restrict__ bits,
-                float *__restrict__ beta)
+                float *__restrict__ beta, uint8_t *__restrict__ bytes, int32_t *__restrict__ row_pop)
 {
+    // bytes / row_pop (both or neither; n a multiple of 32): the byte form of the signs for the tensor-core kernel, in
+    // its element order (see bin_expand_kernel), and the number of +1 elements of each row, written in the same pass
     const int lane = threadIdx.x & 31;
     const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
     for (int64_t t = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; t < T; t += warps) {
         const XT *row = x + t * n;
         uint32_t *out = bits + t * row_words;
         double acc = 0.0;
+        int32_t pop = 0;
         // whole groups of 256 values (8 words) per step; row_words * 32 >= n, words past n are written as zero
         for (int32_t j0 = 0; j0 < row_words * 32; j0 += 256) {
             const int32_t j = j0 + lane * 8;
@@ -73,6 +76,20 @@ binarize_kernel(const XT *__restrict__ x, int64_t T, int32_t n, int32_t row_word
             word |= __shfl_xor_sync(0xffffffffu, word, 2);
             const int32_t w = (j0 >> 5) + (lane >> 2);
             if ((lane & 3) == 0 && w < row_words) out[w] = word;
+            if (bytes != nullptr && w * 32 < n) {
+                // the quad shares the word: lane j of it writes registers s = 2 j and 2 j + 1 of the word's 32 bytes
+                if ((lane & 3) == 0) pop += __popc(word);
+                const uint32_t s0 = 2u * (uint32_t)(lane & 3);
+                uint32_t e0, e1;
+                asm("prmt.b32 %0, %1, %1, 0xBA98;" : "=r"(e0) : "r"(word << s0));
+                asm("prmt.b32 %0, %1, %1, 0xBA98;" : "=r"(e1) : "r"(word << (s0 + 1u)));
+                *reinterpret_cast<uint2 *>(bytes + t * n + (int64_t)w * 32 + 4 * s0) = make_uint2(e0, e1);
+            }
+        }
+        if (row_pop != nullptr) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) pop += __shfl_xor_sync(0xffffffffu, pop, off);
+            if (lane == 0) row_pop[t] = pop;
         }
         if (beta != nullptr) {
 #pragma unroll
@@ -217,20 +234,22 @@ cudaError_t launch_bin_expand(const uint32_t *bits, int64_t T, int32_t n, int32_
     return cudaGetLastError();
 }
 
-cudaError_t launch_binarize(const void *x, int x_dtype, int64_t T, int32_t n, uint32_t *bits, float *beta, cudaStream_t s)
+cudaError_t launch_binarize(const void *x, int x_dtype, int64_t T, int32_t n, uint32_t *bits, float *beta, void *bytes_out,
+                            int32_t *row_pop, cudaStream_t s)
 {
+    uint8_t *bytes = static_cast<uint8_t *>(bytes_out);
     const int32_t rw = (int32_t)tbn_row_words(n);
     const int64_t blocks_needed = (T + 7) / 8;
     const unsigned grid = (unsigned)(blocks_needed < 148 * 16 ? (blocks_needed > 0 ? blocks_needed : 1) : 148 * 16);
     const bool vec = (n % 8 == 0) && (reinterpret_cast<uintptr_t>(x) & 15) == 0;
     if (x_dtype == TBN_BF16) {
         const __nv_bfloat16 *xp = static_cast<const __nv_bfloat16 *>(x);
-        if (vec) binarize_kernel<__nv_bfloat16, true><<<grid, 256, 0, s>>>(xp, T, n, rw, bits, beta);
-        else binarize_kernel<__nv_bfloat16, false><<<grid, 256, 0, s>>>(xp, T, n, rw, bits, beta);
+        if (vec) binarize_kernel<__nv_bfloat16, true><<<grid, 256, 0, s>>>(xp, T, n, rw, bits, beta, bytes, row_pop);
+        else binarize_kernel<__nv_bfloat16, false><<<grid, 256, 0, s>>>(xp, T, n, rw, bits, beta, bytes, row_pop);
     } else {
         const float *xp = static_cast<const float *>(x);
-        if (vec) binarize_kernel<float, true><<<grid, 256, 0, s>>>(xp, T, n, rw, bits, beta);
-        else binarize_kernel<float, false><<<grid, 256, 0, s>>>(xp, T, n, rw, bits, beta);
+        if (vec) binarize_kernel<float, true><<<grid, 256, 0, s>>>(xp, T, n, rw, bits, beta, bytes, row_pop);
+        else binarize_kernel<float, false><<<grid, 256, 0, s>>>(xp, T, n, rw, bits, beta, bytes, row_pop);
     }
     return cudaGetLastError();
 }

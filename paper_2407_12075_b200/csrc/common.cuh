@@ -160,7 +160,8 @@ struct BinArgs {
     int32_t n, m, k;
     int alpha_mode, act, y_dtype;   // y_dtype TBN_I32: the raw integer accumulators
 };
-cudaError_t launch_binarize(const void *x, int x_dtype, int64_t T, int32_t n, uint32_t *bits, float *beta, cudaStream_t s);
+cudaError_t launch_binarize(const void *x, int x_dtype, int64_t T, int32_t n, uint32_t *bits, float *beta, void *bytes_out,
+                            int32_t *row_pop, cudaStream_t s);
 cudaError_t launch_bin_expand(const uint32_t *bits, int64_t T, int32_t n, int32_t row_words, void *bytes, int32_t *row_pop,
                               cudaStream_t s);
 bool bin_popc_supported(const BinArgs &a);

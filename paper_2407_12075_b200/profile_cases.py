@@ -4,6 +4,7 @@ of launches):
     python -m paper_2407_12075_b200.profile_cases <case> [--reps N]
 
 Cases: linear_k2, linear_k16 (8192 x 8192, T = 8192), bin_k2, bin_k16 (binary activations, 8192 x 8192, T = 4096),
+binbytes_k2, binbytes_k16 (the same with the activation signs as bytes),
 conv_s2 (64 -> 128, 32 x 32, batch 64), attention (64 images x 12 heads x 197 tokens), binarize, tile_bwd,
 compact_gelu (second MLP layer of a ViT-B block fed the first layer's 384 distinct pre-activations, T = 25,216).
 Inputs are seeded device-side random values of the benchmark's shapes; every run checks the device status word.
@@ -38,7 +39,7 @@ def main():
         tile, alpha = rand_tile(n * m // k), torch.rand(k, device=dev, generator=gen) * 0.02
         ws = torch.empty(max(B.tbn_linear_workspace_bytes(T, n, m, k, B.BF16), 16), dtype=torch.uint8, device=dev)
         run = lambda: B.tbn_linear_fwd(x, m, tile, k, alpha, B.ALPHA_PER_TILE, y=y, workspace=ws)
-    elif args.case in ("bin_k2", "bin_k16", "binarize"):
+    elif args.case in ("bin_k2", "bin_k16", "binarize", "binbytes_k2", "binbytes_k16"):
         T = 4096
         x = torch.randn(T, n, device=dev, generator=gen).to(torch.bfloat16)
         xb, beta = B.tbn_binarize_fwd(x)
@@ -48,7 +49,11 @@ def main():
             k = int(args.case.split("_k")[1])
             y = torch.empty(T, m, device=dev, dtype=torch.bfloat16)
             tile, alpha = rand_tile(n * m // k), torch.rand(k, device=dev, generator=gen) * 0.02
-            run = lambda: B.tbn_linear_bin_fwd(xb, n, m, tile, k, alpha, B.ALPHA_PER_TILE, beta=beta, y=y)
+            if args.case.startswith("binbytes"):
+                xbytes, xpop = B.tbn_bin_expand_fwd(xb, n)
+                run = lambda: B.tbn_linear_bin_bytes_fwd(xbytes, xpop, n, m, tile, k, alpha, B.ALPHA_PER_TILE, beta=beta, y=y)
+            else:
+                run = lambda: B.tbn_linear_bin_fwd(xb, n, m, tile, k, alpha, B.ALPHA_PER_TILE, beta=beta, y=y)
     elif args.case == "conv_s2":
         xc = torch.rand(64, 64, 32, 32, device=dev, generator=gen).to(torch.bfloat16)
         tile, alpha = rand_tile(128 * 64 * 9 // 4), torch.rand(4, device=dev, generator=gen) * 0.05

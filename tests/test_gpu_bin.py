@@ -162,6 +162,18 @@ def test_expand_to_bytes_matches_the_documented_order(T, n):
     assert e.value.status == -3
 
 
+@pytest.mark.parametrize("T,n,bf16", [(3, 32, True), (70, 992, True), (130, 768, False), (33, 8192, True)])
+def test_one_pass_binarize_with_bytes_equals_the_two_passes(T, n, bf16):
+    x = synth.normal(80 + n, 0, T * n).reshape(T, n)
+    x[0, :4] = [0.0, -0.0, 1e-30, -1.0]
+    xin = to_dev(synth.to_bf16_bits(x) if bf16 else x)
+    xb, beta = B.tbn_binarize_fwd(xin)
+    xbytes, xpop = B.tbn_bin_expand_fwd(xb, n)
+    xb1, beta1, xbytes1, xpop1 = B.tbn_binarize_bytes_fwd(xin)
+    torch.cuda.synchronize()
+    assert torch.equal(xb, xb1) and torch.equal(beta, beta1) and torch.equal(xbytes, xbytes1) and torch.equal(xpop, xpop1)
+
+
 @pytest.mark.parametrize("T,m,n,k", TENSOR)
 def test_byte_form_integers_exact_every_tile_shape(T, m, n, k):
     x, words, al, abits, beta = _case(64, T, m, n, k, True)
