@@ -369,7 +369,7 @@ int tbn_mlp_fwd(const void *x, int x_dtype, int64_t T, int32_t L, const int32_t 
  *   variance, statistics in fp32); gamma, beta: d floats each or NULL.  x, y: T x d, fp32 or bf16.
  * tbn_attention_fwd: qkv: (Nb*S) x (3*heads*d_head) bf16, columns (q | k | v), head h at h*d_head inside each third;
  *   out: (Nb*S) x (heads*d_head) bf16.  bf16 operands, fp32 accumulation and softmax.  d_head must be 64 and
- *   S <= 208 (TBN_ERR_UNSUPPORTED otherwise).
+ *   S <= 208 (TBN_ERR_UNSUPPORTED otherwise).  Both pointers 16-byte aligned.
  * tbn_vit_block_fwd: x, y: (Nb*S) x d bf16.  tiles / ks / alphas / alpha_modes: HOST arrays of 4 entries in the order
  *   qkv (d -> 3d), proj (d -> d), fc1 (d -> mlp_dim), fc2 (mlp_dim -> d); tiles and alphas hold DEVICE pointers.
  *   workspace: tbn_vit_block_workspace_bytes(...) bytes (the block's intermediate tensors in bf16 plus the linears'
@@ -415,6 +415,7 @@ int tbn_debug_force_linear_config(int candidate, int splits);
 int tbn_debug_force_mlp_layerwise(int on);
 /* Same for the tile shape of the binary-activation tensor-core kernel (candidate < 0: automatic). */
 int tbn_debug_force_bin_config(int candidate);
+int tbn_debug_force_attention_path(int path); /* 0 automatic, 1 the warp-level MMA kernel, 2 the tcgen05 kernel; tests */
 
 #ifdef __cplusplus
 }

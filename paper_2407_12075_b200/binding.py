@@ -73,6 +73,7 @@ SIGNATURES = {
     "tbn_binarize_fwd": (c_int, [c_vp, c_int, c_i64, c_i32, c_vp, c_vp, c_vp]),
     "tbn_linear_bin_fwd": (c_int, [c_vp, c_i64, c_i32, c_i32, c_vp, c_i32, c_vp, c_int, c_vp, c_vp, c_int, c_vp, c_int,
                                    c_vp, c_int]),
+    "tbn_debug_force_attention_path": (c_int, [c_int]),
     "tbn_bin_expand_fwd": (c_int, [c_vp, c_i64, c_i32, c_vp, c_vp, c_vp]),
     "tbn_binarize_bytes_fwd": (c_int, [c_vp, c_int, c_i64, c_i32, c_vp, c_vp, c_vp, c_vp, c_vp]),
     "tbn_linear_bin_bytes_fwd": (c_int, [c_vp, c_vp, c_i64, c_i32, c_i32, c_vp, c_i32, c_vp, c_int, c_vp, c_vp, c_int, c_vp,
@@ -428,8 +429,9 @@ def tbn_layernorm_fwd(x: torch.Tensor, gamma: torch.Tensor | None = None, beta: 
     return y
 
 
-def tbn_attention_fwd(qkv: torch.Tensor, Nb: int, S: int, heads: int, d_head: int) -> torch.Tensor:
-    out = torch.empty((Nb * S, heads * d_head), dtype=torch.bfloat16, device=qkv.device)
+def tbn_attention_fwd(qkv: torch.Tensor, Nb: int, S: int, heads: int, d_head: int, out: torch.Tensor | None = None) -> torch.Tensor:
+    if out is None:
+        out = torch.empty((Nb * S, heads * d_head), dtype=torch.bfloat16, device=qkv.device)
     _check(lib().tbn_attention_fwd(_ptr(qkv), Nb, S, heads, d_head, _ptr(out), _stream()), "tbn_attention_fwd")
     return out
 

@@ -848,8 +848,7 @@ int tbn_attention_fwd(const void *qkv, int32_t Nb, int32_t S, int32_t heads, int
     if (Nb == 0) return TBN_OK;
     if (!qkv || !out || !aligned16(qkv) || !aligned16(out)) return TBN_ERR_INVALID_ARG;
     if (!attention_supported(S, heads, d_head) || (int64_t)Nb * heads > 0x7fffffffLL) return TBN_ERR_UNSUPPORTED;
-    return launch_attention(qkv, Nb, S, heads, d_head, out, static_cast<cudaStream_t>(stream)) == cudaSuccess ? TBN_OK
-                                                                                                               : TBN_ERR_CUDA;
+    return launch_attention(qkv, Nb, S, heads, d_head, out, device_status_ptr(), static_cast<cudaStream_t>(stream));
 }
 
 // workspace layout of the encoder block: [h: T x d][qkv: T x 3d][att: T x d][x1: T x d][f: T x mlp] bf16, then the
@@ -902,7 +901,8 @@ int tbn_vit_block_fwd(const void *x, int32_t Nb, int32_t S, int32_t d, int32_t h
     rc = tbn_linear_fwd_path(h, B16, T, d, 3 * d, tiles[0], ks[0], alphas[0], alpha_modes[0], nullptr, TBN_ACT_NONE, qkv, B16,
                              scratch, scratch_bytes, stream, AUTO);
     if (rc != TBN_OK) return rc;
-    if (launch_attention(qkv, Nb, S, heads, d / heads, att, s) != cudaSuccess) return TBN_ERR_CUDA;
+    rc = launch_attention(qkv, Nb, S, heads, d / heads, att, device_status_ptr(), s);
+    if (rc != TBN_OK) return rc;
     if (add_layernorm_supported(d)) {
         // the projection writes into x1; one pass then forms x1 = x + projection and h = LayerNorm(x1)
         rc = tbn_linear_fwd_path(att, B16, T, d, d, tiles[1], ks[1], alphas[1], alpha_modes[1], nullptr, TBN_ACT_NONE, x1, B16,
@@ -1044,6 +1044,8 @@ int tbn_linear_bin_bytes_fwd(const void *x_bytes, const int32_t *x_pop, int64_t 
 }
 
 int tbn_debug_force_bin_config(int candidate) { return force_bin_config(candidate); }
+
+int tbn_debug_force_attention_path(int path) { return force_attention_path(path); }
 
 int tbn_last_device_status(void *stream, int *code, int *detail)
 {

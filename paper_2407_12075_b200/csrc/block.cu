@@ -2,6 +2,8 @@
 // feed-forward layers of Vision Transformers; Sec. 5.2 profiles the kernel inside one): LayerNorm and multi-head
 // softmax attention.  Neither is a tiled layer and neither is specific to the paper; they exist so that the block
 // runs end to end on the device with activations produced by the previous kernel.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace tbn {
@@ -324,14 +326,31 @@ bool attention_supported(int32_t S, int32_t heads, int32_t d_head)
     return d_head == kAttD && S >= 1 && S <= 208 && heads >= 1;
 }
 
-cudaError_t launch_attention(const void *qkv, int32_t Nb, int32_t S, int32_t heads, int32_t d_head, void *out, cudaStream_t s)
+namespace {
+std::atomic<int> g_attention_path{0};
+}
+
+int force_attention_path(int path)
 {
-    (void)d_head;
+    if (path < 0 || path > 2) return TBN_ERR_INVALID_ARG;
+    g_attention_path.store(path);
+    return TBN_OK;
+}
+
+int launch_attention(const void *qkv, int32_t Nb, int32_t S, int32_t heads, int32_t d_head, void *out, int *device_status,
+                     cudaStream_t s)
+{
+    const int forced = g_attention_path.load(std::memory_order_relaxed);
+    if (forced != 1 && device_status && tc_attention_supported(Nb, S, heads, d_head))
+        return launch_tc_attention(qkv, Nb, S, heads, d_head, out, device_status, s);
+    if (forced == 2) return TBN_ERR_UNSUPPORTED;
     const __nv_bfloat16 *q = static_cast<const __nv_bfloat16 *>(qkv);
     __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(out);
-    if (S <= 64) return launch_attention_nt<4>(q, Nb, S, heads, o, s);
-    if (S <= 128) return launch_attention_nt<8>(q, Nb, S, heads, o, s);
-    return launch_attention_nt<13>(q, Nb, S, heads, o, s);
+    cudaError_t e;
+    if (S <= 64) e = launch_attention_nt<4>(q, Nb, S, heads, o, s);
+    else if (S <= 128) e = launch_attention_nt<8>(q, Nb, S, heads, o, s);
+    else e = launch_attention_nt<13>(q, Nb, S, heads, o, s);
+    return e == cudaSuccess ? TBN_OK : TBN_ERR_CUDA;
 }
 
 }  // namespace tbn

@@ -187,7 +187,13 @@ cudaError_t launch_add_layernorm(const void *a, const void *b, void *sum_out, in
 cudaError_t launch_layernorm(const void *x, int x_dtype, int64_t T, int32_t d, const float *gamma, const float *beta, float eps,
                              void *y, int y_dtype, cudaStream_t s);
 bool attention_supported(int32_t S, int32_t heads, int32_t d_head);
-cudaError_t launch_attention(const void *qkv, int32_t Nb, int32_t S, int32_t heads, int32_t d_head, void *out, cudaStream_t s);
+// returns a tbn_status; the tcgen05 kernel (tc_attention.cu) unless forced otherwise, the warp-level MMA kernel as the other path
+int launch_attention(const void *qkv, int32_t Nb, int32_t S, int32_t heads, int32_t d_head, void *out, int *device_status,
+                     cudaStream_t s);
+int force_attention_path(int path);                            // testing aid: 0 automatic, 1 warp-level MMA, 2 tcgen05
+bool tc_attention_supported(int32_t Nb, int32_t S, int32_t heads, int32_t d_head);
+int launch_tc_attention(const void *qkv, int32_t Nb, int32_t S, int32_t heads, int32_t d_head, void *out, int *device_status,
+                        cudaStream_t s);
 
 // ---- full-precision ends of a convolution stack (dense_ends.cu) ---------------------------------------------
 bool dense_conv_supported(int32_t Cin, int32_t kh, int32_t kw);

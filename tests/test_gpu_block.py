@@ -27,13 +27,21 @@ def test_layernorm_matches_oracle(T, d, bf16, affine):
     assert_close(to_np64(y), ref, "layernorm")
 
 
-@pytest.mark.parametrize("Nb,S,heads", [(2, 197, 12), (3, 64, 2), (1, 17, 1), (2, 128, 3), (1, 208, 1), (2, 1, 2), (2, 65, 1)])
-def test_attention_matches_oracle(Nb, S, heads):
+@pytest.mark.parametrize("path", [1, 2])          # 1: the warp-level MMA kernel, 2: the tcgen05 kernel
+@pytest.mark.parametrize("Nb,S,heads", [(2, 197, 12), (3, 64, 2), (1, 17, 1), (2, 128, 3), (1, 208, 1), (2, 1, 2), (2, 65, 1),
+                                        (3, 129, 2), (5, 16, 1), (2, 200, 2)])
+def test_attention_matches_oracle(Nb, S, heads, path):
     qkv = synth.to_bf16_bits(synth.normal(81, 0, Nb * S * 3 * heads * 64, 1.2).reshape(Nb * S, 3 * heads * 64))
     ref = O.attention(qkv, Nb, S, heads, 64)
-    out = B.tbn_attention_fwd(to_dev(qkv), Nb, S, heads, 64)
-    torch.cuda.synchronize()
-    assert_close(to_np64(out), ref, "attention")
+    assert B.lib().tbn_debug_force_attention_path(path) == 0
+    try:
+        out = torch.full((Nb * S, heads * 64), float("nan"), dtype=torch.bfloat16, device=DEV)
+        B.tbn_attention_fwd(to_dev(qkv), Nb, S, heads, 64, out=out)
+        torch.cuda.synchronize()
+    finally:
+        B.lib().tbn_debug_force_attention_path(0)
+    assert_close(to_np64(out), ref, f"attention, path {path}")
+    assert B.tbn_last_device_status() == (0, 0)
 
 
 def test_attention_rejects_unsupported_shapes():
