@@ -50,10 +50,10 @@ def algorithmic_bytes(T: int, k: int) -> float:
 
 
 # DRAM traffic of the dominant launch (k = 2) from an ncu capture of that kernel at T = 8192 (dram bytes read +
-# written: 235.1 MB); traffic is proportional to T.  The figure is only valid for the kernel source it was taken
+# written: 235.9 MB); traffic is proportional to T.  The figure is only valid for the kernel source it was taken
 # from: the hash below covers the code (comments stripped) of tc_linear.cu and tc_common.cuh.
-TRAFFIC_BYTES_AT_T8192 = 138.643200e6 + 96.431872e6
-TRAFFIC_SOURCE_HASH = "97eb7ca1eacc71f3"
+TRAFFIC_BYTES_AT_T8192 = 138.699520e6 + 97.207040e6
+TRAFFIC_SOURCE_HASH = "142aa7ff97fc3d03"
 
 
 def kernel_source_hash() -> str:
