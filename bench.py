@@ -343,10 +343,20 @@ def measure_other_configs(B, torch, dev, peaks):
                                          includes="LN + qkv + attention + proj(+res) + LN + fc1(GELU) + fc2(+res)")
     qkv_ = torch.randn(Nb * S, 3 * d, device=dev, generator=gen).to(torch.bfloat16)
     us = graph_us(lambda: B.tbn_attention_fwd(qkv_, Nb, S, heads, 64), reps=3, iters=3)
-    out["vit_attention_only"] = dict(us=us, dense_tflops=4.0 * Nb * heads * S * S * 64 / us / 1e6, note="warp-level MMA, not a tiled layer")
+    out["vit_attention_only"] = dict(us=us, dense_tflops=4.0 * Nb * heads * S * S * 64 / us / 1e6, note="tcgen05 kernel; glue of the block, not a tiled layer")
     us = graph_us(lambda: B.tbn_layernorm_fwd(xb_), reps=3, iters=3)
     out["vit_layernorm_only"] = dict(us=us, alg_gbs=2.0 * xb_.numel() * 2 / us / 1e3)
-    del bws, qkv_, by, xb_
+    # the block's MLP with the first layer in compact form (its 384 distinct pre-activations only) and the second layer
+    # rebuilding gelu(alpha_j z) on chip, against the full form timed above (fc1 with GELU + fc2)
+    zc = torch.empty(Nb * S, mlp // 8, device=dev, dtype=torch.bfloat16)
+    one = torch.ones(1, device=dev)
+    us1 = graph_us(lambda: B.tbn_linear_fwd(xb_, mlp // 8, btiles[2], 1, one, B.ALPHA_PER_LAYER, y=zc), reps=3, iters=3)
+    us2 = graph_us(lambda: B.tbn_linear_compact_fwd(zc, 8, balphas[2], B.ALPHA_PER_TILE, B.ACT_GELU, d, btiles[3], 8, balphas[3],
+                                                    B.ALPHA_PER_TILE, y=by), reps=3, iters=3)
+    out["vit_mlp_compact_gelu_chain"] = dict(us=us1 + us2, first_layer_us=us1, second_layer_us=us2,
+                                             full_form_us=out["vit_fc1_768_3072_gelu"]["us"] + out["vit_fc2_3072_768"]["us"],
+                                             note="measured slower than the full form, which the block therefore uses")
+    del bws, qkv_, by, xb_, zc
     xc0 = torch.rand(256, 3, 32, 32, device=dev, generator=gen).to(torch.bfloat16)
     W0 = torch.randn(64, 3, 3, 3, device=dev, generator=gen) * 0.27
     ct1, ca1 = rand_tile(128 * 64 * 9 // 4), torch.rand(4, device=dev, generator=gen) * 0.05
