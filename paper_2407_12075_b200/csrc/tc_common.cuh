@@ -217,7 +217,7 @@ static __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, vol
 }
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
                                          int detail) {
-    // every lane of the calling warp waits; the verdict is made warp-uniform so that the warp stays
+    // every lane of the calling warp waits; the outcome is made warp-uniform so that the warp stays
     // converged for the .sync.aligned tcgen05 instructions that follow
     bool r = mbar_try_wait(bar, parity) != 0;
     if (!r) r = wait_slow(bar, parity, abort_flag, status, detail);
