@@ -321,13 +321,18 @@ int tbn_conv2d_fwd_path(const void *x, int x_dtype, int32_t Nb, int32_t Cin, int
  * tbn_conv2d_dense_fwd: the convolution above with an explicit fp32 weight (Cout, Cin, kh, kw) instead of a tile, for
  *   short contractions (Cin*kh*kw <= 512; TBN_ERR_UNSUPPORTED beyond); x, y NCHW, fp32 or bf16; bias Cout floats or NULL.
  * tbn_global_avgpool_fwd: y[b][c] = mean over the H*Wd positions of x[b][c]; x NCHW, y (Nb, C); fp32 accumulation.
- * (A full-precision classifier is tbn_linear_fp_tile_fwd with k = 1.)  Neither is defined by the paper; both are
- * ordinary layers that the stack needs to run end to end. */
+ * tbn_avgpool_linear_fwd: the pooling above followed by a full-precision classifier in one launch:
+ *   y[b][o] = sum_c weight[o][c] * mean(x[b][c]) + bias[o]; weight (out_f, C) fp32 row-major, bias out_f floats or NULL,
+ *   y (Nb, out_f) fp32; C <= 4096 (TBN_ERR_UNSUPPORTED beyond).
+ * (A full-precision classifier on its own is tbn_linear_fp_tile_fwd with k = 1.)  None of these is defined by the paper;
+ * they are ordinary layers that the stack needs to run end to end. */
 int tbn_conv2d_dense_fwd(const void *x, int x_dtype, int32_t Nb, int32_t Cin, int32_t H, int32_t Wd, int32_t Cout, int32_t kh,
                          int32_t kw, int32_t stride, int32_t pad, const float *weight, const float *bias, int act, void *y,
                          int y_dtype, void *stream);
 int tbn_global_avgpool_fwd(const void *x, int x_dtype, int32_t Nb, int32_t C, int32_t H, int32_t Wd, void *y, int y_dtype,
                            void *stream);
+int tbn_avgpool_linear_fwd(const void *x, int x_dtype, int32_t Nb, int32_t C, int32_t H, int32_t Wd, const float *weight,
+                           const float *bias, int32_t out_f, float *y, void *stream);
 
 /* ------------------------------------------------------------------------------------------------
  * Chain of L fully-connected tiled layers (Sec. 5.1: an MLP with a fused ReLU):

@@ -74,6 +74,7 @@ SIGNATURES = {
     "tbn_linear_bin_fwd": (c_int, [c_vp, c_i64, c_i32, c_i32, c_vp, c_i32, c_vp, c_int, c_vp, c_vp, c_int, c_vp, c_int,
                                    c_vp, c_int]),
     "tbn_debug_force_attention_path": (c_int, [c_int]),
+    "tbn_avgpool_linear_fwd": (c_int, [c_vp, c_int, c_i32, c_i32, c_i32, c_i32, c_vp, c_vp, c_i32, c_vp, c_vp]),
     "tbn_bin_expand_fwd": (c_int, [c_vp, c_i64, c_i32, c_vp, c_vp, c_vp]),
     "tbn_binarize_bytes_fwd": (c_int, [c_vp, c_int, c_i64, c_i32, c_vp, c_vp, c_vp, c_vp, c_vp]),
     "tbn_linear_bin_bytes_fwd": (c_int, [c_vp, c_vp, c_i64, c_i32, c_i32, c_vp, c_i32, c_vp, c_int, c_vp, c_vp, c_int, c_vp,
@@ -477,6 +478,16 @@ def tbn_global_avgpool_fwd(x: torch.Tensor, y_dtype=None) -> torch.Tensor:
     yd = xd if y_dtype is None else y_dtype
     y = torch.empty((Nb, C), dtype=_torch_dtype(yd), device=x.device)
     _check(lib().tbn_global_avgpool_fwd(_ptr(x), xd, Nb, C, H, Wd, _ptr(y), yd, _stream()), "tbn_global_avgpool_fwd")
+    return y
+
+
+def tbn_avgpool_linear_fwd(x: torch.Tensor, weight: torch.Tensor, bias: torch.Tensor | None = None) -> torch.Tensor:
+    """Global average pooling followed by a dense fp32 classifier (weight: out_f x C) in one launch; y: Nb x out_f fp32."""
+    Nb, C, H, Wd = x.shape
+    out_f = weight.shape[0]
+    y = torch.empty((Nb, out_f), dtype=torch.float32, device=x.device)
+    _check(lib().tbn_avgpool_linear_fwd(_ptr(x), _dtype_code(x), Nb, C, H, Wd, _ptr(weight), _ptr(bias), out_f, _ptr(y),
+                                        _stream()), "tbn_avgpool_linear_fwd")
     return y
 
 

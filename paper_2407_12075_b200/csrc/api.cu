@@ -946,6 +946,17 @@ int tbn_global_avgpool_fwd(const void *x, int x_dtype, int32_t Nb, int32_t C, in
                ? TBN_OK : TBN_ERR_CUDA;
 }
 
+int tbn_avgpool_linear_fwd(const void *x, int x_dtype, int32_t Nb, int32_t C, int32_t H, int32_t Wd, const float *weight,
+                           const float *bias, int32_t out_f, float *y, void *stream)
+{
+    if (Nb < 0 || C <= 0 || H <= 0 || Wd <= 0 || out_f <= 0 || !valid_dtype(x_dtype) || !weight) return TBN_ERR_INVALID_ARG;
+    if (Nb == 0) return TBN_OK;
+    if (!x || !y) return TBN_ERR_INVALID_ARG;
+    if ((int64_t)H * Wd > 0x7fffffffLL || !avgpool_linear_supported(C)) return TBN_ERR_UNSUPPORTED;
+    return launch_avgpool_linear(x, x_dtype, Nb, C, H * Wd, weight, bias, out_f, y, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? TBN_OK : TBN_ERR_CUDA;
+}
+
 int64_t tbn_row_words(int32_t n) { return tbn_tile_words(n); }
 
 int tbn_binarize_fwd(const void *x, int x_dtype, int64_t T, int32_t in_f, uint32_t *x_bits, float *beta, void *stream)

@@ -200,6 +200,9 @@ bool dense_conv_supported(int32_t Cin, int32_t kh, int32_t kw);
 cudaError_t launch_dense_conv(const void *x, int x_dtype, const float *w, const float *bias, void *y, int y_dtype, int32_t Nb,
                               int32_t Cin, int32_t H, int32_t Wd, int32_t Cout, int32_t kh, int32_t kw, int32_t stride, int32_t pad,
                               int act, cudaStream_t s);
+bool avgpool_linear_supported(int32_t C);
+cudaError_t launch_avgpool_linear(const void *x, int x_dtype, int32_t Nb, int32_t C, int32_t hw, const float *w, const float *bias,
+                                  int32_t out_f, float *y, cudaStream_t s);
 cudaError_t launch_global_avgpool(const void *x, int x_dtype, int64_t planes, int32_t hw, void *y, int y_dtype, cudaStream_t s);
 
 // ---- layer fed with the compact form of the previous tiled layer's output (tc_linear_compact.cu) ---------

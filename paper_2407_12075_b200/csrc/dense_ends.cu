@@ -160,6 +160,64 @@ global_avgpool_kernel(const XT *__restrict__ x, int64_t planes, int32_t hw, YT *
 
 }  // namespace
 
+// Global average pooling and a dense classifier in one launch: a block per image first leaves the C channel means (fp32) in
+// shared memory, then its warps take the classes in turn (lanes split the channels, shuffle tree, bias added last).
+constexpr int kPlMaxC = 4096;
+template <typename XT>
+__global__ void __launch_bounds__(256)
+avgpool_linear_kernel(const XT *__restrict__ x, int32_t C, int32_t hw, const float *__restrict__ w, const float *__restrict__ bias,
+                      int32_t out_f, float *__restrict__ y)
+{
+    __shared__ float pooled[kPlMaxC];
+    const int64_t b = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (sizeof(XT) == 2 && hw % 8 == 0 && hw <= 512 && (reinterpret_cast<uintptr_t>(x) & 15u) == 0) {
+        // short bf16 planes (a few 16-byte pieces): a thread per channel, 16-byte loads
+        for (int32_t c = threadIdx.x; c < C; c += blockDim.x) {
+            const uint4 *plane = reinterpret_cast<const uint4 *>(x + (b * C + c) * (int64_t)hw);
+            float s = 0.0f;
+            for (int32_t i = 0; i < hw / 8; ++i) {
+                const uint4 u = __ldg(plane + i);
+                const uint32_t wv[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) s += __uint_as_float(wv[e] << 16) + __uint_as_float(wv[e] & 0xffff0000u);
+            }
+            pooled[c] = s / (float)hw;
+        }
+    } else
+    // a warp per channel plane: consecutive lanes read consecutive positions
+    for (int32_t c = warp; c < C; c += 8) {
+        const XT *plane = x + (b * C + c) * (int64_t)hw;
+        float s = 0.0f;
+        for (int32_t i = lane; i < hw; i += 32) s += load_as_float(plane, i);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+        if (lane == 0) pooled[c] = s / (float)hw;
+    }
+    __syncthreads();
+    for (int32_t o = warp; o < out_f; o += 8) {
+        const float *wr = w + (int64_t)o * C;
+        float s = 0.0f;
+        for (int32_t c = lane; c < C; c += 32) s = fmaf(__ldg(wr + c), pooled[c], s);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+        if (lane == 0) y[b * out_f + o] = s + (bias ? __ldg(bias + o) : 0.0f);
+    }
+}
+
+bool avgpool_linear_supported(int32_t C) { return C > 0 && C <= kPlMaxC; }
+
+cudaError_t launch_avgpool_linear(const void *x, int x_dtype, int32_t Nb, int32_t C, int32_t hw, const float *w, const float *bias,
+                                  int32_t out_f, float *y, cudaStream_t s)
+{
+    if (!avgpool_linear_supported(C)) return cudaErrorInvalidValue;
+    if (x_dtype == TBN_BF16)
+        avgpool_linear_kernel<<<(unsigned)Nb, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(x), C, hw, w, bias, out_f, y);
+    else
+        avgpool_linear_kernel<<<(unsigned)Nb, 256, 0, s>>>(static_cast<const float *>(x), C, hw, w, bias, out_f, y);
+    return cudaGetLastError();
+}
+
 bool dense_conv_supported(int32_t Cin, int32_t kh, int32_t kw) { return (int64_t)Cin * kh * kw * kDcCo <= kDcMaxW; }
 
 cudaError_t launch_dense_conv(const void *x, int x_dtype, const float *w, const float *bias, void *y, int y_dtype, int32_t Nb,

@@ -36,10 +36,30 @@ def test_global_avgpool_matches_numpy_mean(Nb, C, H, W):
     assert np.allclose(to_np64(y), ref, rtol=1e-5, atol=1e-6)
 
 
-def run_stack(x_dev, W0_dev, convs_dev, Wfc_dev):
+@pytest.mark.parametrize("Nb,C,H,W,out_f,bf16", [(3, 5, 1, 1, 2, True), (2, 256, 8, 8, 10, True), (1, 7, 5, 9, 33, False), (4, 300, 4, 4, 10, True)])
+def test_avgpool_plus_classifier_in_one_launch(Nb, C, H, W, out_f, bf16):
+    x = synth.normal(93, 0, Nb * C * H * W).reshape(Nb, C, H, W)
+    xin = synth.to_bf16_bits(x) if bf16 else x
+    Wfc = synth.normal(93, 1, out_f * C, C ** -0.5).reshape(out_f, C)
+    bias = synth.normal(93, 2, out_f, 0.1)
+    ref = O.widen(xin).mean(axis=(2, 3)) @ Wfc.astype(np.float64).T + bias.astype(np.float64)
+    y = B.tbn_avgpool_linear_fwd(to_dev(xin), to_dev(Wfc), to_dev(bias))
+    y0 = B.tbn_avgpool_linear_fwd(to_dev(xin), to_dev(Wfc))
+    torch.cuda.synchronize()
+    assert np.allclose(to_np64(y), ref, rtol=1e-5, atol=1e-5)
+    assert np.allclose(to_np64(y0), ref - bias.astype(np.float64), rtol=1e-5, atol=1e-5)
+    # and it agrees with the two separate calls (whose classifier rounds its operands to bf16 on the tensor path)
+    two = B.tbn_linear_fp_tile_fwd(B.tbn_global_avgpool_fwd(to_dev(xin), y_dtype=B.F32), out_f, to_dev(Wfc).reshape(-1), 1, y_dtype=B.F32)
+    torch.cuda.synchronize()
+    assert_close(to_np64(two), to_np64(y0), "separate calls against the fused one")
+
+
+def run_stack(x_dev, W0_dev, convs_dev, Wfc_dev, fused_tail=False):
     h = B.tbn_conv2d_dense_fwd(x_dev, W0_dev, 1, 1, act=B.ACT_RELU)
     for (tile, alpha, Cout, k, stride) in convs_dev:
         h = B.tbn_conv2d_fwd(h, Cout, 3, 3, stride, 1, tile, k, alpha, B.ALPHA_PER_TILE, act=B.ACT_RELU)
+    if fused_tail:
+        return B.tbn_avgpool_linear_fwd(h, Wfc_dev)
     pooled = B.tbn_global_avgpool_fwd(h, y_dtype=B.F32)
     return B.tbn_linear_fp_tile_fwd(pooled, Wfc_dev.shape[0], Wfc_dev.reshape(-1), 1, y_dtype=B.F32)
 
@@ -64,8 +84,10 @@ def test_small_stack_matches_oracle(Nb, H, chans, k):
     W0, convs, convs_dev, Wfc = make_stack(92, chans, k)
     ref = O.conv_stack(x, W0, convs, Wfc)
     y = run_stack(to_dev(x), to_dev(W0), convs_dev, to_dev(Wfc))
+    yf = run_stack(to_dev(x), to_dev(W0), convs_dev, to_dev(Wfc), fused_tail=True)
     torch.cuda.synchronize()
     assert_close(to_np64(y), ref, "conv stack")
+    assert_close(to_np64(yf), ref, "conv stack, pooling and classifier in one launch")
 
 
 def test_conv_stack_config_sampled_images():
