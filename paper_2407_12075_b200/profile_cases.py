@@ -6,7 +6,7 @@ of launches):
 Cases: linear_k2, linear_k16 (8192 x 8192, T = 8192), bin_k2, bin_k16 (binary activations, 8192 x 8192, T = 4096),
 binbytes_k2, binbytes_k16 (the same with the activation signs as bytes),
 conv_s2 (64 -> 128, 32 x 32, batch 64), attention (64 images x 12 heads x 197 tokens), binarize, tile_bwd,
-compact_gelu (second MLP layer of a ViT-B block fed the first layer's 384 distinct pre-activations, T = 25,216).
+first_conv (dense 3 -> 64, 32 x 32, batch 256), compact_gelu (second MLP layer of a ViT-B block fed the first layer's 384 distinct pre-activations, T = 25,216).
 Inputs are seeded device-side random values of the benchmark's shapes; every run checks the device status word.
 """
 from __future__ import annotations
@@ -68,6 +68,10 @@ def main():
         tile = rand_tile(d * mlp // k)
         a1, a2 = torch.rand(k, device=dev, generator=gen) * 0.05, torch.rand(k, device=dev, generator=gen) * 0.02
         run = lambda: B.tbn_linear_compact_fwd(z, k, a1, B.ALPHA_PER_TILE, B.ACT_GELU, d, tile, k, a2, B.ALPHA_PER_TILE, y=y)
+    elif args.case == "first_conv":
+        xc = torch.rand(256, 3, 32, 32, device=dev, generator=gen).to(torch.bfloat16)
+        W0 = torch.randn(64, 3, 3, 3, device=dev, generator=gen) * 0.27
+        run = lambda: B.tbn_conv2d_dense_fwd(xc, W0, 1, 1, act=B.ACT_RELU)
     elif args.case == "tile_bwd":
         N, k = 4096 * 4096, 4
         W = torch.randn(N, device=dev, generator=gen) * 0.02
