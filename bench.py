@@ -196,15 +196,29 @@ def oracle_sample(x_bits: np.ndarray, W: np.ndarray, k: int, rows: int, seed: in
 def run_reference(args, T: int):
     """--impl reference: the oracle as it stands, on the host cores, on a bounded sample per step."""
     from paper_2407_12075_b200 import synth
-    rows = 64
-    x = synth.to_bf16_bits(synth.normal(SEED, 0, rows * N_FEAT).reshape(rows, N_FEAT))
     W = synth.normal(SEED, 1, N_FEAT * N_FEAT, 0.02).reshape(N_FEAT, N_FEAT)
-    times, cores = [], 1
-    for step in range(args.warmup + args.steps):
+    # Tiles are prepared once (not part of a step).  The sample per step is sized so that all steps together take about two
+    # minutes: an untimed probe of 4 rows gives the oracle's time per token row on this host, then 1..64 rows per step.
+    from oracle import tbn_oracle as O
+    prepared = {k: O.prepare(W, k, True) for k in KS}
+
+    def step_seconds(xs):
         t = 0.0
         for k in KS:
-            dt, n, cores = oracle_sample(x, W, k, rows)[:3]
-            t += dt
+            words, al = prepared[k]
+            t0 = time.perf_counter()
+            O.linear(xs, words, k, al, True, N_FEAT, N_FEAT)
+            t += time.perf_counter() - t0
+        return t
+
+    probe = synth.to_bf16_bits(synth.normal(SEED, 2, 4 * N_FEAT).reshape(4, N_FEAT))
+    per_row = step_seconds(probe) / 4.0
+    rows = int(max(1, min(64, 120.0 / ((args.warmup + args.steps) * max(per_row, 1e-6)))))
+    x = synth.to_bf16_bits(synth.normal(SEED, 0, rows * N_FEAT).reshape(rows, N_FEAT))
+    cores = O.num_threads()
+    times = []
+    for step in range(args.warmup + args.steps):
+        t = step_seconds(x)
         if step >= args.warmup:
             times.append(t)
     ms = 1e3 * float(np.mean(times))
