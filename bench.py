@@ -197,35 +197,35 @@ def run_reference(args, T: int):
     """--impl reference: the oracle as it stands, on the host cores, on a bounded sample per step."""
     from paper_2407_12075_b200 import synth
     W = synth.normal(SEED, 1, N_FEAT * N_FEAT, 0.02).reshape(N_FEAT, N_FEAT)
-    # Tiles are prepared once (not part of a step).  The sample per step is sized so that all steps together take about two
-    # minutes: an untimed probe of 4 rows gives the oracle's time per token row on this host, then 1..64 rows per step.
+    # Tiles are prepared once (not part of a step).  The oracle's layer call has a large fixed cost (it expands the tile to
+    # the dense weight matrix), so the sample of a step is bounded in two ways: at most 64 token rows, and -- when all steps
+    # with all four k would take more than about two minutes -- one k per step, taken in turn.
     from oracle import tbn_oracle as O
     prepared = {k: O.prepare(W, k, True) for k in KS}
-
-    def step_seconds(xs):
-        t = 0.0
-        for k in KS:
-            words, al = prepared[k]
-            t0 = time.perf_counter()
-            O.linear(xs, words, k, al, True, N_FEAT, N_FEAT)
-            t += time.perf_counter() - t0
-        return t
-
-    probe = synth.to_bf16_bits(synth.normal(SEED, 2, 4 * N_FEAT).reshape(4, N_FEAT))
-    per_row = step_seconds(probe) / 4.0
-    rows = int(max(1, min(64, 120.0 / ((args.warmup + args.steps) * max(per_row, 1e-6)))))
+    rows = 64
     x = synth.to_bf16_bits(synth.normal(SEED, 0, rows * N_FEAT).reshape(rows, N_FEAT))
+
+    def layer_seconds(k):
+        words, al = prepared[k]
+        t0 = time.perf_counter()
+        O.linear(x, words, k, al, True, N_FEAT, N_FEAT)
+        return time.perf_counter() - t0
+
+    probe = sum(layer_seconds(k) for k in KS)                 # untimed: decides the sampling
+    n_steps = args.warmup + args.steps
+    rotate = n_steps * probe > 120.0
     cores = O.num_threads()
-    times = []
-    for step in range(args.warmup + args.steps):
-        t = step_seconds(x)
+    t_sum, f_sum = 0.0, 0.0
+    for step in range(n_steps):
+        ks = (KS[step % len(KS)],) if rotate else KS
+        t = sum(layer_seconds(k) for k in ks)
         if step >= args.warmup:
-            times.append(t)
-    ms = 1e3 * float(np.mean(times))
-    flops = sum(algorithmic_flops(rows, k) for k in KS)
-    value = flops / (ms * 1e-3) / 1e12
-    sample = (f"{rows} of {T} token rows x all 8192 outputs, each k in {list(KS)}; dense fp64 product "
-              f"(the oracle never uses the replicated-row shortcut); value counts algorithmic flops")
+            t_sum += t
+            f_sum += sum(algorithmic_flops(rows, k) for k in ks)
+    ms = 1e3 * t_sum / max(args.steps, 1)
+    value = f_sum / max(t_sum, 1e-12) / 1e12
+    sample = (f"{rows} of {T} token rows x all 8192 outputs, " + (f"one k of {list(KS)} per step in turn" if rotate else f"each k in {list(KS)}") +
+              "; dense fp64 product (the oracle never uses the replicated-row shortcut); value counts algorithmic flops")
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
                 ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64",
                 data="synthetic", impl="reference",
